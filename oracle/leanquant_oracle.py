@@ -1,0 +1,341 @@
+"""Float64 CPU oracle for the LeanQuant per-linear-layer pass (Algorithm 1).
+
+TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what the
+pass computes; the CUDA library is checked against it.  It shares no code with
+the CUDA path and must never be imported by it: only tests, the smoke check and
+the benchmark's CPU-baseline leg call it.
+
+Everything is numpy float64.  Inputs in a narrower type (bf16 / fp32) are widened
+exactly by the caller.  Notation follows the paper: W is r x c, X is c x n,
+H = 2 X X^T, K = 2^b grid points, B the block width of the column loop.
+
+Where the paper leaves a detail open this file takes one reading and says so at
+the spot; the design notes list all of them.
+
+Pinned by tests/test_oracle_pins.py against: brute-force fixed-order OBQ with the
+explicit inverse-Hessian downdate (column loop), the trace identity of the damped
+proxy loss, H = I giving round-to-nearest, dynamic-programming optimal weighted
+1-D k-means, an independently written plain Lloyd for p = 0, the worked 2-bit grid
+example of Appendix A, a triple-loop affine search, textbook library inverses and
+Cholesky factors, and scale / permutation / row-subset invariances.  The numbers
+it produces on the benchmark configurations themselves are not printed anywhere in
+the paper: for those, parity is "unpinned" beyond these properties.
+"""
+from __future__ import annotations
+
+import numpy as np
+import scipy.linalg as sla
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------- #
+# Stage 1 -- Algorithm 1 line 3, Section 2.2: H = 2 X X^T
+# --------------------------------------------------------------------------- #
+def hessian(X_chunks, alpha: float = 2.0, H: np.ndarray | None = None) -> np.ndarray:
+    """H (+)= alpha * sum_chunks X_chunk X_chunk^T.  ``X_chunks`` is one c x n array
+    or an iterable of c x n_i arrays (tokens may arrive in pieces; the sum is the same)."""
+    if isinstance(X_chunks, np.ndarray):
+        X_chunks = [X_chunks]
+    for Xc in X_chunks:
+        Xc = np.asarray(Xc, dtype=F64)
+        G = alpha * (Xc @ Xc.T)
+        H = G if H is None else H + G
+    return H
+
+
+# --------------------------------------------------------------------------- #
+# Stage 2 -- Algorithm 1 line 4 and the "Cholesky and Dampening" paragraph
+# --------------------------------------------------------------------------- #
+def prepare_hinv(H: np.ndarray, damp_frac: float = 0.01, W: np.ndarray | None = None):
+    """Dampen, invert, factor.
+
+    Returns (U, dinv, H_d, W_fixed):
+      H_d  = H + damp_frac * mean(diag H) * I           (1 % of the average diagonal)
+      dinv = diag(H_d^-1)
+      U    = the upper-triangular Cholesky factor of H_d^-1, H_d^-1 = U^T U, U_jj > 0.
+
+    Reading: the factor is the *upper* one.  Only then do the rows "H^-1[j, j:]" used
+    by lines 17-20 of Algorithm 1 reproduce Eq. 3 with the Eq. 9 downdate.
+    Reading (the paper is silent; GPTQ's convention, on which the method builds): an
+    input channel that never fires (H_ii = 0) gets H_ii = 1 and its weight column is
+    zeroed before anything else.
+    """
+    H = np.array(H, dtype=F64, copy=True)
+    c = H.shape[0]
+    dead = np.diag(H) == 0.0
+    if dead.any():
+        H[dead, dead] = 1.0
+    if W is not None:
+        W = np.array(W, dtype=F64, copy=True)
+        W[:, dead] = 0.0
+    damp = damp_frac * np.mean(np.diag(H))
+    H_d = H + damp * np.eye(c)
+    Hinv = sla.inv(H_d)
+    dinv = np.diag(Hinv).copy()
+    U = sla.cholesky(Hinv, lower=False)
+    return U, dinv, H_d, W
+
+
+# --------------------------------------------------------------------------- #
+# Stage 3 -- loss-error-aware grids
+# --------------------------------------------------------------------------- #
+def sample_weights(dinv: np.ndarray, p: float) -> np.ndarray:
+    """s_j = (H^-1_jj)^(-p), Eq. 5 / Eq. 7, divided by its geometric mean.
+
+    Reading: the common factor changes neither the arg-min of Eq. 5 / Eq. 7 nor any
+    Lloyd centroid; it is taken out so that p = 4 cannot overflow a narrow float."""
+    ld = np.log(np.asarray(dinv, dtype=F64))
+    return np.exp(-p * (ld - ld.mean()))
+
+
+def grid_init_uniform(w_min, w_max, K: int) -> np.ndarray:
+    """Eq. 6: K evenly spaced points from min(w) to max(w), per row."""
+    t = np.arange(K, dtype=F64)
+    w_min = np.asarray(w_min, dtype=F64)[..., None]
+    w_max = np.asarray(w_max, dtype=F64)[..., None]
+    return w_min + (w_max - w_min) * t / (K - 1)
+
+
+def grid_init_weighted_quantile(W: np.ndarray, s: np.ndarray, K: int) -> np.ndarray:
+    """Alternative deterministic init: per row, sort ascending, accumulate sample
+    weight, and take the value at the first position whose cumulative weight reaches
+    (k + 1/2)/K of the total, k = 0..K-1."""
+    W = np.asarray(W, dtype=F64)
+    r, c = W.shape
+    G = np.empty((r, K), dtype=F64)
+    for i in range(r):
+        order = np.argsort(W[i], kind="stable")
+        cw = np.cumsum(s[order])
+        for k in range(K):
+            pos = int(np.searchsorted(cw, (k + 0.5) / K * cw[-1], side="left"))
+            G[i, k] = W[i, order[min(pos, c - 1)]]
+    return G
+
+
+def assign_nu(w: np.ndarray, grid: np.ndarray) -> np.ndarray:
+    """quant_nu's arg-min as an index.  ``grid`` is ascending along its last axis;
+    the nearest point is found by counting the midpoints m_k = (g_k + g_{k+1})/2 that
+    lie strictly below w, so a weight exactly on a midpoint takes the lower point.
+    w: (..., c), grid: (..., K) -> codes (..., c) in 0..K-1."""
+    mid = 0.5 * (grid[..., :-1] + grid[..., 1:])
+    return (w[..., :, None] > mid[..., None, :]).sum(axis=-1)
+
+
+def fit_grid_nonuniform(W, dinv, bits: int, p: float = 4.0, n_iter: int = 20,
+                        init: str = "uniform", return_trace: bool = False):
+    """Eq. 5 by Lloyd's algorithm, one independent problem per row.
+
+    K = 2^bits centroids, sample weights ``sample_weights(dinv, p)`` shared by all rows,
+    start from Eq. 6 (or the weighted-quantile alternative), then exactly ``n_iter``
+    rounds of: assign every weight to its nearest centroid (``assign_nu``), move each
+    centroid to the weighted mean of its members.  Readings: a fixed iteration count
+    with no early stop; a centroid whose members carry zero total weight stays where
+    it was.  Centroids remain ascending.
+    """
+    W = np.asarray(W, dtype=F64)
+    r, c = W.shape
+    K = 1 << bits
+    s = sample_weights(dinv, p)
+    if init == "uniform":
+        G = grid_init_uniform(W.min(axis=1), W.max(axis=1), K)
+    elif init == "weighted_quantile":
+        G = grid_init_weighted_quantile(W, s, K)
+    else:
+        raise ValueError(init)
+    trace = []
+    for _ in range(n_iter):
+        a = assign_nu(W, G)
+        if return_trace:
+            trace.append(float((s * (np.take_along_axis(G, a, 1) - W) ** 2).sum()))
+        for k in range(K):
+            member = a == k
+            den = (member * s).sum(axis=1)
+            num = (member * (s * W)).sum(axis=1)
+            ok = den > 0.0
+            G[ok, k] = num[ok] / den[ok]
+    if return_trace:
+        a = assign_nu(W, G)
+        trace.append(float((s * (np.take_along_axis(G, a, 1) - W) ** 2).sum()))
+        return G, trace
+    return G
+
+
+def affine_codes(w, S, Z, K: int):
+    """w_int = clip(round(w / S) + Z, 0, K - 1) with round-half-to-even."""
+    return np.clip(np.rint(w / S) + Z, 0, K - 1)
+
+
+def quant_aff(w, S, Z, K: int):
+    """quant_aff(w, S, Z) = (w_int - Z) * S."""
+    return (affine_codes(w, S, Z, K) - Z) * S
+
+
+def affine_candidate(mn: float, mx: float, t_min: int, t_max: int, T: int, K: int):
+    """One element of the search space of Eq. 7: shrink the range by t_min*R/T from
+    below and t_max*R/T from above; S = (hi - lo)/(K-1), Z = -round(lo/S).
+    Reading for a constant group (R = 0): widen the range to include 0; if it is
+    still empty use S = 1, Z = 0 (the constant is then reproduced exactly when it is
+    an integer in range, and this only matters for all-equal groups)."""
+    R = mx - mn
+    if R == 0.0:
+        lo, hi = min(mn, 0.0), max(mx, 0.0)
+        if hi == lo:
+            return 1.0, 0.0
+        S = (hi - lo) / (K - 1)
+        return S, -np.rint(lo / S)
+    lo = mn + t_min * R / T
+    hi = mx - t_max * R / T
+    S = (hi - lo) / (K - 1)
+    if not S > 0.0:
+        return None
+    return S, -np.rint(lo / S)
+
+
+def fit_grid_affine(W, dinv, bits: int, p: float = 4.0, group: int = 0,
+                    T: int = 2048, t: int | None = None):
+    """Eq. 7: enumerate (t_min, t_max) in {0..t}^2 per (row, group) and keep the pair
+    (S, Z) with the least weighted squared error; ties keep the first candidate in
+    t_min-major, t_max-minor order.  ``group`` = 0 means one group per row.
+    Appendix B: t = 0.2T / 0.3T / 0.4T for 4 / 3 / 2 bits (floored to an integer).
+    Returns scale (r x n_groups) and zero (r x n_groups, integer-valued float64)."""
+    W = np.asarray(W, dtype=F64)
+    r, c = W.shape
+    K = 1 << bits
+    if t is None:
+        t = int(np.floor({4: 0.2, 3: 0.3, 2: 0.4}[bits] * T))
+    g = c if group in (0, None) else group
+    if c % g:
+        raise ValueError("c must be a multiple of the group size")
+    ng = c // g
+    s = sample_weights(dinv, p)
+    scale = np.empty((r, ng), dtype=F64)
+    zero = np.empty((r, ng), dtype=F64)
+    for gi in range(ng):
+        w = W[:, gi * g:(gi + 1) * g]
+        sg = s[gi * g:(gi + 1) * g]
+        mn = w.min(axis=1)
+        mx = w.max(axis=1)
+        R = mx - mn
+        best = np.full(r, np.inf)
+        bS = np.ones(r)
+        bZ = np.zeros(r)
+        flat = R == 0.0
+        for i in np.nonzero(flat)[0]:
+            bS[i], bZ[i] = affine_candidate(mn[i], mx[i], 0, 0, T, K)
+        live = ~flat
+        if live.any():
+            wl, mnl, mxl, Rl = w[live], mn[live], mx[live], R[live]
+            bl = np.full(wl.shape[0], np.inf)
+            Sl = np.ones(wl.shape[0])
+            Zl = np.zeros(wl.shape[0])
+            for t_min in range(t + 1):
+                lo = mnl + t_min * Rl / T
+                for t_max in range(t + 1):
+                    hi = mxl - t_max * Rl / T
+                    S = (hi - lo) / (K - 1)
+                    valid = S > 0.0
+                    Ssafe = np.where(valid, S, 1.0)
+                    Z = -np.rint(lo / Ssafe)
+                    q = quant_aff(wl, Ssafe[:, None], Z[:, None], K)
+                    loss = (sg * (q - wl) ** 2).sum(axis=1)
+                    better = valid & (loss < bl)
+                    bl[better] = loss[better]
+                    Sl[better] = S[better]
+                    Zl[better] = Z[better]
+            bS[live], bZ[live] = Sl, Zl
+        scale[:, gi], zero[:, gi] = bS, bZ
+    return scale, zero
+
+
+# --------------------------------------------------------------------------- #
+# Stage 4 -- Algorithm 1 lines 10-21: block-wise column loop with error feedback
+# --------------------------------------------------------------------------- #
+def quantize_layer(W, U, *, grid=None, scale=None, zero=None, bits: int = 4,
+                   group: int = 0, block: int = 128):
+    """The iterative loss-error-based loop on a learned grid.
+
+    For each block of ``block`` columns, for each column j in it: quantise W[:, j] for
+    all rows (nearest point of the row's grid, or quant_aff with the parameters of
+    group j // group), E[:, j-i] = (W[:, j] - What[:, j]) / U[j, j], and
+    W[:, j:i+B] -= E[:, j-i] * U[j, j:i+B] inside the block; after the block
+    W[:, i+B:] -= E @ U[i:i+B, i+B:].
+
+    Returns codes (r x c, int64), W_hat (r x c) and loss = 1/2 * sum(E^2), the summed
+    loss error of Eq. 3 with the damped inverse."""
+    Wc = np.array(W, dtype=F64, copy=True)
+    U = np.asarray(U, dtype=F64)
+    r, c = Wc.shape
+    K = 1 << bits
+    codes = np.zeros((r, c), dtype=np.int64)
+    What = np.zeros((r, c), dtype=F64)
+    loss = 0.0
+    g = c if group in (0, None) else group
+    for i in range(0, c, block):
+        e_end = min(i + block, c)
+        E = np.zeros((r, e_end - i), dtype=F64)
+        for j in range(i, e_end):
+            w = Wc[:, j]
+            if grid is not None:
+                a = assign_nu(w[:, None], grid)[:, 0]
+                q = np.take_along_axis(grid, a[:, None], 1)[:, 0]
+            else:
+                S = scale[:, j // g]
+                Z = zero[:, j // g]
+                a = affine_codes(w, S, Z, K)
+                q = (a - Z) * S
+            codes[:, j] = a
+            What[:, j] = q
+            e = (w - q) / U[j, j]
+            E[:, j - i] = e
+            Wc[:, j:e_end] -= np.outer(e, U[j, j:e_end])
+        loss += 0.5 * float((E * E).sum())
+        if e_end < c:
+            Wc[:, e_end:] -= E @ U[i:e_end, e_end:]
+    return codes, What, loss
+
+
+def proxy_loss(W, What, H) -> float:
+    """tr((W - What) H (W - What)^T); with the undamped H = 2XX^T this is
+    2 * ||W X - What X||_F^2, the layer objective of Eq. 1 up to the factor 2."""
+    D = np.asarray(W, dtype=F64) - np.asarray(What, dtype=F64)
+    return float(np.einsum("ij,ij->", D @ np.asarray(H, dtype=F64), D))
+
+
+# --------------------------------------------------------------------------- #
+# Baseline grids used for the loss comparison of ablation Q1
+# --------------------------------------------------------------------------- #
+def minmax_affine_params(W, bits: int, group: int = 0):
+    """Plain min-max asymmetric affine grid of Section 2.1: S = (max - min)/(K-1),
+    Z = -round(min / S), per (row, group)."""
+    W = np.asarray(W, dtype=F64)
+    r, c = W.shape
+    K = 1 << bits
+    g = c if group in (0, None) else group
+    ng = c // g
+    scale = np.empty((r, ng))
+    zero = np.empty((r, ng))
+    for gi in range(ng):
+        w = W[:, gi * g:(gi + 1) * g]
+        for i in range(r):
+            scale[i, gi], zero[i, gi] = affine_candidate(w[i].min(), w[i].max(), 0, 0, 1, K)
+    return scale, zero
+
+
+def run_pass(W, X, *, grid_type="nonuniform", bits=4, p=4.0, block=128, damp=0.01,
+             n_iter=20, init="uniform", group=0, T=2048, t=None, alpha=2.0):
+    """Algorithm 1 end to end; returns a dict with every intermediate."""
+    H = hessian(X, alpha)
+    U, dinv, H_d, Wf = prepare_hinv(H, damp, W)
+    out = dict(H=H, U=U, dinv=dinv, H_d=H_d)
+    if grid_type == "nonuniform":
+        G = fit_grid_nonuniform(Wf, dinv, bits, p, n_iter, init)
+        codes, What, loss = quantize_layer(Wf, U, grid=G, bits=bits, block=block)
+        out.update(grid=G)
+    else:
+        S, Z = fit_grid_affine(Wf, dinv, bits, p, group, T, t)
+        codes, What, loss = quantize_layer(Wf, U, scale=S, zero=Z, bits=bits, group=group, block=block)
+        out.update(scale=S, zero=Z)
+    out.update(codes=codes, W_hat=What, loss=loss, proxy=proxy_loss(Wf, What, H),
+               proxy_d=proxy_loss(Wf, What, H_d))
+    return out

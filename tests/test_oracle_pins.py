@@ -1,0 +1,395 @@
+"""Pins for the float64 oracle: each test checks it against something that is not
+the oracle itself -- a brute-force statement of the paper's equations, a closed
+form, a value the paper prints, or a textbook library routine.  CPU only."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import synth
+from oracle import leanquant_oracle as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def rng(seed):
+    return np.random.default_rng(seed)
+
+
+def spd(c, seed, cond=1e3):
+    """Random symmetric positive definite matrix with a prescribed spectrum."""
+    g = rng(seed)
+    Q, _ = np.linalg.qr(g.standard_normal((c, c)))
+    lam = np.logspace(0, np.log10(cond), c)
+    return (Q * lam) @ Q.T
+
+
+# ------------------------------------------------------------------ P1 ---- #
+def obq_fixed_order(W, Hinv, quant_row):
+    """Eq. 3 and Eq. 9 taken literally, column by column in fixed order:
+    quantise w_j, w <- w - (w_j - q)/Hinv_jj * Hinv[:, j], then remove row/column j
+    from the inverse by Hinv <- Hinv - Hinv[:, j] Hinv[j, :]/Hinv_jj."""
+    W = W.copy()
+    Hinv = Hinv.copy()
+    r, c = W.shape
+    Q = np.zeros_like(W)
+    eps = 0.0
+    for j in range(c):
+        d = Hinv[j, j]
+        for k in range(r):
+            q = quant_row(k, j, W[k, j])
+            Q[k, j] = q
+            delta = (q - W[k, j]) / d * Hinv[:, j]
+            eps += 0.5 * (q - W[k, j]) ** 2 / d
+            W[k, :] += delta
+            W[k, j] = q
+        Hinv = Hinv - np.outer(Hinv[:, j], Hinv[j, :]) / d
+    return Q, eps
+
+
+@pytest.mark.parametrize("c,block", [(8, 3), (24, 8), (48, 128), (64, 16)])
+def test_p1_column_loop_equals_explicit_obq(c, block):
+    g = rng(c)
+    r = 5
+    W = g.standard_normal((r, c)) * 0.05
+    H = spd(c, 7 + c, 1e2)
+    U, dinv, H_d, _ = O.prepare_hinv(H, 0.01)
+    grid = np.sort(g.standard_normal((r, 4)) * 0.05, axis=1)
+
+    def quant_row(k, j, w):
+        return grid[k, np.argmin(np.abs(grid[k] - w))]
+
+    Q_ref, eps_ref = obq_fixed_order(W, np.linalg.inv(H_d), quant_row)
+    codes, What, loss = O.quantize_layer(W, U, grid=grid, bits=2, block=block)
+    assert np.array_equal(np.take_along_axis(grid, codes, 1), What)
+    np.testing.assert_allclose(What, Q_ref, rtol=0, atol=1e-10)
+    np.testing.assert_allclose(loss, eps_ref, rtol=1e-9)
+
+
+def test_p1b_block_size_does_not_matter():
+    g = rng(3)
+    r, c = 6, 40
+    W = g.standard_normal((r, c))
+    U, *_ = O.prepare_hinv(spd(c, 11, 1e3), 0.01)
+    grid = O.grid_init_uniform(W.min(1), W.max(1), 8)
+    ref = O.quantize_layer(W, U, grid=grid, bits=3, block=c)
+    for B in (1, 7, 16, 128):
+        out = O.quantize_layer(W, U, grid=grid, bits=3, block=B)
+        assert np.array_equal(out[0], ref[0])
+        np.testing.assert_allclose(out[2], ref[2], rtol=1e-12)
+
+
+# ------------------------------------------------------------------ P2 ---- #
+def test_p2_damped_proxy_equals_twice_loss():
+    g = rng(5)
+    r, c = 7, 32
+    W = g.standard_normal((r, c)) * 0.1
+    X = g.standard_normal((c, 100)) * np.exp(g.standard_normal(c))[:, None]
+    out = O.run_pass(W, X, bits=3, block=8, n_iter=5)
+    np.testing.assert_allclose(out["proxy_d"], 2.0 * out["loss"], rtol=1e-9)
+
+
+# ------------------------------------------------------------------ P3 ---- #
+def test_p3_identity_hessian_is_round_to_nearest():
+    g = rng(9)
+    r, c = 9, 50
+    W = g.standard_normal((r, c))
+    U, dinv, _, _ = O.prepare_hinv(np.eye(c), 0.01)
+    assert np.allclose(U, np.diag(np.diag(U)))
+    G = O.fit_grid_nonuniform(W, dinv, 3, 4.0, 10)
+    codes, What, _ = O.quantize_layer(W, U, grid=G, bits=3, block=16)
+    nearest = np.abs(W[:, :, None] - G[:, None, :]).argmin(-1)
+    assert np.array_equal(codes, nearest)
+    assert np.array_equal(What, np.take_along_axis(G, nearest, 1))
+
+
+# ------------------------------------------------------------------ P4 ---- #
+def kmeans_dp_optimum(w, s, K):
+    """Optimal weighted 1-D K-means cost by dynamic programming over sorted points:
+    clusters of a 1-D optimum are contiguous in sorted order."""
+    order = np.argsort(w)
+    w, s = w[order], s[order]
+    n = len(w)
+
+    def cost(a, b):  # points a..b-1 in one cluster
+        ss = s[a:b].sum()
+        mu = (s[a:b] * w[a:b]).sum() / ss
+        return (s[a:b] * (w[a:b] - mu) ** 2).sum()
+
+    D = np.full((K + 1, n + 1), np.inf)
+    D[0, 0] = 0.0
+    for k in range(1, K + 1):
+        for b in range(1, n + 1):
+            for a in range(k - 1, b):
+                if D[k - 1, a] < np.inf:
+                    D[k, b] = min(D[k, b], D[k - 1, a] + cost(a, b))
+    return D[1:, n].min()
+
+
+def objective(w, s, grid):
+    return float((s * (np.abs(w[:, None] - grid[None, :]).min(1)) ** 2).sum())
+
+
+def test_p4_lloyd_vs_dp_optimum():
+    g = rng(21)
+    for trial in range(6):
+        c, K = 20, 4
+        w = g.standard_normal(c)
+        dinv = np.exp(g.standard_normal(c))
+        s = O.sample_weights(dinv, 2.0)
+        G, trace = O.fit_grid_nonuniform(w[None], dinv, 2, 2.0, 30, return_trace=True)
+        opt = kmeans_dp_optimum(w, s, K)
+        assert objective(w, s, G[0]) >= opt * (1 - 1e-12)
+        assert all(b <= a * (1 + 1e-12) for a, b in zip(trace, trace[1:]))
+        np.testing.assert_allclose(trace[-1], objective(w, s, G[0]), rtol=1e-12)
+    # four well-separated clumps: Lloyd from the evenly spaced start reaches the optimum
+    centres = np.array([-3.0, -1.0, 1.0, 3.0])
+    w = (centres[:, None] + 0.05 * g.standard_normal((4, 6))).ravel()
+    dinv = np.exp(0.3 * g.standard_normal(w.size))
+    s = O.sample_weights(dinv, 4.0)
+    G = O.fit_grid_nonuniform(w[None], dinv, 2, 4.0, 20)
+    np.testing.assert_allclose(objective(w, s, G[0]), kmeans_dp_optimum(w, s, 4), rtol=1e-10)
+
+
+# ------------------------------------------------------------------ P5 ---- #
+def plain_lloyd(w, K, n_iter):
+    """Unweighted Lloyd from evenly spaced centres, written with explicit loops."""
+    lo, hi = min(w), max(w)
+    g = [lo + (hi - lo) * t / (K - 1) for t in range(K)]
+    for _ in range(n_iter):
+        members = [[] for _ in range(K)]
+        for x in w:
+            best = 0
+            for k in range(1, K):
+                if abs(x - g[k]) < abs(x - g[best]):
+                    best = k
+            members[best].append(x)
+        g = [sum(m) / len(m) if m else g[k] for k, m in enumerate(members)]
+    return g
+
+
+def test_p5_p_zero_is_plain_lloyd():
+    g = rng(33)
+    W = g.standard_normal((4, 200))
+    dinv = np.exp(2 * g.standard_normal(200))
+    G = O.fit_grid_nonuniform(W, dinv, 3, 0.0, 12)
+    for i in range(4):
+        np.testing.assert_allclose(G[i], plain_lloyd(list(W[i]), 8, 12), rtol=1e-12, atol=1e-14)
+    assert np.allclose(O.sample_weights(dinv, 0.0), 1.0)
+
+
+# ------------------------------------------------------------------ P6 ---- #
+def test_p6_appendix_a_worked_example():
+    rows = {}
+    for line in open(os.path.join(GOLDEN, "appendix_a_grid.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        key, *vals = line.split()
+        rows[key] = [float(v) for v in vals]
+    mn, mx, bits = rows["range"]
+    G = O.grid_init_uniform([mn], [mx], 1 << int(bits))[0]
+    np.testing.assert_allclose(G, rows["grid"], atol=0.005)      # printed to 2 decimals
+    w, nearest = rows["nearest"]
+    code = O.assign_nu(np.array([[w]]), G[None])[0, 0]
+    assert abs(G[code] - nearest) < 0.005
+    assert abs(G[code] - 1 / 3) < 1e-15
+
+
+def test_p6b_appendix_b_shrink_defaults():
+    spec = {}
+    for line in open(os.path.join(GOLDEN, "appendix_b_shrink.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        k, v = line.split()
+        spec[k] = float(v)
+    T = int(spec.pop("T"))
+    g = rng(2)
+    w = g.standard_normal((1, 16))
+    dinv = np.ones(16)
+    for bits, frac in spec.items():
+        bits = int(bits)
+        # the default t equals floor(frac*T): compare on a coarse T where the search is cheap
+        Tc = 40
+        a = O.fit_grid_affine(w, dinv, bits, 0.0, 0, T=Tc, t=None)
+        b = O.fit_grid_affine(w, dinv, bits, 0.0, 0, T=Tc, t=int(np.floor(frac * Tc)))
+        assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+
+
+# ------------------------------------------------------------------ P7 ---- #
+def affine_bruteforce(w, s, bits, T, t):
+    """Eq. 7 with explicit scalar loops (Python round() is round-half-to-even)."""
+    K = (1 << bits) - 1
+    mn, mx = min(w), max(w)
+    R = mx - mn
+    best = (float("inf"), None, None)
+    for t_min in range(t + 1):
+        for t_max in range(t + 1):
+            lo = mn + t_min * R / T
+            hi = mx - t_max * R / T
+            S = (hi - lo) / K
+            if S <= 0:
+                continue
+            Z = -round(lo / S)
+            loss = 0.0
+            for wi, si in zip(w, s):
+                q = min(max(round(wi / S) + Z, 0), K)
+                loss += si * ((q - Z) * S - wi) ** 2
+            if loss < best[0]:
+                best = (loss, S, Z)
+    return best
+
+
+def test_p7_affine_search():
+    g = rng(41)
+    r, c, group = 5, 32, 16
+    W = g.standard_normal((r, c)) * 0.03
+    W[0, 3] = 0.4          # an outlier the search should clip away from
+    dinv = np.exp(g.standard_normal(c))
+    s = O.sample_weights(dinv, 2.0)
+    for bits in (2, 4):
+        S, Z = O.fit_grid_affine(W, dinv, bits, 2.0, group, T=24, t=6)
+        S0, Z0 = O.fit_grid_affine(W, dinv, bits, 2.0, group, T=24, t=0)
+        Sm, Zm = O.minmax_affine_params(W, bits, group)
+        np.testing.assert_allclose(S0, Sm, rtol=1e-15)
+        assert np.array_equal(Z0, Zm)
+        K = 1 << bits
+        for i in range(r):
+            for gi in range(c // group):
+                w = W[i, gi * group:(gi + 1) * group]
+                sg = s[gi * group:(gi + 1) * group]
+                loss_b, S_b, Z_b = affine_bruteforce(list(w), list(sg), bits, 24, 6)
+                np.testing.assert_allclose(S[i, gi], S_b, rtol=1e-14)
+                assert Z[i, gi] == Z_b
+                mine = float((sg * (O.quant_aff(w, S[i, gi], Z[i, gi], K) - w) ** 2).sum())
+                mm = float((sg * (O.quant_aff(w, Sm[i, gi], Zm[i, gi], K) - w) ** 2).sum())
+                np.testing.assert_allclose(mine, loss_b, rtol=1e-12)
+                assert mine <= mm * (1 + 1e-12)
+                # min-max formulas of Section 2.1
+                assert np.isclose(Sm[i, gi], (w.max() - w.min()) / (K - 1))
+                assert Zm[i, gi] == -round(w.min() / Sm[i, gi])
+    # constant group: reproduced exactly
+    Wc = np.full((1, 8), 0.25)
+    S, Z = O.fit_grid_affine(Wc, np.ones(8), 4, 1.0, 0, T=8, t=2)
+    np.testing.assert_allclose(O.quant_aff(Wc, S, Z, 16), Wc, atol=1e-15)
+
+
+def test_quant_aff_round_half_even_and_clip():
+    w = np.array([0.5, 1.5, 2.5, -0.5, 100.0, -100.0])
+    assert list(O.affine_codes(w, 1.0, 3.0, 16)) == [3, 5, 5, 3, 15, 0]
+    np.testing.assert_allclose(O.quant_aff(w, 1.0, 3.0, 16), [0, 2, 2, 0, 12, -3])
+
+
+# ------------------------------------------------------------------ P8 ---- #
+def test_p8_loss_ordering_on_ill_conditioned_layer():
+    L = synth.make_layer("c1", 96, 128, 1024, seed=4)
+    W = L.W.double().numpy()
+    X = L.X.double().numpy()
+    bits = 3
+    lean = O.run_pass(W, X, bits=bits, p=4.0, block=32, n_iter=20)
+    H, U = lean["H"], lean["U"]
+    Sm, Zm = O.minmax_affine_params(W, bits)
+    _, What_mm_loop, loss_mm_loop = O.quantize_layer(W, U, scale=Sm, zero=Zm, bits=bits, block=32)
+    What_rtn = O.quant_aff(W, Sm, Zm, 1 << bits)
+    p_lean = lean["proxy"]
+    p_loop = O.proxy_loss(W, What_mm_loop, H)
+    p_rtn = O.proxy_loss(W, What_rtn, H)
+    assert p_lean < p_loop < p_rtn
+    assert lean["loss"] < loss_mm_loop
+    # affine loss-error-aware grid also beats min-max inside the same loop
+    aff = O.run_pass(W, X, grid_type="affine", bits=bits, p=4.0, block=32, T=40, t=12)
+    assert aff["proxy"] < p_loop
+
+
+# ------------------------------------------------------------------ P9 ---- #
+def test_p9_invariances():
+    L = synth.make_layer("c1", 24, 48, 256, seed=8)
+    W = L.W.double().numpy()
+    X = L.X.double().numpy()
+    a = O.run_pass(W, X, bits=3, block=16, n_iter=8)
+    b = O.run_pass(W, 4.0 * X, bits=3, block=16, n_iter=8)          # exact power-of-two scaling
+    assert np.array_equal(a["codes"], b["codes"])
+    np.testing.assert_allclose(a["grid"], b["grid"], rtol=1e-9)
+    np.testing.assert_allclose(b["proxy"], 16.0 * a["proxy"], rtol=1e-8)
+    perm = rng(1).permutation(24)
+    cperm = O.run_pass(W[perm], X, bits=3, block=16, n_iter=8)
+    assert np.array_equal(cperm["codes"], a["codes"][perm])
+    sub = O.run_pass(W[5:11], X, bits=3, block=16, n_iter=8)
+    assert np.array_equal(sub["codes"], a["codes"][5:11])
+    np.testing.assert_allclose(sub["grid"], a["grid"][5:11], rtol=0, atol=0)
+    # tokens arriving in chunks give the same Hessian
+    Hc = O.hessian([X[:, :100], X[:, 100:]])
+    np.testing.assert_allclose(Hc, a["H"], rtol=1e-12, atol=1e-12 * np.abs(a["H"]).max())
+
+
+# ------------------------------------------------------------------ P10 --- #
+def test_p10_library_and_residuals():
+    g = rng(17)
+    c, n = 40, 300
+    X = g.standard_normal((c, n)) * np.exp(g.standard_normal(c))[:, None]
+    H = O.hessian(X)
+    ref = np.zeros((c, c))
+    for tkn in range(n):
+        ref += 2.0 * np.outer(X[:, tkn], X[:, tkn])
+    np.testing.assert_allclose(H, ref, rtol=1e-12, atol=1e-12 * np.abs(ref).max())
+    U, dinv, H_d, _ = O.prepare_hinv(H, 0.01)
+    np.testing.assert_allclose(H_d - H, 0.01 * np.trace(H) / c * np.eye(c), atol=1e-9 * np.trace(H))
+    assert np.allclose(U, np.triu(U)) and (np.diag(U) > 0).all()
+    np.testing.assert_allclose(U.T @ U @ H_d, np.eye(c), atol=1e-8)
+    np.testing.assert_allclose(dinv, np.diag(np.linalg.inv(H_d)), rtol=1e-10)
+    np.testing.assert_allclose(dinv, (U * U).sum(axis=0), rtol=1e-10)
+    # second route to the same factor: H_d = R R^T with R upper, then U = R^-1
+    J = np.eye(c)[::-1]
+    R = J @ np.linalg.cholesky(J @ H_d @ J) @ J
+    np.testing.assert_allclose(np.linalg.inv(R), U, rtol=1e-8, atol=1e-12)
+    # Eq. 9: U[j, j:] is the j-th row of the downdated inverse over sqrt of its diagonal,
+    # and the remaining inverse diagonals only decrease along the downdate
+    Hinv = np.linalg.inv(H_d)
+    for j in range(c):
+        np.testing.assert_allclose(U[j, j:], Hinv[j, j:] / np.sqrt(Hinv[j, j]), rtol=1e-7, atol=1e-13)
+        new = Hinv - np.outer(Hinv[:, j], Hinv[j, :]) / Hinv[j, j]
+        assert (np.diag(new)[j + 1:] <= np.diag(Hinv)[j + 1:] * (1 + 1e-12)).all()
+        Hinv = new
+
+
+def test_dead_channel_convention():
+    g = rng(6)
+    c = 12
+    X = g.standard_normal((c, 60))
+    X[4] = 0.0
+    W = g.standard_normal((3, c))
+    U, dinv, H_d, Wf = O.prepare_hinv(O.hessian(X), 0.01, W)
+    assert (Wf[:, 4] == 0).all() and np.array_equal(np.delete(Wf, 4, 1), np.delete(W, 4, 1))
+    assert np.isfinite(U).all() and np.isfinite(dinv).all()
+
+
+def test_weighted_quantile_init_is_deterministic_and_sorted():
+    g = rng(12)
+    W = g.standard_normal((3, 64))
+    dinv = np.exp(g.standard_normal(64))
+    s = O.sample_weights(dinv, 1.0)
+    G = O.grid_init_weighted_quantile(W, s, 8)
+    assert (np.diff(G, axis=1) >= 0).all()
+    # brute force for one row
+    order = sorted(range(64), key=lambda j: W[0, j])
+    acc_total = 0.0
+    for j in order:
+        acc_total += s[j]
+    for k in range(8):
+        acc = 0.0
+        for j in order:
+            acc += s[j]
+            if acc >= (k + 0.5) / 8 * acc_total:
+                assert G[0, k] == W[0, j]
+                break
+    G2 = O.fit_grid_nonuniform(W, dinv, 3, 1.0, 5, init="weighted_quantile")
+    assert (np.diff(G2, axis=1) >= 0).all()
+
+
+def test_sample_weights_definition():
+    dinv = np.array([0.5, 2.0, 8.0])
+    s = O.sample_weights(dinv, 2.0)
+    raw = dinv ** -2.0
+    np.testing.assert_allclose(s / s[0], raw / raw[0], rtol=1e-13)
+    np.testing.assert_allclose(np.prod(s), 1.0, rtol=1e-12)
