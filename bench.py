@@ -1,0 +1,320 @@
+#!/usr/bin/env python
+"""Benchmark of the LeanQuant per-linear-layer pass on B200.
+
+A "step" is one pass of all four stages (Hessian, dampen/invert/factor, grid fit, column
+loop) over one synthetic layer of the chosen workload.  Default workload: the
+Llama-3-8B-shaped q_proj (W 4096 x 4096 bf16, X 4096 x 262144 bf16, 4-bit non-uniform,
+p = 4, 20 k-means iterations, 128-column blocks).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 (under torchrun): every rank quantises its own layer (layers are independent
+problems, no collective on the data path); value = weights of all ranks / max time.
+--impl reference times the float64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth  # noqa: E402
+
+WORKLOADS = {
+    # name: (recipe, r, c, n, settings)
+    "llama3-8b-q_proj-nu4": ("c2", 4096, 4096, 262144, dict(grid="nonuniform", bits=4, p=4.0, n_iter=20)),
+    "c1-512": ("c1", 512, 512, 8192, dict(grid="nonuniform", bits=4, p=4.0, n_iter=20)),
+}
+L2_BYTES = 126 * 1024 * 1024
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm=p["hbm_gbs"], tf_burst=p["bf16_tflops"], tf_sust=p["bf16_tflops_sustained"], src="measured")
+    return dict(hbm=6650.0, tf_burst=1590.0, tf_sust=1400.0, src="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(mx)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+# ------------------------------------------------------------------ reference arm ----
+def oracle_sample(name, seed=0, n_tokens=8192, n_rows=256, device="cpu", layer=None):
+    """Times the float64 oracle on a bounded sample of the workload: stage 1 on `n_tokens`
+    tokens (scaled up linearly), stage 2 in full, stages 3-4 on `n_rows` rows (scaled up
+    linearly: rows are independent problems).  Returns (seconds for the full layer,
+    description, cores)."""
+    from oracle import leanquant_oracle as O
+    recipe, r, c, n, st = WORKLOADS[name]
+    n_tokens = min(n_tokens, n)
+    n_rows = min(n_rows, r)
+    if layer is None:
+        layer = synth.make_layer(recipe, n_rows, c, n_tokens, seed=seed, device=device)
+        Xs = layer.X.double().cpu().numpy()
+        Ws = layer.W.double().cpu().numpy()
+    else:
+        Xs = layer.X[:, :n_tokens].double().cpu().numpy()
+        Ws = layer.W[:n_rows].double().cpu().numpy()
+    t0 = time.perf_counter()
+    H = O.hessian(Xs)
+    t1 = time.perf_counter()
+    U, dinv, _, Wf = O.prepare_hinv(H, 0.01, Ws)
+    t2 = time.perf_counter()
+    G = O.fit_grid_nonuniform(Wf, dinv, st["bits"], st["p"], st["n_iter"])
+    t3 = time.perf_counter()
+    O.quantize_layer(Wf, U, grid=G, bits=st["bits"], block=128)
+    t4 = time.perf_counter()
+    full = (t1 - t0) * (n / n_tokens) + (t2 - t1) + ((t3 - t2) + (t4 - t3)) * (r / n_rows)
+    cores = len(os.sched_getaffinity(0))
+    desc = (f"float64 oracle: stage 1 on {n_tokens} of {n} tokens (scaled x{n / n_tokens:g}), stage 2 in full, "
+            f"stages 3-4 on {n_rows} of {r} rows (scaled x{r / n_rows:g}); measured "
+            f"{t1 - t0:.2f}+{t2 - t1:.2f}+{t3 - t2:.2f}+{t4 - t3:.2f} s, extrapolated to the full layer")
+    return full, desc, cores
+
+
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    recipe, r, c, n, st = WORKLOADS[args.workload]
+    times = []
+    desc, cores = "", 0
+    for i in range(args.warmup + args.steps):
+        t, desc, cores = oracle_sample(args.workload, seed=i, n_tokens=args.ref_tokens, n_rows=args.ref_rows)
+        if i >= args.warmup:
+            times.append(t)
+    sec = float(np.mean(times))
+    val = r * c / sec
+    line = {"impl": "reference", "metric": "weights quantized/sec per linear layer", "value": val,
+            "unit": "weights/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic", "config": {"workload": args.workload, "r": r, "c": c, "n_tokens": n, **st},
+            "cpu_baseline": {"value": val, "unit": "weights/s", "cores": cores, "kind": "oracle", "sample": desc},
+            "e2e": {"value": val, "unit": "weights/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------ our arm ----
+def run_ours(args):
+    import paper_2407_10032_b200 as lq
+    rank, world, local = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    recipe, r, c, n, st = WORKLOADS[args.workload]
+    cfg = lq.Config.make(**st)
+    h = lq.lq_create(local)
+    layer = synth.make_layer(recipe, r, c, n, seed=1000 + rank, device=dev)
+    W, X = layer.W, layer.X
+    P = lq.LayerPass(h, r, c, cfg, w_dtype=W.dtype, x_dtype=X.dtype, n_chunk=n, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def one_step(events=None):
+        ev = events
+        P.H.zero_()
+        if ev: ev[0].record(stream)
+        lq.lq_hessian_accumulate(h, X, P.H, 2.0, P.ws)
+        if ev: ev[1].record(stream)
+        lq.lq_hessian_finalize(h, P.H)
+        lq.lq_prepare_hinv(h, P.H, P.U, P.dinv, P.ws, 0.01, W)
+        if ev: ev[2].record(stream)
+        lq.lq_fit_grid(h, cfg, W, P.dinv, P.ws, P.grid, P.scale, P.zero)
+        if ev: ev[3].record(stream)
+        lq.lq_quantize_layer(h, cfg, W, P.U, P.codes, P.ws, P.grid, P.scale, P.zero, P.W_hat, P.loss)
+        if ev: ev[4].record(stream)
+
+    for _ in range(args.warmup):
+        one_step()
+    lq.lq_sync_status(h)
+    barrier()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.25)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(args.steps)]
+    e_beg, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = lq.lq_launch_count()
+    barrier()
+    e_beg.record(stream)
+    for i in range(args.steps):
+        one_step(evs[i])
+    e_end.record(stream)
+    barrier()
+    launches = lq.lq_launch_count() - launches0
+    total_ms = e_beg.elapsed_time(e_end)
+    clocks = sampler.stop() if rank == 0 else None
+    lq.lq_sync_status(h)
+
+    stage_ms = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(4)] for e in evs]).mean(axis=0)
+
+    # ---- end to end through the public API with host buffers -------------------------------
+    e2e_steps = max(1, min(args.steps, 3))
+    Xh = torch.empty(X.shape, dtype=X.dtype, pin_memory=True)
+    Wh = torch.empty(W.shape, dtype=W.dtype, pin_memory=True)
+    Xh.copy_(X)
+    Wh.copy_(W)
+    codes_h = torch.empty(P.codes.shape, dtype=torch.uint8, pin_memory=True)
+    grid_h = torch.empty(P.grid.shape, dtype=torch.float32, pin_memory=True)
+    loss_h = torch.empty((1,), dtype=torch.float64, pin_memory=True)
+    Xd, Wd = torch.empty_like(X), torch.empty_like(W)
+    barrier()
+    b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    b0.record(stream)
+    for _ in range(e2e_steps):
+        Xd.copy_(Xh, non_blocking=True)
+        Wd.copy_(Wh, non_blocking=True)
+        P.H.zero_()
+        lq.lq_hessian_accumulate(h, Xd, P.H, 2.0, P.ws)
+        lq.lq_hessian_finalize(h, P.H)
+        lq.lq_prepare_hinv(h, P.H, P.U, P.dinv, P.ws, 0.01, Wd)
+        lq.lq_fit_grid(h, cfg, Wd, P.dinv, P.ws, P.grid, P.scale, P.zero)
+        lq.lq_quantize_layer(h, cfg, Wd, P.U, P.codes, P.ws, P.grid, P.scale, P.zero, None, P.loss)
+        codes_h.copy_(P.codes, non_blocking=True)
+        grid_h.copy_(P.grid, non_blocking=True)
+        loss_h.copy_(P.loss, non_blocking=True)
+    b1.record(stream)
+    barrier()
+    e2e_ms = b0.elapsed_time(b1) / e2e_steps
+    h2d = Xh.numel() * Xh.element_size() + Wh.numel() * Wh.element_size()
+    d2h = codes_h.numel() + grid_h.numel() * 4 + 8
+
+    t = torch.tensor([total_ms, e2e_ms], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(t[0]), float(t[1])
+    ms_per_step = total_ms / args.steps
+    weights = r * c * world
+    value = weights / (ms_per_step * 1e-3)
+
+    if rank == 0:
+        pk = peaks()
+        # dominant kernel: the stage-1 tensor-core contraction.  Algorithmic work with the
+        # symmetry used: c^2 * n flops (n tokens, c(c+1)/2 outputs, 2 flops each).
+        flops = float(c) * c * n
+        ach = flops / (stage_ms[0] * 1e-3) / 1e12
+        peak = pk["tf_burst"]
+        roof = {"bound": "tensor", "kernel": "lq_tc_gemm_kernel (stage 1, H += 2XX^T)", "achieved": ach, "peak": peak,
+                "unit": "TFLOP/s", "frac": ach / peak, "traffic": None, "peak_source": pk["src"] + " burst bf16",
+                "frac_of_sustained": ach / pk["tf_sust"], "flops_per_launch": flops}
+        cpu = None
+        if world == 1:
+            sec, desc, cores = oracle_sample(args.workload, n_tokens=args.ref_tokens, n_rows=args.ref_rows, layer=layer)
+            cpu = {"value": r * c / sec, "unit": "weights/s", "cores": cores, "kind": "oracle", "sample": desc}
+        line = {
+            "metric": "weights quantized/sec per linear layer", "value": value, "unit": "weights/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic",
+            "config": {"workload": args.workload, "r": r, "c": c, "n_tokens": n, **st, "block": 128, "damp": 0.01,
+                       "l2": f"inputs per step ({(X.numel() * X.element_size()) >> 20} MiB X) exceed the 126 MiB L2",
+                       "parallelism": "one layer per GPU, no collective"},
+            "stage_ms": {"hessian": float(stage_ms[0]), "prepare_hinv": float(stage_ms[1]),
+                         "fit_grid": float(stage_ms[2]), "quantize_layer": float(stage_ms[3])},
+            "roofline": roof, "cpu_baseline": cpu,
+            "e2e": {"value": weights / (e2e_ms * 1e-3), "unit": "weights/s", "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+            "gpu_launches": int(launches), "clocks": clocks,
+        }
+        print(json.dumps(line))
+    lq.lq_destroy(h)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama3-8b-q_proj-nu4", choices=sorted(WORKLOADS))
+    ap.add_argument("--ref-tokens", type=int, default=32768)
+    ap.add_argument("--ref-rows", type=int, default=512)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

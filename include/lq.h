@@ -1,0 +1,151 @@
+/*
+ * lq.h -- C ABI of the B200 (sm_100a) LeanQuant per-linear-layer quantisation pass.
+ *
+ * The pass is Algorithm 1 of the paper ("LeanQuant for LLM quantization"), split
+ * into its four stages.  Notation is the paper's: W is r x c (r output rows, c input
+ * columns), X is c x n (n calibration tokens), H = 2 X X^T is c x c, b bits give
+ * K = 2^b grid points, B is the block width of the column loop.
+ *
+ * Conventions for every call
+ *   - Returns LQ_OK or an lq_status error code.  Argument errors are found on the host
+ *     before anything is launched; nothing is enqueued when a call fails.
+ *   - All pointers named "device" are device pointers owned by the caller; they must stay
+ *     valid until the stream has executed the call.  The library allocates nothing per
+ *     call: scratch memory is a caller-allocated workspace sized by the matching
+ *     *_workspace query (256-byte aligned).
+ *   - Work is enqueued on the given CUDA stream (a cudaStream_t passed as void*) and is
+ *     asynchronous.  Failures found on the device (a non-positive pivot, a non-finite
+ *     value, a wait that ran out) are recorded in the handle and read by lq_sync_status.
+ *   - Matrices are row-major with a leading dimension in elements.
+ *   - There is no CPU fallback: without a CUDA device every compute call fails.
+ */
+#ifndef LQ_H_
+#define LQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    LQ_OK = 0,
+    LQ_ERR_INVALID_ARG = 1,
+    LQ_ERR_UNSUPPORTED = 2,
+    LQ_ERR_WORKSPACE_TOO_SMALL = 3,
+    LQ_ERR_NOT_POSITIVE_DEFINITE = 4,  /* device: pivot <= 0 in the factorisation; info = column */
+    LQ_ERR_NONFINITE = 5,              /* device: NaN/Inf met; info = index */
+    LQ_ERR_CUDA = 6,                   /* a CUDA runtime / driver call failed */
+    LQ_ERR_TIMEOUT = 7                 /* device: a bounded wait inside a kernel ran out */
+} lq_status;
+
+typedef enum { LQ_F32 = 0, LQ_BF16 = 1 } lq_dtype;
+typedef enum { LQ_FEATURE_MAJOR = 0 /* X is c x n, tokens contiguous */ } lq_layout;
+typedef enum { LQ_GRID_NONUNIFORM = 0, LQ_GRID_AFFINE = 1 } lq_grid_type;
+typedef enum { LQ_INIT_UNIFORM = 0 /* Eq. 6 */ } lq_init;
+
+typedef struct lq_handle lq_handle;
+
+/* Settings of stages 3 and 4 (inputs of Algorithm 1 plus the search parameters of Eq. 7). */
+typedef struct {
+    int32_t bits;        /* b: 2, 3 or 4                                                    */
+    int32_t grid_type;   /* lq_grid_type                                                    */
+    float   p;           /* outlier-preservation strength of Eq. 5 / Eq. 7 (paper: 4)       */
+    int32_t n_iter;      /* Lloyd iterations, fixed count, no early stop                    */
+    int32_t init;        /* lq_init                                                         */
+    int32_t group_size;  /* affine: weights per (S, Z) group along a row; 0 = whole row     */
+    int32_t T;           /* affine: partitions of the range R (paper: 2048)                 */
+    int32_t t_count;     /* affine: t, t_min and t_max run over 0..t (Appendix B)           */
+    int32_t block;       /* B: columns per block of the column loop; must be 128            */
+    int32_t reserved;
+} lq_config;
+
+/* ---- handle ------------------------------------------------------------------------- */
+
+/* Creates a handle bound to CUDA device `device` (allocates a few bytes of device memory
+ * for the status word).  Fails with LQ_ERR_CUDA when no such device exists. */
+int lq_create(lq_handle** out, int device);
+int lq_destroy(lq_handle* h);
+
+/* Waits for `stream`, then returns the first device-detected failure recorded since the
+ * last call (LQ_OK if none) in *status with its detail in *info, and clears it. */
+int lq_sync_status(lq_handle* h, void* stream, int32_t* status, int64_t* info);
+
+/* ---- stage 1: Algorithm 1 line 3 (H <- 2 X X^T), Section 2.2 ------------------------- */
+
+/* H[0:c,0:c] += alpha * X X^T for one chunk of tokens; call once per chunk, H (device,
+ * fp32, ldh >= c, ldh % 4 == 0, 16-byte aligned) is the in/out accumulator and must be
+ * zeroed by the caller before the first chunk.  Only tiles touching the upper triangle are
+ * updated: entries strictly below the diagonal are unspecified until lq_hessian_finalize.
+ * X: device, c x n_chunk, feature-major (ldx >= n_chunk elements; ldx*sizeof(x) % 16 == 0,
+ * 16-byte aligned), bf16 or fp32.  bf16 products are exact in the fp32 accumulator; fp32
+ * input is split into three bf16 terms (workspace needed) and keeps fp32-level accuracy.
+ * workspace: lq_hessian_workspace bytes (0 for bf16 input; ws may then be NULL). */
+int lq_hessian_workspace(int32_t x_dtype, int64_t c, int64_t n_chunk, size_t* bytes);
+int lq_hessian_accumulate(lq_handle* h, void* stream, const void* X, int32_t x_dtype,
+                          int32_t layout, int64_t c, int64_t n_chunk, int64_t ldx,
+                          float* H, int64_t ldh, float alpha, void* ws, size_t ws_bytes);
+/* Copies the upper triangle of H onto the lower one. */
+int lq_hessian_finalize(lq_handle* h, void* stream, float* H, int64_t c, int64_t ldh);
+
+/* ---- stage 2: Algorithm 1 line 4, "Cholesky and Dampening" --------------------------- */
+
+/* H_d = H + damp_frac * mean(diag H) * I;  U = upper Cholesky factor of H_d^-1
+ * (H_d^-1 = U^T U, U_jj > 0; strictly lower part of U is written as 0);
+ * dinv = diag(H_d^-1).  Only the upper triangle of H is read.  A zero diagonal entry of H
+ * (an input channel that never fired) is replaced by 1 and, when W is given, that column of
+ * W is zeroed in place (W: device r x c of w_dtype, may be NULL).
+ * H: device fp32 c x c (not modified unless U aliases it, which is allowed).
+ * U: device fp32 c x c, ldu >= c.  dinv: device fp32[c].
+ * Internally factorises in fp64 (blocked, tensor-core FP64 MMA trailing updates).
+ * A non-positive pivot records LQ_ERR_NOT_POSITIVE_DEFINITE (info = column). */
+int lq_prepare_hinv_workspace(int64_t c, size_t* bytes);
+int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64_t c, int64_t ldh,
+                    float damp_frac, float* U, int64_t ldu, float* dinv,
+                    void* W, int32_t w_dtype, int64_t r, int64_t ldw,
+                    void* ws, size_t ws_bytes);
+
+/* ---- stage 3: loss-error-aware grid, Eq. 5 (non-uniform) / Eq. 7 (affine) ------------ */
+
+/* Non-uniform: for every row k, K = 2^bits centroids by weighted 1-D k-means with sample
+ * weights dinv^(-p) (normalised by their geometric mean), started from Eq. 6 and run for
+ * exactly n_iter Lloyd iterations; grid (device fp32, r x K) gets the ascending centroids.
+ * Affine: for every (row, group) the pair (S, Z) of Eq. 7 with least weighted squared
+ * error over (t_min, t_max) in {0..t_count}^2, first minimum in t_min-major order;
+ * scale (device fp32) and zero (device int32) are r x (c / group).
+ * W: device r x c (bf16 or fp32).  dinv: device fp32[c] from stage 2. */
+int lq_fit_grid_workspace(const lq_config* cfg, int64_t r, int64_t c, size_t* bytes);
+int lq_fit_grid(lq_handle* h, void* stream, const lq_config* cfg, const void* W,
+                int32_t w_dtype, int64_t r, int64_t c, int64_t ldw, const float* dinv,
+                float* grid, float* scale, int32_t* zero, void* ws, size_t ws_bytes);
+
+/* ---- stage 4: Algorithm 1 lines 10-21, the block-wise column loop -------------------- */
+
+/* For each block of B = 128 columns: quantise column j of every row to its grid
+ * (quant_nu: nearest centroid, a weight exactly on a midpoint takes the lower one;
+ * quant_aff: clip(round(w/S) + Z, 0, K-1) with the group's (S, Z)),
+ * E[:, j-i] = (W[:, j] - What[:, j]) / U[j, j], feed the error back inside the block, then
+ * W[:, i+B:] -= E U[i:i+B, i+B:] on the tensor cores.  W is not modified (a fp32 working
+ * copy lives in the workspace).
+ * codes: device uint8 r x c (ld = c), one code per byte.  W_hat: device, what_dtype, r x c
+ * with ldwh, or NULL.  loss_out: device double[1] = 1/2 * sum E^2 (Eq. 3), or NULL. */
+int lq_quantize_layer_workspace(const lq_config* cfg, int64_t r, int64_t c, size_t* bytes);
+int lq_quantize_layer(lq_handle* h, void* stream, const lq_config* cfg, const void* W,
+                      int32_t w_dtype, int64_t r, int64_t c, int64_t ldw,
+                      const float* U, int64_t ldu,
+                      const float* grid, const float* scale, const int32_t* zero,
+                      uint8_t* codes, void* W_hat, int32_t what_dtype, int64_t ldwh,
+                      double* loss_out, void* ws, size_t ws_bytes);
+
+/* Number of CUDA kernels this library has launched in this process so far (host counter,
+ * not thread-safe; for benchmarks and tests that want to see that the kernels ran). */
+uint64_t lq_launch_count(void);
+
+/* Library version string (static storage). */
+const char* lq_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LQ_H_ */

@@ -1,0 +1,237 @@
+"""ctypes binding of liblq.so: the same entry points as include/lq.h, taking torch tensors.
+
+Only argument marshalling happens here (pointers, sizes, strides, dtypes).  Every step of
+the pass runs in the library's CUDA kernels; if the library cannot be loaded, or a call
+fails, an exception is raised -- there is no fallback path."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "liblq.so")
+_lib = None
+
+LQ_F32, LQ_BF16 = 0, 1
+LQ_GRID_NONUNIFORM, LQ_GRID_AFFINE = 0, 1
+STATUS_NAMES = {0: "LQ_OK", 1: "LQ_ERR_INVALID_ARG", 2: "LQ_ERR_UNSUPPORTED", 3: "LQ_ERR_WORKSPACE_TOO_SMALL",
+                4: "LQ_ERR_NOT_POSITIVE_DEFINITE", 5: "LQ_ERR_NONFINITE", 6: "LQ_ERR_CUDA", 7: "LQ_ERR_TIMEOUT"}
+
+
+class LQError(RuntimeError):
+    def __init__(self, code, where, info=None):
+        self.code, self.info = code, info
+        extra = f" (info={info})" if info is not None else ""
+        super().__init__(f"{where}: {STATUS_NAMES.get(code, code)}{extra}")
+
+
+class Config(C.Structure):
+    """Mirror of lq_config."""
+    _fields_ = [("bits", C.c_int32), ("grid_type", C.c_int32), ("p", C.c_float), ("n_iter", C.c_int32),
+                ("init", C.c_int32), ("group_size", C.c_int32), ("T", C.c_int32), ("t_count", C.c_int32),
+                ("block", C.c_int32), ("reserved", C.c_int32)]
+
+    @classmethod
+    def make(cls, grid="nonuniform", bits=4, p=4.0, n_iter=20, group=0, T=2048, t=None, block=128, **_):
+        if t is None:
+            t = int({4: 0.2, 3: 0.3, 2: 0.4}[bits] * T)
+        gt = LQ_GRID_NONUNIFORM if grid == "nonuniform" else LQ_GRID_AFFINE
+        return cls(bits, gt, float(p), n_iter, 0, group or 0, T, t, block, 0)
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def LQ():
+    """The loaded library (loads it on first use; raises if it has not been built)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise LQError(6, f"liblq.so not built at {_LIB_PATH} (run paper_2407_10032_b200/build.py)")
+        lib = C.CDLL(_LIB_PATH)
+        vp, i32, i64, f32, sz = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_size_t
+        P = C.POINTER
+        sig = {
+            "lq_create": [P(vp), C.c_int],
+            "lq_destroy": [vp],
+            "lq_sync_status": [vp, vp, P(i32), P(i64)],
+            "lq_hessian_workspace": [i32, i64, i64, P(sz)],
+            "lq_hessian_accumulate": [vp, vp, vp, i32, i32, i64, i64, i64, vp, i64, f32, vp, sz],
+            "lq_hessian_finalize": [vp, vp, vp, i64, i64],
+            "lq_prepare_hinv_workspace": [i64, P(sz)],
+            "lq_prepare_hinv": [vp, vp, vp, i64, i64, f32, vp, i64, vp, vp, i32, i64, i64, vp, sz],
+            "lq_fit_grid_workspace": [P(Config), i64, i64, P(sz)],
+            "lq_fit_grid": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, sz],
+            "lq_quantize_layer_workspace": [P(Config), i64, i64, P(sz)],
+            "lq_quantize_layer": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, i64, vp, vp, vp, vp, vp, i32, i64,
+                                  vp, vp, sz],
+        }
+        for name, args in sig.items():
+            fn = getattr(lib, name)
+            fn.argtypes = args
+            fn.restype = C.c_int
+        lib.lq_launch_count.restype = C.c_uint64
+        lib.lq_launch_count.argtypes = []
+        lib.lq_version.restype = C.c_char_p
+        lib.lq_version.argtypes = []
+        _lib = lib
+    return _lib
+
+
+def _check(code, where):
+    if code != 0:
+        raise LQError(code, where)
+
+
+def _dt(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return LQ_F32
+    if t.dtype == torch.bfloat16:
+        return LQ_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def _rowmajor(t: torch.Tensor):
+    assert t.dim() == 2 and t.stride(1) == 1, "row-major 2-D tensor expected"
+    return t.stride(0)
+
+
+def lq_version() -> str:
+    return LQ().lq_version().decode()
+
+
+def lq_launch_count() -> int:
+    return int(LQ().lq_launch_count())
+
+
+def lq_create(device: int = 0):
+    h = C.c_void_p()
+    _check(LQ().lq_create(C.byref(h), device), "lq_create")
+    return h
+
+
+def lq_destroy(h):
+    _check(LQ().lq_destroy(h), "lq_destroy")
+
+
+def lq_sync_status(h, stream=None, raise_on_error=True):
+    st, info = C.c_int32(0), C.c_int64(0)
+    _check(LQ().lq_sync_status(h, _stream(stream), C.byref(st), C.byref(info)), "lq_sync_status")
+    if st.value and raise_on_error:
+        raise LQError(st.value, "device status", info.value)
+    return st.value, info.value
+
+
+def lq_hessian_workspace(x_dtype, c, n_chunk) -> int:
+    b = C.c_size_t(0)
+    dt = x_dtype if isinstance(x_dtype, int) else (LQ_F32 if x_dtype == torch.float32 else LQ_BF16)
+    _check(LQ().lq_hessian_workspace(dt, c, n_chunk, C.byref(b)), "lq_hessian_workspace")
+    return b.value
+
+
+def lq_hessian_accumulate(h, X, H, alpha=2.0, ws=None, stream=None):
+    c, n = X.shape
+    _check(LQ().lq_hessian_accumulate(h, _stream(stream), _ptr(X), _dt(X), 0, c, n, _rowmajor(X), _ptr(H),
+                                      _rowmajor(H), alpha, _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size()),
+           "lq_hessian_accumulate")
+
+
+def lq_hessian_finalize(h, H, stream=None):
+    _check(LQ().lq_hessian_finalize(h, _stream(stream), _ptr(H), H.shape[0], _rowmajor(H)), "lq_hessian_finalize")
+
+
+def lq_prepare_hinv_workspace(c) -> int:
+    b = C.c_size_t(0)
+    _check(LQ().lq_prepare_hinv_workspace(c, C.byref(b)), "lq_prepare_hinv_workspace")
+    return b.value
+
+
+def lq_prepare_hinv(h, H, U, dinv, ws, damp_frac=0.01, W=None, stream=None):
+    c = H.shape[0]
+    r, ldw, wdt = (0, 0, 0) if W is None else (W.shape[0], _rowmajor(W), _dt(W))
+    _check(LQ().lq_prepare_hinv(h, _stream(stream), _ptr(H), c, _rowmajor(H), damp_frac, _ptr(U), _rowmajor(U),
+                                _ptr(dinv), _ptr(W), wdt, r, ldw, _ptr(ws), ws.numel() * ws.element_size()),
+           "lq_prepare_hinv")
+
+
+def lq_fit_grid_workspace(cfg, r, c) -> int:
+    b = C.c_size_t(0)
+    _check(LQ().lq_fit_grid_workspace(C.byref(cfg), r, c, C.byref(b)), "lq_fit_grid_workspace")
+    return b.value
+
+
+def lq_fit_grid(h, cfg, W, dinv, ws, grid=None, scale=None, zero=None, stream=None):
+    r, c = W.shape
+    _check(LQ().lq_fit_grid(h, _stream(stream), C.byref(cfg), _ptr(W), _dt(W), r, c, _rowmajor(W), _ptr(dinv),
+                            _ptr(grid), _ptr(scale), _ptr(zero), _ptr(ws), ws.numel() * ws.element_size()),
+           "lq_fit_grid")
+
+
+def lq_quantize_layer_workspace(cfg, r, c) -> int:
+    b = C.c_size_t(0)
+    _check(LQ().lq_quantize_layer_workspace(C.byref(cfg), r, c, C.byref(b)), "lq_quantize_layer_workspace")
+    return b.value
+
+
+def lq_quantize_layer(h, cfg, W, U, codes, ws, grid=None, scale=None, zero=None, W_hat=None, loss_out=None, stream=None):
+    r, c = W.shape
+    whdt, ldwh = (0, 0) if W_hat is None else (_dt(W_hat), _rowmajor(W_hat))
+    _check(LQ().lq_quantize_layer(h, _stream(stream), C.byref(cfg), _ptr(W), _dt(W), r, c, _rowmajor(W), _ptr(U),
+                                  _rowmajor(U), _ptr(grid), _ptr(scale), _ptr(zero), _ptr(codes), _ptr(W_hat), whdt,
+                                  ldwh, _ptr(loss_out), _ptr(ws), ws.numel() * ws.element_size()),
+           "lq_quantize_layer")
+
+
+class LayerPass:
+    """Buffers for one layer shape plus the four calls in Algorithm 1's order.
+
+    Allocation only (through torch's allocator); all arithmetic is in liblq."""
+
+    def __init__(self, handle, r, c, cfg: Config, w_dtype=torch.bfloat16, x_dtype=torch.bfloat16, n_chunk=0,
+                 device="cuda", want_w_hat=True):
+        self.h, self.r, self.c, self.cfg = handle, r, c, cfg
+        dev = torch.device(device)
+        K = 1 << cfg.bits
+        f32 = dict(device=dev, dtype=torch.float32)
+        self.H = torch.zeros((c, c), **f32)
+        self.U = torch.empty((c, c), **f32)
+        self.dinv = torch.empty((c,), **f32)
+        self.affine = cfg.grid_type == LQ_GRID_AFFINE
+        ng = 1 if cfg.group_size == 0 else c // cfg.group_size
+        self.grid = None if self.affine else torch.empty((r, K), **f32)
+        self.scale = torch.empty((r, ng), **f32) if self.affine else None
+        self.zero = torch.empty((r, ng), device=dev, dtype=torch.int32) if self.affine else None
+        self.codes = torch.empty((r, c), device=dev, dtype=torch.uint8)
+        self.W_hat = torch.empty((r, c), device=dev, dtype=w_dtype) if want_w_hat else None
+        self.loss = torch.zeros((1,), device=dev, dtype=torch.float64)
+        nbytes = max(lq_hessian_workspace(x_dtype, c, n_chunk), lq_prepare_hinv_workspace(c),
+                     lq_fit_grid_workspace(cfg, r, c), lq_quantize_layer_workspace(cfg, r, c), 256)
+        self.ws = torch.empty((nbytes,), device=dev, dtype=torch.uint8)
+
+    def accumulate(self, X, alpha=2.0):
+        lq_hessian_accumulate(self.h, X, self.H, alpha, self.ws)
+
+    def finish(self, W, damp_frac=0.01):
+        """Stages 2-4 after all chunks were accumulated."""
+        lq_hessian_finalize(self.h, self.H)
+        lq_prepare_hinv(self.h, self.H, self.U, self.dinv, self.ws, damp_frac, W)
+        lq_fit_grid(self.h, self.cfg, W, self.dinv, self.ws, self.grid, self.scale, self.zero)
+        lq_quantize_layer(self.h, self.cfg, W, self.U, self.codes, self.ws, self.grid, self.scale, self.zero,
+                          self.W_hat, self.loss)
+
+    def run(self, W, X, damp_frac=0.01, alpha=2.0):
+        self.H.zero_()
+        self.accumulate(X, alpha)
+        self.finish(W, damp_frac)

@@ -1,0 +1,77 @@
+// Shared internals of liblq: handle layout, device status word, small helpers.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "lq.h"
+
+struct lq_dev_status {
+    int32_t code;      // first failure recorded on the device (lq_status), 0 = none
+    int32_t pad;
+    long long info;    // detail of that failure
+};
+
+struct lq_handle {
+    int device;
+    int sm_count;
+    lq_dev_status* dstatus;   // device memory
+};
+
+// Record the first device-side failure; later ones are dropped.
+__device__ __forceinline__ void lq_report(lq_dev_status* st, int code, long long info) {
+    if (atomicCAS(&st->code, 0, code) == 0) st->info = info;
+}
+
+#define LQ_CUDA_TRY(expr)                                   \
+    do {                                                    \
+        cudaError_t _e = (expr);                            \
+        if (_e != cudaSuccess) return LQ_ERR_CUDA;          \
+    } while (0)
+
+// Every kernel launch of the library goes through this: it counts the launch (see
+// lq_launch_count) and turns a launch failure into LQ_ERR_CUDA.
+extern unsigned long long lq_launches_total;
+#define LQ_LAUNCH_CHECK()                                   \
+    do {                                                    \
+        ++lq_launches_total;                                \
+        if (cudaGetLastError() != cudaSuccess) return LQ_ERR_CUDA; \
+    } while (0)
+
+static inline size_t lq_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline int64_t lq_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+// ---- bf16 tensor-core GEMM (lq_gemm_tc.cu) -------------------------------------------
+// D[M x N] (fp32, row-major, ldd) (+)= alpha * sum_p A_p[M x K] * B_p[N x K]^T
+// A_p and B_p are bf16, K contiguous.  The operands of all passes live in one matrix
+// each: pass p reads rows [a_row_off[p], a_row_off[p] + M) of A_all and rows
+// [b_row_off[p], b_row_off[p] + N) of B_all.  accumulate != 0 adds into D (a reduction
+// done by the copy engine), otherwise D is overwritten.  upper_only != 0 skips the
+// 128 x 256 tiles that lie strictly below the diagonal (symmetric results).
+// The tensor core adds into its fp32 accumulator with truncation, so a long K is cut into
+// segments whose partial sums are added to D with round-to-nearest (seg_iters).
+struct lq_tc_gemm_args {
+    const __nv_bfloat16* A_all; int64_t a_rows; int64_t lda;   // a_rows = total rows of A_all
+    const __nv_bfloat16* B_all; int64_t b_rows; int64_t ldb;
+    float* D; int64_t ldd;
+    int64_t M, N, K;
+    int n_pass;
+    int64_t a_row_off[6];
+    int64_t b_row_off[6];
+    float alpha;
+    int accumulate;
+    int upper_only;
+    int seg_iters;   // flush the TMEM partial sum into D every seg_iters 64-wide k-steps (0 = only at the end)
+};
+int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a);
+
+// Split fp32 into three bf16 terms hi + mid + lo (each the bf16 rounding of what is left).
+__device__ __forceinline__ void lq_split3(float x, __nv_bfloat16& hi, __nv_bfloat16& mid, __nv_bfloat16& lo) {
+    hi = __float2bfloat16_rn(x);
+    float r1 = x - __bfloat162float(hi);
+    mid = __float2bfloat16_rn(r1);
+    float r2 = r1 - __bfloat162float(mid);
+    lo = __float2bfloat16_rn(r2);
+}

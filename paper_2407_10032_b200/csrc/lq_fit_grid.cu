@@ -1,0 +1,368 @@
+// Stage 3 -- the loss-error-aware grid (Section 3.2, Algorithm 1 lines 5-9).
+//
+// Non-uniform (Eq. 5): one weighted 1-D k-means per output row.  One CTA per row, the row
+// staged once (registers for short rows, shared memory for long ones), the sample weights
+// s_j = dinv_j^(-p) / geometric mean shared by all rows.  Assignment compares and the
+// per-cluster sums run in fp64: a weight that sits next to a midpoint must fall on the same
+// side as in a float64 evaluation, or the centroids drift apart by far more than rounding.
+//
+// Affine (Eq. 7): one CTA per (row, group); every thread evaluates whole candidates
+// (t_min, t_max) over the group's weights held in shared memory, then the CTA takes the
+// arg-min (first minimum in t_min-major order).  Also fp64, for the same reason.
+#include <math.h>
+
+#include "lq_common.cuh"
+
+namespace {
+
+constexpr int KM_THREADS = 256;
+constexpr int KM_WARPS = KM_THREADS / 32;
+
+// scal[1] = mean_j ln(dinv_j)
+__global__ void log_mean_kernel(const float* __restrict__ dinv, int64_t c, double* __restrict__ scal, lq_dev_status* st) {
+    __shared__ double red[1024];
+    double s = 0.0;
+    for (int64_t j = threadIdx.x; j < c; j += blockDim.x) {
+        float d = dinv[j];
+        if (!(d > 0.0f) || !isfinite(d)) { lq_report(st, LQ_ERR_NONFINITE, j); d = 1.0f; }
+        s += log(static_cast<double>(d));
+    }
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = blockDim.x / 2; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) scal[1] = red[0] / static_cast<double>(c);
+}
+
+// s_j = exp(-p (ln dinv_j - mean ln dinv))
+__global__ void sample_weights_kernel(const float* __restrict__ dinv, int64_t c, double p, const double* __restrict__ scal,
+                                      double* __restrict__ s) {
+    const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (j >= c) return;
+    float d = dinv[j];
+    if (!(d > 0.0f) || !isfinite(d)) d = 1.0f;
+    s[j] = exp(-p * (log(static_cast<double>(d)) - scal[1]));
+}
+
+__device__ __forceinline__ float load_w(const float* p) { return *p; }
+__device__ __forceinline__ float load_w(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+// EPT > 0: each thread keeps EPT weights and their sample weights in registers
+// (c <= EPT * KM_THREADS).  EPT == 0: the row lives in dynamic shared memory as fp32 and
+// the sample weights are re-read (L1/L2) every iteration.
+template <int K, int EPT, typename T>
+__global__ void __launch_bounds__(KM_THREADS)
+kmeans_rows_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int64_t c, const double* __restrict__ s64,
+                   float* __restrict__ grid, int n_iter) {
+    extern __shared__ float wrow[];                      // EPT == 0 only
+    __shared__ double g[K];
+    __shared__ double mid[K];
+    __shared__ double red[KM_WARPS][2 * K];
+    __shared__ float redf[2][KM_WARPS];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    constexpr int NREG = EPT > 0 ? EPT : 1;
+    float wr[NREG];
+    double sr[NREG];
+    if (EPT > 0) {
+#pragma unroll
+        for (int e = 0; e < NREG; ++e) {
+            const int64_t j = tid + (int64_t)e * KM_THREADS;
+            sr[e] = j < c ? s64[j] : 0.0;
+        }
+    }
+
+    for (int64_t row = blockIdx.x; row < r; row += gridDim.x) {
+        const T* wp = W + row * ldw;
+        float mn = INFINITY, mx = -INFINITY;
+        if (EPT > 0) {
+#pragma unroll
+            for (int e = 0; e < NREG; ++e) {
+                const int64_t j = tid + (int64_t)e * KM_THREADS;
+                if (j < c) {
+                    wr[e] = load_w(wp + j);
+                    mn = fminf(mn, wr[e]);
+                    mx = fmaxf(mx, wr[e]);
+                } else {
+                    wr[e] = 0.0f;      // carries zero sample weight
+                }
+            }
+        } else {
+            for (int64_t j = tid; j < c; j += KM_THREADS) {
+                float w = load_w(wp + j);
+                wrow[j] = w;
+                mn = fminf(mn, w);
+                mx = fmaxf(mx, w);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        }
+        if (lane == 0) { redf[0][warp] = mn; redf[1][warp] = mx; }
+        __syncthreads();
+        if (tid < K) {
+            float a = redf[0][0], b = redf[1][0];
+            for (int w = 1; w < KM_WARPS; ++w) { a = fminf(a, redf[0][w]); b = fmaxf(b, redf[1][w]); }
+            const double lo = a, hi = b;
+            g[tid] = lo + (hi - lo) * static_cast<double>(tid) / static_cast<double>(K - 1);   // Eq. 6
+        }
+        __syncthreads();
+
+        for (int it = 0; it < n_iter; ++it) {
+            if (tid < K - 1) mid[tid] = 0.5 * (g[tid] + g[tid + 1]);
+            __syncthreads();
+            double ns[K], nsw[K];
+#pragma unroll
+            for (int k = 0; k < K; ++k) ns[k] = nsw[k] = 0.0;
+
+            auto visit = [&](float wf, double sv) {
+                const double w = static_cast<double>(wf);
+                int a = 0;
+#pragma unroll
+                for (int step = K / 2; step > 0; step >>= 1)
+                    if (w > mid[a + step - 1]) a += step;          // count of midpoints below w
+                const double sw = sv * w;
+#pragma unroll
+                for (int k = 0; k < K; ++k) {
+                    ns[k] += (a == k) ? sv : 0.0;
+                    nsw[k] += (a == k) ? sw : 0.0;
+                }
+            };
+            if (EPT > 0) {
+#pragma unroll
+                for (int e = 0; e < NREG; ++e) visit(wr[e], sr[e]);
+            } else {
+                for (int64_t j = tid; j < c; j += KM_THREADS) visit(wrow[j], s64[j]);
+            }
+#pragma unroll
+            for (int k = 0; k < K; ++k) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    ns[k] += __shfl_xor_sync(0xffffffffu, ns[k], o);
+                    nsw[k] += __shfl_xor_sync(0xffffffffu, nsw[k], o);
+                }
+            }
+            if (lane == 0) {
+#pragma unroll
+                for (int k = 0; k < K; ++k) { red[warp][k] = ns[k]; red[warp][K + k] = nsw[k]; }
+            }
+            __syncthreads();
+            if (tid < K) {
+                double den = 0.0, num = 0.0;
+                for (int w = 0; w < KM_WARPS; ++w) { den += red[w][tid]; num += red[w][K + tid]; }
+                if (den > 0.0) g[tid] = num / den;      // an empty / weightless cluster keeps its centroid
+            }
+            __syncthreads();
+        }
+        if (tid < K) grid[row * K + tid] = static_cast<float>(g[tid]);
+        __syncthreads();
+    }
+}
+
+template <int K, typename T>
+int launch_kmeans(cudaStream_t st, int sms, const T* W, int64_t ldw, int64_t r, int64_t c, const double* s64, float* grid,
+                  int n_iter) {
+    const unsigned blocks = static_cast<unsigned>(r < (int64_t)sms * 8 ? r : (int64_t)sms * 8);
+    if (c <= 1 * KM_THREADS) kmeans_rows_kernel<K, 1, T><<<blocks, KM_THREADS, 0, st>>>(W, ldw, r, c, s64, grid, n_iter);
+    else if (c <= 2 * KM_THREADS) kmeans_rows_kernel<K, 2, T><<<blocks, KM_THREADS, 0, st>>>(W, ldw, r, c, s64, grid, n_iter);
+    else if (c <= 4 * KM_THREADS) kmeans_rows_kernel<K, 4, T><<<blocks, KM_THREADS, 0, st>>>(W, ldw, r, c, s64, grid, n_iter);
+    else if (c <= 8 * KM_THREADS) kmeans_rows_kernel<K, 8, T><<<blocks, KM_THREADS, 0, st>>>(W, ldw, r, c, s64, grid, n_iter);
+    else if (c <= 16 * KM_THREADS) kmeans_rows_kernel<K, 16, T><<<blocks, KM_THREADS, 0, st>>>(W, ldw, r, c, s64, grid, n_iter);
+    else {
+        const size_t smem = static_cast<size_t>(c) * sizeof(float);
+        if (smem > 200 * 1024) return LQ_ERR_UNSUPPORTED;
+        static bool attr_set = false;
+        if (!attr_set) {
+            LQ_CUDA_TRY(cudaFuncSetAttribute(kmeans_rows_kernel<K, 0, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+            attr_set = true;
+        }
+        const unsigned b2 = static_cast<unsigned>(r < sms ? r : sms);
+        kmeans_rows_kernel<K, 0, T><<<b2, KM_THREADS, smem, st>>>(W, ldw, r, c, s64, grid, n_iter);
+    }
+    LQ_LAUNCH_CHECK();
+    return LQ_OK;
+}
+
+// ------------------------------------------------------------------- affine search --
+constexpr int AF_THREADS = 128;
+
+template <typename T>
+__global__ void __launch_bounds__(AF_THREADS)
+affine_search_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, int group, int n_groups,
+                     const double* __restrict__ s64, int K, int Tparts, int t_count,
+                     float* __restrict__ scale, int32_t* __restrict__ zero) {
+    extern __shared__ float wg[];                 // group weights
+    __shared__ float redf[2][AF_THREADS / 32];
+    __shared__ double best_loss[AF_THREADS / 32];
+    __shared__ int best_idx[AF_THREADS / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t row = blockIdx.x / n_groups;
+    const int gi = blockIdx.x % n_groups;
+    const T* wp = W + row * ldw + (int64_t)gi * group;
+    const double* sp = s64 + (int64_t)gi * group;
+
+    float mn = INFINITY, mx = -INFINITY;
+    for (int j = tid; j < group; j += AF_THREADS) {
+        float w = load_w(wp + j);
+        wg[j] = w;
+        mn = fminf(mn, w);
+        mx = fmaxf(mx, w);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    }
+    if (lane == 0) { redf[0][warp] = mn; redf[1][warp] = mx; }
+    __syncthreads();
+    mn = redf[0][0]; mx = redf[1][0];
+    for (int w = 1; w < AF_THREADS / 32; ++w) { mn = fminf(mn, redf[0][w]); mx = fmaxf(mx, redf[1][w]); }
+    const double dmn = mn, dmx = mx, R = dmx - dmn;
+    const double Km1 = static_cast<double>(K - 1);
+    const int64_t out = row * n_groups + gi;
+
+    if (R == 0.0) {                                // constant group
+        if (tid == 0) {
+            double lo = fmin(dmn, 0.0), hi = fmax(dmx, 0.0);
+            double S = 1.0, Z = 0.0;
+            if (hi != lo) { S = (hi - lo) / Km1; Z = -rint(lo / S); }
+            scale[out] = static_cast<float>(S);
+            zero[out] = static_cast<int32_t>(Z);
+        }
+        return;
+    }
+
+    const int side = t_count + 1;
+    const int n_cand = side * side;
+    double my_loss = INFINITY;
+    int my_idx = 0x7fffffff;
+    for (int cand = tid; cand < n_cand; cand += AF_THREADS) {
+        const int t_min = cand / side, t_max = cand - t_min * side;
+        const double lo = dmn + static_cast<double>(t_min) * R / static_cast<double>(Tparts);
+        const double hi = dmx - static_cast<double>(t_max) * R / static_cast<double>(Tparts);
+        const double S = (hi - lo) / Km1;
+        if (!(S > 0.0)) continue;
+        const double Z = -rint(lo / S);
+        double loss = 0.0;
+        for (int j = 0; j < group; ++j) {
+            const double w = static_cast<double>(wg[j]);
+            double q = rint(w / S) + Z;
+            q = fmin(fmax(q, 0.0), Km1);
+            const double d = (q - Z) * S - w;
+            loss += sp[j] * (d * d);
+        }
+        if (loss < my_loss) { my_loss = loss; my_idx = cand; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const double ol = __shfl_xor_sync(0xffffffffu, my_loss, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, my_idx, o);
+        if (ol < my_loss || (ol == my_loss && oi < my_idx)) { my_loss = ol; my_idx = oi; }
+    }
+    if (lane == 0) { best_loss[warp] = my_loss; best_idx[warp] = my_idx; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < AF_THREADS / 32; ++w)
+            if (best_loss[w] < my_loss || (best_loss[w] == my_loss && best_idx[w] < my_idx)) {
+                my_loss = best_loss[w]; my_idx = best_idx[w];
+            }
+        double S = 1.0, Z = 0.0;
+        if (my_idx != 0x7fffffff) {
+            const int t_min = my_idx / side, t_max = my_idx - t_min * side;
+            const double lo = dmn + static_cast<double>(t_min) * R / static_cast<double>(Tparts);
+            const double hi = dmx - static_cast<double>(t_max) * R / static_cast<double>(Tparts);
+            S = (hi - lo) / Km1;
+            Z = -rint(lo / S);
+        }
+        scale[out] = static_cast<float>(S);
+        zero[out] = static_cast<int32_t>(Z);
+    }
+}
+
+int check_cfg(const lq_config* cfg) {
+    if (!cfg) return LQ_ERR_INVALID_ARG;
+    if (cfg->bits < 2 || cfg->bits > 4) return LQ_ERR_INVALID_ARG;
+    if (cfg->grid_type != LQ_GRID_NONUNIFORM && cfg->grid_type != LQ_GRID_AFFINE) return LQ_ERR_INVALID_ARG;
+    if (cfg->grid_type == LQ_GRID_NONUNIFORM && (cfg->n_iter < 0 || cfg->init != LQ_INIT_UNIFORM)) return LQ_ERR_INVALID_ARG;
+    if (cfg->grid_type == LQ_GRID_AFFINE &&
+        (cfg->T <= 0 || cfg->t_count < 0 || 2 * (int64_t)cfg->t_count > cfg->T || cfg->group_size < 0 || cfg->t_count > 4095))
+        return LQ_ERR_INVALID_ARG;
+    return LQ_OK;
+}
+
+}  // namespace
+
+extern "C" int lq_fit_grid_workspace(const lq_config* cfg, int64_t r, int64_t c, size_t* bytes) {
+    int e = check_cfg(cfg);
+    if (e) return e;
+    if (!bytes || r <= 0 || c <= 0) return LQ_ERR_INVALID_ARG;
+    *bytes = 256 + lq_align_up(static_cast<size_t>(c) * sizeof(double), 256);
+    return LQ_OK;
+}
+
+extern "C" int lq_fit_grid(lq_handle* h, void* stream, const lq_config* cfg, const void* W, int32_t w_dtype, int64_t r,
+                           int64_t c, int64_t ldw, const float* dinv, float* grid, float* scale, int32_t* zero, void* ws,
+                           size_t ws_bytes) {
+    int e = check_cfg(cfg);
+    if (e) return e;
+    if (!h || !W || !dinv || r <= 0 || c <= 0 || ldw < c) return LQ_ERR_INVALID_ARG;
+    if (w_dtype != LQ_F32 && w_dtype != LQ_BF16) return LQ_ERR_INVALID_ARG;
+    size_t need = 0;
+    lq_fit_grid_workspace(cfg, r, c, &need);
+    if (!ws || ws_bytes < need) return LQ_ERR_WORKSPACE_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(ws) & 255) return LQ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    double* scal = static_cast<double*>(ws);
+    double* s64 = reinterpret_cast<double*>(static_cast<char*>(ws) + 256);
+
+    if (cfg->grid_type == LQ_GRID_NONUNIFORM) {
+        if (!grid) return LQ_ERR_INVALID_ARG;
+    } else {
+        if (!scale || !zero) return LQ_ERR_INVALID_ARG;
+        const int64_t g = cfg->group_size == 0 ? c : cfg->group_size;
+        if (c % g) return LQ_ERR_INVALID_ARG;
+        if (g * sizeof(float) > 200 * 1024) return LQ_ERR_UNSUPPORTED;
+        if (r * (c / g) > 0x7fffffffLL) return LQ_ERR_UNSUPPORTED;
+    }
+
+    log_mean_kernel<<<1, 1024, 0, st>>>(dinv, c, scal, h->dstatus);
+    LQ_LAUNCH_CHECK();
+    sample_weights_kernel<<<static_cast<unsigned>(lq_ceil_div(c, 256)), 256, 0, st>>>(dinv, c, static_cast<double>(cfg->p), scal, s64);
+    LQ_LAUNCH_CHECK();
+
+    if (cfg->grid_type == LQ_GRID_NONUNIFORM) {
+#define LQ_KM(KK)                                                                                                     \
+    (w_dtype == LQ_F32 ? launch_kmeans<KK, float>(st, h->sm_count, static_cast<const float*>(W), ldw, r, c, s64, grid, cfg->n_iter) \
+                       : launch_kmeans<KK, __nv_bfloat16>(st, h->sm_count, static_cast<const __nv_bfloat16*>(W), ldw, r, c, s64, grid, cfg->n_iter))
+        switch (cfg->bits) {
+            case 2: return LQ_KM(4);
+            case 3: return LQ_KM(8);
+            default: return LQ_KM(16);
+        }
+#undef LQ_KM
+    }
+
+    const int64_t g = cfg->group_size == 0 ? c : cfg->group_size;
+    const int n_groups = static_cast<int>(c / g);
+    const size_t smem = static_cast<size_t>(g) * sizeof(float);
+    const unsigned blocks = static_cast<unsigned>(r * n_groups);
+    const int K = 1 << cfg->bits;
+    static bool attr_set = false;
+    if (!attr_set) {
+        LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        attr_set = true;
+    }
+    if (w_dtype == LQ_F32)
+        affine_search_kernel<float><<<blocks, AF_THREADS, smem, st>>>(static_cast<const float*>(W), ldw, c, (int)g, n_groups, s64, K,
+                                                                       cfg->T, cfg->t_count, scale, zero);
+    else
+        affine_search_kernel<__nv_bfloat16><<<blocks, AF_THREADS, smem, st>>>(static_cast<const __nv_bfloat16*>(W), ldw, c, (int)g,
+                                                                               n_groups, s64, K, cfg->T, cfg->t_count, scale, zero);
+    LQ_LAUNCH_CHECK();
+    return LQ_OK;
+}

@@ -1,0 +1,472 @@
+// bf16 x bf16 -> fp32 "NT" GEMM on the sm_100a tensor cores.
+//
+//   D[M x N] (+)= alpha * sum_p A_p[M x K] * B_p[N x K]^T        (all row-major, K contiguous)
+//
+// Used by stage 1 (H += 2 X X^T, Algorithm 1 line 3) and by the lazy trailing update of
+// the column loop (Algorithm 1 line 20).  fp32 operands are fed as several bf16 passes
+// (hi/mid/lo terms), which is what n_pass > 1 is for.
+//
+// One persistent CTA per SM, 128 x 256 output tiles, K consumed 64 at a time.
+//   warp 0      : TMA producer (cp.async.bulk.tensor, 128-byte swizzle, 4-stage ring)
+//   warp 1      : issues tcgen05.mma (one thread), accumulators in TMEM (2 x 256 columns,
+//                 so the epilogue of one tile overlaps the main loop of the next)
+//   warps 2..9  : epilogue.  The tensor core adds into its fp32 accumulator with truncation,
+//                 which over a long K biases every sum low; so K is consumed in short
+//                 segments, and after each one these warps tcgen05.ld the partial sum and
+//                 add it (round-to-nearest) to running sums held in registers.  After the
+//                 tile's last segment: scale -> swizzled smem slab -> TMA store, or a TMA
+//                 reduce-add when accumulating into D (no read of D by the SM).
+// Every wait on an mbarrier is bounded: when the time limit passes the CTA records
+// LQ_ERR_TIMEOUT in the handle's status word, stops issuing work and leaves.
+#include <cuda.h>
+
+#include "lq_common.cuh"
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BN = 256;
+constexpr int BK = 64;                 // 64 bf16 = 128 bytes = one swizzle row
+constexpr int UMMA_K = 16;
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = BM * BK * 2;
+constexpr int B_STAGE_BYTES = BN * BK * 2;
+constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+constexpr int EPI_COLS = 32;           // 32 fp32 = 128 bytes = one swizzle row
+constexpr int EPI_BUF_BYTES = BM * EPI_COLS * 4;
+constexpr int EPI_BUFS = 2;
+constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BUFS * EPI_BUF_BYTES + 1024;
+constexpr int NUM_THREADS = 320;
+constexpr int TMEM_COLS = 512;
+
+struct KParams {
+    int M, N, K;
+    int n_pass;
+    int a_off[6];
+    int b_off[6];
+    float alpha;
+    int accumulate;
+    int upper_only;
+    int tiles_m, tiles_n;
+    int num_tiles;
+    int seg_iters;            // k-iterations accumulated in TMEM before the partial sum is flushed to D
+    lq_dev_status* status;
+    unsigned long long timeout_ns;
+};
+
+// ---------------------------------------------------------------- PTX wrappers ----
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ unsigned long long global_timer() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          const KParams& p, int where) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer();
+    uint32_t spins = 0;
+    for (;;) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((++spins & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer() - t0 > p.timeout_ns) {
+                *abort_flag = 1;
+                lq_report(p.status, LQ_ERR_TIMEOUT, where);
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void tma_reduce_add_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
+    asm volatile("cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+template <int N> __device__ __forceinline__ void bulk_wait() {
+    asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t acc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(acc) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void group_bar_sync(uint32_t id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
+
+// Shared-memory matrix descriptor for a K-major bf16 tile stored by TMA with the 128-byte
+// swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_desc_sw128(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);       // start address / 16
+    d |= static_cast<uint64_t>(1) << 16;                        // leading byte offset / 16 (fixed for swizzled K-major)
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;                // stride byte offset / 16
+    d |= static_cast<uint64_t>(1) << 46;                        // descriptor version of this architecture
+    d |= static_cast<uint64_t>(2) << 61;                        // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 256.
+constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(BN >> 3) << 17) | (uint32_t(BM >> 4) << 24);
+
+// Map the idx-th scheduled tile to (tile row, tile column).  With upper_only, row tm keeps
+// the columns tn with (tn + 1) * BN > tm * BM.
+__device__ __forceinline__ void tile_coords(const KParams& p, int idx, int& tm, int& tn) {
+    if (!p.upper_only) {
+        tm = idx / p.tiles_n;
+        tn = idx - tm * p.tiles_n;
+        return;
+    }
+    int m = 0;
+    for (;; ++m) {
+        int first = (m * BM) / BN;
+        int cnt = p.tiles_n - first;
+        if (cnt < 0) cnt = 0;
+        if (idx < cnt) { tm = m; tn = first + idx; return; }
+        idx -= cnt;
+    }
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                  const __grid_constant__ CUtensorMap map_d, const __grid_constant__ KParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) uint64_t bars[2 * STAGES + 4];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const uint32_t warp_idx = threadIdx.x >> 5;
+    const uint32_t lane = threadIdx.x & 31;
+
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+    const uint32_t epi_base = smem_base + STAGES * STAGE_BYTES;
+    uint8_t* epi_gen = smem_gen + STAGES * STAGE_BYTES;
+
+    const uint32_t bar_full = smem_u32(&bars[0]);
+    const uint32_t bar_empty = smem_u32(&bars[STAGES]);
+    const uint32_t bar_tfull = smem_u32(&bars[2 * STAGES]);
+    const uint32_t bar_tempty = smem_u32(&bars[2 * STAGES + 2]);
+
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(bar_tfull + 8 * a, 1);
+            mbar_init(bar_tempty + 8 * a, 8);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp_idx == 1) {
+        tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_base_slot);
+    volatile int* abortp = &abort_flag;
+
+    const int k_blocks = (p.K + BK - 1) / BK;
+    const int k_iters = k_blocks * p.n_pass;
+
+    if (warp_idx == 0) {
+        // ------------------------------------------------------------ TMA producer
+        uint32_t stage = 0, phase = 0;
+        bool alive = true;
+        for (int t = blockIdx.x; t < p.num_tiles && alive; t += gridDim.x) {
+            int tm, tn;
+            tile_coords(p, t, tm, tn);
+            const int m0 = tm * BM, n0 = tn * BN;
+            for (int kit = 0; kit < k_iters; ++kit) {       // segments only matter to the consumers
+                if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abortp, p, 1)) { alive = false; break; }
+                if (lane == 0) {
+                    const int pass = kit / k_blocks;
+                    const int k0 = (kit - pass * k_blocks) * BK;
+                    const uint32_t sa = smem_base + stage * STAGE_BYTES;
+                    const uint32_t sb = sa + A_STAGE_BYTES;
+                    mbar_arrive_expect_tx(bar_full + 8 * stage, STAGE_BYTES);
+                    tma_load_2d(sa, &map_a, bar_full + 8 * stage, k0, p.a_off[pass] + m0);
+                    tma_load_2d(sb, &map_b, bar_full + 8 * stage, k0, p.b_off[pass] + n0);
+                }
+                __syncwarp();
+                if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
+    } else if (warp_idx == 1) {
+        // ------------------------------------------------------------ MMA issuer
+        uint32_t stage = 0, phase = 0;
+        int it = 0;                                  // counts (tile, segment) units: one TMEM accumulator each
+        bool alive = true;
+        for (int t = blockIdx.x; t < p.num_tiles && alive; t += gridDim.x) {
+            for (int k_lo = 0; k_lo < k_iters && alive; k_lo += p.seg_iters, ++it) {
+                const int k_hi = min(k_iters, k_lo + p.seg_iters);
+                const uint32_t acc = it & 1;
+                const uint32_t acc_phase = (it >> 1) & 1;
+                if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abortp, p, 2)) { alive = false; break; }
+                tc_fence_after();
+                const uint32_t tmem_d = tmem_base + acc * BN;
+                for (int kit = k_lo; kit < k_hi; ++kit) {
+                    if (!mbar_wait(bar_full + 8 * stage, phase, abortp, p, 3)) { alive = false; break; }
+                    tc_fence_after();
+                    if (lane == 0) {
+                        const uint32_t sa = smem_base + stage * STAGE_BYTES;
+                        const uint64_t da = make_desc_sw128(sa);
+                        const uint64_t db = make_desc_sw128(sa + A_STAGE_BYTES);
+#pragma unroll
+                        for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+                            // advancing 16 bf16 = 32 bytes inside the swizzle row: +2 in the address field
+                            umma_bf16(tmem_d, da + 2 * kk, db + 2 * kk, kInstrDesc, (kit > k_lo || kk > 0) ? 1u : 0u);
+                        }
+                        umma_commit(bar_empty + 8 * stage);
+                    }
+                    __syncwarp();
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!alive) break;
+                if (lane == 0) umma_commit(bar_tfull + 8 * acc);
+                __syncwarp();
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue (warps 2..9)
+        // Two groups of four warps; group hf owns columns [128*hf, 128*hf + 128) of the tile.
+        // Each thread keeps its row's 128 running sums in registers: after every segment
+        // the TMEM partial sum is added in with round-to-nearest, and the tile is written
+        // to D once, after its last segment.
+        const uint32_t q = warp_idx & 3;              // TMEM lane quarter this warp may read
+        const uint32_t hf = (warp_idx - 2) >> 2;
+        const uint32_t row = q * 32 + lane;           // row inside the tile
+        const bool leader = (lane == 0) && (warp_idx == 2 + 4 * hf);
+        uint8_t* my_buf = epi_gen + hf * EPI_BUF_BYTES;
+        const uint32_t my_buf_s = epi_base + hf * EPI_BUF_BYTES;
+        float accr[BN / 2];
+        int it = 0;
+        bool alive = true;
+        for (int t = blockIdx.x; t < p.num_tiles && alive; t += gridDim.x) {
+            int tm, tn;
+            tile_coords(p, t, tm, tn);
+            const int m0 = tm * BM, n0 = tn * BN;
+            for (int k_lo = 0; k_lo < k_iters; k_lo += p.seg_iters, ++it) {
+                const uint32_t acc = it & 1;
+                const uint32_t acc_phase = (it >> 1) & 1;
+                if (!mbar_wait(bar_tfull + 8 * acc, acc_phase, abortp, p, 4)) { alive = false; break; }
+                tc_fence_after();
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem_base + ((q * 32u) << 16) + acc * BN + hf * (BN / 2) + ch * EPI_COLS, v);
+                    tmem_wait_ld();
+                    if (k_lo == 0) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) accr[ch * 32 + i] = __uint_as_float(v[i]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) accr[ch * 32 + i] += __uint_as_float(v[i]);
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+            }
+            if (!alive) break;
+#pragma unroll
+            for (int ch = 0; ch < 4; ++ch) {
+                const int col0 = n0 + hf * (BN / 2) + ch * EPI_COLS;
+                if (col0 < p.N) {
+                    if (leader) bulk_wait_read<0>();          // the slab buffer has been read out
+                    group_bar_sync(1 + hf);
+                    uint8_t* rowp = my_buf + row * 128u;
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        float4 o;
+                        o.x = p.alpha * accr[ch * 32 + 4 * j + 0];
+                        o.y = p.alpha * accr[ch * 32 + 4 * j + 1];
+                        o.z = p.alpha * accr[ch * 32 + 4 * j + 2];
+                        o.w = p.alpha * accr[ch * 32 + 4 * j + 3];
+                        *reinterpret_cast<float4*>(rowp + ((j ^ (row & 7u)) << 4)) = o;
+                    }
+                    fence_async_smem();
+                    group_bar_sync(1 + hf);
+                    if (leader) {
+                        if (p.accumulate) tma_reduce_add_2d(&map_d, my_buf_s, col0, m0);
+                        else tma_store_2d(&map_d, my_buf_s, col0, m0);
+                        bulk_commit();
+                    }
+                }
+            }
+        }
+        if (leader) bulk_wait<0>();
+    }
+
+    if (*abortp) {
+        // give copies that were already issued time to land before the smem is released
+        const unsigned long long t0 = global_timer();
+        while (global_timer() - t0 < 200000ull) __nanosleep(1000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp_idx == 1) {
+        tc_fence_after();
+        __syncwarp();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------- host side ----
+typedef CUresult (*encode_tiled_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+encode_tiled_fn get_encode_fn() {
+    static encode_tiled_fn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<encode_tiled_fn>(ptr);
+    }
+    return fn;
+}
+
+bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const void* base, uint64_t inner,
+                 uint64_t outer, uint64_t ld_elems, uint32_t box_inner, uint32_t box_outer) {
+    encode_tiled_fn fn = get_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {ld_elems * static_cast<uint64_t>(elem_bytes)};
+    cuuint32_t box[2] = {box_inner, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
+    if (a.M <= 0 || a.N <= 0) return LQ_OK;
+    if (a.K <= 0) return LQ_OK;
+    if (a.n_pass < 1 || a.n_pass > 6) return LQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(a.A_all) & 15) || (reinterpret_cast<uintptr_t>(a.B_all) & 15) ||
+        (reinterpret_cast<uintptr_t>(a.D) & 15) || (a.lda % 8) || (a.ldb % 8) || (a.ldd % 4))
+        return LQ_ERR_INVALID_ARG;
+    if (a.a_rows > 0x7fffffffLL || a.b_rows > 0x7fffffffLL || a.K > 0x7fffffffLL || a.M > 0x7fffffffLL ||
+        a.N > 0x7fffffffLL)
+        return LQ_ERR_UNSUPPORTED;
+
+    static bool attr_set = false;
+    if (!attr_set) {
+        LQ_CUDA_TRY(cudaFuncSetAttribute(lq_tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+        attr_set = true;
+    }
+
+    CUtensorMap map_a, map_b, map_d;
+    if (!make_map_2d(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.A_all, a.K, a.a_rows, a.lda, BK, BM) ||
+        !make_map_2d(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.B_all, a.K, a.b_rows, a.ldb, BK, BN) ||
+        !make_map_2d(&map_d, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.D, a.N, a.M, a.ldd, EPI_COLS, BM))
+        return LQ_ERR_CUDA;
+
+    KParams p;
+    p.M = static_cast<int>(a.M);
+    p.N = static_cast<int>(a.N);
+    p.K = static_cast<int>(a.K);
+    p.n_pass = a.n_pass;
+    for (int i = 0; i < 6; ++i) {
+        p.a_off[i] = static_cast<int>(a.a_row_off[i]);
+        p.b_off[i] = static_cast<int>(a.b_row_off[i]);
+    }
+    p.alpha = a.alpha;
+    p.accumulate = a.accumulate;
+    p.upper_only = a.upper_only;
+    p.tiles_m = static_cast<int>(lq_ceil_div(a.M, BM));
+    p.tiles_n = static_cast<int>(lq_ceil_div(a.N, BN));
+    if (a.upper_only) {
+        int cnt = 0;
+        for (int m = 0; m < p.tiles_m; ++m) {
+            int c = p.tiles_n - (m * BM) / BN;
+            if (c > 0) cnt += c;
+        }
+        p.num_tiles = cnt;
+    } else {
+        p.num_tiles = p.tiles_m * p.tiles_n;
+    }
+    p.status = h->dstatus;
+    p.timeout_ns = 5ull * 1000ull * 1000ull * 1000ull;
+    if (p.num_tiles == 0) return LQ_OK;
+    {
+        const int k_iters = static_cast<int>(lq_ceil_div(a.K, BK)) * a.n_pass;
+        p.seg_iters = (a.seg_iters > 0 && a.seg_iters < k_iters) ? a.seg_iters : k_iters;
+    }
+
+    int grid = p.num_tiles < h->sm_count ? p.num_tiles : h->sm_count;
+    lq_tc_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, map_d, p);
+    LQ_LAUNCH_CHECK();
+    return LQ_OK;
+}

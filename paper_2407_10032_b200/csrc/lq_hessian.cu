@@ -1,0 +1,104 @@
+// Stage 1 -- Algorithm 1 line 3: H <- 2 X X^T, accumulated chunk by chunk.
+// The contraction itself is lq_tc_gemm (tcgen05 + TMA); this file holds the entry points,
+// the fp32 -> 3 x bf16 operand split and the upper -> lower mirror.
+#include "lq_common.cuh"
+
+#include <stdlib.h>
+namespace {
+
+// Tokens are summed in TMEM 64 * kSegIters at a time; see lq_tc_gemm_args::seg_iters.
+constexpr int kSegIters = 8;
+
+// src: rows x cols fp32 (ld).  dst: 3 stacked bf16 matrices of rows x dst_ld (hi, mid, lo).
+__global__ void split3_kernel(const float* __restrict__ src, int64_t ld, int64_t rows, int64_t cols,
+                              __nv_bfloat16* __restrict__ dst, int64_t dst_ld) {
+    const int64_t row = blockIdx.y;
+    const float* s = src + row * ld;
+    __nv_bfloat16* d0 = dst + row * dst_ld;
+    __nv_bfloat16* d1 = d0 + rows * dst_ld;
+    __nv_bfloat16* d2 = d1 + rows * dst_ld;
+    for (int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < dst_ld; j += (int64_t)gridDim.x * blockDim.x) {
+        float x = j < cols ? s[j] : 0.0f;
+        __nv_bfloat16 a, b, c;
+        lq_split3(x, a, b, c);
+        d0[j] = a; d1[j] = b; d2[j] = c;
+    }
+}
+
+// H[j][i] = H[i][j] for j > i, 32 x 32 tiles through shared memory.
+__global__ void mirror_upper_kernel(float* __restrict__ H, int64_t c, int64_t ldh) {
+    __shared__ float tile[32][33];
+    const int bi = blockIdx.y, bj = blockIdx.x;     // source tile (rows bi, cols bj), bj >= bi
+    if (bj < bi) return;
+    const int tx = threadIdx.x, ty = threadIdx.y;   // 32 x 8
+    for (int k = ty; k < 32; k += 8) {
+        int64_t i = (int64_t)bi * 32 + k, j = (int64_t)bj * 32 + tx;
+        tile[k][tx] = (i < c && j < c) ? H[i * ldh + j] : 0.0f;
+    }
+    __syncthreads();
+    for (int k = ty; k < 32; k += 8) {
+        int64_t j = (int64_t)bj * 32 + k, i = (int64_t)bi * 32 + tx;   // destination H[j][i]
+        if (j < c && i < c && j > i) H[j * ldh + i] = tile[tx][k];
+    }
+}
+
+}  // namespace
+
+extern "C" int lq_hessian_workspace(int32_t x_dtype, int64_t c, int64_t n_chunk, size_t* bytes) {
+    if (!bytes || c <= 0 || n_chunk < 0) return LQ_ERR_INVALID_ARG;
+    if (x_dtype == LQ_BF16) { *bytes = 0; return LQ_OK; }
+    if (x_dtype != LQ_F32) return LQ_ERR_INVALID_ARG;
+    int64_t ld = lq_ceil_div(n_chunk, 8) * 8;
+    *bytes = lq_align_up(static_cast<size_t>(3) * c * ld * sizeof(__nv_bfloat16), 256);
+    return LQ_OK;
+}
+
+extern "C" int lq_hessian_accumulate(lq_handle* h, void* stream, const void* X, int32_t x_dtype, int32_t layout,
+                                     int64_t c, int64_t n_chunk, int64_t ldx, float* H, int64_t ldh, float alpha,
+                                     void* ws, size_t ws_bytes) {
+    if (!h || !X || !H || c <= 0 || n_chunk < 0 || ldx < n_chunk || ldh < c) return LQ_ERR_INVALID_ARG;
+    if (layout != LQ_FEATURE_MAJOR) return LQ_ERR_UNSUPPORTED;
+    if (x_dtype != LQ_BF16 && x_dtype != LQ_F32) return LQ_ERR_INVALID_ARG;
+    if (ldh % 4 || (reinterpret_cast<uintptr_t>(H) & 15) || (reinterpret_cast<uintptr_t>(X) & 15)) return LQ_ERR_INVALID_ARG;
+    if (n_chunk == 0) return LQ_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    lq_tc_gemm_args g = {};
+    g.D = H; g.ldd = ldh; g.M = c; g.N = c; g.K = n_chunk;
+    g.alpha = alpha; g.accumulate = 1; g.upper_only = 1;
+    g.seg_iters = kSegIters;
+    if (const char* e = getenv("LQ_HESSIAN_SEG")) g.seg_iters = atoi(e);
+    if (x_dtype == LQ_BF16) {
+        if (ldx % 8) return LQ_ERR_INVALID_ARG;
+        g.A_all = g.B_all = static_cast<const __nv_bfloat16*>(X);
+        g.a_rows = g.b_rows = c; g.lda = g.ldb = ldx;
+        g.n_pass = 1;
+    } else {
+        size_t need = 0;
+        lq_hessian_workspace(x_dtype, c, n_chunk, &need);
+        if (!ws || ws_bytes < need) return LQ_ERR_WORKSPACE_TOO_SMALL;
+        if (reinterpret_cast<uintptr_t>(ws) & 15) return LQ_ERR_INVALID_ARG;
+        const int64_t ld = lq_ceil_div(n_chunk, 8) * 8;
+        __nv_bfloat16* split = static_cast<__nv_bfloat16*>(ws);
+        dim3 grid(static_cast<unsigned>(lq_ceil_div(ld, 256) < 64 ? lq_ceil_div(ld, 256) : 64), static_cast<unsigned>(c));
+        split3_kernel<<<grid, 256, 0, st>>>(static_cast<const float*>(X), ldx, c, n_chunk, split, ld);
+        LQ_LAUNCH_CHECK();
+        g.A_all = g.B_all = split;
+        g.a_rows = g.b_rows = 3 * c; g.lda = g.ldb = ld;
+        // (hi,hi) (hi,mid) (mid,hi) (hi,lo) (lo,hi) (mid,mid): every product term above 2^-24 relative
+        const int64_t ao[6] = {0, 0, c, 0, 2 * c, c};
+        const int64_t bo[6] = {0, c, 0, 2 * c, 0, c};
+        for (int i = 0; i < 6; ++i) { g.a_row_off[i] = ao[i]; g.b_row_off[i] = bo[i]; }
+        g.n_pass = 6;
+    }
+    return lq_tc_gemm(h, st, g);
+}
+
+extern "C" int lq_hessian_finalize(lq_handle* h, void* stream, float* H, int64_t c, int64_t ldh) {
+    if (!h || !H || c <= 0 || ldh < c) return LQ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned nb = static_cast<unsigned>(lq_ceil_div(c, 32));
+    mirror_upper_kernel<<<dim3(nb, nb), dim3(32, 8), 0, st>>>(H, c, ldh);
+    LQ_LAUNCH_CHECK();
+    return LQ_OK;
+}

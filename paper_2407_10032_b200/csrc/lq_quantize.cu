@@ -1,0 +1,415 @@
+// Stage 4 -- Algorithm 1 lines 10-21: the block-wise column loop with error feedback.
+//
+// Per block of B = 128 columns:
+//   in-block kernel  : one thread per output row keeps the row's 128 block weights in
+//                      registers and walks the columns in order (quantise, E = (w - q)/U_jj,
+//                      w[k] -= E * U[j][k]); the 128 x 128 diagonal block of U sits in shared
+//                      memory and is read as warp-wide broadcasts.  The walk is organised as
+//                      8 sub-blocks of 16 columns so that the register file is indexed
+//                      statically while the code stays small.
+//   trailing update  : W[:, i+B:] -= E U[i:i+B, i+B:] on the tensor cores (lq_tc_gemm), fp32
+//                      operands fed as three bf16 terms each (six products), accumulated into
+//                      the fp32 working copy by the copy engine's reduce-add.
+#include <math.h>
+
+#include "lq_common.cuh"
+
+namespace {
+
+constexpr int B = 128;      // block width of the column loop
+constexpr int SB = 16;      // sub-block width
+constexpr int NSB = B / SB;
+
+template <typename T>
+__global__ void to_f32_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, float* __restrict__ Wc, int64_t ldc) {
+    const int64_t row = blockIdx.y;
+    for (int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < ldc; j += (int64_t)gridDim.x * blockDim.x) {
+        float v = 0.0f;
+        if (j < c) {
+            if (sizeof(T) == 4) v = reinterpret_cast<const float*>(W)[row * ldw + j];
+            else v = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(W)[row * ldw + j]);
+        }
+        Wc[row * ldc + j] = v;
+    }
+}
+
+// UT[s][n][k] = s-th bf16 term of U[k][n]   (three stacked c x ldt matrices)
+__global__ void split_transpose_kernel(const float* __restrict__ U, int64_t ldu, int64_t c,
+                                       __nv_bfloat16* __restrict__ UT, int64_t ldt) {
+    __shared__ float tile[32][33];
+    const int64_t k0 = (int64_t)blockIdx.y * 32, n0 = (int64_t)blockIdx.x * 32;
+    const int tx = threadIdx.x, ty = threadIdx.y;       // 32 x 8
+    for (int a = ty; a < 32; a += 8) {
+        const int64_t k = k0 + a, n = n0 + tx;
+        tile[a][tx] = (k < c && n < c) ? U[k * ldu + n] : 0.0f;
+    }
+    __syncthreads();
+    for (int a = ty; a < 32; a += 8) {
+        const int64_t n = n0 + a, k = k0 + tx;
+        if (n < c && k < ldt) {
+            __nv_bfloat16 h, m, l;
+            lq_split3(k < c ? tile[tx][a] : 0.0f, h, m, l);
+            UT[n * ldt + k] = h;
+            UT[(c + n) * ldt + k] = m;
+            UT[(2 * c + n) * ldt + k] = l;
+        }
+    }
+}
+
+template <int K>
+struct NuGrid {
+    float g[K];
+    float m[K - 1];
+    __device__ __forceinline__ void load(const float* grid_row) {
+#pragma unroll
+        for (int k = 0; k < K; ++k) g[k] = grid_row[k];
+#pragma unroll
+        for (int k = 0; k < K - 1; ++k) m[k] = 0.5f * (g[k] + g[k + 1]);
+    }
+    // nearest grid point: code = number of midpoints strictly below w
+    __device__ __forceinline__ void quant(float w, int& code, float& q) const {
+        int cnt = 0;
+#pragma unroll
+        for (int k = 0; k < K - 1; ++k) cnt += (w > m[k]) ? 1 : 0;
+        code = cnt;
+        float sel[K];
+#pragma unroll
+        for (int k = 0; k < K; ++k) sel[k] = g[k];
+#pragma unroll
+        for (int width = K / 2, bit = 1; width >= 1; width >>= 1, bit <<= 1) {
+#pragma unroll
+            for (int k = 0; k < width; ++k) sel[k] = (cnt & bit) ? sel[2 * k + 1] : sel[2 * k];
+        }
+        q = sel[0];
+    }
+};
+
+struct QuantOut {
+    uint8_t* codes;          // r x c
+    void* what;              // r x ldwh or null
+    int what_bf16;
+    int64_t ldwh;
+    __nv_bfloat16* esplit;   // 3 x r x B
+    double* loss_rows;       // r
+};
+
+template <int K, bool AFFINE>
+__global__ void __launch_bounds__(128)
+inblock_kernel(float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, int64_t i0, const float* __restrict__ U,
+               int64_t ldu, const float* __restrict__ grid, const float* __restrict__ scale,
+               const int32_t* __restrict__ zero, int group, int n_groups, QuantOut out) {
+    extern __shared__ float Us[];          // B x B block of U, then B reciprocals of its diagonal
+    float* invd = Us + B * B;
+    const int tid = threadIdx.x;
+    const int bw = (c - i0) < B ? static_cast<int>(c - i0) : B;
+
+    for (int idx = tid; idx < B * B / 4; idx += 128) {
+        const int jj = idx / (B / 4), k4 = (idx % (B / 4)) * 4;
+        float4 v;
+        if (jj < bw && k4 + 3 < bw && (ldu % 4 == 0)) {
+            v = *reinterpret_cast<const float4*>(U + (i0 + jj) * ldu + i0 + k4);
+        } else {
+            float t[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int kk = k4 + u;
+                t[u] = (jj < bw && kk < bw) ? U[(i0 + jj) * ldu + i0 + kk] : (jj == kk ? 1.0f : 0.0f);
+            }
+            v = make_float4(t[0], t[1], t[2], t[3]);
+        }
+        *reinterpret_cast<float4*>(Us + jj * B + k4) = v;
+    }
+    __syncthreads();
+    if (tid < B) invd[tid] = 1.0f / Us[tid * B + tid];
+    __syncthreads();
+
+    const int64_t row = (int64_t)blockIdx.x * 128 + tid;
+    if (row >= r) return;
+
+    float w[B];
+    {
+        const float* wp = Wc + row * ldc + i0;
+#pragma unroll
+        for (int k = 0; k < B; k += 4) {
+            if (k + 3 < bw) {
+                const float4 v = *reinterpret_cast<const float4*>(wp + k);
+                w[k] = v.x; w[k + 1] = v.y; w[k + 2] = v.z; w[k + 3] = v.w;
+            } else {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) w[k + u] = (k + u < bw) ? wp[k + u] : 0.0f;
+            }
+        }
+    }
+
+    NuGrid<K> ng;
+    if (!AFFINE) ng.load(grid + row * K);
+    double loss = 0.0;
+
+#pragma unroll 1
+    for (int s = 0; s < NSB; ++s) {
+        float ws[SB];
+#pragma unroll
+        for (int kb = 0; kb < NSB; ++kb)
+            if (kb == s) {
+#pragma unroll
+                for (int t = 0; t < SB; ++t) ws[t] = w[kb * SB + t];
+            }
+        float S = 1.0f, Zf = 0.0f;
+        if (AFFINE) {
+            const int64_t gi = (i0 + s * SB) / group;
+            const int64_t gidx = row * n_groups + (gi < n_groups ? gi : n_groups - 1);
+            S = scale[gidx];
+            Zf = static_cast<float>(zero[gidx]);
+        }
+        float e[SB];
+        float qv[SB];
+        uint32_t cpack[SB / 4];
+#pragma unroll
+        for (int t = 0; t < SB / 4; ++t) cpack[t] = 0;
+        const float* urow = Us + (s * SB) * B + s * SB;
+#pragma unroll
+        for (int t = 0; t < SB; ++t) {
+            int code;
+            float q;
+            if (AFFINE) {
+                float qi = rintf(__fdiv_rn(ws[t], S)) + Zf;
+                qi = fminf(fmaxf(qi, 0.0f), static_cast<float>(K - 1));
+                code = static_cast<int>(qi);
+                q = (qi - Zf) * S;
+            } else {
+                ng.quant(ws[t], code, q);
+            }
+            const bool live = (s * SB + t) < bw;
+            const float et = live ? (ws[t] - q) * invd[s * SB + t] : 0.0f;
+            e[t] = et;
+            qv[t] = q;
+            cpack[t >> 2] |= static_cast<uint32_t>(code) << (8 * (t & 3));
+            loss += static_cast<double>(et) * static_cast<double>(et);
+#pragma unroll
+            for (int u = t + 1; u < SB; ++u) ws[u] = fmaf(-et, urow[t * B + u], ws[u]);
+        }
+        // feed the 16 errors forward to the later sub-blocks of this block
+#pragma unroll
+        for (int kb = 1; kb < NSB; ++kb) {
+            if (kb > s) {
+#pragma unroll
+                for (int t = 0; t < SB; ++t) {
+                    const float4* up = reinterpret_cast<const float4*>(Us + (s * SB + t) * B + kb * SB);
+#pragma unroll
+                    for (int u4 = 0; u4 < SB / 4; ++u4) {
+                        const float4 uv = up[u4];
+                        w[kb * SB + 4 * u4 + 0] = fmaf(-e[t], uv.x, w[kb * SB + 4 * u4 + 0]);
+                        w[kb * SB + 4 * u4 + 1] = fmaf(-e[t], uv.y, w[kb * SB + 4 * u4 + 1]);
+                        w[kb * SB + 4 * u4 + 2] = fmaf(-e[t], uv.z, w[kb * SB + 4 * u4 + 2]);
+                        w[kb * SB + 4 * u4 + 3] = fmaf(-e[t], uv.w, w[kb * SB + 4 * u4 + 3]);
+                    }
+                }
+            }
+        }
+        // outputs of this sub-block
+        const int col0 = s * SB;
+        if (col0 < bw) {
+            const int64_t gcol = i0 + col0;
+            if (col0 + SB <= bw && (c % 16 == 0)) {
+                *reinterpret_cast<uint4*>(out.codes + row * c + gcol) = make_uint4(cpack[0], cpack[1], cpack[2], cpack[3]);
+            } else {
+#pragma unroll
+                for (int t = 0; t < SB; ++t)
+                    if (col0 + t < bw) out.codes[row * c + gcol + t] = static_cast<uint8_t>((cpack[t >> 2] >> (8 * (t & 3))) & 0xff);
+            }
+            if (out.what) {
+#pragma unroll
+                for (int t = 0; t < SB; ++t)
+                    if (col0 + t < bw) {
+                        if (out.what_bf16) static_cast<__nv_bfloat16*>(out.what)[row * out.ldwh + gcol + t] = __float2bfloat16_rn(qv[t]);
+                        else static_cast<float*>(out.what)[row * out.ldwh + gcol + t] = qv[t];
+                    }
+            }
+        }
+        {
+            uint32_t ph[SB / 2], pm[SB / 2], pl[SB / 2];
+#pragma unroll
+            for (int t = 0; t < SB; t += 2) {
+                __nv_bfloat16 h0, m0, l0, h1, m1, l1;
+                lq_split3(e[t], h0, m0, l0);
+                lq_split3(e[t + 1], h1, m1, l1);
+                ph[t / 2] = static_cast<uint32_t>(__bfloat16_as_ushort(h0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(h1)) << 16);
+                pm[t / 2] = static_cast<uint32_t>(__bfloat16_as_ushort(m0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(m1)) << 16);
+                pl[t / 2] = static_cast<uint32_t>(__bfloat16_as_ushort(l0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(l1)) << 16);
+            }
+            __nv_bfloat16* e0 = out.esplit + row * B + col0;
+            __nv_bfloat16* e1 = e0 + r * B;
+            __nv_bfloat16* e2 = e1 + r * B;
+            *reinterpret_cast<uint4*>(e0) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
+            *reinterpret_cast<uint4*>(e0 + 8) = make_uint4(ph[4], ph[5], ph[6], ph[7]);
+            *reinterpret_cast<uint4*>(e1) = make_uint4(pm[0], pm[1], pm[2], pm[3]);
+            *reinterpret_cast<uint4*>(e1 + 8) = make_uint4(pm[4], pm[5], pm[6], pm[7]);
+            *reinterpret_cast<uint4*>(e2) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
+            *reinterpret_cast<uint4*>(e2 + 8) = make_uint4(pl[4], pl[5], pl[6], pl[7]);
+        }
+    }
+    out.loss_rows[row] += loss;
+}
+
+__global__ void zero_doubles_kernel(double* p, int64_t n) {
+    const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (i < n) p[i] = 0.0;
+}
+
+// loss_out[0] = 1/2 * sum_rows loss_rows
+__global__ void loss_reduce_kernel(const double* __restrict__ loss_rows, int64_t r, double* __restrict__ loss_out) {
+    __shared__ double red[1024];
+    double s = 0.0;
+    for (int64_t i = threadIdx.x; i < r; i += blockDim.x) s += loss_rows[i];
+    red[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = blockDim.x / 2; o > 0; o >>= 1) {
+        if (threadIdx.x < o) red[threadIdx.x] += red[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) loss_out[0] = 0.5 * red[0];
+}
+
+struct WsLayout {
+    size_t wc, ut, es, loss, total;
+    int64_t ldc, ldt;
+};
+WsLayout ws_layout(int64_t r, int64_t c) {
+    WsLayout L;
+    L.ldc = lq_ceil_div(c, 4) * 4;
+    L.ldt = lq_ceil_div(c, 8) * 8;
+    size_t off = 0;
+    L.wc = off; off += lq_align_up(static_cast<size_t>(r) * L.ldc * sizeof(float), 256);
+    L.ut = off; off += lq_align_up(static_cast<size_t>(3) * c * L.ldt * sizeof(__nv_bfloat16), 256);
+    L.es = off; off += lq_align_up(static_cast<size_t>(3) * r * B * sizeof(__nv_bfloat16), 256);
+    L.loss = off; off += lq_align_up(static_cast<size_t>(r) * sizeof(double), 256);
+    L.total = off;
+    return L;
+}
+
+int check_cfg4(const lq_config* cfg) {
+    if (!cfg) return LQ_ERR_INVALID_ARG;
+    if (cfg->bits < 2 || cfg->bits > 4) return LQ_ERR_INVALID_ARG;
+    if (cfg->block != B) return LQ_ERR_UNSUPPORTED;
+    if (cfg->grid_type != LQ_GRID_NONUNIFORM && cfg->grid_type != LQ_GRID_AFFINE) return LQ_ERR_INVALID_ARG;
+    return LQ_OK;
+}
+
+template <int K, bool AFFINE>
+int launch_inblock(cudaStream_t st, float* Wc, int64_t ldc, int64_t r, int64_t c, int64_t i0, const float* U, int64_t ldu,
+                   const float* grid, const float* scale, const int32_t* zero, int group, int n_groups, const QuantOut& out) {
+    const int smem = (B * B + B) * sizeof(float);
+    static bool attr_set = false;
+    if (!attr_set) {
+        LQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel<K, AFFINE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        attr_set = true;
+    }
+    inblock_kernel<K, AFFINE><<<static_cast<unsigned>(lq_ceil_div(r, 128)), 128, smem, st>>>(
+        Wc, ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out);
+    LQ_LAUNCH_CHECK();
+    return LQ_OK;
+}
+
+}  // namespace
+
+extern "C" int lq_quantize_layer_workspace(const lq_config* cfg, int64_t r, int64_t c, size_t* bytes) {
+    int e = check_cfg4(cfg);
+    if (e) return e;
+    if (!bytes || r <= 0 || c <= 0) return LQ_ERR_INVALID_ARG;
+    *bytes = ws_layout(r, c).total;
+    return LQ_OK;
+}
+
+extern "C" int lq_quantize_layer(lq_handle* h, void* stream, const lq_config* cfg, const void* W, int32_t w_dtype,
+                                 int64_t r, int64_t c, int64_t ldw, const float* U, int64_t ldu, const float* grid,
+                                 const float* scale, const int32_t* zero, uint8_t* codes, void* W_hat,
+                                 int32_t what_dtype, int64_t ldwh, double* loss_out, void* ws, size_t ws_bytes) {
+    int e = check_cfg4(cfg);
+    if (e) return e;
+    if (!h || !W || !U || !codes || r <= 0 || c <= 0 || ldw < c || ldu < c) return LQ_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(U) & 15) || (reinterpret_cast<uintptr_t>(codes) & 15)) return LQ_ERR_INVALID_ARG;
+    if (w_dtype != LQ_F32 && w_dtype != LQ_BF16) return LQ_ERR_INVALID_ARG;
+    if (W_hat && (ldwh < c || (what_dtype != LQ_F32 && what_dtype != LQ_BF16))) return LQ_ERR_INVALID_ARG;
+    const bool affine = cfg->grid_type == LQ_GRID_AFFINE;
+    int group = 0, n_groups = 1;
+    if (affine) {
+        if (!scale || !zero) return LQ_ERR_INVALID_ARG;
+        const int64_t g = cfg->group_size == 0 ? c : cfg->group_size;
+        if (c % g) return LQ_ERR_INVALID_ARG;
+        if (g != c && (g % SB)) return LQ_ERR_UNSUPPORTED;     // (S, Z) may change only between 16-column sub-blocks
+        if (g > 0x7fffffffLL) return LQ_ERR_UNSUPPORTED;
+        group = static_cast<int>(g);
+        n_groups = static_cast<int>(c / g);
+    } else if (!grid) {
+        return LQ_ERR_INVALID_ARG;
+    }
+    const WsLayout L = ws_layout(r, c);
+    if (!ws || ws_bytes < L.total) return LQ_ERR_WORKSPACE_TOO_SMALL;
+    if (reinterpret_cast<uintptr_t>(ws) & 255) return LQ_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char* wsp = static_cast<char*>(ws);
+    float* Wc = reinterpret_cast<float*>(wsp + L.wc);
+    __nv_bfloat16* UT = reinterpret_cast<__nv_bfloat16*>(wsp + L.ut);
+    __nv_bfloat16* ES = reinterpret_cast<__nv_bfloat16*>(wsp + L.es);
+    double* loss_rows = reinterpret_cast<double*>(wsp + L.loss);
+
+    {
+        dim3 g(static_cast<unsigned>(lq_ceil_div(L.ldc, 256) < 32 ? lq_ceil_div(L.ldc, 256) : 32), static_cast<unsigned>(r));
+        if (w_dtype == LQ_F32) to_f32_kernel<float><<<g, 256, 0, st>>>(static_cast<const float*>(W), ldw, c, Wc, L.ldc);
+        else to_f32_kernel<__nv_bfloat16><<<g, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(W), ldw, c, Wc, L.ldc);
+        LQ_LAUNCH_CHECK();
+    }
+    if (c > B) {
+        dim3 g(static_cast<unsigned>(lq_ceil_div(c, 32)), static_cast<unsigned>(lq_ceil_div(L.ldt, 32)));
+        split_transpose_kernel<<<g, dim3(32, 8), 0, st>>>(U, ldu, c, UT, L.ldt);
+        LQ_LAUNCH_CHECK();
+    }
+    zero_doubles_kernel<<<static_cast<unsigned>(lq_ceil_div(r, 256)), 256, 0, st>>>(loss_rows, r);
+    LQ_LAUNCH_CHECK();
+
+    QuantOut out;
+    out.codes = codes;
+    out.what = W_hat;
+    out.what_bf16 = (what_dtype == LQ_BF16);
+    out.ldwh = ldwh;
+    out.esplit = ES;
+    out.loss_rows = loss_rows;
+
+    for (int64_t i0 = 0; i0 < c; i0 += B) {
+        int rc;
+        if (affine) {
+            switch (cfg->bits) {
+                case 2: rc = launch_inblock<4, true>(st, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
+                case 3: rc = launch_inblock<8, true>(st, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
+                default: rc = launch_inblock<16, true>(st, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
+            }
+        } else {
+            switch (cfg->bits) {
+                case 2: rc = launch_inblock<4, false>(st, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
+                case 3: rc = launch_inblock<8, false>(st, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
+                default: rc = launch_inblock<16, false>(st, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
+            }
+        }
+        if (rc) return rc;
+        const int64_t rest = c - (i0 + B);
+        if (rest > 0) {
+            lq_tc_gemm_args g = {};
+            g.A_all = ES; g.a_rows = 3 * r; g.lda = B;
+            g.B_all = UT + (i0 + B) * L.ldt + i0; g.b_rows = 3 * c - (i0 + B); g.ldb = L.ldt;
+            g.D = Wc + (i0 + B); g.ldd = L.ldc;
+            g.M = r; g.N = rest; g.K = B;
+            g.n_pass = 6;
+            const int64_t ao[6] = {0, 0, r, 0, 2 * r, r};
+            const int64_t bo[6] = {0, c, 0, 2 * c, 0, c};
+            for (int i = 0; i < 6; ++i) { g.a_row_off[i] = ao[i]; g.b_row_off[i] = bo[i]; }
+            g.alpha = -1.0f; g.accumulate = 1; g.upper_only = 0;
+            rc = lq_tc_gemm(h, st, g);
+            if (rc) return rc;
+        }
+    }
+    if (loss_out) {
+        loss_reduce_kernel<<<1, 1024, 0, st>>>(loss_rows, r, loss_out);
+        LQ_LAUNCH_CHECK();
+    }
+    return LQ_OK;
+}
