@@ -98,6 +98,19 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
+def layer_seed(rank: int) -> int:
+    """Every rank quantises a different synthetic layer."""
+    return 1000 + rank
+
+
+def max_over_ranks(t: torch.Tensor, world: int) -> torch.Tensor:
+    """Multi-rank timings are reported as the maximum over ranks."""
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t
+
+
 def dist_env():
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -177,7 +190,7 @@ def run_ours(args):
     recipe, r, c, n, st = WORKLOADS[args.workload]
     cfg = lq.Config.make(**st)
     h = lq.lq_create(local)
-    layer = synth.make_layer(recipe, r, c, n, seed=1000 + rank, device=dev)
+    layer = synth.make_layer(recipe, r, c, n, seed=layer_seed(rank), device=dev)
     W, X = layer.W, layer.X
     P = lq.LayerPass(h, r, c, cfg, w_dtype=W.dtype, x_dtype=X.dtype, n_chunk=n, device=dev)
     stream = torch.cuda.current_stream()
@@ -257,9 +270,7 @@ def run_ours(args):
     h2d = Xh.numel() * Xh.element_size() + Wh.numel() * Wh.element_size()
     d2h = codes_h.numel() + grid_h.numel() * 4 + 8
 
-    t = torch.tensor([total_ms, e2e_ms], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    t = max_over_ranks(torch.tensor([total_ms, e2e_ms], device=dev, dtype=torch.float64), world)
     total_ms, e2e_ms = float(t[0]), float(t[1])
     ms_per_step = total_ms / args.steps
     weights = r * c * world

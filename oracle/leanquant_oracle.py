@@ -252,7 +252,7 @@ def fit_grid_affine(W, dinv, bits: int, p: float = 4.0, group: int = 0,
 # Stage 4 -- Algorithm 1 lines 10-21: block-wise column loop with error feedback
 # --------------------------------------------------------------------------- #
 def quantize_layer(W, U, *, grid=None, scale=None, zero=None, bits: int = 4,
-                   group: int = 0, block: int = 128):
+                   group: int = 0, block: int = 128, return_pre: bool = False):
     """The iterative loss-error-based loop on a learned grid.
 
     For each block of ``block`` columns, for each column j in it: quantise W[:, j] for
@@ -262,13 +262,15 @@ def quantize_layer(W, U, *, grid=None, scale=None, zero=None, bits: int = 4,
     W[:, i+B:] -= E @ U[i:i+B, i+B:].
 
     Returns codes (r x c, int64), W_hat (r x c) and loss = 1/2 * sum(E^2), the summed
-    loss error of Eq. 3 with the damped inverse."""
+    loss error of Eq. 3 with the damped inverse.  With ``return_pre`` a fourth array holds
+    every weight as it stood at the moment it was quantised (for tie analysis in tests)."""
     Wc = np.array(W, dtype=F64, copy=True)
     U = np.asarray(U, dtype=F64)
     r, c = Wc.shape
     K = 1 << bits
     codes = np.zeros((r, c), dtype=np.int64)
     What = np.zeros((r, c), dtype=F64)
+    Wpre = np.zeros((r, c), dtype=F64) if return_pre else None
     loss = 0.0
     g = c if group in (0, None) else group
     for i in range(0, c, block):
@@ -276,6 +278,8 @@ def quantize_layer(W, U, *, grid=None, scale=None, zero=None, bits: int = 4,
         E = np.zeros((r, e_end - i), dtype=F64)
         for j in range(i, e_end):
             w = Wc[:, j]
+            if return_pre:
+                Wpre[:, j] = w
             if grid is not None:
                 a = assign_nu(w[:, None], grid)[:, 0]
                 q = np.take_along_axis(grid, a[:, None], 1)[:, 0]
@@ -292,6 +296,8 @@ def quantize_layer(W, U, *, grid=None, scale=None, zero=None, bits: int = 4,
         loss += 0.5 * float((E * E).sum())
         if e_end < c:
             Wc[:, e_end:] -= E @ U[i:e_end, e_end:]
+    if return_pre:
+        return codes, What, loss, Wpre
     return codes, What, loss
 
 

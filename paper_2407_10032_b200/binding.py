@@ -36,7 +36,7 @@ class Config(C.Structure):
     @classmethod
     def make(cls, grid="nonuniform", bits=4, p=4.0, n_iter=20, group=0, T=2048, t=None, block=128, **_):
         if t is None:
-            t = int({4: 0.2, 3: 0.3, 2: 0.4}[bits] * T)
+            t = int({4: 0.2, 3: 0.3, 2: 0.4}.get(bits, 0.2) * T)
         gt = LQ_GRID_NONUNIFORM if grid == "nonuniform" else LQ_GRID_AFFINE
         return cls(bits, gt, float(p), n_iter, 0, group or 0, T, t, block, 0)
 

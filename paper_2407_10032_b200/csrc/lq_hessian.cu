@@ -56,11 +56,12 @@ extern "C" int lq_hessian_workspace(int32_t x_dtype, int64_t c, int64_t n_chunk,
 extern "C" int lq_hessian_accumulate(lq_handle* h, void* stream, const void* X, int32_t x_dtype, int32_t layout,
                                      int64_t c, int64_t n_chunk, int64_t ldx, float* H, int64_t ldh, float alpha,
                                      void* ws, size_t ws_bytes) {
-    if (!h || !X || !H || c <= 0 || n_chunk < 0 || ldx < n_chunk || ldh < c) return LQ_ERR_INVALID_ARG;
+    if (!h || !H || c <= 0 || n_chunk < 0 || ldh < c) return LQ_ERR_INVALID_ARG;
+    if (n_chunk == 0) return LQ_OK;                  // an empty chunk adds nothing
+    if (!X || ldx < n_chunk) return LQ_ERR_INVALID_ARG;
     if (layout != LQ_FEATURE_MAJOR) return LQ_ERR_UNSUPPORTED;
     if (x_dtype != LQ_BF16 && x_dtype != LQ_F32) return LQ_ERR_INVALID_ARG;
     if (ldh % 4 || (reinterpret_cast<uintptr_t>(H) & 15) || (reinterpret_cast<uintptr_t>(X) & 15)) return LQ_ERR_INVALID_ARG;
-    if (n_chunk == 0) return LQ_OK;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
     lq_tc_gemm_args g = {};
