@@ -37,7 +37,8 @@ typedef enum {
     LQ_ERR_NOT_POSITIVE_DEFINITE = 4,  /* device: pivot <= 0 in the factorisation; info = column */
     LQ_ERR_NONFINITE = 5,              /* device: NaN/Inf met; info = index */
     LQ_ERR_CUDA = 6,                   /* a CUDA runtime / driver call failed */
-    LQ_ERR_TIMEOUT = 7                 /* device: a bounded wait inside a kernel ran out */
+    LQ_ERR_TIMEOUT = 7,                /* device: a bounded wait inside a kernel ran out */
+    LQ_ERR_STATIC_SCRATCH_TOO_SMALL = 8 /* lq_fit_grid_noalloc: the problem needs more than the built-in scratch */
 } lq_status;
 
 typedef enum { LQ_F32 = 0, LQ_BF16 = 1 } lq_dtype;
@@ -119,6 +120,35 @@ int lq_fit_grid_workspace(const lq_config* cfg, int64_t r, int64_t c, size_t* by
 int lq_fit_grid(lq_handle* h, void* stream, const lq_config* cfg, const void* W,
                 int32_t w_dtype, int64_t r, int64_t c, int64_t ldw, const float* dinv,
                 float* grid, float* scale, int32_t* zero, void* ws, size_t ws_bytes);
+
+/* The paper has no counterpart for this entry point; it exists for callers that must not
+ * allocate device memory.  Examples: a process in which a framework's caching allocator or a
+ * serving engine has already reserved all of HBM, so that cudaMalloc fails or fragments its
+ * pool; a latency-critical section that cannot afford the device-wide synchronisation that
+ * cudaMalloc / cudaFree imply; a plug-in or callback context whose host forbids allocation.
+ * It computes exactly what lq_fit_grid computes (same kernels, same results) but takes no
+ * workspace: the scratch (the per-column sample weights and two scalars) lives in an array
+ * of 256 + 8 * LQ_FIT_GRID_NOALLOC_MAX_C bytes (128.25 KiB) that is part of the library image,
+ * so every GPU on which the library's kernels are loaded holds it until the process exits.
+ * The call itself calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - h may be NULL, so that not even lq_create (which allocates the 16-byte status word) is
+ *     needed; device-detected failures (a non-finite or non-positive dinv entry) are then
+ *     recorded in an internal word that no call reads.  With a handle they are reported by
+ *     lq_sync_status as usual.  The handle's device must be the current device.
+ *   - c > LQ_FIT_GRID_NOALLOC_MAX_C (or any future setting whose scratch need exceeds the
+ *     array) fails with LQ_ERR_STATIC_SCRATCH_TOO_SMALL before anything is launched.
+ *   - The first call on each device looks up the array's device address (one-time set-up,
+ *     guarded by a mutex) with that device current; make that first call before any stream
+ *     capture begins.  Later calls only launch kernels.
+ *   - All calls on one device share the one array.  It keeps whatever the previous call left
+ *     there; nothing has to be cleared because every word a call reads it has written first.
+ *     Two calls whose kernels may overlap on the GPU (different streams, no ordering between
+ *     them) race on it: order them on one stream or with events.
+ * All other arguments, layouts and results are those of lq_fit_grid. */
+#define LQ_FIT_GRID_NOALLOC_MAX_C 16384
+int lq_fit_grid_noalloc(lq_handle* h, void* stream, const lq_config* cfg, const void* W,
+                        int32_t w_dtype, int64_t r, int64_t c, int64_t ldw, const float* dinv,
+                        float* grid, float* scale, int32_t* zero);
 
 /* ---- stage 4: Algorithm 1 lines 10-21, the block-wise column loop -------------------- */
 

@@ -17,7 +17,8 @@ _lib = None
 LQ_F32, LQ_BF16 = 0, 1
 LQ_GRID_NONUNIFORM, LQ_GRID_AFFINE = 0, 1
 STATUS_NAMES = {0: "LQ_OK", 1: "LQ_ERR_INVALID_ARG", 2: "LQ_ERR_UNSUPPORTED", 3: "LQ_ERR_WORKSPACE_TOO_SMALL",
-                4: "LQ_ERR_NOT_POSITIVE_DEFINITE", 5: "LQ_ERR_NONFINITE", 6: "LQ_ERR_CUDA", 7: "LQ_ERR_TIMEOUT"}
+                4: "LQ_ERR_NOT_POSITIVE_DEFINITE", 5: "LQ_ERR_NONFINITE", 6: "LQ_ERR_CUDA", 7: "LQ_ERR_TIMEOUT",
+                8: "LQ_ERR_STATIC_SCRATCH_TOO_SMALL"}
 
 
 class LQError(RuntimeError):
@@ -65,6 +66,7 @@ def LQ():
             "lq_prepare_hinv": [vp, vp, vp, i64, i64, f32, vp, i64, vp, vp, i32, i64, i64, vp, sz],
             "lq_fit_grid_workspace": [P(Config), i64, i64, P(sz)],
             "lq_fit_grid": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, sz],
+            "lq_fit_grid_noalloc": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, vp, vp, vp],
             "lq_quantize_layer_workspace": [P(Config), i64, i64, P(sz)],
             "lq_quantize_layer": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, i64, vp, vp, vp, vp, vp, i32, i64,
                                   vp, vp, sz],
@@ -177,6 +179,14 @@ def lq_fit_grid(h, cfg, W, dinv, ws, grid=None, scale=None, zero=None, stream=No
     _check(LQ().lq_fit_grid(h, _stream(stream), C.byref(cfg), _ptr(W), _dt(W), r, c, _rowmajor(W), _ptr(dinv),
                             _ptr(grid), _ptr(scale), _ptr(zero), _ptr(ws), ws.numel() * ws.element_size()),
            "lq_fit_grid")
+
+
+def lq_fit_grid_noalloc(h, cfg, W, dinv, grid=None, scale=None, zero=None, stream=None):
+    """lq_fit_grid without a workspace: the scratch is an array built into the library, for callers
+    that must not allocate device memory.  `h` may be None."""
+    r, c = W.shape
+    _check(LQ().lq_fit_grid_noalloc(h, _stream(stream), C.byref(cfg), _ptr(W), _dt(W), r, c, _rowmajor(W), _ptr(dinv),
+                                    _ptr(grid), _ptr(scale), _ptr(zero)), "lq_fit_grid_noalloc")
 
 
 def lq_quantize_layer_workspace(cfg, r, c) -> int:

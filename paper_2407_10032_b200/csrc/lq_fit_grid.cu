@@ -11,6 +11,8 @@
 // arg-min (first minimum in t_min-major order).  Also fp64, for the same reason.
 #include <math.h>
 
+#include <mutex>
+
 #include "lq_common.cuh"
 
 namespace {
@@ -365,4 +367,72 @@ extern "C" int lq_fit_grid(lq_handle* h, void* stream, const lq_config* cfg, con
                                                                                n_groups, s64, K, cfg->T, cfg->t_count, scale, zero);
     LQ_LAUNCH_CHECK();
     return LQ_OK;
+}
+
+// ---------------------------------------------------- entry point without allocation --
+// Same computation as lq_fit_grid, with the scratch in an array that is part of the library
+// image instead of a caller workspace (for callers that must not allocate device memory).
+namespace {
+
+constexpr size_t kNoAllocScratchBytes = 256 + static_cast<size_t>(LQ_FIT_GRID_NOALLOC_MAX_C) * sizeof(double);
+static __device__ __align__(256) unsigned char lq_noalloc_scratch[kNoAllocScratchBytes];
+static __device__ __align__(256) lq_dev_status lq_noalloc_status;    // used when the caller has no handle
+
+// In host code the two names above are only stand-ins for the device arrays; their device
+// addresses are looked up once per device and kept here.
+constexpr int kMaxDevices = 64;
+struct NoAllocDevice {
+    bool ready = false;
+    void* scratch = nullptr;
+    lq_dev_status* status = nullptr;
+    int sm_count = 0;
+};
+NoAllocDevice g_noalloc[kMaxDevices];
+std::mutex g_noalloc_mutex;
+
+int noalloc_setup(int dev, NoAllocDevice& out) {
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    NoAllocDevice& d = g_noalloc[dev];
+    if (!d.ready) {
+        void* sp = nullptr;
+        void* tp = nullptr;
+        int sms = 0;
+        LQ_CUDA_TRY(cudaGetSymbolAddress(&sp, lq_noalloc_scratch));
+        LQ_CUDA_TRY(cudaGetSymbolAddress(&tp, lq_noalloc_status));
+        LQ_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        if (!sp || !tp || sms <= 0) return LQ_ERR_CUDA;
+        d.scratch = sp;
+        d.status = static_cast<lq_dev_status*>(tp);
+        d.sm_count = sms;
+        d.ready = true;
+    }
+    out = d;
+    return LQ_OK;
+}
+
+}  // namespace
+
+extern "C" int lq_fit_grid_noalloc(lq_handle* h, void* stream, const lq_config* cfg, const void* W, int32_t w_dtype,
+                                   int64_t r, int64_t c, int64_t ldw, const float* dinv, float* grid, float* scale,
+                                   int32_t* zero) {
+    int e = check_cfg(cfg);
+    if (e) return e;
+    if (r <= 0 || c <= 0) return LQ_ERR_INVALID_ARG;
+    size_t need = 0;
+    e = lq_fit_grid_workspace(cfg, r, c, &need);
+    if (e) return e;
+    if (c > LQ_FIT_GRID_NOALLOC_MAX_C || need > kNoAllocScratchBytes) return LQ_ERR_STATIC_SCRATCH_TOO_SMALL;
+    int dev = -1;
+    LQ_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return LQ_ERR_UNSUPPORTED;
+    if (h && h->device != dev) return LQ_ERR_INVALID_ARG;
+    NoAllocDevice d;
+    e = noalloc_setup(dev, d);
+    if (e) return e;
+    lq_handle local;
+    local.device = dev;
+    local.sm_count = d.sm_count;
+    local.dstatus = d.status;
+    return lq_fit_grid(h ? h : &local, stream, cfg, W, w_dtype, r, c, ldw, dinv, grid, scale, zero, d.scratch,
+                       kNoAllocScratchBytes);
 }
