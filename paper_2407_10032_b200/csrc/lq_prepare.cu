@@ -8,16 +8,25 @@
 // That is one factorisation plus one triangular inversion (2/3 c^3 flops) instead of
 // factor + invert + factor again.
 //
+// The two are run as ONE sweep over 128-wide block columns k = last .. 0.  R is inverted in
+// place by block Gauss-Jordan elimination with the pivots taken in the same descending order,
+// so that step k needs exactly what the factorisation has produced by then:
+//   diag   : A[k][k] (symmetric positive definite) -> V_k = R_kk^-1            (one CTA)
+//   panel  : P_i = A[i][k] V_k^T = R[i][k]  (i < k);   A[k][j] <- V_k A[k][j]  (j > k, final U)
+//   update : A[i][j] -= P_i P_j^T   (i <= j < k, the Cholesky trailing update)
+//            A[i][j] -= P_i A[k][j] (i < k < j, the Gauss-Jordan update)
+//            A[i][k]  = -P_i V_k    (i < k)
+// Every product has inner dimension 128 and all of a step's updates form one launch over the
+// whole width, so the grid stays large from the first step to the last.
+//
 // Everything is fp64 (fp32 factors of an ill-conditioned H move too many quantisation
-// decisions): a blocked right-looking factorisation with 128-wide panels, the diagonal
-// blocks handled by one CTA in shared memory, and all panel / trailing updates done by an
-// FP64 tensor-core GEMM (mma.sync m8n8k4 f64).
+// decisions); all products run on the FP64 tensor-core MMA (mma.sync m8n8k4 f64) fed by a
+// cp.async ring.
 #include "lq_common.cuh"
 
 namespace {
 
-constexpr int NB = 128;          // panel width
-constexpr int DP = NB + 1;       // shared-memory pitch of the diagonal block (bank-conflict free columns)
+constexpr int NB = 128;          // block width
 
 // ------------------------------------------------------------------ set-up kernels --
 // scal[0] = damp = damp_frac * mean(diag H), dead (zero) diagonal entries counted as 1.
@@ -70,109 +79,59 @@ __global__ void load_damped_kernel(const float* __restrict__ H, int64_t c, int64
     }
 }
 
-// --------------------------------------------------------- diagonal block kernel ----
-// In place on the NB x NB diagonal block at A + off: reads its upper triangle (a symmetric
-// positive definite block), computes the upper R with block = R R^T, inverts it, and writes
-// V = R^-1 (upper; zeros below the diagonal).  One CTA of 1024 threads.
-__global__ void __launch_bounds__(1024, 1)
-diag_block_kernel(double* __restrict__ A, int64_t cp, int64_t blk, int64_t c_real, lq_dev_status* st) {
-    extern __shared__ double S[];          // NB x DP
-    __shared__ double colbuf[2][NB];
-    __shared__ double vd[NB];
-    __shared__ double piv[2];              // sqrt of the current pivot and its reciprocal
-    double* base = A + blk * NB * cp + blk * NB;
-    const int tid = threadIdx.x;
-    const int tx = tid & 31, ty = tid >> 5;      // 32 x 32
-    for (int i = ty; i < NB; i += 32)
-        for (int j = tx; j < NB; j += 32) S[i * DP + j] = base[(int64_t)i * cp + j];
-    __syncthreads();
-
-    // Only one thread ever does the fp64 square root / division of a step.
-    auto set_pivot = [&](int j) {
-        double d = S[j * DP + j];
-        if (!(d > 0.0) || !isfinite(d)) {
-            if (blk * NB + j < c_real) lq_report(st, LQ_ERR_NOT_POSITIVE_DEFINITE, blk * NB + j);
-            d = 1.0;
-        }
-        const double rjj = sqrt(d);
-        piv[0] = rjj;
-        piv[1] = 1.0 / rjj;
-    };
-    if (tid == 0) set_pivot(NB - 1);
-    __syncthreads();
-
-    // R R^T factorisation, last column first.
-    for (int j = NB - 1; j >= 0; --j) {
-        const double rjj = piv[0], rinv = piv[1];
-        if (tid < j) {
-            const double v = S[tid * DP + j] * rinv;
-            colbuf[0][tid] = v;
-            S[tid * DP + j] = v;
-        } else if (tid == j) {
-            S[j * DP + j] = rjj;
-        }
-        __syncthreads();
-        for (int i = ty; i < j; i += 32) {
-            const double ci = colbuf[0][i];
-            for (int k = tx; k < j; k += 32)
-                if (k >= i) S[i * DP + k] -= ci * colbuf[0][k];
-        }
-        // the thread that just finished the next pivot entry prepares its square root
-        if (j > 0 && ty == ((j - 1) & 31) && tx == ((j - 1) & 31)) set_pivot(j - 1);
-        __syncthreads();
-    }
-
-    // In-place inversion of the upper-triangular R, one column at a time:
-    // V[j][j] = 1/R[j][j]; V[i][j] = -V[j][j] * sum_{k=i}^{j-1} V[i][k] R[k][j]  (i < j).
-    if (tid < NB) vd[tid] = 1.0 / S[tid * DP + tid];
-    for (int j = 0; j < NB; ++j) {
-        double* cb = colbuf[j & 1];
-        if (tid < j) cb[tid] = S[tid * DP + j];
-        __syncthreads();                   // column j staged; column j-1 of V complete
-        const int i = tid >> 3, part = tid & 7;      // 8 threads per row
-        double acc = 0.0;
-        if (i < j)
-            for (int k = i + part; k < j; k += 8) acc += S[i * DP + k] * cb[k];
-        acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-        acc += __shfl_xor_sync(0xffffffffu, acc, 2);
-        acc += __shfl_xor_sync(0xffffffffu, acc, 4);
-        if (part == 0) {
-            if (i < j) S[i * DP + j] = -vd[j] * acc;
-            else if (i == j) S[j * DP + j] = vd[j];
-        }
-    }
-    __syncthreads();
-
-    for (int i = ty; i < NB; i += 32)
-        for (int j = tx; j < NB; j += 32) base[(int64_t)i * cp + j] = (j >= i) ? S[i * DP + j] : 0.0;
-}
-
-// -------------------------------------------------------------- FP64 MMA GEMM -------
-// C[M x N] = alpha * A[M x K] * op(B) + beta * C, all fp64 row-major, M and N multiples of
-// 64, K a multiple of 16.  TRANS_B: B is N x K (C = A B^T); otherwise B is K x N.
-// a_tri: A is block upper triangular (entries left of the 64-aligned row start are zero and
-// are skipped).  c_upper: tiles strictly below the diagonal are skipped.
+// ------------------------------------------------------------------ FP64 MMA -------
 __device__ __forceinline__ void dmma(double& c0, double& c1, double a, double b) {
     asm volatile("mma.sync.aligned.m8n8k4.row.col.f64.f64.f64.f64 {%0, %1}, {%2}, {%3}, {%0, %1};"
                  : "+d"(c0), "+d"(c1) : "d"(a), "d"(b));
 }
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
+    const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
 
-constexpr int GT = 64;    // tile
-constexpr int GK = 16;
-constexpr int GKP = 20;   // padded k pitch: conflict-free fragment loads
+// ---------------------------------------------------- 128 x 64 tile product, K = 128 --
+// C[128 x 64] = beta * C + alpha * A[128 x 128] * B[128 x 64], all fp64 row-major.
+// 256 threads = 8 warps in a 4 x 2 arrangement, each owning a 32 x 32 patch as 4 x 4 MMA tiles.
+// K is streamed 16 at a time through a 3-stage cp.async ring; the shared-memory pitches make
+// every fragment load conflict-free.  The output may alias B (all of B has been read before
+// the first store).  Optional extra outputs: a plain copy (C2) and a transposed copy (Ct).
+constexpr int TM = 128, TN = 64, TK = 16, NST = 3;
+constexpr int AP = 20;                       // pitch (doubles) of an A chunk row: 16 + 4
+constexpr int BP = 68;                       // pitch of a B chunk row: 64 + 4
+constexpr int STAGE_DOUBLES = TM * AP + TK * BP;
+constexpr int GEMM_SMEM = NST * STAGE_DOUBLES * 8;
+constexpr int GEMM_THREADS = 256;
 
-template <bool TRANS_B>
-__global__ void __launch_bounds__(128)
-dgemm_kernel(const double* __restrict__ A, int64_t lda, const double* __restrict__ B, int64_t ldb,
-             double* __restrict__ C, int64_t ldc, int M, int N, int K, double alpha, double beta,
-             int a_tri, int c_upper) {
-    const int bi = blockIdx.y, bj = blockIdx.x;
-    if (c_upper && bj < bi) return;
-    __shared__ double As[GT * GKP];
-    __shared__ double Bs[GT * GKP];
+struct TileOut {
+    double* C;  int64_t ldc;
+    double* C2; int64_t ldc2;     // optional copy of the result
+    double* Ct; int64_t ldct;     // optional transposed copy: Ct[col * ldct + row]
+};
+
+__device__ __forceinline__ void gemm_tile(const double* __restrict__ A, int64_t lda, const double* B, int64_t ldb,
+                                          double alpha, double beta, const TileOut& o, double* smem) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int wm0 = (warp >> 1) * 32, wn0 = (warp & 1) * 32;
-    const int m0 = bi * GT, n0 = bj * GT;
+    const int wm = warp >> 1, wn = warp & 1;
+    const int fr = lane >> 2, fk = lane & 3;
+
+    auto issue = [&](int kc) {
+        double* as = smem + (kc % NST) * STAGE_DOUBLES;
+        double* bs = as + TM * AP;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int idx = tid + GEMM_THREADS * u, row = idx >> 3, seg = idx & 7;
+            cp_async16(as + row * AP + seg * 2, A + (int64_t)row * lda + kc * TK + seg * 2);
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int idx = tid + GEMM_THREADS * u, row = idx >> 5, seg = idx & 31;
+            cp_async16(bs + row * BP + seg * 2, B + (int64_t)(kc * TK + row) * ldb + seg * 2);
+        }
+    };
 
     double acc[4][4][2];
 #pragma unroll
@@ -180,126 +139,342 @@ dgemm_kernel(const double* __restrict__ A, int64_t lda, const double* __restrict
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
 
-    // global -> register staging
-    const int a_row = tid >> 1, a_k = (tid & 1) * 8;
-    const int bt_k = tid >> 3, bt_n = (tid & 7) * 8;     // non-transposed B: 16 x 64 tile
-    double ra[8], rb[8];
-    const int k_begin = a_tri ? m0 : 0;
-
-    auto load_tile = [&](int k0) {
-        const double* ap = A + (int64_t)(m0 + a_row) * lda + k0 + a_k;
-#pragma unroll
-        for (int u = 0; u < 8; u += 2) {
-            double2 v = *reinterpret_cast<const double2*>(ap + u);
-            ra[u] = v.x; ra[u + 1] = v.y;
-        }
-        if (TRANS_B) {
-            const double* bp = B + (int64_t)(n0 + a_row) * ldb + k0 + a_k;
-#pragma unroll
-            for (int u = 0; u < 8; u += 2) {
-                double2 v = *reinterpret_cast<const double2*>(bp + u);
-                rb[u] = v.x; rb[u + 1] = v.y;
-            }
-        } else {
-            const double* bp = B + (int64_t)(k0 + bt_k) * ldb + n0 + bt_n;
-#pragma unroll
-            for (int u = 0; u < 8; u += 2) {
-                double2 v = *reinterpret_cast<const double2*>(bp + u);
-                rb[u] = v.x; rb[u + 1] = v.y;
-            }
-        }
-    };
-    auto store_tile = [&]() {
-#pragma unroll
-        for (int u = 0; u < 8; ++u) As[a_row * GKP + a_k + u] = ra[u];
-        if (TRANS_B) {
-#pragma unroll
-            for (int u = 0; u < 8; ++u) Bs[a_row * GKP + a_k + u] = rb[u];
-        } else {
-#pragma unroll
-            for (int u = 0; u < 8; ++u) Bs[(bt_n + u) * GKP + bt_k] = rb[u];
-        }
-    };
-
-    if (k_begin < K) load_tile(k_begin);
-    for (int k0 = k_begin; k0 < K; k0 += GK) {
+    constexpr int NCHUNK = NB / TK;
+    issue(0); cp_async_commit();
+    issue(1); cp_async_commit();
+#pragma unroll 1
+    for (int kc = 0; kc < NCHUNK; ++kc) {
+        cp_async_wait<NST - 2>();
         __syncthreads();
-        store_tile();
-        __syncthreads();
-        if (k0 + GK < K) load_tile(k0 + GK);
-        const int fr = lane >> 2, fk = lane & 3;
+        if (kc + NST - 1 < NCHUNK) issue(kc + NST - 1);
+        cp_async_commit();
+        const double* as = smem + (kc % NST) * STAGE_DOUBLES + (wm * 32 + fr) * AP + fk;
+        const double* bs = smem + (kc % NST) * STAGE_DOUBLES + TM * AP + fk * BP + wn * 32 + fr;
 #pragma unroll
-        for (int kk = 0; kk < GK; kk += 4) {
+        for (int kk = 0; kk < TK / 4; ++kk) {
             double a[4], b[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) a[i] = As[(wm0 + 8 * i + fr) * GKP + kk + fk];
+            for (int i = 0; i < 4; ++i) a[i] = as[8 * i * AP + kk * 4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) b[j] = Bs[(wn0 + 8 * j + fr) * GKP + kk + fk];
+            for (int j = 0; j < 4; ++j) b[j] = bs[kk * 4 * BP + 8 * j];
 #pragma unroll
             for (int i = 0; i < 4; ++i)
 #pragma unroll
                 for (int j = 0; j < 4; ++j) dmma(acc[i][j][0], acc[i][j][1], a[i], b[j]);
         }
     }
+    cp_async_wait<0>();
+    __syncthreads();      // every thread's copies have landed: B may now be overwritten
 
-    const int cr = lane >> 2, cc = (lane & 3) * 2;
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < 4; ++i) {
+        const int row = wm * 32 + 8 * i + fr;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            double* cp = C + (int64_t)(m0 + wm0 + 8 * i + cr) * ldc + n0 + wn0 + 8 * j + cc;
-            double2 o;
+            const int col = wn * 32 + 8 * j + 2 * fk;
+            double2 v;
+            v.x = alpha * acc[i][j][0];
+            v.y = alpha * acc[i][j][1];
+            double* cp = o.C + (int64_t)row * o.ldc + col;
             if (beta != 0.0) {
-                double2 old = *reinterpret_cast<double2*>(cp);
-                o.x = alpha * acc[i][j][0] + beta * old.x;
-                o.y = alpha * acc[i][j][1] + beta * old.y;
-            } else {
-                o.x = alpha * acc[i][j][0];
-                o.y = alpha * acc[i][j][1];
+                const double2 old = *reinterpret_cast<const double2*>(cp);
+                v.x += beta * old.x;
+                v.y += beta * old.y;
             }
-            *reinterpret_cast<double2*>(cp) = o;
+            *reinterpret_cast<double2*>(cp) = v;
+            if (o.C2) *reinterpret_cast<double2*>(o.C2 + (int64_t)row * o.ldc2 + col) = v;
+            if (o.Ct) {
+                o.Ct[(int64_t)col * o.ldct + row] = v.x;
+                o.Ct[(int64_t)(col + 1) * o.ldct + row] = v.y;
+            }
         }
-}
-
-void dgemm(cudaStream_t st, bool trans_b, const double* A, int64_t lda, const double* B, int64_t ldb, double* C,
-           int64_t ldc, int64_t M, int64_t N, int64_t K, double alpha, double beta, int a_tri, int c_upper) {
-    if (M <= 0 || N <= 0) return;
-    dim3 grid(static_cast<unsigned>(N / GT), static_cast<unsigned>(M / GT));
-    if (trans_b)
-        dgemm_kernel<true><<<grid, 128, 0, st>>>(A, lda, B, ldb, C, ldc, (int)M, (int)N, (int)K, alpha, beta, a_tri, c_upper);
-    else
-        dgemm_kernel<false><<<grid, 128, 0, st>>>(A, lda, B, ldb, C, ldc, (int)M, (int)N, (int)K, alpha, beta, a_tri, c_upper);
-}
-
-// copy rows x NB doubles from P (pitch NB) into A's panel (pitch cp)
-__global__ void copy_panel_kernel(const double* __restrict__ P, double* __restrict__ dst, int64_t rows, int64_t cp) {
-    const int64_t i = blockIdx.x;
-    for (int j = threadIdx.x; j < NB; j += blockDim.x) dst[i * cp + j] = P[i * NB + j];
-}
-
-// U (fp32, c x c, upper, zeros below) and dinv[j] = sum_k U64[k][j]^2.
-__global__ void finalize_u_kernel(const double* __restrict__ A, int64_t cp, int64_t c, float* __restrict__ U, int64_t ldu) {
-    const int64_t i = blockIdx.y;
-    for (int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < c; j += (int64_t)gridDim.x * blockDim.x)
-        U[i * ldu + j] = (j >= i) ? static_cast<float>(A[i * cp + j]) : 0.0f;
-}
-__global__ void dinv_kernel(const double* __restrict__ A, int64_t cp, int64_t c, float* __restrict__ dinv) {
-    const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (j >= c) return;
-    double s = 0.0;
-    for (int64_t k = 0; k <= j; ++k) {
-        double u = A[k * cp + j];
-        s += u * u;
     }
-    dinv[j] = static_cast<float>(s);
+}
+
+// Step k, panel: blocks [0, 2k) compute P_i = A[i][k] V_k^T (to Pbuf, and transposed into Q's
+// columns of block i); blocks [2k, 2(nblk-1)) scale row k: A[k][j] <- V_k A[k][j] for j > k
+// (in place: these are final entries of U) with a copy in Q's columns of block j.
+// Q is 128 x cp: the right-hand operand of the step's update for every block column.
+__global__ void __launch_bounds__(GEMM_THREADS, 2)
+panel_kernel(double* __restrict__ A, int64_t cp, int k, const double* __restrict__ VT, double* __restrict__ Pbuf,
+             double* __restrict__ Q) {
+    extern __shared__ double smem[];
+    const int t = blockIdx.x >> 1, h = blockIdx.x & 1;
+    TileOut o = {};
+    if (t < k) {
+        const int i = t;
+        o.C = Pbuf + (int64_t)i * NB * NB + h * TN; o.ldc = NB;
+        o.Ct = Q + (int64_t)(h * TN) * cp + (int64_t)i * NB; o.ldct = cp;
+        gemm_tile(A + (int64_t)i * NB * cp + (int64_t)k * NB, cp, VT + h * TN, NB, 1.0, 0.0, o, smem);
+    } else {
+        const int j = t + 1;
+        double* row = A + (int64_t)k * NB * cp + (int64_t)j * NB + h * TN;
+        o.C = row; o.ldc = cp;
+        o.C2 = Q + (int64_t)j * NB + h * TN; o.ldc2 = cp;
+        gemm_tile(A + (int64_t)k * NB * cp + (int64_t)k * NB, cp, row, cp, 1.0, 0.0, o, smem);
+    }
+}
+
+// Step k, update of block rows i < k over the whole width (grid: 2 * nblk x k).
+__global__ void __launch_bounds__(GEMM_THREADS, 2)
+update_kernel(double* __restrict__ A, int64_t cp, int k, const double* __restrict__ Pbuf, const double* __restrict__ Q) {
+    extern __shared__ double smem[];
+    const int j = blockIdx.x >> 1, h = blockIdx.x & 1, i = blockIdx.y;
+    if (j < i) return;                                  // strictly lower tiles of the symmetric part
+    const double* Pi = Pbuf + (int64_t)i * NB * NB;
+    TileOut o = {};
+    o.C = A + (int64_t)i * NB * cp + (int64_t)j * NB + h * TN; o.ldc = cp;
+    if (j == k)     // A[i][k] = -P_i V_k
+        gemm_tile(Pi, NB, A + (int64_t)k * NB * cp + (int64_t)k * NB + h * TN, cp, -1.0, 0.0, o, smem);
+    else            // A[i][j] -= P_i Q[:, j]
+        gemm_tile(Pi, NB, Q + (int64_t)j * NB + h * TN, cp, -1.0, 1.0, o, smem);
+}
+
+// --------------------------------------------------------- diagonal block kernel ----
+// In place on the 128 x 128 diagonal block k of A: reads its upper triangle (symmetric positive
+// definite), computes the upper R with block = R R^T and writes V = R^-1 (upper, zeros below)
+// back, plus V^T to VT.  One CTA of 256 threads.  The block is handled as 4 x 4 sub-blocks of
+// 32 with the same sweep as the outer algorithm: warp 0 factorises and inverts a 32 x 32
+// diagonal sub-block in registers (one row per lane), then all warps do the panel, update and
+// scaling products with the FP64 MMA out of shared memory.
+constexpr int SB = 32;
+constexpr int DP = 132;          // pitch of the block in shared memory (conflict-free fragments)
+constexpr int PP = 36;           // pitch of the panel buffer
+constexpr int DIAG_THREADS = 256;
+constexpr int DIAG_SMEM = (NB * DP + (NB - SB) * PP + 2 * SB + SB) * 8;
+
+// 32 x 32 sub-block at S (pitch DP): upper triangle in, V = R^-1 out (upper, zeros below).
+__device__ __forceinline__ void warp_factor_invert(double* S, double* colbuf, double* rinvb, int lane,
+                                                   long long col_global, long long c_real, lq_dev_status* st) {
+    double a[SB];
+#pragma unroll
+    for (int t = 0; t < SB; ++t) a[t] = (t >= lane) ? S[lane * DP + t] : 0.0;
+    // R R^T factorisation, last column first; lane i holds row i.
+#pragma unroll
+    for (int j = SB - 1; j >= 0; --j) {
+        double d = __shfl_sync(0xffffffffu, a[j], j);
+        if (!(d > 0.0) || !isfinite(d)) {
+            if (lane == 0 && col_global + j < c_real) lq_report(st, LQ_ERR_NOT_POSITIVE_DEFINITE, col_global + j);
+            d = 1.0;
+        }
+        const double rinv = rsqrt(d);
+        const double l = (lane < j) ? a[j] * rinv : ((lane == j) ? d * rinv : 0.0);   // R[i][j]; sqrt(d) on the diagonal
+        a[j] = l;
+        if (lane == j) rinvb[j] = rinv;
+        double* cb = colbuf + (j & 1) * SB;
+        cb[lane] = (lane < j) ? l : 0.0;
+        __syncwarp();
+#pragma unroll
+        for (int t = 0; t < j; ++t) a[t] -= l * cb[t];            // meaningful for lane <= t
+    }
+    // R to shared memory (rows), then V = R^-1 row by row: V[i][j] = (delta_ij - sum_{t<j} V[i][t] R[t][j]) / R[j][j]
+#pragma unroll
+    for (int t = 0; t < SB; ++t) S[lane * DP + t] = (t >= lane) ? a[t] : 0.0;
+    __syncwarp();
+    double v[SB];
+#pragma unroll
+    for (int j = 0; j < SB; ++j) {
+        double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+#pragma unroll
+        for (int t = 0; t < j; ++t) {
+            const double rt = S[t * DP + j];
+            if ((t & 3) == 0) s0 = fma(v[t], rt, s0);
+            else if ((t & 3) == 1) s1 = fma(v[t], rt, s1);
+            else if ((t & 3) == 2) s2 = fma(v[t], rt, s2);
+            else s3 = fma(v[t], rt, s3);
+        }
+        const double rhs = ((lane == j) ? 1.0 : 0.0) - ((s0 + s1) + (s2 + s3));
+        v[j] = (lane <= j) ? rhs * rinvb[j] : 0.0;
+    }
+    __syncwarp();
+#pragma unroll
+    for (int t = 0; t < SB; ++t) S[lane * DP + t] = v[t];
+}
+
+// 16 x 16 output patch, K = 32, out of shared memory.  a(r, t): left operand, row r of the patch;
+// B is given either as rows of K (NT: Bt[n * ldb + t]) or as K rows (NN: Bn[t * ldb + n]).
+template <bool NT>
+__device__ __forceinline__ void patch16(const double* Ap, int lda, const double* Bp, int ldb, int lane, double (&acc)[2][2][2]) {
+    const int fr = lane >> 2, fk = lane & 3;
+#pragma unroll
+    for (int i = 0; i < 2; ++i)
+#pragma unroll
+        for (int j = 0; j < 2; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
+#pragma unroll
+    for (int kk = 0; kk < SB / 4; ++kk) {
+        double a[2], b[2];
+#pragma unroll
+        for (int i = 0; i < 2; ++i) a[i] = Ap[(8 * i + fr) * lda + kk * 4 + fk];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) b[j] = NT ? Bp[(8 * j + fr) * ldb + kk * 4 + fk] : Bp[(kk * 4 + fk) * ldb + 8 * j + fr];
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int j = 0; j < 2; ++j) dmma(acc[i][j][0], acc[i][j][1], a[i], b[j]);
+    }
+}
+
+__global__ void __launch_bounds__(DIAG_THREADS, 1)
+diag_block_kernel(double* __restrict__ A, int64_t cp, int64_t blk, int64_t c_real, double* __restrict__ VT,
+                  lq_dev_status* st) {
+    extern __shared__ double sm[];
+    double* S = sm;                       // NB x DP
+    double* Pb = S + NB * DP;             // (NB - SB) x PP
+    double* colbuf = Pb + (NB - SB) * PP; // 2 x SB
+    double* rinvb = colbuf + 2 * SB;      // SB
+    double* base = A + blk * NB * cp + blk * NB;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int fr = lane >> 2, fk = lane & 3;
+    constexpr int NW = DIAG_THREADS / 32;
+
+    for (int idx = tid; idx < NB * (NB / 2); idx += DIAG_THREADS) {
+        const int row = idx >> 6, c2 = (idx & 63) * 2;
+        const double2 v = *reinterpret_cast<const double2*>(base + (int64_t)row * cp + c2);
+        S[row * DP + c2] = v.x;
+        S[row * DP + c2 + 1] = v.y;
+    }
+    __syncthreads();
+
+#pragma unroll 1
+    for (int kb = NB / SB - 1; kb >= 0; --kb) {
+        const int c0 = kb * SB;
+        const int right = NB - c0 - SB;               // columns to the right of this sub-block
+        double* D = S + c0 * DP + c0;                 // diagonal sub-block
+        if (warp == 0) warp_factor_invert(D, colbuf, rinvb, lane, blk * NB + c0, c_real, st);
+        __syncthreads();
+        // panel: Pb[m][q] = sum_t S[m][c0 + t] V[q][t]   (m < c0); row scaling: S[c0 + q][j] <- sum_t V[q][t] S[c0 + t][j]  (j > c0 + 32)
+        {
+            const int nP = (c0 / 16) * 2;
+            const int nR = right / 8;
+            for (int item = warp; item < nP + nR; item += NW) {
+                if (item < nP) {
+                    const int m0 = (item >> 1) * 16, q0 = (item & 1) * 16;
+                    double acc[2][2][2];
+                    patch16<true>(S + m0 * DP + c0, DP, D + q0 * DP, DP, lane, acc);
+#pragma unroll
+                    for (int i = 0; i < 2; ++i)
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            double* p = Pb + (m0 + 8 * i + fr) * PP + q0 + 8 * j + 2 * fk;
+                            p[0] = acc[i][j][0];
+                            p[1] = acc[i][j][1];
+                        }
+                } else {
+                    // one warp owns an 8-column strip over all 32 rows, so the in-place update is safe
+                    const int j0 = c0 + SB + (item - nP) * 8;
+                    double acc[4][2];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[i][0] = acc[i][1] = 0.0;
+#pragma unroll
+                    for (int kk = 0; kk < SB / 4; ++kk) {
+                        const double b = S[(c0 + kk * 4 + fk) * DP + j0 + fr];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) dmma(acc[i][0], acc[i][1], D[(8 * i + fr) * DP + kk * 4 + fk], b);
+                    }
+                    __syncwarp();
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        double* p = S + (c0 + 8 * i + fr) * DP + j0 + 2 * fk;
+                        p[0] = acc[i][0];
+                        p[1] = acc[i][1];
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        // update of the rows above: 16 x 16 patches over the whole width
+        {
+            const int nRow = c0 / 16;
+            for (int item = warp; item < nRow * 8; item += NW) {
+                const int rg = item >> 3, cg = item & 7;
+                const int m0 = rg * 16, n0 = cg * 16;
+                double acc[2][2][2];
+                double sign_old;
+                if (n0 < c0) {
+                    if (cg < rg) continue;                                   // symmetric part: upper patches only
+                    patch16<true>(Pb + m0 * PP, PP, Pb + n0 * PP, PP, lane, acc);          // P_m P_n^T
+                    sign_old = 1.0;
+                } else if (n0 < c0 + SB) {
+                    patch16<false>(Pb + m0 * PP, PP, D + (n0 - c0), DP, lane, acc);        // P_m V
+                    sign_old = 0.0;
+                } else {
+                    patch16<false>(Pb + m0 * PP, PP, S + c0 * DP + n0, DP, lane, acc);     // P_m (scaled row)
+                    sign_old = 1.0;
+                }
+#pragma unroll
+                for (int i = 0; i < 2; ++i)
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        double* p = S + (m0 + 8 * i + fr) * DP + n0 + 8 * j + 2 * fk;
+                        p[0] = sign_old * p[0] - acc[i][j][0];
+                        p[1] = sign_old * p[1] - acc[i][j][1];
+                    }
+            }
+        }
+        __syncthreads();
+    }
+
+    for (int idx = tid; idx < NB * NB; idx += DIAG_THREADS) {
+        const int row = idx >> 7, col = idx & 127;
+        base[(int64_t)row * cp + col] = (col >= row) ? S[row * DP + col] : 0.0;
+    }
+    for (int idx = tid; idx < NB * NB; idx += DIAG_THREADS) {
+        const int col = idx >> 7, row = idx & 127;                           // VT[col][row] = V[row][col]
+        VT[col * NB + row] = (col >= row) ? S[row * DP + col] : 0.0;
+    }
+}
+
+// U (fp32, c x c, upper, zeros below) and dinv[j] = sum_k U64[k][j]^2: one CTA per 32 columns.
+__global__ void __launch_bounds__(256)
+finalize_kernel(const double* __restrict__ A, int64_t cp, int64_t c, float* __restrict__ U, int64_t ldu,
+                float* __restrict__ dinv) {
+    __shared__ double red[8][33];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int64_t j = (int64_t)blockIdx.x * 32 + tx;
+    double s = 0.0;
+    if (j < c) {
+        for (int64_t i = ty; i < c; i += 8) {
+            double u = 0.0;
+            if (i <= j) {
+                u = A[i * cp + j];
+                s = fma(u, u, s);
+            }
+            U[i * ldu + j] = static_cast<float>(u);
+        }
+    }
+    red[ty][tx] = s;
+    __syncthreads();
+    if (ty == 0 && j < c) {
+        double t = 0.0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) t += red[w][tx];
+        dinv[j] = static_cast<float>(t);
+    }
+}
+
+struct PrepLayout {
+    int64_t nblk, cp;
+    size_t scal, a, pbuf, q, vt, total;
+};
+PrepLayout prep_layout(int64_t c) {
+    PrepLayout L;
+    L.nblk = lq_ceil_div(c, NB);
+    L.cp = L.nblk * NB;
+    size_t off = 0;
+    L.scal = off; off += 256;
+    L.a = off;    off += lq_align_up(static_cast<size_t>(L.cp) * L.cp * sizeof(double), 256);
+    L.pbuf = off; off += lq_align_up(static_cast<size_t>(L.cp) * NB * sizeof(double), 256);
+    L.q = off;    off += lq_align_up(static_cast<size_t>(L.cp) * NB * sizeof(double), 256);
+    L.vt = off;   off += lq_align_up(static_cast<size_t>(NB) * NB * sizeof(double), 256);
+    L.total = off;
+    return L;
 }
 
 }  // namespace
 
 extern "C" int lq_prepare_hinv_workspace(int64_t c, size_t* bytes) {
     if (!bytes || c <= 0) return LQ_ERR_INVALID_ARG;
-    const size_t cp = static_cast<size_t>(lq_ceil_div(c, NB)) * NB;
-    *bytes = 256 + lq_align_up(cp * cp * sizeof(double), 256) + lq_align_up(cp * NB * sizeof(double), 256);
+    *bytes = prep_layout(c).total;
     return LQ_OK;
 }
 
@@ -308,23 +483,25 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
                                void* ws, size_t ws_bytes) {
     if (!h || !H || !U || !dinv || c <= 0 || ldh < c || ldu < c || !(damp_frac >= 0.0f)) return LQ_ERR_INVALID_ARG;
     if (W && (r <= 0 || ldw < c || (w_dtype != LQ_F32 && w_dtype != LQ_BF16))) return LQ_ERR_INVALID_ARG;
-    size_t need = 0;
-    lq_prepare_hinv_workspace(c, &need);
-    if (!ws || ws_bytes < need) return LQ_ERR_WORKSPACE_TOO_SMALL;
+    const PrepLayout L = prep_layout(c);
+    if (!ws || ws_bytes < L.total) return LQ_ERR_WORKSPACE_TOO_SMALL;
     if (reinterpret_cast<uintptr_t>(ws) & 255) return LQ_ERR_INVALID_ARG;
+    if (L.nblk > 32767) return LQ_ERR_UNSUPPORTED;            // grid.y of the update launch
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-    const int64_t nblk = lq_ceil_div(c, NB);
-    const int64_t cp = nblk * NB;
+    const int64_t nblk = L.nblk, cp = L.cp;
     char* wsp = static_cast<char*>(ws);
-    double* scal = reinterpret_cast<double*>(wsp);
-    double* A = reinterpret_cast<double*>(wsp + 256);
-    double* P = reinterpret_cast<double*>(wsp + 256 + lq_align_up(static_cast<size_t>(cp) * cp * sizeof(double), 256));
+    double* scal = reinterpret_cast<double*>(wsp + L.scal);
+    double* A = reinterpret_cast<double*>(wsp + L.a);
+    double* Pbuf = reinterpret_cast<double*>(wsp + L.pbuf);
+    double* Q = reinterpret_cast<double*>(wsp + L.q);
+    double* VT = reinterpret_cast<double*>(wsp + L.vt);
 
     static bool attr_set = false;
-    const int diag_smem = NB * DP * sizeof(double);
     if (!attr_set) {
-        LQ_CUDA_TRY(cudaFuncSetAttribute(diag_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, diag_smem));
+        LQ_CUDA_TRY(cudaFuncSetAttribute(diag_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DIAG_SMEM));
+        LQ_CUDA_TRY(cudaFuncSetAttribute(panel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
+        LQ_CUDA_TRY(cudaFuncSetAttribute(update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
         attr_set = true;
     }
 
@@ -344,41 +521,21 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
         LQ_LAUNCH_CHECK();
     }
 
-    // Phase A: A = R R^T, R upper, last block column first.  Afterwards the off-diagonal
-    // blocks of A hold R and every diagonal block holds the inverse of its R block.
     for (int64_t k = nblk - 1; k >= 0; --k) {
-        diag_block_kernel<<<1, 1024, diag_smem, st>>>(A, cp, k, c, h->dstatus);
+        diag_block_kernel<<<1, DIAG_THREADS, DIAG_SMEM, st>>>(A, cp, k, c, VT, h->dstatus);
         LQ_LAUNCH_CHECK();
-        if (k == 0) break;
-        const int64_t rows = k * NB;
-        double* panel = A + k * NB;                         // rows 0..rows-1, columns of block k
-        const double* Vkk = A + k * NB * cp + k * NB;
-        // R[0:k, k] = A[0:k, k] * Vkk^T
-        dgemm(st, true, panel, cp, Vkk, cp, P, NB, rows, NB, NB, 1.0, 0.0, 0, 0);
-        LQ_LAUNCH_CHECK();
-        copy_panel_kernel<<<static_cast<unsigned>(rows), 128, 0, st>>>(P, panel, rows, cp);
-        LQ_LAUNCH_CHECK();
-        // A[0:k, 0:k] -= R[0:k, k] R[0:k, k]^T   (upper tiles only)
-        dgemm(st, true, P, NB, P, NB, A, cp, rows, rows, NB, -1.0, 1.0, 0, 1);
-        LQ_LAUNCH_CHECK();
+        if (nblk > 1) {
+            panel_kernel<<<static_cast<unsigned>(2 * (nblk - 1)), GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, static_cast<int>(k), VT,
+                                                                                                Pbuf, Q);
+            LQ_LAUNCH_CHECK();
+        }
+        if (k > 0) {
+            dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(k));
+            update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, static_cast<int>(k), Pbuf, Q);
+            LQ_LAUNCH_CHECK();
+        }
     }
-    // Phase B: U = R^-1 block column by block column:
-    // U[0:k, k] = -(U[0:k, 0:k] * R[0:k, k]) * Vkk,  U[k, k] = Vkk.
-    for (int64_t k = 1; k < nblk; ++k) {
-        const int64_t rows = k * NB;
-        double* panel = A + k * NB;
-        const double* Vkk = A + k * NB * cp + k * NB;
-        dgemm(st, false, A, cp, panel, cp, P, NB, rows, NB, rows, 1.0, 0.0, 1, 0);
-        LQ_LAUNCH_CHECK();
-        dgemm(st, false, P, NB, Vkk, cp, panel, cp, rows, NB, NB, -1.0, 0.0, 0, 0);
-        LQ_LAUNCH_CHECK();
-    }
-    {
-        dim3 g(static_cast<unsigned>(lq_ceil_div(c, 256) < 32 ? lq_ceil_div(c, 256) : 32), static_cast<unsigned>(c));
-        finalize_u_kernel<<<g, 256, 0, st>>>(A, cp, c, U, ldu);
-        LQ_LAUNCH_CHECK();
-        dinv_kernel<<<static_cast<unsigned>(lq_ceil_div(c, 128)), 128, 0, st>>>(A, cp, c, dinv);
-        LQ_LAUNCH_CHECK();
-    }
+    finalize_kernel<<<static_cast<unsigned>(lq_ceil_div(c, 32)), 256, 0, st>>>(A, cp, c, U, ldu, dinv);
+    LQ_LAUNCH_CHECK();
     return LQ_OK;
 }
