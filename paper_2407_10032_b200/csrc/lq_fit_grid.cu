@@ -1,10 +1,11 @@
 // Stage 3 -- the loss-error-aware grid (Section 3.2, Algorithm 1 lines 5-9).
 //
-// Non-uniform (Eq. 5): one weighted 1-D k-means per output row.  One CTA per row, the row
-// staged once (registers for short rows, shared memory for long ones), the sample weights
-// s_j = dinv_j^(-p) / geometric mean shared by all rows.  Assignment compares and the
-// per-cluster sums run in fp64: a weight that sits next to a midpoint must fall on the same
-// side as in a float64 evaluation, or the centroids drift apart by far more than rounding.
+// Non-uniform (Eq. 5): one weighted 1-D k-means per output row, one CTA per row, the sample
+// weights s_j = dinv_j^(-p) / geometric mean shared by all rows.  The row is sorted once in
+// shared memory; Lloyd iterations then work on boundaries and prefix sums (see below).
+// Centroids, midpoints and cluster sums are fp64: a weight that sits next to a midpoint must
+// fall on the same side as in a float64 evaluation, or the centroids drift apart by far more
+// than rounding.
 //
 // Affine (Eq. 7): one CTA per (row, group); every thread evaluates whole candidates
 // (t_min, t_max) over the group's weights held in shared memory, then the CTA takes the
@@ -51,53 +52,230 @@ __global__ void sample_weights_kernel(const float* __restrict__ dinv, int64_t c,
 __device__ __forceinline__ float load_w(const float* p) { return *p; }
 __device__ __forceinline__ float load_w(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 
-// EPT > 0: each thread keeps EPT weights and their sample weights in registers
-// (c <= EPT * KM_THREADS).  EPT == 0: the row lives in dynamic shared memory as fp32 and
-// the sample weights are re-read (L1/L2) every iteration.
-template <int K, int EPT, typename T>
+// ---------------------------------------------------------------- sorted k-means ----
+// In one dimension the members of a cluster are a contiguous range of the sorted row, so the
+// row is sorted once and every Lloyd iteration reduces to K-1 boundary searches plus
+// differences of prefix sums: the per-iteration cost no longer depends on the row length.
+//   keys   : (order-preserving bits of w) << 32 | column index, bitonic-sorted in shared memory;
+//   coarse : exclusive prefix sums of s and s*w at every 8th element, kept as double-double
+//            (hi, lo) pairs so that a light cluster next to a very heavy weight (the sample
+//            weights span many decades at p = 4) loses nothing to cancellation;
+//   F(b)   : prefix up to element b = coarse[b / 8] plus at most 7 terms added one by one.
+// Cluster k of an iteration is [ub(m_{k-1}), ub(m_k)) with ub(m) the first sorted position
+// whose weight exceeds m: exactly "code = number of midpoints strictly below w".
+struct dd { double hi, lo; };
+// Error-free additions: written with the _rn intrinsics, which the compiler never fuses with a
+// neighbouring multiplication (a fused multiply-add in place of the first sum breaks the
+// error term by up to an ulp of the large operand).
+__device__ __forceinline__ dd dd_add_d(dd a, double b) {
+    const double s = __dadd_rn(a.hi, b);
+    const double bb = __dsub_rn(s, a.hi);
+    double e = __dadd_rn(__dsub_rn(a.hi, __dsub_rn(s, bb)), __dsub_rn(b, bb));
+    e = __dadd_rn(e, a.lo);
+    dd r;
+    r.hi = __dadd_rn(s, e);
+    r.lo = __dsub_rn(e, __dsub_rn(r.hi, s));
+    return r;
+}
+__device__ __forceinline__ dd dd_add(dd a, dd b) {
+    const double s = __dadd_rn(a.hi, b.hi);
+    const double bb = __dsub_rn(s, a.hi);
+    double e = __dadd_rn(__dsub_rn(a.hi, __dsub_rn(s, bb)), __dsub_rn(b.hi, bb));
+    e = __dadd_rn(e, __dadd_rn(a.lo, b.lo));
+    dd r;
+    r.hi = __dadd_rn(s, e);
+    r.lo = __dsub_rn(e, __dsub_rn(r.hi, s));
+    return r;
+}
+__device__ __forceinline__ double dd_diff(dd a, dd b) {       // a - b, rounded to double
+    const double nb = -b.hi;
+    const double s = __dadd_rn(a.hi, nb);
+    const double bb = __dsub_rn(s, a.hi);
+    double e = __dadd_rn(__dsub_rn(a.hi, __dsub_rn(s, bb)), __dsub_rn(nb, bb));
+    e = __dadd_rn(e, __dsub_rn(a.lo, b.lo));
+    return __dadd_rn(s, e);
+}
+__device__ __forceinline__ float key_weight(unsigned long long key) {
+    uint32_t u = static_cast<uint32_t>(key >> 32);
+    u ^= (u & 0x80000000u) ? 0x80000000u : 0xffffffffu;
+    return __uint_as_float(u);
+}
+
+constexpr int KS_THREADS = 256;
+constexpr int KS_CHUNK = 8;
+constexpr int KS_MAX_N = 16384;        // rows up to this length are sorted in shared memory
+
+struct dd2 { dd s, sw; };              // prefix of the sample weights and of s * w
+
+template <int K, typename T>
+__global__ void __launch_bounds__(KS_THREADS, 4)
+kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int n, const double* __restrict__ s64,
+                     float* __restrict__ grid, int n_iter) {
+    extern __shared__ unsigned long long keys[];               // n keys, then n / 8 + 1 coarse prefixes
+    dd2* coarse = reinterpret_cast<dd2*>(keys + n);
+    __shared__ dd2 tot[KS_THREADS];                            // per-thread totals, then their exclusive scan
+    __shared__ double g[K];
+    __shared__ dd2 F[K + 1];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nch = n / KS_CHUNK;
+    const int cpt = nch > KS_THREADS ? nch / KS_THREADS : 1;   // chunks per thread
+
+    for (int64_t row = blockIdx.x; row < r; row += gridDim.x) {
+        const T* wp = W + row * ldw;
+        for (int i = tid; i < n; i += KS_THREADS) {
+            unsigned long long key = ~0ull;
+            if (i < c) {
+                uint32_t u = __float_as_uint(load_w(wp + i));
+                u ^= (u & 0x80000000u) ? 0xffffffffu : 0x80000000u;
+                key = (static_cast<unsigned long long>(u) << 32) | static_cast<uint32_t>(i);
+            }
+            keys[i] = key;
+        }
+        __syncthreads();
+        // bitonic sort, ascending
+        for (int k = 2; k <= n; k <<= 1) {
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                for (int t = tid; t < (n >> 1); t += KS_THREADS) {
+                    const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+                    const int l = i | j;
+                    const unsigned long long a = keys[i], b = keys[l];
+                    const bool up = (i & k) == 0;
+                    if ((a > b) == up) { keys[i] = b; keys[l] = a; }
+                }
+                __syncthreads();
+            }
+        }
+        // chunk totals, thread-local exclusive prefixes
+        dd2 run;
+        run.s.hi = run.s.lo = run.sw.hi = run.sw.lo = 0.0;
+        for (int q = tid * cpt; q < (tid + 1) * cpt && q < nch; ++q) {
+            coarse[q] = run;
+#pragma unroll
+            for (int e = 0; e < KS_CHUNK; ++e) {
+                const int i = q * KS_CHUNK + e;
+                if (i < c) {
+                    const unsigned long long key = keys[i];
+                    const double sv = s64[static_cast<uint32_t>(key)];
+                    run.s = dd_add_d(run.s, sv);                 // same order and arithmetic as F(b) below
+                    run.sw = dd_add_d(run.sw, __dmul_rn(sv, static_cast<double>(key_weight(key))));
+                }
+            }
+        }
+        tot[tid] = run;
+        __syncthreads();
+        if (warp == 0) {       // exclusive scan of the 256 thread totals: 8 per lane, then across the warp
+            dd2 loc[KS_THREADS / 32];
+            dd2 acc;
+            acc.s.hi = acc.s.lo = acc.sw.hi = acc.sw.lo = 0.0;
+#pragma unroll
+            for (int e = 0; e < KS_THREADS / 32; ++e) {
+                loc[e] = acc;
+                const dd2 v = tot[lane * (KS_THREADS / 32) + e];
+                acc.s = dd_add(acc.s, v.s);
+                acc.sw = dd_add(acc.sw, v.sw);
+            }
+            dd2 inc = acc;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                dd2 up;
+                up.s.hi = __shfl_up_sync(0xffffffffu, inc.s.hi, o);
+                up.s.lo = __shfl_up_sync(0xffffffffu, inc.s.lo, o);
+                up.sw.hi = __shfl_up_sync(0xffffffffu, inc.sw.hi, o);
+                up.sw.lo = __shfl_up_sync(0xffffffffu, inc.sw.lo, o);
+                if (lane >= o) { inc.s = dd_add(up.s, inc.s); inc.sw = dd_add(up.sw, inc.sw); }
+            }
+            dd2 excl;                                           // sum of the lanes before this one
+            excl.s.hi = __shfl_up_sync(0xffffffffu, inc.s.hi, 1);
+            excl.s.lo = __shfl_up_sync(0xffffffffu, inc.s.lo, 1);
+            excl.sw.hi = __shfl_up_sync(0xffffffffu, inc.sw.hi, 1);
+            excl.sw.lo = __shfl_up_sync(0xffffffffu, inc.sw.lo, 1);
+            if (lane == 0) excl.s.hi = excl.s.lo = excl.sw.hi = excl.sw.lo = 0.0;
+#pragma unroll
+            for (int e = 0; e < KS_THREADS / 32; ++e) {
+                dd2 v;
+                v.s = dd_add(excl.s, loc[e].s);
+                v.sw = dd_add(excl.sw, loc[e].sw);
+                tot[lane * (KS_THREADS / 32) + e] = v;
+            }
+            if (lane == 31) coarse[nch] = inc;                  // grand total
+        }
+        __syncthreads();
+        {
+            const dd2 off = tot[tid];
+            for (int q = tid * cpt; q < (tid + 1) * cpt && q < nch; ++q) {
+                dd2 v = coarse[q];
+                v.s = dd_add(off.s, v.s);
+                v.sw = dd_add(off.sw, v.sw);
+                coarse[q] = v;
+            }
+        }
+        __syncthreads();
+
+        if (warp == 0) {
+            const double lo = static_cast<double>(key_weight(keys[0]));
+            const double hi = static_cast<double>(key_weight(keys[c - 1]));
+            if (lane < K) g[lane] = lo + (hi - lo) * static_cast<double>(lane) / static_cast<double>(K - 1);   // Eq. 6
+            if (lane == 0) {
+                F[0].s.hi = F[0].s.lo = F[0].sw.hi = F[0].sw.lo = 0.0;
+                F[K] = coarse[nch];
+            }
+            __syncwarp();
+            for (int it = 0; it < n_iter; ++it) {
+                if (lane < K - 1) {
+                    const double m = 0.5 * (g[lane] + g[lane + 1]);
+                    int b0 = 0, b1 = c;                        // first position whose weight exceeds m
+                    while (b0 < b1) {
+                        const int mid = (b0 + b1) >> 1;
+                        if (static_cast<double>(key_weight(keys[mid])) > m) b1 = mid; else b0 = mid + 1;
+                    }
+                    const int q = b0 / KS_CHUNK, rem = b0 % KS_CHUNK;
+                    dd2 f = coarse[q];
+                    for (int e = 0; e < rem; ++e) {
+                        const unsigned long long key = keys[q * KS_CHUNK + e];
+                        const double sv = s64[static_cast<uint32_t>(key)];
+                        f.s = dd_add_d(f.s, sv);
+                        f.sw = dd_add_d(f.sw, __dmul_rn(sv, static_cast<double>(key_weight(key))));
+                    }
+                    F[lane + 1] = f;
+                }
+                __syncwarp();
+                if (lane < K) {
+                    const double den = dd_diff(F[lane + 1].s, F[lane].s);
+                    const double num = dd_diff(F[lane + 1].sw, F[lane].sw);
+                    if (den > 0.0) g[lane] = num / den;         // an empty cluster keeps its centroid
+                }
+                __syncwarp();
+            }
+            if (lane < K) grid[row * K + lane] = static_cast<float>(g[lane]);
+        }
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------- long rows: direct k-means --------
+// Rows too long to sort in shared memory: the row is staged once in shared memory in its own
+// type and every iteration visits every weight (compares and cluster sums in fp64).
+template <int K, typename T>
 __global__ void __launch_bounds__(KM_THREADS)
 kmeans_rows_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int64_t c, const double* __restrict__ s64,
                    float* __restrict__ grid, int n_iter) {
-    extern __shared__ float wrow[];                      // EPT == 0 only
+    extern __shared__ unsigned char wrow_raw[];
+    T* wrow = reinterpret_cast<T*>(wrow_raw);
     __shared__ double g[K];
     __shared__ double mid[K];
     __shared__ double red[KM_WARPS][2 * K];
     __shared__ float redf[2][KM_WARPS];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    constexpr int NREG = EPT > 0 ? EPT : 1;
-    float wr[NREG];
-    double sr[NREG];
-    if (EPT > 0) {
-#pragma unroll
-        for (int e = 0; e < NREG; ++e) {
-            const int64_t j = tid + (int64_t)e * KM_THREADS;
-            sr[e] = j < c ? s64[j] : 0.0;
-        }
-    }
-
     for (int64_t row = blockIdx.x; row < r; row += gridDim.x) {
         const T* wp = W + row * ldw;
         float mn = INFINITY, mx = -INFINITY;
-        if (EPT > 0) {
-#pragma unroll
-            for (int e = 0; e < NREG; ++e) {
-                const int64_t j = tid + (int64_t)e * KM_THREADS;
-                if (j < c) {
-                    wr[e] = load_w(wp + j);
-                    mn = fminf(mn, wr[e]);
-                    mx = fmaxf(mx, wr[e]);
-                } else {
-                    wr[e] = 0.0f;      // carries zero sample weight
-                }
-            }
-        } else {
-            for (int64_t j = tid; j < c; j += KM_THREADS) {
-                float w = load_w(wp + j);
-                wrow[j] = w;
-                mn = fminf(mn, w);
-                mx = fmaxf(mx, w);
-            }
+        for (int64_t j = tid; j < c; j += KM_THREADS) {
+            const T raw = wp[j];
+            wrow[j] = raw;
+            const float w = load_w(&raw);
+            mn = fminf(mn, w);
+            mx = fmaxf(mx, w);
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
@@ -120,9 +298,9 @@ kmeans_rows_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int64_t c, c
             double ns[K], nsw[K];
 #pragma unroll
             for (int k = 0; k < K; ++k) ns[k] = nsw[k] = 0.0;
-
-            auto visit = [&](float wf, double sv) {
-                const double w = static_cast<double>(wf);
+            for (int64_t j = tid; j < c; j += KM_THREADS) {
+                const double w = static_cast<double>(load_w(wrow + j));
+                const double sv = s64[j];
                 int a = 0;
 #pragma unroll
                 for (int step = K / 2; step > 0; step >>= 1)
@@ -133,12 +311,6 @@ kmeans_rows_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int64_t c, c
                     ns[k] += (a == k) ? sv : 0.0;
                     nsw[k] += (a == k) ? sw : 0.0;
                 }
-            };
-            if (EPT > 0) {
-#pragma unroll
-                for (int e = 0; e < NREG; ++e) visit(wr[e], sr[e]);
-            } else {
-                for (int64_t j = tid; j < c; j += KM_THREADS) visit(wrow[j], s64[j]);
             }
 #pragma unroll
             for (int k = 0; k < K; ++k) {
@@ -168,22 +340,29 @@ kmeans_rows_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int64_t c, c
 template <int K, typename T>
 int launch_kmeans(cudaStream_t st, int sms, const T* W, int64_t ldw, int64_t r, int64_t c, const double* s64, float* grid,
                   int n_iter) {
-    const unsigned blocks = static_cast<unsigned>(r < (int64_t)sms * 8 ? r : (int64_t)sms * 8);
-    if (c <= 1 * KM_THREADS) kmeans_rows_kernel<K, 1, T><<<blocks, KM_THREADS, 0, st>>>(W, ldw, r, c, s64, grid, n_iter);
-    else if (c <= 2 * KM_THREADS) kmeans_rows_kernel<K, 2, T><<<blocks, KM_THREADS, 0, st>>>(W, ldw, r, c, s64, grid, n_iter);
-    else if (c <= 4 * KM_THREADS) kmeans_rows_kernel<K, 4, T><<<blocks, KM_THREADS, 0, st>>>(W, ldw, r, c, s64, grid, n_iter);
-    else if (c <= 8 * KM_THREADS) kmeans_rows_kernel<K, 8, T><<<blocks, KM_THREADS, 0, st>>>(W, ldw, r, c, s64, grid, n_iter);
-    else if (c <= 16 * KM_THREADS) kmeans_rows_kernel<K, 16, T><<<blocks, KM_THREADS, 0, st>>>(W, ldw, r, c, s64, grid, n_iter);
-    else {
-        const size_t smem = static_cast<size_t>(c) * sizeof(float);
+    if (c <= KS_MAX_N) {
+        int n = 64;
+        while (n < c) n <<= 1;
+        const size_t smem = static_cast<size_t>(n) * 8 + (static_cast<size_t>(n) / KS_CHUNK + 1) * sizeof(dd2);
+        static bool attr_set = false;
+        if (!attr_set) {
+            LQ_CUDA_TRY(cudaFuncSetAttribute(kmeans_sorted_kernel<K, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+            attr_set = true;
+        }
+        int per_sm = static_cast<int>((228 * 1024) / (smem + 10 * 1024));      // static shared memory and the per-CTA reserve
+        per_sm = per_sm < 1 ? 1 : (per_sm > 4 ? 4 : per_sm);                    // 64 registers x 256 threads: four CTAs per SM
+        const int64_t cap = static_cast<int64_t>(sms) * per_sm;
+        kmeans_sorted_kernel<K, T><<<static_cast<unsigned>(r < cap ? r : cap), KS_THREADS, smem, st>>>(
+            W, ldw, r, static_cast<int>(c), n, s64, grid, n_iter);
+    } else {
+        const size_t smem = static_cast<size_t>(c) * sizeof(T);
         if (smem > 200 * 1024) return LQ_ERR_UNSUPPORTED;
         static bool attr_set = false;
         if (!attr_set) {
-            LQ_CUDA_TRY(cudaFuncSetAttribute(kmeans_rows_kernel<K, 0, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+            LQ_CUDA_TRY(cudaFuncSetAttribute(kmeans_rows_kernel<K, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
             attr_set = true;
         }
-        const unsigned b2 = static_cast<unsigned>(r < sms ? r : sms);
-        kmeans_rows_kernel<K, 0, T><<<b2, KM_THREADS, smem, st>>>(W, ldw, r, c, s64, grid, n_iter);
+        kmeans_rows_kernel<K, T><<<static_cast<unsigned>(r < sms ? r : sms), KM_THREADS, smem, st>>>(W, ldw, r, c, s64, grid, n_iter);
     }
     LQ_LAUNCH_CHECK();
     return LQ_OK;
