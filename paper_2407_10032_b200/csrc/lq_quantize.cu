@@ -1,12 +1,9 @@
 // Stage 4 -- Algorithm 1 lines 10-21: the block-wise column loop with error feedback.
 //
 // Per block of B = 128 columns:
-//   in-block kernel  : one thread per output row keeps the row's 128 block weights in
-//                      registers and walks the columns in order (quantise, E = (w - q)/U_jj,
-//                      w[k] -= E * U[j][k]); the 128 x 128 diagonal block of U sits in shared
-//                      memory and is read as warp-wide broadcasts.  The walk is organised as
-//                      8 sub-blocks of 16 columns so that the register file is indexed
-//                      statically while the code stays small.
+//   in-block kernel  : one warp per output row, four block columns per lane, walks the columns
+//                      in order (quantise, E = (w - q)/U_jj, w[k] -= E * U[j][k]); the
+//                      128 x 128 diagonal block of U sits in shared memory.
 //   trailing update  : W[:, i+B:] -= E U[i:i+B, i+B:] on the tensor cores (lq_tc_gemm), fp32
 //                      operands fed as three bf16 terms each (six products), accumulated into
 //                      the fp32 working copy by the copy engine's reduce-add.
@@ -17,8 +14,6 @@
 namespace {
 
 constexpr int B = 128;      // block width of the column loop
-constexpr int SB = 16;      // sub-block width
-constexpr int NSB = B / SB;
 
 template <typename T>
 __global__ void to_f32_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, float* __restrict__ Wc, int64_t ldc) {
@@ -56,34 +51,6 @@ __global__ void split_transpose_kernel(const float* __restrict__ U, int64_t ldu,
     }
 }
 
-template <int K>
-struct NuGrid {
-    float g[K];
-    float m[K - 1];
-    __device__ __forceinline__ void load(const float* grid_row) {
-#pragma unroll
-        for (int k = 0; k < K; ++k) g[k] = grid_row[k];
-#pragma unroll
-        for (int k = 0; k < K - 1; ++k) m[k] = 0.5f * (g[k] + g[k + 1]);
-    }
-    // nearest grid point: code = number of midpoints strictly below w
-    __device__ __forceinline__ void quant(float w, int& code, float& q) const {
-        int cnt = 0;
-#pragma unroll
-        for (int k = 0; k < K - 1; ++k) cnt += (w > m[k]) ? 1 : 0;
-        code = cnt;
-        float sel[K];
-#pragma unroll
-        for (int k = 0; k < K; ++k) sel[k] = g[k];
-#pragma unroll
-        for (int width = K / 2, bit = 1; width >= 1; width >>= 1, bit <<= 1) {
-#pragma unroll
-            for (int k = 0; k < width; ++k) sel[k] = (cnt & bit) ? sel[2 * k + 1] : sel[2 * k];
-        }
-        q = sel[0];
-    }
-};
-
 struct QuantOut {
     uint8_t* codes;          // r x c
     void* what;              // r x ldwh or null
@@ -93,17 +60,27 @@ struct QuantOut {
     double* loss_rows;       // r
 };
 
+// One warp per output row, lane l owning columns 4l .. 4l+3 of the block.  Column step j:
+// the owning lane's weight is broadcast; the nearest grid point is found by every lane
+// comparing the weight with "its" midpoint (lane k holds g_k and m_k = (g_k + g_{k+1})/2) and a
+// ballot -- code = number of midpoints strictly below w -- and the grid value comes back from
+// lane `code`; then E = (w - q) / U_jj and every lane feeds it into its four weights with one
+// 16-byte read of row j of the block of U held in shared memory.  Entries of that row left of
+// the diagonal are zero, so no lane needs a predicate.
+constexpr int IB_WARPS = 16;
+constexpr int IB_THREADS = IB_WARPS * 32;
+
 template <int K, bool AFFINE>
-__global__ void __launch_bounds__(128)
-inblock_kernel(float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, int64_t i0, const float* __restrict__ U,
+__global__ void __launch_bounds__(IB_THREADS)
+inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, int64_t i0, const float* __restrict__ U,
                int64_t ldu, const float* __restrict__ grid, const float* __restrict__ scale,
                const int32_t* __restrict__ zero, int group, int n_groups, QuantOut out) {
     extern __shared__ float Us[];          // B x B block of U, then B reciprocals of its diagonal
     float* invd = Us + B * B;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bw = (c - i0) < B ? static_cast<int>(c - i0) : B;
 
-    for (int idx = tid; idx < B * B / 4; idx += 128) {
+    for (int idx = tid; idx < B * B / 4; idx += IB_THREADS) {
         const int jj = idx / (B / 4), k4 = (idx % (B / 4)) * 4;
         float4 v;
         if (jj < bw && k4 + 3 < bw && (ldu % 4 == 0)) {
@@ -123,132 +100,114 @@ inblock_kernel(float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, int64_
     if (tid < B) invd[tid] = 1.0f / Us[tid * B + tid];
     __syncthreads();
 
-    const int64_t row = (int64_t)blockIdx.x * 128 + tid;
+    const int64_t row = (int64_t)blockIdx.x * IB_WARPS + warp;
     if (row >= r) return;
 
-    float w[B];
+    const int col0 = 4 * lane;             // first of this lane's columns inside the block
+    float w[4];
     {
-        const float* wp = Wc + row * ldc + i0;
+        const float* wp = Wc + row * ldc + i0 + col0;
+        if (col0 + 3 < bw) {
+            const float4 v = *reinterpret_cast<const float4*>(wp);
+            w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+        } else {
 #pragma unroll
-        for (int k = 0; k < B; k += 4) {
-            if (k + 3 < bw) {
-                const float4 v = *reinterpret_cast<const float4*>(wp + k);
-                w[k] = v.x; w[k + 1] = v.y; w[k + 2] = v.z; w[k + 3] = v.w;
-            } else {
-#pragma unroll
-                for (int u = 0; u < 4; ++u) w[k + u] = (k + u < bw) ? wp[k + u] : 0.0f;
-            }
+            for (int u = 0; u < 4; ++u) w[u] = (col0 + u < bw) ? wp[u] : 0.0f;
         }
     }
+    float gl = 0.0f, ml = INFINITY;        // this lane's grid point and the midpoint above it
+    float S_mine = 1.0f, Z_mine = 0.0f;    // affine parameters of this lane's columns
+    if (!AFFINE) {
+        if (lane < K) gl = grid[row * K + lane];
+        const float gn = __shfl_down_sync(0xffffffffu, gl, 1);
+        if (lane < K - 1) ml = 0.5f * (gl + gn);
+    } else if (col0 < bw) {
+        const int64_t gi = (i0 + col0) / group;
+        const int64_t gidx = row * n_groups + (gi < n_groups ? gi : n_groups - 1);
+        S_mine = scale[gidx];
+        Z_mine = static_cast<float>(zero[gidx]);
+    }
 
-    NuGrid<K> ng;
-    if (!AFFINE) ng.load(grid + row * K);
-    double loss = 0.0;
-
+    float qkeep[4] = {0.0f, 0.0f, 0.0f, 0.0f}, ekeep[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    uint32_t cpack = 0;
+    float loss = 0.0f;
+    const int n_owner = (bw + 3) / 4;
 #pragma unroll 1
-    for (int s = 0; s < NSB; ++s) {
-        float ws[SB];
-#pragma unroll
-        for (int kb = 0; kb < NSB; ++kb)
-            if (kb == s) {
-#pragma unroll
-                for (int t = 0; t < SB; ++t) ws[t] = w[kb * SB + t];
-            }
+    for (int jj = 0; jj < n_owner; ++jj) {
         float S = 1.0f, Zf = 0.0f;
         if (AFFINE) {
-            const int64_t gi = (i0 + s * SB) / group;
-            const int64_t gidx = row * n_groups + (gi < n_groups ? gi : n_groups - 1);
-            S = scale[gidx];
-            Zf = static_cast<float>(zero[gidx]);
+            S = __shfl_sync(0xffffffffu, S_mine, jj);
+            Zf = __shfl_sync(0xffffffffu, Z_mine, jj);
         }
-        float e[SB];
-        float qv[SB];
-        uint32_t cpack[SB / 4];
+        const bool mine = lane == jj;
 #pragma unroll
-        for (int t = 0; t < SB / 4; ++t) cpack[t] = 0;
-        const float* urow = Us + (s * SB) * B + s * SB;
-#pragma unroll
-        for (int t = 0; t < SB; ++t) {
+        for (int u = 0; u < 4; ++u) {
+            const int j = 4 * jj + u;
+            const float wj = __shfl_sync(0xffffffffu, w[u], jj);
             int code;
             float q;
             if (AFFINE) {
-                float qi = rintf(__fdiv_rn(ws[t], S)) + Zf;
+                float qi = rintf(__fdiv_rn(wj, S)) + Zf;
                 qi = fminf(fmaxf(qi, 0.0f), static_cast<float>(K - 1));
                 code = static_cast<int>(qi);
                 q = (qi - Zf) * S;
             } else {
-                ng.quant(ws[t], code, q);
+                code = __popc(__ballot_sync(0xffffffffu, wj > ml));
+                q = __shfl_sync(0xffffffffu, gl, code);
             }
-            const bool live = (s * SB + t) < bw;
-            const float et = live ? (ws[t] - q) * invd[s * SB + t] : 0.0f;
-            e[t] = et;
-            qv[t] = q;
-            cpack[t >> 2] |= static_cast<uint32_t>(code) << (8 * (t & 3));
-            loss += static_cast<double>(et) * static_cast<double>(et);
-#pragma unroll
-            for (int u = t + 1; u < SB; ++u) ws[u] = fmaf(-et, urow[t * B + u], ws[u]);
-        }
-        // feed the 16 errors forward to the later sub-blocks of this block
-#pragma unroll
-        for (int kb = 1; kb < NSB; ++kb) {
-            if (kb > s) {
-#pragma unroll
-                for (int t = 0; t < SB; ++t) {
-                    const float4* up = reinterpret_cast<const float4*>(Us + (s * SB + t) * B + kb * SB);
-#pragma unroll
-                    for (int u4 = 0; u4 < SB / 4; ++u4) {
-                        const float4 uv = up[u4];
-                        w[kb * SB + 4 * u4 + 0] = fmaf(-e[t], uv.x, w[kb * SB + 4 * u4 + 0]);
-                        w[kb * SB + 4 * u4 + 1] = fmaf(-e[t], uv.y, w[kb * SB + 4 * u4 + 1]);
-                        w[kb * SB + 4 * u4 + 2] = fmaf(-e[t], uv.z, w[kb * SB + 4 * u4 + 2]);
-                        w[kb * SB + 4 * u4 + 3] = fmaf(-e[t], uv.w, w[kb * SB + 4 * u4 + 3]);
-                    }
-                }
+            const float e = (j < bw) ? (wj - q) * invd[j] : 0.0f;
+            loss = fmaf(e, e, loss);
+            if (mine) {
+                qkeep[u] = q;
+                ekeep[u] = e;
+                cpack |= static_cast<uint32_t>(code) << (8 * u);
             }
-        }
-        // outputs of this sub-block
-        const int col0 = s * SB;
-        if (col0 < bw) {
-            const int64_t gcol = i0 + col0;
-            if (col0 + SB <= bw && (c % 16 == 0)) {
-                *reinterpret_cast<uint4*>(out.codes + row * c + gcol) = make_uint4(cpack[0], cpack[1], cpack[2], cpack[3]);
-            } else {
-#pragma unroll
-                for (int t = 0; t < SB; ++t)
-                    if (col0 + t < bw) out.codes[row * c + gcol + t] = static_cast<uint8_t>((cpack[t >> 2] >> (8 * (t & 3))) & 0xff);
-            }
-            if (out.what) {
-#pragma unroll
-                for (int t = 0; t < SB; ++t)
-                    if (col0 + t < bw) {
-                        if (out.what_bf16) static_cast<__nv_bfloat16*>(out.what)[row * out.ldwh + gcol + t] = __float2bfloat16_rn(qv[t]);
-                        else static_cast<float*>(out.what)[row * out.ldwh + gcol + t] = qv[t];
-                    }
-            }
-        }
-        {
-            uint32_t ph[SB / 2], pm[SB / 2], pl[SB / 2];
-#pragma unroll
-            for (int t = 0; t < SB; t += 2) {
-                __nv_bfloat16 h0, m0, l0, h1, m1, l1;
-                lq_split3(e[t], h0, m0, l0);
-                lq_split3(e[t + 1], h1, m1, l1);
-                ph[t / 2] = static_cast<uint32_t>(__bfloat16_as_ushort(h0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(h1)) << 16);
-                pm[t / 2] = static_cast<uint32_t>(__bfloat16_as_ushort(m0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(m1)) << 16);
-                pl[t / 2] = static_cast<uint32_t>(__bfloat16_as_ushort(l0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(l1)) << 16);
-            }
-            __nv_bfloat16* e0 = out.esplit + row * B + col0;
-            __nv_bfloat16* e1 = e0 + r * B;
-            __nv_bfloat16* e2 = e1 + r * B;
-            *reinterpret_cast<uint4*>(e0) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
-            *reinterpret_cast<uint4*>(e0 + 8) = make_uint4(ph[4], ph[5], ph[6], ph[7]);
-            *reinterpret_cast<uint4*>(e1) = make_uint4(pm[0], pm[1], pm[2], pm[3]);
-            *reinterpret_cast<uint4*>(e1 + 8) = make_uint4(pm[4], pm[5], pm[6], pm[7]);
-            *reinterpret_cast<uint4*>(e2) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
-            *reinterpret_cast<uint4*>(e2 + 8) = make_uint4(pl[4], pl[5], pl[6], pl[7]);
+            const float4 uv = *reinterpret_cast<const float4*>(Us + j * B + col0);
+            w[0] = fmaf(-e, uv.x, w[0]);
+            w[1] = fmaf(-e, uv.y, w[1]);
+            w[2] = fmaf(-e, uv.z, w[2]);
+            w[3] = fmaf(-e, uv.w, w[3]);
         }
     }
-    out.loss_rows[row] += loss;
+
+    // outputs of this lane's four columns
+    if (col0 < bw) {
+        const int64_t gcol = i0 + col0;
+        if (col0 + 3 < bw && (c % 4 == 0)) {
+            *reinterpret_cast<uint32_t*>(out.codes + row * c + gcol) = cpack;
+        } else {
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (col0 + u < bw) out.codes[row * c + gcol + u] = static_cast<uint8_t>((cpack >> (8 * u)) & 0xff);
+        }
+        if (out.what) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (col0 + u < bw) {
+                    if (out.what_bf16) static_cast<__nv_bfloat16*>(out.what)[row * out.ldwh + gcol + u] = __float2bfloat16_rn(qkeep[u]);
+                    else static_cast<float*>(out.what)[row * out.ldwh + gcol + u] = qkeep[u];
+                }
+        }
+    }
+    {
+        uint32_t ph[2], pm[2], pl[2];
+#pragma unroll
+        for (int t = 0; t < 4; t += 2) {
+            __nv_bfloat16 h0, m0, l0, h1, m1, l1;
+            lq_split3(ekeep[t], h0, m0, l0);
+            lq_split3(ekeep[t + 1], h1, m1, l1);
+            ph[t / 2] = static_cast<uint32_t>(__bfloat16_as_ushort(h0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(h1)) << 16);
+            pm[t / 2] = static_cast<uint32_t>(__bfloat16_as_ushort(m0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(m1)) << 16);
+            pl[t / 2] = static_cast<uint32_t>(__bfloat16_as_ushort(l0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(l1)) << 16);
+        }
+        __nv_bfloat16* e0 = out.esplit + row * B + col0;
+        __nv_bfloat16* e1 = e0 + r * B;
+        __nv_bfloat16* e2 = e1 + r * B;
+        *reinterpret_cast<uint2*>(e0) = make_uint2(ph[0], ph[1]);
+        *reinterpret_cast<uint2*>(e1) = make_uint2(pm[0], pm[1]);
+        *reinterpret_cast<uint2*>(e2) = make_uint2(pl[0], pl[1]);
+    }
+    if (lane == 0) out.loss_rows[row] += static_cast<double>(loss);
 }
 
 __global__ void zero_doubles_kernel(double* p, int64_t n) {
@@ -304,7 +263,7 @@ int launch_inblock(cudaStream_t st, float* Wc, int64_t ldc, int64_t r, int64_t c
         LQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel<K, AFFINE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         attr_set = true;
     }
-    inblock_kernel<K, AFFINE><<<static_cast<unsigned>(lq_ceil_div(r, 128)), 128, smem, st>>>(
+    inblock_kernel<K, AFFINE><<<static_cast<unsigned>(lq_ceil_div(r, IB_WARPS)), IB_THREADS, smem, st>>>(
         Wc, ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out);
     LQ_LAUNCH_CHECK();
     return LQ_OK;
@@ -336,7 +295,7 @@ extern "C" int lq_quantize_layer(lq_handle* h, void* stream, const lq_config* cf
         if (!scale || !zero) return LQ_ERR_INVALID_ARG;
         const int64_t g = cfg->group_size == 0 ? c : cfg->group_size;
         if (c % g) return LQ_ERR_INVALID_ARG;
-        if (g != c && (g % SB)) return LQ_ERR_UNSUPPORTED;     // (S, Z) may change only between 16-column sub-blocks
+        if (g != c && (g % 4)) return LQ_ERR_UNSUPPORTED;      // a lane's four columns share one (S, Z)
         if (g > 0x7fffffffLL) return LQ_ERR_UNSUPPORTED;
         group = static_cast<int>(g);
         n_groups = static_cast<int>(c / g);
