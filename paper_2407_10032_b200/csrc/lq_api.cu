@@ -20,9 +20,26 @@ extern "C" int lq_create(lq_handle** out, int device) {
     h->device = device;
     h->sm_count = prop.multiProcessorCount;
     h->dstatus = nullptr;
+    h->aux = nullptr;
+    h->ev_fork = h->ev_next = h->ev_rest = nullptr;
+    if (cudaStreamCreateWithFlags(&h->aux, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_next, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_rest, cudaEventDisableTiming) != cudaSuccess) {
+        if (h->ev_rest) cudaEventDestroy(h->ev_rest);
+        if (h->ev_next) cudaEventDestroy(h->ev_next);
+        if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+        if (h->aux) cudaStreamDestroy(h->aux);
+        delete h;
+        return LQ_ERR_CUDA;
+    }
     if (cudaMalloc(&h->dstatus, sizeof(lq_dev_status)) != cudaSuccess ||
         cudaMemset(h->dstatus, 0, sizeof(lq_dev_status)) != cudaSuccess) {
         if (h->dstatus) cudaFree(h->dstatus);
+        cudaEventDestroy(h->ev_rest);
+        cudaEventDestroy(h->ev_next);
+        cudaEventDestroy(h->ev_fork);
+        cudaStreamDestroy(h->aux);
         delete h;
         return LQ_ERR_CUDA;
     }
@@ -33,6 +50,13 @@ extern "C" int lq_create(lq_handle** out, int device) {
 extern "C" int lq_destroy(lq_handle* h) {
     if (!h) return LQ_ERR_INVALID_ARG;
     cudaFree(h->dstatus);
+    if (h->aux) {
+        cudaStreamSynchronize(h->aux);
+        cudaEventDestroy(h->ev_rest);
+        cudaEventDestroy(h->ev_next);
+        cudaEventDestroy(h->ev_fork);
+        cudaStreamDestroy(h->aux);
+    }
     delete h;
     return LQ_OK;
 }

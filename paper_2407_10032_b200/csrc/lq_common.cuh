@@ -18,6 +18,11 @@ struct lq_handle {
     int device;
     int sm_count;
     lq_dev_status* dstatus;   // device memory
+    // Fork/join helpers of stage 2: the bulk of a step's update runs on `aux` while the caller's
+    // stream already works on the next block column.  Null in a handle that owns no stream
+    // (everything then runs on the caller's stream).
+    cudaStream_t aux;
+    cudaEvent_t ev_fork, ev_next, ev_rest;
 };
 
 // Record the first device-side failure; later ones are dropped.

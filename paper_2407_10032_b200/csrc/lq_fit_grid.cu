@@ -612,6 +612,8 @@ extern "C" int lq_fit_grid_noalloc(lq_handle* h, void* stream, const lq_config* 
     local.device = dev;
     local.sm_count = d.sm_count;
     local.dstatus = d.status;
+    local.aux = nullptr;
+    local.ev_fork = local.ev_next = local.ev_rest = nullptr;
     return lq_fit_grid(h ? h : &local, stream, cfg, W, w_dtype, r, c, ldw, dinv, grid, scale, zero, d.scratch,
                        kNoAllocScratchBytes);
 }

@@ -215,11 +215,25 @@ panel_kernel(double* __restrict__ A, int64_t cp, int k, const double* __restrict
     }
 }
 
-// Step k, update of block rows i < k over the whole width (grid: 2 * nblk x k).
+// Step k, update of block rows i < k over the whole width.  The tiles of block column k-1 and
+// of block row k-1 are all that step k-1's diagonal and panel kernels read, so they can be
+// updated first ("next") and the remainder ("rest") left to run beside step k-1:
+//   part 0: everything, grid 2 nblk x k;  part 2: the rest, same grid;
+//   part 1: next only, grid 2 nblk x 1 -- tile t < k is (t, k-1), tile t >= k is (k-1, t).
 __global__ void __launch_bounds__(GEMM_THREADS, 2)
-update_kernel(double* __restrict__ A, int64_t cp, int k, const double* __restrict__ Pbuf, const double* __restrict__ Q) {
+update_kernel(double* __restrict__ A, int64_t cp, int k, int part, const double* __restrict__ Pbuf,
+              const double* __restrict__ Q) {
     extern __shared__ double smem[];
-    const int j = blockIdx.x >> 1, h = blockIdx.x & 1, i = blockIdx.y;
+    const int h = blockIdx.x & 1;
+    int i, j;
+    if (part == 1) {
+        const int t = blockIdx.x >> 1;
+        if (t < k) { i = t; j = k - 1; } else { i = k - 1; j = t; }
+    } else {
+        j = blockIdx.x >> 1;
+        i = blockIdx.y;
+        if (part == 2 && (j == k - 1 || i == k - 1)) return;
+    }
     if (j < i) return;                                  // strictly lower tiles of the symmetric part
     const double* Pi = Pbuf + (int64_t)i * NB * NB;
     TileOut o = {};
@@ -454,7 +468,7 @@ finalize_kernel(const double* __restrict__ A, int64_t cp, int64_t c, float* __re
 
 struct PrepLayout {
     int64_t nblk, cp;
-    size_t scal, a, pbuf, q, vt, total;
+    size_t scal, a, pbuf, q, vt, total, panel_bytes;
 };
 PrepLayout prep_layout(int64_t c) {
     PrepLayout L;
@@ -463,8 +477,9 @@ PrepLayout prep_layout(int64_t c) {
     size_t off = 0;
     L.scal = off; off += 256;
     L.a = off;    off += lq_align_up(static_cast<size_t>(L.cp) * L.cp * sizeof(double), 256);
-    L.pbuf = off; off += lq_align_up(static_cast<size_t>(L.cp) * NB * sizeof(double), 256);
-    L.q = off;    off += lq_align_up(static_cast<size_t>(L.cp) * NB * sizeof(double), 256);
+    L.panel_bytes = lq_align_up(static_cast<size_t>(L.cp) * NB * sizeof(double), 256);
+    L.pbuf = off; off += 2 * L.panel_bytes;            // P and Q are double-buffered: one step's
+    L.q = off;    off += 2 * L.panel_bytes;            // update may still read them while the next is written
     L.vt = off;   off += lq_align_up(static_cast<size_t>(NB) * NB * sizeof(double), 256);
     L.total = off;
     return L;
@@ -493,8 +508,6 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
     char* wsp = static_cast<char*>(ws);
     double* scal = reinterpret_cast<double*>(wsp + L.scal);
     double* A = reinterpret_cast<double*>(wsp + L.a);
-    double* Pbuf = reinterpret_cast<double*>(wsp + L.pbuf);
-    double* Q = reinterpret_cast<double*>(wsp + L.q);
     double* VT = reinterpret_cast<double*>(wsp + L.vt);
 
     static bool attr_set = false;
@@ -521,20 +534,48 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
         LQ_LAUNCH_CHECK();
     }
 
+    // The sweep.  With an auxiliary stream: step k's diagonal and panel kernels and the "next"
+    // part of its update stay on the caller's stream; the rest of the update goes to the
+    // auxiliary stream and overlaps step k-1's diagonal and panel kernels.
+    cudaStream_t aux = h->aux;
+    const bool fork = aux != nullptr && nblk > 2;
+    if (fork) {
+        LQ_CUDA_TRY(cudaEventRecord(h->ev_fork, st));
+        LQ_CUDA_TRY(cudaStreamWaitEvent(aux, h->ev_fork, 0));
+    }
+    bool rest_pending = false;
     for (int64_t k = nblk - 1; k >= 0; --k) {
+        double* Pk = reinterpret_cast<double*>(wsp + L.pbuf + (k & 1) * L.panel_bytes);
+        double* Qk = reinterpret_cast<double*>(wsp + L.q + (k & 1) * L.panel_bytes);
         diag_block_kernel<<<1, DIAG_THREADS, DIAG_SMEM, st>>>(A, cp, k, c, VT, h->dstatus);
         LQ_LAUNCH_CHECK();
         if (nblk > 1) {
             panel_kernel<<<static_cast<unsigned>(2 * (nblk - 1)), GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, static_cast<int>(k), VT,
-                                                                                                Pbuf, Q);
+                                                                                                Pk, Qk);
             LQ_LAUNCH_CHECK();
         }
-        if (k > 0) {
+        if (k == 0) break;
+        if (!fork) {
             dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(k));
-            update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, static_cast<int>(k), Pbuf, Q);
+            update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, static_cast<int>(k), 0, Pk, Qk);
             LQ_LAUNCH_CHECK();
+            continue;
+        }
+        if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_rest, 0));     // step k+1's rest touched the same tiles
+        update_kernel<<<static_cast<unsigned>(2 * nblk), GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, static_cast<int>(k), 1, Pk, Qk);
+        LQ_LAUNCH_CHECK();
+        rest_pending = false;
+        if (k > 1) {
+            LQ_CUDA_TRY(cudaEventRecord(h->ev_next, st));
+            LQ_CUDA_TRY(cudaStreamWaitEvent(aux, h->ev_next, 0));
+            dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(k - 1));
+            update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, aux>>>(A, cp, static_cast<int>(k), 2, Pk, Qk);
+            LQ_LAUNCH_CHECK();
+            LQ_CUDA_TRY(cudaEventRecord(h->ev_rest, aux));
+            rest_pending = true;
         }
     }
+    if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_rest, 0));
     finalize_kernel<<<static_cast<unsigned>(lq_ceil_div(c, 32)), 256, 0, st>>>(A, cp, c, U, ldu, dinv);
     LQ_LAUNCH_CHECK();
     return LQ_OK;
