@@ -93,18 +93,21 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
-// ---------------------------------------------------- 128 x 64 tile product, K = 128 --
-// C[128 x 64] = beta * C + alpha * A[128 x 128] * B[128 x 64], all fp64 row-major.
-// 256 threads = 8 warps in a 4 x 2 arrangement, each owning a 32 x 32 patch as 4 x 4 MMA tiles.
-// K is streamed 16 at a time through a 3-stage cp.async ring; the shared-memory pitches make
-// every fragment load conflict-free.  The output may alias B (all of B has been read before
-// the first store).  Optional extra outputs: a plain copy (C2) and a transposed copy (Ct).
-constexpr int TM = 128, TN = 64, TK = 16, NST = 3;
-constexpr int AP = 20;                       // pitch (doubles) of an A chunk row: 16 + 4
-constexpr int BP = 68;                       // pitch of a B chunk row: 64 + 4
-constexpr int STAGE_DOUBLES = TM * AP + TK * BP;
-constexpr int GEMM_SMEM = NST * STAGE_DOUBLES * 8;
+// ------------------------------------------------------------ tile product, K = 128 --
+// C[TM x TN] = beta * C + alpha * A[TM x 128] * op(B), all fp64 row-major, by 256 threads = 8 warps
+// arranged WMW x (8 / WMW); each warp owns an (8 MI) x 32 patch as MI x 4 MMA tiles, so
+// TM = 8 MI WMW and TN = 32 (8 / WMW).  NT: B is given as TN rows of K (C = A B^T), otherwise as
+// K rows of TN.  K is streamed 16 at a time through a 3-stage cp.async ring; the shared-memory
+// pitches make every fragment load conflict-free.  The output may alias B when the tile spans
+// all of B's rows and columns that it reads (all of B has been read before the first store).
+// Optional extra outputs: a plain copy (C2) and a transposed copy (Ct).
+//   <4, 4, *>  128 x 64   the bulk of the updates (two CTAs per SM)
+//   <2, 4, *>   64 x 64   panel and "next" tiles: short launches that sit on the critical path
+//   <2, 8, *>  128 x 32   row scaling in place (a CTA owns whole columns)
+constexpr int TK = 16, NST = 3;
+constexpr int AP = 20;                       // pitch (doubles) of a K-major chunk row: 16 + 4
 constexpr int GEMM_THREADS = 256;
+constexpr int GEMM_SMEM = NST * (128 * AP + TK * (64 + 4)) * 8;     // the largest instantiation
 
 struct TileOut {
     double* C;  int64_t ldc;
@@ -112,30 +115,45 @@ struct TileOut {
     double* Ct; int64_t ldct;     // optional transposed copy: Ct[col * ldct + row]
 };
 
+template <int MI, int WMW, bool NT>
 __device__ __forceinline__ void gemm_tile(const double* __restrict__ A, int64_t lda, const double* B, int64_t ldb,
                                           double alpha, double beta, const TileOut& o, double* smem) {
+    constexpr int WNW = 8 / WMW;
+    constexpr int TMR = 8 * MI * WMW, TNC = 32 * WNW;
+    constexpr int BP = TNC + 4;                               // pitch of an N-major chunk row (NN form)
+    constexpr int STAGE = TMR * AP + (NT ? TNC * AP : TK * BP);
+    static_assert(NST * STAGE * 8 <= GEMM_SMEM, "shared memory");
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int wm = warp >> 1, wn = warp & 1;
+    const int wm = warp / WNW, wn = warp % WNW;
     const int fr = lane >> 2, fk = lane & 3;
 
     auto issue = [&](int kc) {
-        double* as = smem + (kc % NST) * STAGE_DOUBLES;
-        double* bs = as + TM * AP;
+        double* as = smem + (kc % NST) * STAGE;
+        double* bs = as + TMR * AP;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < TMR * 8 / GEMM_THREADS; ++u) {
             const int idx = tid + GEMM_THREADS * u, row = idx >> 3, seg = idx & 7;
             cp_async16(as + row * AP + seg * 2, A + (int64_t)row * lda + kc * TK + seg * 2);
         }
+        if (NT) {
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
-            const int idx = tid + GEMM_THREADS * u, row = idx >> 5, seg = idx & 31;
-            cp_async16(bs + row * BP + seg * 2, B + (int64_t)(kc * TK + row) * ldb + seg * 2);
+            for (int u = 0; u < TNC * 8 / GEMM_THREADS; ++u) {
+                const int idx = tid + GEMM_THREADS * u, row = idx >> 3, seg = idx & 7;
+                cp_async16(bs + row * AP + seg * 2, B + (int64_t)row * ldb + kc * TK + seg * 2);
+            }
+        } else {
+            constexpr int SEGS = TNC / 2;                     // 16-byte pieces per row
+#pragma unroll
+            for (int u = 0; u < TK * SEGS / GEMM_THREADS; ++u) {
+                const int idx = tid + GEMM_THREADS * u, row = idx / SEGS, seg = idx % SEGS;
+                cp_async16(bs + row * BP + seg * 2, B + (int64_t)(kc * TK + row) * ldb + seg * 2);
+            }
         }
     };
 
-    double acc[4][4][2];
+    double acc[MI][4][2];
 #pragma unroll
-    for (int i = 0; i < 4; ++i)
+    for (int i = 0; i < MI; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j][0] = acc[i][j][1] = 0.0;
 
@@ -148,17 +166,17 @@ __device__ __forceinline__ void gemm_tile(const double* __restrict__ A, int64_t 
         __syncthreads();
         if (kc + NST - 1 < NCHUNK) issue(kc + NST - 1);
         cp_async_commit();
-        const double* as = smem + (kc % NST) * STAGE_DOUBLES + (wm * 32 + fr) * AP + fk;
-        const double* bs = smem + (kc % NST) * STAGE_DOUBLES + TM * AP + fk * BP + wn * 32 + fr;
+        const double* as = smem + (kc % NST) * STAGE + (wm * 8 * MI + fr) * AP + fk;
+        const double* bs = smem + (kc % NST) * STAGE + TMR * AP + (NT ? (wn * 32 + fr) * AP + fk : fk * BP + wn * 32 + fr);
 #pragma unroll
         for (int kk = 0; kk < TK / 4; ++kk) {
-            double a[4], b[4];
+            double a[MI], b[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) a[i] = as[8 * i * AP + kk * 4];
+            for (int i = 0; i < MI; ++i) a[i] = as[8 * i * AP + kk * 4];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) b[j] = bs[kk * 4 * BP + 8 * j];
+            for (int j = 0; j < 4; ++j) b[j] = NT ? bs[8 * j * AP + kk * 4] : bs[kk * 4 * BP + 8 * j];
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < MI; ++i)
 #pragma unroll
                 for (int j = 0; j < 4; ++j) dmma(acc[i][j][0], acc[i][j][1], a[i], b[j]);
         }
@@ -167,8 +185,8 @@ __device__ __forceinline__ void gemm_tile(const double* __restrict__ A, int64_t 
     __syncthreads();      // every thread's copies have landed: B may now be overwritten
 
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int row = wm * 32 + 8 * i + fr;
+    for (int i = 0; i < MI; ++i) {
+        const int row = wm * 8 * MI + 8 * i + fr;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int col = wn * 32 + 8 * j + 2 * fk;
@@ -191,63 +209,70 @@ __device__ __forceinline__ void gemm_tile(const double* __restrict__ A, int64_t 
     }
 }
 
-// Step k, panel: blocks [0, 2k) compute P_i = A[i][k] V_k^T (to Pbuf, and transposed into Q's
-// columns of block i); blocks [2k, 2(nblk-1)) scale row k: A[k][j] <- V_k A[k][j] for j > k
-// (in place: these are final entries of U) with a copy in Q's columns of block j.
-// Q is 128 x cp: the right-hand operand of the step's update for every block column.
+// Step k, panel.  Blocks [0, 4k): 64 x 64 tiles of P_i = A[i][k] V_k^T (to Pbuf, and transposed
+// into Q's columns of block i).  Blocks [4k, 4(nblk-1)): 128 x 32 tiles of the row scaling
+// A[k][j] <- V_k A[k][j] for j > k (in place: these are final entries of U) with a copy in Q's
+// columns of block j.  Q is 128 x cp: the right-hand operand of the step's update for every
+// block column.
 __global__ void __launch_bounds__(GEMM_THREADS, 2)
-panel_kernel(double* __restrict__ A, int64_t cp, int k, const double* __restrict__ VT, double* __restrict__ Pbuf,
-             double* __restrict__ Q) {
+panel_kernel(double* __restrict__ A, int64_t cp, int k, double* __restrict__ Pbuf, double* __restrict__ Q) {
     extern __shared__ double smem[];
-    const int t = blockIdx.x >> 1, h = blockIdx.x & 1;
+    const int t = blockIdx.x >> 2, q = blockIdx.x & 3;
+    const double* Vk = A + (int64_t)k * NB * cp + (int64_t)k * NB;
     TileOut o = {};
     if (t < k) {
-        const int i = t;
-        o.C = Pbuf + (int64_t)i * NB * NB + h * TN; o.ldc = NB;
-        o.Ct = Q + (int64_t)(h * TN) * cp + (int64_t)i * NB; o.ldct = cp;
-        gemm_tile(A + (int64_t)i * NB * cp + (int64_t)k * NB, cp, VT + h * TN, NB, 1.0, 0.0, o, smem);
+        const int i = t, mh = q >> 1, h = q & 1;
+        o.C = Pbuf + (int64_t)i * NB * NB + (int64_t)(mh * 64) * NB + h * 64; o.ldc = NB;
+        o.Ct = Q + (int64_t)(h * 64) * cp + (int64_t)i * NB + mh * 64; o.ldct = cp;
+        gemm_tile<2, 4, true>(A + ((int64_t)i * NB + mh * 64) * cp + (int64_t)k * NB, cp, Vk + (int64_t)(h * 64) * cp, cp, 1.0,
+                              0.0, o, smem);
     } else {
         const int j = t + 1;
-        double* row = A + (int64_t)k * NB * cp + (int64_t)j * NB + h * TN;
+        double* row = A + (int64_t)k * NB * cp + (int64_t)j * NB + q * 32;
         o.C = row; o.ldc = cp;
-        o.C2 = Q + (int64_t)j * NB + h * TN; o.ldc2 = cp;
-        gemm_tile(A + (int64_t)k * NB * cp + (int64_t)k * NB, cp, row, cp, 1.0, 0.0, o, smem);
+        o.C2 = Q + (int64_t)j * NB + q * 32; o.ldc2 = cp;
+        gemm_tile<2, 8, false>(Vk, cp, row, cp, 1.0, 0.0, o, smem);
     }
 }
 
 // Step k, update of block rows i < k over the whole width.  The tiles of block column k-1 and
 // of block row k-1 are all that step k-1's diagonal and panel kernels read, so they can be
 // updated first ("next") and the remainder ("rest") left to run beside step k-1:
-//   part 0: everything, grid 2 nblk x k;  part 2: the rest, same grid;
-//   part 1: next only, grid 2 nblk x 1 -- tile t < k is (t, k-1), tile t >= k is (k-1, t).
+//   part 0: everything, grid 2 nblk x k, 128 x 64 tiles;  part 2: the rest, same grid;
+//   part 1: next only, grid 4 nblk x 1, 64 x 64 tiles -- block tile t < k is (t, k-1),
+//           t >= k is (k-1, t).
 __global__ void __launch_bounds__(GEMM_THREADS, 2)
 update_kernel(double* __restrict__ A, int64_t cp, int k, int part, const double* __restrict__ Pbuf,
               const double* __restrict__ Q) {
     extern __shared__ double smem[];
-    const int h = blockIdx.x & 1;
-    int i, j;
+    int i, j, r0, c0;
     if (part == 1) {
-        const int t = blockIdx.x >> 1;
+        const int t = blockIdx.x >> 2;
         if (t < k) { i = t; j = k - 1; } else { i = k - 1; j = t; }
+        r0 = ((blockIdx.x >> 1) & 1) * 64;
+        c0 = (blockIdx.x & 1) * 64;
     } else {
         j = blockIdx.x >> 1;
         i = blockIdx.y;
         if (part == 2 && (j == k - 1 || i == k - 1)) return;
+        r0 = 0;
+        c0 = (blockIdx.x & 1) * 64;
     }
     if (j < i) return;                                  // strictly lower tiles of the symmetric part
-    const double* Pi = Pbuf + (int64_t)i * NB * NB;
+    const double* Pi = Pbuf + (int64_t)i * NB * NB + (int64_t)r0 * NB;
     TileOut o = {};
-    o.C = A + (int64_t)i * NB * cp + (int64_t)j * NB + h * TN; o.ldc = cp;
-    if (j == k)     // A[i][k] = -P_i V_k
-        gemm_tile(Pi, NB, A + (int64_t)k * NB * cp + (int64_t)k * NB + h * TN, cp, -1.0, 0.0, o, smem);
-    else            // A[i][j] -= P_i Q[:, j]
-        gemm_tile(Pi, NB, Q + (int64_t)j * NB + h * TN, cp, -1.0, 1.0, o, smem);
+    o.C = A + ((int64_t)i * NB + r0) * cp + (int64_t)j * NB + c0; o.ldc = cp;
+    // A[i][k] = -P_i V_k;  A[i][j] -= P_i Q[:, j] otherwise
+    const double* Bsrc = (j == k) ? A + (int64_t)k * NB * cp + (int64_t)k * NB + c0 : Q + (int64_t)j * NB + c0;
+    const double beta = (j == k) ? 0.0 : 1.0;
+    if (part == 1) gemm_tile<2, 4, false>(Pi, NB, Bsrc, cp, -1.0, beta, o, smem);
+    else gemm_tile<4, 4, false>(Pi, NB, Bsrc, cp, -1.0, beta, o, smem);
 }
 
 // --------------------------------------------------------- diagonal block kernel ----
 // In place on the 128 x 128 diagonal block k of A: reads its upper triangle (symmetric positive
 // definite), computes the upper R with block = R R^T and writes V = R^-1 (upper, zeros below)
-// back, plus V^T to VT.  One CTA of 256 threads.  The block is handled as 4 x 4 sub-blocks of
+// back.  One CTA of 256 threads.  The block is handled as 4 x 4 sub-blocks of
 // 32 with the same sweep as the outer algorithm: warp 0 factorises and inverts a 32 x 32
 // diagonal sub-block in registers (one row per lane), then all warps do the panel, update and
 // scaling products with the FP64 MMA out of shared memory.
@@ -329,8 +354,7 @@ __device__ __forceinline__ void patch16(const double* Ap, int lda, const double*
 }
 
 __global__ void __launch_bounds__(DIAG_THREADS, 1)
-diag_block_kernel(double* __restrict__ A, int64_t cp, int64_t blk, int64_t c_real, double* __restrict__ VT,
-                  lq_dev_status* st) {
+diag_block_kernel(double* __restrict__ A, int64_t cp, int64_t blk, int64_t c_real, lq_dev_status* st) {
     extern __shared__ double sm[];
     double* S = sm;                       // NB x DP
     double* Pb = S + NB * DP;             // (NB - SB) x PP
@@ -343,10 +367,10 @@ diag_block_kernel(double* __restrict__ A, int64_t cp, int64_t blk, int64_t c_rea
 
     for (int idx = tid; idx < NB * (NB / 2); idx += DIAG_THREADS) {
         const int row = idx >> 6, c2 = (idx & 63) * 2;
-        const double2 v = *reinterpret_cast<const double2*>(base + (int64_t)row * cp + c2);
-        S[row * DP + c2] = v.x;
-        S[row * DP + c2 + 1] = v.y;
+        cp_async16(S + row * DP + c2, base + (int64_t)row * cp + c2);
     }
+    cp_async_commit();
+    cp_async_wait<0>();
     __syncthreads();
 
 #pragma unroll 1
@@ -428,13 +452,12 @@ diag_block_kernel(double* __restrict__ A, int64_t cp, int64_t blk, int64_t c_rea
         __syncthreads();
     }
 
-    for (int idx = tid; idx < NB * NB; idx += DIAG_THREADS) {
-        const int row = idx >> 7, col = idx & 127;
-        base[(int64_t)row * cp + col] = (col >= row) ? S[row * DP + col] : 0.0;
-    }
-    for (int idx = tid; idx < NB * NB; idx += DIAG_THREADS) {
-        const int col = idx >> 7, row = idx & 127;                           // VT[col][row] = V[row][col]
-        VT[col * NB + row] = (col >= row) ? S[row * DP + col] : 0.0;
+    for (int idx = tid; idx < NB * (NB / 2); idx += DIAG_THREADS) {
+        const int row = idx >> 6, c2 = (idx & 63) * 2;
+        double2 v;
+        v.x = (c2 >= row) ? S[row * DP + c2] : 0.0;
+        v.y = (c2 + 1 >= row) ? S[row * DP + c2 + 1] : 0.0;
+        *reinterpret_cast<double2*>(base + (int64_t)row * cp + c2) = v;
     }
 }
 
@@ -468,7 +491,7 @@ finalize_kernel(const double* __restrict__ A, int64_t cp, int64_t c, float* __re
 
 struct PrepLayout {
     int64_t nblk, cp;
-    size_t scal, a, pbuf, q, vt, total, panel_bytes;
+    size_t scal, a, pbuf, q, total, panel_bytes;
 };
 PrepLayout prep_layout(int64_t c) {
     PrepLayout L;
@@ -480,7 +503,6 @@ PrepLayout prep_layout(int64_t c) {
     L.panel_bytes = lq_align_up(static_cast<size_t>(L.cp) * NB * sizeof(double), 256);
     L.pbuf = off; off += 2 * L.panel_bytes;            // P and Q are double-buffered: one step's
     L.q = off;    off += 2 * L.panel_bytes;            // update may still read them while the next is written
-    L.vt = off;   off += lq_align_up(static_cast<size_t>(NB) * NB * sizeof(double), 256);
     L.total = off;
     return L;
 }
@@ -508,7 +530,6 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
     char* wsp = static_cast<char*>(ws);
     double* scal = reinterpret_cast<double*>(wsp + L.scal);
     double* A = reinterpret_cast<double*>(wsp + L.a);
-    double* VT = reinterpret_cast<double*>(wsp + L.vt);
 
     static bool attr_set = false;
     if (!attr_set) {
@@ -547,11 +568,10 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
     for (int64_t k = nblk - 1; k >= 0; --k) {
         double* Pk = reinterpret_cast<double*>(wsp + L.pbuf + (k & 1) * L.panel_bytes);
         double* Qk = reinterpret_cast<double*>(wsp + L.q + (k & 1) * L.panel_bytes);
-        diag_block_kernel<<<1, DIAG_THREADS, DIAG_SMEM, st>>>(A, cp, k, c, VT, h->dstatus);
+        diag_block_kernel<<<1, DIAG_THREADS, DIAG_SMEM, st>>>(A, cp, k, c, h->dstatus);
         LQ_LAUNCH_CHECK();
         if (nblk > 1) {
-            panel_kernel<<<static_cast<unsigned>(2 * (nblk - 1)), GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, static_cast<int>(k), VT,
-                                                                                                Pk, Qk);
+            panel_kernel<<<static_cast<unsigned>(4 * (nblk - 1)), GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, static_cast<int>(k), Pk, Qk);
             LQ_LAUNCH_CHECK();
         }
         if (k == 0) break;
@@ -562,7 +582,7 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
             continue;
         }
         if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_rest, 0));     // step k+1's rest touched the same tiles
-        update_kernel<<<static_cast<unsigned>(2 * nblk), GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, static_cast<int>(k), 1, Pk, Qk);
+        update_kernel<<<static_cast<unsigned>(4 * nblk), GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, static_cast<int>(k), 1, Pk, Qk);
         LQ_LAUNCH_CHECK();
         rest_pending = false;
         if (k > 1) {
