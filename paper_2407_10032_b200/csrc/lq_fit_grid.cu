@@ -95,11 +95,43 @@ __device__ __forceinline__ double dd_diff(dd a, dd b) {       // a - b, rounded 
     e = __dadd_rn(e, __dsub_rn(a.lo, b.lo));
     return __dadd_rn(s, e);
 }
+// Sort keys: the order-preserving bits of the weight above the column index.  bf16 rows fit a
+// 32-bit key (16 + 16 bits), fp32 rows take 64 bits (32 + 32).
+template <typename T> struct KeyOf;
+template <> struct KeyOf<__nv_bfloat16> {
+    typedef uint32_t type;
+    static __device__ __forceinline__ type make(__nv_bfloat16 w, int i) {
+        uint32_t u = __bfloat16_as_ushort(w);
+        u ^= (u & 0x8000u) ? 0xffffu : 0x8000u;
+        return (u << 16) | static_cast<uint32_t>(i);
+    }
+    static __device__ __forceinline__ type pad() { return 0xffffffffu; }
+};
+template <> struct KeyOf<float> {
+    typedef unsigned long long type;
+    static __device__ __forceinline__ type make(float w, int i) {
+        uint32_t u = __float_as_uint(w);
+        u ^= (u & 0x80000000u) ? 0xffffffffu : 0x80000000u;
+        return (static_cast<unsigned long long>(u) << 32) | static_cast<uint32_t>(i);
+    }
+    static __device__ __forceinline__ type pad() { return ~0ull; }
+};
 __device__ __forceinline__ float key_weight(unsigned long long key) {
     uint32_t u = static_cast<uint32_t>(key >> 32);
     u ^= (u & 0x80000000u) ? 0x80000000u : 0xffffffffu;
     return __uint_as_float(u);
 }
+__device__ __forceinline__ float key_weight(uint32_t key) {
+    uint32_t u = key >> 16;
+    u ^= (u & 0x8000u) ? 0x8000u : 0xffffu;
+    return __uint_as_float(u << 16);
+}
+__device__ __forceinline__ uint32_t key_index(unsigned long long key) { return static_cast<uint32_t>(key); }
+__device__ __forceinline__ uint32_t key_index(uint32_t key) { return key & 0xffffu; }
+
+// Shared-memory slot of sorted position i: one pad slot per 32, so that the strided accesses of
+// the register-blocked sort spread over the banks.
+__device__ __forceinline__ int ks_slot(int i) { return i + (i >> 5); }
 
 constexpr int KS_THREADS = 256;
 constexpr int KS_CHUNK = 8;
@@ -107,12 +139,82 @@ constexpr int KS_MAX_N = 16384;        // rows up to this length are sorted in s
 
 struct dd2 { dd s, sw; };              // prefix of the sample weights and of s * w
 
+// Compare-exchange sub-stages of a bitonic network on 16 keys held in registers: sub-stage s
+// pairs registers that differ in bit s of their number; NST sub-stages, highest bit first.
+template <typename KeyT, int NST>
+__device__ __forceinline__ void ce_stages(KeyT (&e)[16], bool up) {
+#pragma unroll
+    for (int s = NST - 1; s >= 0; --s) {
+#pragma unroll
+        for (int m = 0; m < 16; ++m) {
+            if ((m >> s) & 1) continue;
+            const KeyT a = e[m], b = e[m | (1 << s)];
+            const KeyT lo = a < b ? a : b, hi = a < b ? b : a;
+            e[m] = up ? lo : hi;
+            e[m | (1 << s)] = up ? hi : lo;
+        }
+    }
+}
+
+// Ascending bitonic sort of n keys (a power of two >= 64) in shared memory.  Every pass through
+// shared memory moves 16 keys per thread into registers and runs up to four sub-stages there.
+template <typename KeyT>
+__device__ __forceinline__ void bitonic_sort(KeyT* keys, int n, int tid) {
+    const int logn = 31 - __clz(n);
+    // levels k = 2, 4, 8, 16 on 16 consecutive keys
+    for (int vt = tid; vt < (n >> 4); vt += KS_THREADS) {
+        KeyT e[16];
+#pragma unroll
+        for (int m = 0; m < 16; ++m) e[m] = keys[ks_slot(16 * vt + m)];
+#pragma unroll
+        for (int lk = 1; lk <= 4; ++lk) {
+#pragma unroll
+            for (int s = lk - 1; s >= 0; --s) {
+#pragma unroll
+                for (int m = 0; m < 16; ++m) {
+                    if ((m >> s) & 1) continue;
+                    const bool up = lk < 4 ? ((m >> lk) & 1) == 0 : (vt & 1) == 0;
+                    const KeyT a = e[m], b = e[m | (1 << s)];
+                    const KeyT lo = a < b ? a : b, hi = a < b ? b : a;
+                    e[m] = up ? lo : hi;
+                    e[m | (1 << s)] = up ? hi : lo;
+                }
+            }
+        }
+#pragma unroll
+        for (int m = 0; m < 16; ++m) keys[ks_slot(16 * vt + m)] = e[m];
+    }
+    __syncthreads();
+    for (int L = 5; L <= logn; ++L) {                 // level k = 2^L: sub-stages j = 2^(L-1) .. 1
+        for (int bhi = L - 1; bhi >= 0; bhi -= 4) {
+            const int lo = bhi >= 3 ? bhi - 3 : 0;
+            const int nst = bhi - lo + 1;
+            for (int vt = tid; vt < (n >> 4); vt += KS_THREADS) {
+                const int base = ((vt >> lo) << (lo + 4)) | (vt & ((1 << lo) - 1));
+                const bool up = ((base >> L) & 1) == 0;
+                KeyT e[16];
+#pragma unroll
+                for (int m = 0; m < 16; ++m) e[m] = keys[ks_slot(base | (m << lo))];
+                if (nst == 4) ce_stages<KeyT, 4>(e, up);
+                else if (nst == 3) ce_stages<KeyT, 3>(e, up);
+                else if (nst == 2) ce_stages<KeyT, 2>(e, up);
+                else ce_stages<KeyT, 1>(e, up);
+#pragma unroll
+                for (int m = 0; m < 16; ++m) keys[ks_slot(base | (m << lo))] = e[m];
+            }
+            __syncthreads();
+        }
+    }
+}
+
 template <int K, typename T>
 __global__ void __launch_bounds__(KS_THREADS, 4)
 kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int n, const double* __restrict__ s64,
                      float* __restrict__ grid, int n_iter) {
-    extern __shared__ unsigned long long keys[];               // n keys, then n / 8 + 1 coarse prefixes
-    dd2* coarse = reinterpret_cast<dd2*>(keys + n);
+    typedef typename KeyOf<T>::type KeyT;
+    extern __shared__ __align__(16) unsigned char ks_smem[];
+    dd2* coarse = reinterpret_cast<dd2*>(ks_smem);            // n / 8 + 1 coarse prefixes, then the n keys (padded slots)
+    KeyT* keys = reinterpret_cast<KeyT*>(coarse + (n / KS_CHUNK + 1));
     __shared__ dd2 tot[KS_THREADS];                            // per-thread totals, then their exclusive scan
     __shared__ double g[K];
     __shared__ dd2 F[K + 1];
@@ -122,29 +224,9 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
 
     for (int64_t row = blockIdx.x; row < r; row += gridDim.x) {
         const T* wp = W + row * ldw;
-        for (int i = tid; i < n; i += KS_THREADS) {
-            unsigned long long key = ~0ull;
-            if (i < c) {
-                uint32_t u = __float_as_uint(load_w(wp + i));
-                u ^= (u & 0x80000000u) ? 0xffffffffu : 0x80000000u;
-                key = (static_cast<unsigned long long>(u) << 32) | static_cast<uint32_t>(i);
-            }
-            keys[i] = key;
-        }
+        for (int i = tid; i < n; i += KS_THREADS) keys[ks_slot(i)] = i < c ? KeyOf<T>::make(wp[i], i) : KeyOf<T>::pad();
         __syncthreads();
-        // bitonic sort, ascending
-        for (int k = 2; k <= n; k <<= 1) {
-            for (int j = k >> 1; j > 0; j >>= 1) {
-                for (int t = tid; t < (n >> 1); t += KS_THREADS) {
-                    const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
-                    const int l = i | j;
-                    const unsigned long long a = keys[i], b = keys[l];
-                    const bool up = (i & k) == 0;
-                    if ((a > b) == up) { keys[i] = b; keys[l] = a; }
-                }
-                __syncthreads();
-            }
-        }
+        bitonic_sort<KeyT>(keys, n, tid);
         // chunk totals, thread-local exclusive prefixes
         dd2 run;
         run.s.hi = run.s.lo = run.sw.hi = run.sw.lo = 0.0;
@@ -154,8 +236,8 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
             for (int e = 0; e < KS_CHUNK; ++e) {
                 const int i = q * KS_CHUNK + e;
                 if (i < c) {
-                    const unsigned long long key = keys[i];
-                    const double sv = s64[static_cast<uint32_t>(key)];
+                    const KeyT key = keys[ks_slot(i)];
+                    const double sv = s64[key_index(key)];
                     run.s = dd_add_d(run.s, sv);                 // same order and arithmetic as F(b) below
                     run.sw = dd_add_d(run.sw, __dmul_rn(sv, static_cast<double>(key_weight(key))));
                 }
@@ -212,27 +294,35 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
         __syncthreads();
 
         if (warp == 0) {
-            const double lo = static_cast<double>(key_weight(keys[0]));
-            const double hi = static_cast<double>(key_weight(keys[c - 1]));
+            const double lo = static_cast<double>(key_weight(keys[ks_slot(0)]));
+            const double hi = static_cast<double>(key_weight(keys[ks_slot(c - 1)]));
             if (lane < K) g[lane] = lo + (hi - lo) * static_cast<double>(lane) / static_cast<double>(K - 1);   // Eq. 6
             if (lane == 0) {
                 F[0].s.hi = F[0].s.lo = F[0].sw.hi = F[0].sw.lo = 0.0;
                 F[K] = coarse[nch];
             }
             __syncwarp();
+            int b_prev = -1;
             for (int it = 0; it < n_iter; ++it) {
+                int b0 = 0;
                 if (lane < K - 1) {
                     const double m = 0.5 * (g[lane] + g[lane + 1]);
-                    int b0 = 0, b1 = c;                        // first position whose weight exceeds m
+                    int b1 = c;                                // first position whose weight exceeds m
                     while (b0 < b1) {
                         const int mid = (b0 + b1) >> 1;
-                        if (static_cast<double>(key_weight(keys[mid])) > m) b1 = mid; else b0 = mid + 1;
+                        if (static_cast<double>(key_weight(keys[ks_slot(mid)])) > m) b1 = mid; else b0 = mid + 1;
                     }
+                }
+                // Unchanged boundaries give back the same centroids, and so would every later
+                // iteration: the fixed point has been reached and the remaining iterations are skipped.
+                if (__all_sync(0xffffffffu, b0 == b_prev)) break;
+                b_prev = b0;
+                if (lane < K - 1) {
                     const int q = b0 / KS_CHUNK, rem = b0 % KS_CHUNK;
                     dd2 f = coarse[q];
                     for (int e = 0; e < rem; ++e) {
-                        const unsigned long long key = keys[q * KS_CHUNK + e];
-                        const double sv = s64[static_cast<uint32_t>(key)];
+                        const KeyT key = keys[ks_slot(q * KS_CHUNK + e)];
+                        const double sv = s64[key_index(key)];
                         f.s = dd_add_d(f.s, sv);
                         f.sw = dd_add_d(f.sw, __dmul_rn(sv, static_cast<double>(key_weight(key))));
                     }
@@ -343,7 +433,8 @@ int launch_kmeans(cudaStream_t st, int sms, const T* W, int64_t ldw, int64_t r, 
     if (c <= KS_MAX_N) {
         int n = 64;
         while (n < c) n <<= 1;
-        const size_t smem = static_cast<size_t>(n) * 8 + (static_cast<size_t>(n) / KS_CHUNK + 1) * sizeof(dd2);
+        const size_t smem = (static_cast<size_t>(n) / KS_CHUNK + 1) * sizeof(dd2) +
+                            static_cast<size_t>(n + n / 32) * sizeof(typename KeyOf<T>::type);
         static bool attr_set = false;
         if (!attr_set) {
             LQ_CUDA_TRY(cudaFuncSetAttribute(kmeans_sorted_kernel<K, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
