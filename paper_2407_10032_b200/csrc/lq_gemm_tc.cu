@@ -6,7 +6,8 @@
 // the column loop (Algorithm 1 line 20).  fp32 operands are fed as several bf16 passes
 // (hi/mid/lo terms), which is what n_pass > 1 is for.
 //
-// One persistent CTA per SM, 128 x 256 output tiles, K consumed 64 at a time.
+// One persistent CTA per SM, 128 x 256 output tiles, K consumed 64 at a time; K may be cut into
+// a few parts so that the schedule's last round is short (see next_piece).
 //   warp 0      : TMA producer (cp.async.bulk.tensor, 128-byte swizzle, 4-stage ring)
 //   warp 1      : issues tcgen05.mma (one thread), accumulators in TMEM (2 x 256 columns,
 //                 so the epilogue of one tile overlaps the main loop of the next)
@@ -50,6 +51,9 @@ struct KParams {
     int tiles_m, tiles_n;
     int num_tiles;
     int seg_iters;            // k-iterations accumulated in TMEM before the partial sum is flushed to D
+    int segs_per_tile;        // ceil(k_iters / seg_iters)
+    int k_parts;              // K is cut into this many parts (<= segs_per_tile)
+    long long total_units;    // num_tiles * k_parts work units, dealt round-robin to the CTAs
     lq_dev_status* status;
     unsigned long long timeout_ns;
 };
@@ -187,6 +191,23 @@ __device__ __forceinline__ void tile_coords(const KParams& p, int idx, int& tm, 
     }
 }
 
+// When the tile count is not a multiple of the CTA count, whole tiles leave some SMs idle in the
+// last round.  K is therefore cut into k_parts equal parts and the launch's work becomes the
+// list of (part, tile) units in part-major order, dealt round-robin to the CTAs: rounds are
+// 1 / k_parts of a tile long, so the idle tail shrinks with them, and at any moment all CTAs
+// still read about the same columns of the operands (they share them through the L2).  A unit
+// leaves a partial sum over its part of K, which is fine because results are added into D.
+struct Piece { int tile, s0, s1; };       // segments [s0, s1) of a tile
+__device__ __forceinline__ bool next_piece(const KParams& p, long long& u, Piece& pc) {
+    if (u >= p.total_units) return false;
+    const int part = static_cast<int>(u / p.num_tiles);
+    pc.tile = static_cast<int>(u - static_cast<long long>(part) * p.num_tiles);
+    pc.s0 = static_cast<int>(static_cast<long long>(p.segs_per_tile) * part / p.k_parts);
+    pc.s1 = static_cast<int>(static_cast<long long>(p.segs_per_tile) * (part + 1) / p.k_parts);
+    u += gridDim.x;
+    return true;
+}
+
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ CUtensorMap map_d, const __grid_constant__ KParams p) {
@@ -232,16 +253,20 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 
     const int k_blocks = (p.K + BK - 1) / BK;
     const int k_iters = k_blocks * p.n_pass;
+    const long long u_begin = blockIdx.x;
 
     if (warp_idx == 0) {
         // ------------------------------------------------------------ TMA producer
         uint32_t stage = 0, phase = 0;
         bool alive = true;
-        for (int t = blockIdx.x; t < p.num_tiles && alive; t += gridDim.x) {
+        long long u = u_begin;
+        Piece pc;
+        while (alive && next_piece(p, u, pc)) {
             int tm, tn;
-            tile_coords(p, t, tm, tn);
+            tile_coords(p, pc.tile, tm, tn);
             const int m0 = tm * BM, n0 = tn * BN;
-            for (int kit = 0; kit < k_iters; ++kit) {       // segments only matter to the consumers
+            const int kit_end = min(k_iters, pc.s1 * p.seg_iters);
+            for (int kit = pc.s0 * p.seg_iters; kit < kit_end; ++kit) {       // segments only matter to the consumers
                 if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abortp, p, 1)) { alive = false; break; }
                 if (lane == 0) {
                     const int pass = kit / k_blocks;
@@ -261,8 +286,11 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         uint32_t stage = 0, phase = 0;
         int it = 0;                                  // counts (tile, segment) units: one TMEM accumulator each
         bool alive = true;
-        for (int t = blockIdx.x; t < p.num_tiles && alive; t += gridDim.x) {
-            for (int k_lo = 0; k_lo < k_iters && alive; k_lo += p.seg_iters, ++it) {
+        long long u = u_begin;
+        Piece pc;
+        while (alive && next_piece(p, u, pc)) {
+            const int piece_end = min(k_iters, pc.s1 * p.seg_iters);
+            for (int k_lo = pc.s0 * p.seg_iters; k_lo < piece_end && alive; k_lo += p.seg_iters, ++it) {
                 const int k_hi = min(k_iters, k_lo + p.seg_iters);
                 const uint32_t acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
@@ -306,11 +334,14 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         float accr[BN / 2];
         int it = 0;
         bool alive = true;
-        for (int t = blockIdx.x; t < p.num_tiles && alive; t += gridDim.x) {
+        long long u = u_begin;
+        Piece pc;
+        while (alive && next_piece(p, u, pc)) {
             int tm, tn;
-            tile_coords(p, t, tm, tn);
+            tile_coords(p, pc.tile, tm, tn);
             const int m0 = tm * BM, n0 = tn * BN;
-            for (int k_lo = 0; k_lo < k_iters; k_lo += p.seg_iters, ++it) {
+            const int piece_lo = pc.s0 * p.seg_iters, piece_end = min(k_iters, pc.s1 * p.seg_iters);
+            for (int k_lo = piece_lo; k_lo < piece_end; k_lo += p.seg_iters, ++it) {
                 const uint32_t acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
                 if (!mbar_wait(bar_tfull + 8 * acc, acc_phase, abortp, p, 4)) { alive = false; break; }
@@ -320,7 +351,7 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     uint32_t v[32];
                     tmem_ld32(tmem_base + ((q * 32u) << 16) + acc * BN + hf * (BN / 2) + ch * EPI_COLS, v);
                     tmem_wait_ld();
-                    if (k_lo == 0) {
+                    if (k_lo == piece_lo) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) accr[ch * 32 + i] = __uint_as_float(v[i]);
                     } else {
@@ -463,9 +494,21 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
     {
         const int k_iters = static_cast<int>(lq_ceil_div(a.K, BK)) * a.n_pass;
         p.seg_iters = (a.seg_iters > 0 && a.seg_iters < k_iters) ? a.seg_iters : k_iters;
+        p.segs_per_tile = static_cast<int>(lq_ceil_div(k_iters, p.seg_iters));
     }
+    // number of K parts: the one that leaves the shortest schedule, ceil(tiles * q / CTAs) / q
+    const int ctas = h->sm_count;
+    p.k_parts = 1;
+    if (a.accumulate && p.num_tiles > ctas) {
+        double best = static_cast<double>(lq_ceil_div(p.num_tiles, ctas));
+        for (int q = 2; q <= 8 && q <= p.segs_per_tile; ++q) {
+            const double t = static_cast<double>(lq_ceil_div(static_cast<int64_t>(p.num_tiles) * q, ctas)) / q;
+            if (t < best * 0.98) { best = t; p.k_parts = q; }
+        }
+    }
+    p.total_units = static_cast<long long>(p.num_tiles) * p.k_parts;
 
-    int grid = p.num_tiles < h->sm_count ? p.num_tiles : h->sm_count;
+    const int grid = p.total_units < ctas ? static_cast<int>(p.total_units) : ctas;
     lq_tc_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, map_d, p);
     LQ_LAUNCH_CHECK();
     return LQ_OK;
