@@ -499,7 +499,7 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
     // number of K parts: the one that leaves the shortest schedule, ceil(tiles * q / CTAs) / q
     const int ctas = h->sm_count;
     p.k_parts = 1;
-    if (a.accumulate && p.num_tiles > ctas) {
+    if (a.accumulate && p.segs_per_tile >= 16) {          // long K only: every unit pays one epilogue
         double best = static_cast<double>(lq_ceil_div(p.num_tiles, ctas));
         for (int q = 2; q <= 8 && q <= p.segs_per_tile; ++q) {
             const double t = static_cast<double>(lq_ceil_div(static_cast<int64_t>(p.num_tiles) * q, ctas)) / q;
