@@ -6,16 +6,22 @@
 // the column loop (Algorithm 1 line 20).  fp32 operands are fed as several bf16 passes
 // (hi/mid/lo terms), which is what n_pass > 1 is for.
 //
-// One persistent CTA per SM, 128 x 256 output tiles, K consumed 64 at a time; K may be cut into
-// a few parts so that the schedule's last round is short (see next_piece).
-//   warp 0      : TMA producer (cp.async.bulk.tensor, 128-byte swizzle, 4-stage ring)
+// One persistent CTA per SM, K consumed 64 at a time; K may be cut into a few parts so that the
+// schedule's last round is short (see next_piece).  Two forms of the same kernel:
+//   CTAS = 1 : one CTA computes a 128 x 256 tile (tcgen05 cta_group::1);
+//   CTAS = 2 : a cluster of two CTAs computes a 256 x 256 tile with the two-SM MMA form
+//              (cta_group::2): each CTA loads its own 128 rows of A and only its half of B, so
+//              the shared-memory traffic per flop drops by a third; the even CTA of the pair
+//              issues the MMAs for both, each CTA drains its own 128 x 256 accumulator.
+//   warp 0      : TMA producer (cp.async.bulk.tensor, 128-byte swizzle, ring of stages)
 //   warp 1      : issues tcgen05.mma (one thread), accumulators in TMEM (2 x 256 columns,
-//                 so the epilogue of one tile overlaps the main loop of the next)
+//                 so the epilogue of one segment overlaps the main loop of the next); in the
+//                 odd CTA of a pair it idles (both CTAs' loads complete on the even CTA's barrier)
 //   warps 2..9  : epilogue.  The tensor core adds into its fp32 accumulator with truncation,
 //                 which over a long K biases every sum low; so K is consumed in short
 //                 segments, and after each one these warps tcgen05.ld the partial sum and
 //                 add it (round-to-nearest) to running sums held in registers.  After the
-//                 tile's last segment: scale -> swizzled smem slab -> TMA store, or a TMA
+//                 piece's last segment: scale -> swizzled smem slab -> TMA store, or a TMA
 //                 reduce-add when accumulating into D (no read of D by the SM).
 // Every wait on an mbarrier is bounded: when the time limit passes the CTA records
 // LQ_ERR_TIMEOUT in the handle's status word, stops issuing work and leaves.
@@ -25,20 +31,28 @@
 
 namespace {
 
-constexpr int BM = 128;
-constexpr int BN = 256;
+constexpr int BM = 128;                // rows of A (and of the accumulator) per CTA
+constexpr int BN = 256;                // tile width
 constexpr int BK = 64;                 // 64 bf16 = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
-constexpr int STAGES = 4;
 constexpr int A_STAGE_BYTES = BM * BK * 2;
-constexpr int B_STAGE_BYTES = BN * BK * 2;
-constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
 constexpr int EPI_COLS = 32;           // 32 fp32 = 128 bytes = one swizzle row
 constexpr int EPI_BUF_BYTES = BM * EPI_COLS * 4;
 constexpr int EPI_BUFS = 2;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BUFS * EPI_BUF_BYTES + 1024;
 constexpr int NUM_THREADS = 320;
 constexpr int TMEM_COLS = 512;
+constexpr int MAX_STAGES = 6;
+
+template <int CTAS> struct Cfg {
+    static constexpr int B_ROWS = BN / CTAS;                     // rows of B a CTA loads
+    static constexpr int B_STAGE_BYTES = B_ROWS * BK * 2;
+    static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+    static constexpr int STAGES = CTAS == 1 ? 4 : 6;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BUFS * EPI_BUF_BYTES + 1024;
+    static constexpr int TILE_M = BM * CTAS;
+    // Instruction descriptor: D fp32, A and B bf16, both K-major, M = TILE_M, N = 256.
+    static constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(BN >> 3) << 17) | (uint32_t(TILE_M >> 4) << 24);
+};
 
 struct KParams {
     int M, N, K;
@@ -48,12 +62,13 @@ struct KParams {
     float alpha;
     int accumulate;
     int upper_only;
+    int tile_m;               // rows of a tile: 128 or 256
     int tiles_m, tiles_n;
     int num_tiles;
     int seg_iters;            // k-iterations accumulated in TMEM before the partial sum is flushed to D
     int segs_per_tile;        // ceil(k_iters / seg_iters)
     int k_parts;              // K is cut into this many parts (<= segs_per_tile)
-    long long total_units;    // num_tiles * k_parts work units, dealt round-robin to the CTAs
+    long long total_units;    // num_tiles * k_parts work units, dealt round-robin to the CTAs (or CTA pairs)
     lq_dev_status* status;
     unsigned long long timeout_ns;
 };
@@ -67,6 +82,15 @@ __device__ __forceinline__ unsigned long long global_timer() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
@@ -76,6 +100,13 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
+// Arrive on the barrier at the same shared-memory offset in CTA `rank` of this cluster.
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t rank) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(bar), "r"(rank));
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
+}
+template <bool CLUSTER>
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -86,13 +117,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).
+template <bool CLUSTER>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           const KParams& p, int where) {
-    if (mbar_try_wait(bar, parity)) return true;
+    if (mbar_try_wait<CLUSTER>(bar, parity)) return true;
     const unsigned long long t0 = global_timer();
     uint32_t spins = 0;
     for (;;) {
-        if (mbar_try_wait(bar, parity)) return true;
+        if (mbar_try_wait<CLUSTER>(bar, parity)) return true;
         if ((++spins & 63u) == 0u) {
             if (*abort_flag) return false;
             if (global_timer() - t0 > p.timeout_ns) {
@@ -107,6 +139,18 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+// The same load issued by either CTA of a pair, completing on a barrier given as a cluster address
+// (the even CTA's): the two-CTA form of the instruction allows the barrier to live in the peer.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ uint32_t cluster_addr(uint32_t addr, uint32_t rank) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(addr), "r"(rank));
+    return remote;
 }
 __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1) {
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];"
@@ -126,23 +170,41 @@ template <int N> __device__ __forceinline__ void bulk_wait() {
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+template <int CTAS> __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols) {
+    if (CTAS == 1) asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+    else asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
 }
-__device__ __forceinline__ void tmem_relinquish() {
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+template <int CTAS> __device__ __forceinline__ void tmem_relinquish() {
+    if (CTAS == 1) asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    else asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+template <int CTAS> __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    if (CTAS == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+    else asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
+template <int CTAS>
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t acc) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(acc) : "memory");
+    if (CTAS == 1)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(acc) : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(acc) : "memory");
 }
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// The barrier is signalled when all MMAs issued so far by this thread have completed; with two
+// CTAs the signal goes to the barrier at this offset in both CTAs of the pair.
+template <int CTAS> __device__ __forceinline__ void umma_commit(uint32_t bar) {
+    if (CTAS == 1) {
+        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    } else {
+        const uint16_t mask = 3;
+        asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                     ::"r"(bar), "h"(mask) : "memory");
+    }
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
@@ -170,11 +232,8 @@ __device__ __forceinline__ uint64_t make_desc_sw128(uint32_t saddr) {
     return d;
 }
 
-// Instruction descriptor: D fp32, A and B bf16, both K-major, M = 128, N = 256.
-constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(BN >> 3) << 17) | (uint32_t(BM >> 4) << 24);
-
 // Map the idx-th scheduled tile to (tile row, tile column).  With upper_only, row tm keeps
-// the columns tn with (tn + 1) * BN > tm * BM.
+// the columns tn with (tn + 1) * BN > tm * tile_m.
 __device__ __forceinline__ void tile_coords(const KParams& p, int idx, int& tm, int& tn) {
     if (!p.upper_only) {
         tm = idx / p.tiles_n;
@@ -183,7 +242,7 @@ __device__ __forceinline__ void tile_coords(const KParams& p, int idx, int& tm, 
     }
     int m = 0;
     for (;; ++m) {
-        int first = (m * BM) / BN;
+        int first = (m * p.tile_m) / BN;
         int cnt = p.tiles_n - first;
         if (cnt < 0) cnt = 0;
         if (idx < cnt) { tm = m; tn = first + idx; return; }
@@ -193,41 +252,47 @@ __device__ __forceinline__ void tile_coords(const KParams& p, int idx, int& tm, 
 
 // When the tile count is not a multiple of the CTA count, whole tiles leave some SMs idle in the
 // last round.  K is therefore cut into k_parts equal parts and the launch's work becomes the
-// list of (part, tile) units in part-major order, dealt round-robin to the CTAs: rounds are
-// 1 / k_parts of a tile long, so the idle tail shrinks with them, and at any moment all CTAs
-// still read about the same columns of the operands (they share them through the L2).  A unit
-// leaves a partial sum over its part of K, which is fine because results are added into D.
+// list of (part, tile) units in part-major order, dealt round-robin to the CTAs (CTA pairs):
+// rounds are 1 / k_parts of a tile long, so the idle tail shrinks with them, and at any moment
+// all CTAs still read about the same columns of the operands (they share them through the L2).
+// A unit leaves a partial sum over its part of K, which is fine because results are added into D.
 struct Piece { int tile, s0, s1; };       // segments [s0, s1) of a tile
-__device__ __forceinline__ bool next_piece(const KParams& p, long long& u, Piece& pc) {
+__device__ __forceinline__ bool next_piece(const KParams& p, long long& u, long long stride, Piece& pc) {
     if (u >= p.total_units) return false;
     const int part = static_cast<int>(u / p.num_tiles);
     pc.tile = static_cast<int>(u - static_cast<long long>(part) * p.num_tiles);
     pc.s0 = static_cast<int>(static_cast<long long>(p.segs_per_tile) * part / p.k_parts);
     pc.s1 = static_cast<int>(static_cast<long long>(p.segs_per_tile) * (part + 1) / p.k_parts);
-    u += gridDim.x;
+    u += stride;
     return true;
 }
 
+template <int CTAS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ CUtensorMap map_d, const __grid_constant__ KParams p) {
+    typedef Cfg<CTAS> C;
+    constexpr int STAGES = C::STAGES;
+    constexpr bool PAIR = CTAS == 2;
     extern __shared__ uint8_t smem_raw[];
-    __shared__ __align__(8) uint64_t bars[2 * STAGES + 4];
+    __shared__ __align__(8) uint64_t bars[3 * MAX_STAGES + 4];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
     const uint32_t warp_idx = threadIdx.x >> 5;
     const uint32_t lane = threadIdx.x & 31;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;      // 0: issues the MMAs; 1: its peer
+    const bool mma_cta = rank == 0;
 
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-    const uint32_t epi_base = smem_base + STAGES * STAGE_BYTES;
-    uint8_t* epi_gen = smem_gen + STAGES * STAGE_BYTES;
+    const uint32_t epi_base = smem_base + STAGES * C::STAGE_BYTES;
+    uint8_t* epi_gen = smem_gen + STAGES * C::STAGE_BYTES;
 
-    const uint32_t bar_full = smem_u32(&bars[0]);
-    const uint32_t bar_empty = smem_u32(&bars[STAGES]);
-    const uint32_t bar_tfull = smem_u32(&bars[2 * STAGES]);
-    const uint32_t bar_tempty = smem_u32(&bars[2 * STAGES + 2]);
+    const uint32_t bar_full = smem_u32(&bars[0]);                      // the TMA loads of a stage have landed (pair: both CTAs', on the even CTA)
+    const uint32_t bar_empty = smem_u32(&bars[MAX_STAGES]);            // the MMAs that read a stage have completed
+    const uint32_t bar_tfull = smem_u32(&bars[3 * MAX_STAGES]);        // an accumulator holds a finished segment
+    const uint32_t bar_tempty = smem_u32(&bars[3 * MAX_STAGES + 2]);   // (even CTA) an accumulator has been drained
 
     if (threadIdx.x == 0) {
         abort_flag = 0;
@@ -237,23 +302,25 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(bar_tfull + 8 * a, 1);
-            mbar_init(bar_tempty + 8 * a, 8);
+            mbar_init(bar_tempty + 8 * a, 8 * CTAS);          // one arrival per epilogue warp of the pair
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp_idx == 1) {
-        tmem_alloc(smem_u32(&tmem_base_slot), TMEM_COLS);
-        tmem_relinquish();
+        tmem_alloc<CTAS>(smem_u32(&tmem_base_slot), TMEM_COLS);
+        tmem_relinquish<CTAS>();
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();           // the peer's barriers are initialised before anything arrives on them
     tc_fence_after();
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_base_slot);
     volatile int* abortp = &abort_flag;
 
     const int k_blocks = (p.K + BK - 1) / BK;
     const int k_iters = k_blocks * p.n_pass;
-    const long long u_begin = blockIdx.x;
+    const long long u_begin = blockIdx.x / CTAS;
+    const long long u_stride = gridDim.x / CTAS;
 
     if (warp_idx == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -261,73 +328,84 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         bool alive = true;
         long long u = u_begin;
         Piece pc;
-        while (alive && next_piece(p, u, pc)) {
+        while (alive && next_piece(p, u, u_stride, pc)) {
             int tm, tn;
             tile_coords(p, pc.tile, tm, tn);
-            const int m0 = tm * BM, n0 = tn * BN;
+            const int m0 = tm * C::TILE_M + static_cast<int>(rank) * BM;
+            const int n0 = tn * BN + static_cast<int>(rank) * C::B_ROWS;
             const int kit_end = min(k_iters, pc.s1 * p.seg_iters);
             for (int kit = pc.s0 * p.seg_iters; kit < kit_end; ++kit) {       // segments only matter to the consumers
-                if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abortp, p, 1)) { alive = false; break; }
+                if (!mbar_wait<PAIR>(bar_empty + 8 * stage, phase ^ 1u, abortp, p, 1)) { alive = false; break; }
                 if (lane == 0) {
                     const int pass = kit / k_blocks;
                     const int k0 = (kit - pass * k_blocks) * BK;
-                    const uint32_t sa = smem_base + stage * STAGE_BYTES;
+                    const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
                     const uint32_t sb = sa + A_STAGE_BYTES;
-                    mbar_arrive_expect_tx(bar_full + 8 * stage, STAGE_BYTES);
-                    tma_load_2d(sa, &map_a, bar_full + 8 * stage, k0, p.a_off[pass] + m0);
-                    tma_load_2d(sb, &map_b, bar_full + 8 * stage, k0, p.b_off[pass] + n0);
+                    if (!PAIR) {
+                        mbar_arrive_expect_tx(bar_full + 8 * stage, C::STAGE_BYTES);
+                        tma_load_2d(sa, &map_a, bar_full + 8 * stage, k0, p.a_off[pass] + m0);
+                        tma_load_2d(sb, &map_b, bar_full + 8 * stage, k0, p.b_off[pass] + n0);
+                    } else {
+                        // both CTAs' loads of a stage complete on the even CTA's barrier, which expects the bytes of both
+                        if (mma_cta) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * C::STAGE_BYTES);
+                        const uint32_t full0 = cluster_addr(bar_full + 8 * stage, 0);
+                        tma_load_2d_pair(sa, &map_a, full0, k0, p.a_off[pass] + m0);
+                        tma_load_2d_pair(sb, &map_b, full0, k0, p.b_off[pass] + n0);
+                    }
                 }
                 __syncwarp();
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
             }
         }
-    } else if (warp_idx == 1) {
+    } else if (warp_idx == 1 && mma_cta) {
         // ------------------------------------------------------------ MMA issuer
         uint32_t stage = 0, phase = 0;
-        int it = 0;                                  // counts (tile, segment) units: one TMEM accumulator each
+        int it = 0;                                  // counts segments: one TMEM accumulator each
         bool alive = true;
         long long u = u_begin;
         Piece pc;
-        while (alive && next_piece(p, u, pc)) {
+        while (alive && next_piece(p, u, u_stride, pc)) {
             const int piece_end = min(k_iters, pc.s1 * p.seg_iters);
             for (int k_lo = pc.s0 * p.seg_iters; k_lo < piece_end && alive; k_lo += p.seg_iters, ++it) {
                 const int k_hi = min(k_iters, k_lo + p.seg_iters);
                 const uint32_t acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
-                if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abortp, p, 2)) { alive = false; break; }
+                if (!mbar_wait<PAIR>(bar_tempty + 8 * acc, acc_phase ^ 1u, abortp, p, 2)) { alive = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + acc * BN;
                 for (int kit = k_lo; kit < k_hi; ++kit) {
-                    if (!mbar_wait(bar_full + 8 * stage, phase, abortp, p, 3)) { alive = false; break; }
+                    if (!mbar_wait<PAIR>(bar_full + 8 * stage, phase, abortp, p, 3)) { alive = false; break; }
                     tc_fence_after();
                     if (lane == 0) {
-                        const uint32_t sa = smem_base + stage * STAGE_BYTES;
+                        const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
                         const uint64_t da = make_desc_sw128(sa);
                         const uint64_t db = make_desc_sw128(sa + A_STAGE_BYTES);
 #pragma unroll
                         for (int kk = 0; kk < BK / UMMA_K; ++kk) {
                             // advancing 16 bf16 = 32 bytes inside the swizzle row: +2 in the address field
-                            umma_bf16(tmem_d, da + 2 * kk, db + 2 * kk, kInstrDesc, (kit > k_lo || kk > 0) ? 1u : 0u);
+                            umma_bf16<CTAS>(tmem_d, da + 2 * kk, db + 2 * kk, C::IDESC, (kit > k_lo || kk > 0) ? 1u : 0u);
                         }
-                        umma_commit(bar_empty + 8 * stage);
+                        umma_commit<CTAS>(bar_empty + 8 * stage);
                     }
                     __syncwarp();
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
                 if (!alive) break;
-                if (lane == 0) umma_commit(bar_tfull + 8 * acc);
+                if (lane == 0) umma_commit<CTAS>(bar_tfull + 8 * acc);
                 __syncwarp();
             }
         }
+    } else if (warp_idx == 1) {
+        // the odd CTA's warp 1 has nothing to issue: the even CTA drives the MMAs of the pair
     } else {
         // ------------------------------------------------------------ epilogue (warps 2..9)
         // Two groups of four warps; group hf owns columns [128*hf, 128*hf + 128) of the tile.
         // Each thread keeps its row's 128 running sums in registers: after every segment
-        // the TMEM partial sum is added in with round-to-nearest, and the tile is written
+        // the TMEM partial sum is added in with round-to-nearest, and the piece is written
         // to D once, after its last segment.
         const uint32_t q = warp_idx & 3;              // TMEM lane quarter this warp may read
         const uint32_t hf = (warp_idx - 2) >> 2;
-        const uint32_t row = q * 32 + lane;           // row inside the tile
+        const uint32_t row = q * 32 + lane;           // row inside this CTA's 128 rows
         const bool leader = (lane == 0) && (warp_idx == 2 + 4 * hf);
         uint8_t* my_buf = epi_gen + hf * EPI_BUF_BYTES;
         const uint32_t my_buf_s = epi_base + hf * EPI_BUF_BYTES;
@@ -336,15 +414,15 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         bool alive = true;
         long long u = u_begin;
         Piece pc;
-        while (alive && next_piece(p, u, pc)) {
+        while (alive && next_piece(p, u, u_stride, pc)) {
             int tm, tn;
             tile_coords(p, pc.tile, tm, tn);
-            const int m0 = tm * BM, n0 = tn * BN;
+            const int m0 = tm * C::TILE_M + static_cast<int>(rank) * BM, n0 = tn * BN;
             const int piece_lo = pc.s0 * p.seg_iters, piece_end = min(k_iters, pc.s1 * p.seg_iters);
             for (int k_lo = piece_lo; k_lo < piece_end; k_lo += p.seg_iters, ++it) {
                 const uint32_t acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
-                if (!mbar_wait(bar_tfull + 8 * acc, acc_phase, abortp, p, 4)) { alive = false; break; }
+                if (!mbar_wait<PAIR>(bar_tfull + 8 * acc, acc_phase, abortp, p, 4)) { alive = false; break; }
                 tc_fence_after();
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) {
@@ -361,13 +439,16 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(bar_tempty + 8 * acc);
+                if (lane == 0) {
+                    if (mma_cta) mbar_arrive(bar_tempty + 8 * acc);
+                    else mbar_arrive_remote(bar_tempty + 8 * acc, 0);
+                }
             }
             if (!alive) break;
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
                 const int col0 = n0 + hf * (BN / 2) + ch * EPI_COLS;
-                if (col0 < p.N) {
+                if (col0 < p.N && m0 < p.M) {
                     if (leader) bulk_wait_read<0>();          // the slab buffer has been read out
                     group_bar_sync(1 + hf);
                     uint8_t* rowp = my_buf + row * 128u;
@@ -400,10 +481,11 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();           // neither CTA frees its TMEM or leaves while the other may still use it
     if (warp_idx == 1) {
         tc_fence_after();
         __syncwarp();
-        tmem_dealloc(tmem_base, TMEM_COLS);
+        tmem_dealloc<CTAS>(tmem_base, TMEM_COLS);
     }
 }
 
@@ -439,6 +521,33 @@ bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const
     return r == CUDA_SUCCESS;
 }
 
+// Number of CTA pairs that can be resident at once (0 when the pair form cannot be launched).
+int max_pairs(int sm_count) {
+    static int cached = -1;
+    if (cached >= 0) return cached;
+    cached = 0;
+    if (cudaFuncSetAttribute(lq_tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::SMEM_BYTES) != cudaSuccess) {
+        cudaGetLastError();
+        return cached;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(sm_count / 2 * 2));
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = Cfg<2>::SMEM_BYTES;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, lq_tc_gemm_kernel<2>, &cfg) != cudaSuccess) {
+        cudaGetLastError();
+        return cached;
+    }
+    cached = n < sm_count / 2 ? n : sm_count / 2;
+    return cached;
+}
+
 }  // namespace
 
 int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
@@ -454,13 +563,17 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
 
     static bool attr_set = false;
     if (!attr_set) {
-        LQ_CUDA_TRY(cudaFuncSetAttribute(lq_tc_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+        LQ_CUDA_TRY(cudaFuncSetAttribute(lq_tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<1>::SMEM_BYTES));
         attr_set = true;
     }
+    // The pair form pays off once there are at least a few 256-row tiles; below that one CTA per tile.
+    const int pairs = (a.M > BM) ? max_pairs(h->sm_count) : 0;
+    const int ctas_per_tile = pairs > 0 ? 2 : 1;
+    const int b_rows_box = BN / ctas_per_tile;
 
     CUtensorMap map_a, map_b, map_d;
     if (!make_map_2d(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.A_all, a.K, a.a_rows, a.lda, BK, BM) ||
-        !make_map_2d(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.B_all, a.K, a.b_rows, a.ldb, BK, BN) ||
+        !make_map_2d(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.B_all, a.K, a.b_rows, a.ldb, BK, b_rows_box) ||
         !make_map_2d(&map_d, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.D, a.N, a.M, a.ldd, EPI_COLS, BM))
         return LQ_ERR_CUDA;
 
@@ -476,12 +589,13 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
     p.alpha = a.alpha;
     p.accumulate = a.accumulate;
     p.upper_only = a.upper_only;
-    p.tiles_m = static_cast<int>(lq_ceil_div(a.M, BM));
+    p.tile_m = BM * ctas_per_tile;
+    p.tiles_m = static_cast<int>(lq_ceil_div(a.M, p.tile_m));
     p.tiles_n = static_cast<int>(lq_ceil_div(a.N, BN));
     if (a.upper_only) {
         int cnt = 0;
         for (int m = 0; m < p.tiles_m; ++m) {
-            int c = p.tiles_n - (m * BM) / BN;
+            int c = p.tiles_n - (m * p.tile_m) / BN;
             if (c > 0) cnt += c;
         }
         p.num_tiles = cnt;
@@ -496,20 +610,38 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
         p.seg_iters = (a.seg_iters > 0 && a.seg_iters < k_iters) ? a.seg_iters : k_iters;
         p.segs_per_tile = static_cast<int>(lq_ceil_div(k_iters, p.seg_iters));
     }
-    // number of K parts: the one that leaves the shortest schedule, ceil(tiles * q / CTAs) / q
-    const int ctas = h->sm_count;
+    // number of K parts: the one that leaves the shortest schedule, ceil(tiles * q / workers) / q
+    const int workers = ctas_per_tile == 2 ? pairs : h->sm_count;
     p.k_parts = 1;
     if (a.accumulate && p.segs_per_tile >= 16) {          // long K only: every unit pays one epilogue
-        double best = static_cast<double>(lq_ceil_div(p.num_tiles, ctas));
+        double best = static_cast<double>(lq_ceil_div(p.num_tiles, workers));
         for (int q = 2; q <= 8 && q <= p.segs_per_tile; ++q) {
-            const double t = static_cast<double>(lq_ceil_div(static_cast<int64_t>(p.num_tiles) * q, ctas)) / q;
+            const double t = static_cast<double>(lq_ceil_div(static_cast<int64_t>(p.num_tiles) * q, workers)) / q;
             if (t < best * 0.98) { best = t; p.k_parts = q; }
         }
     }
     p.total_units = static_cast<long long>(p.num_tiles) * p.k_parts;
+    const int active = p.total_units < workers ? static_cast<int>(p.total_units) : workers;
 
-    const int grid = p.total_units < ctas ? static_cast<int>(p.total_units) : ctas;
-    lq_tc_gemm_kernel<<<grid, NUM_THREADS, SMEM_BYTES, stream>>>(map_a, map_b, map_d, p);
-    LQ_LAUNCH_CHECK();
+    if (ctas_per_tile == 2) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(static_cast<unsigned>(2 * active));
+        cfg.blockDim = dim3(NUM_THREADS);
+        cfg.dynamicSmemBytes = Cfg<2>::SMEM_BYTES;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, lq_tc_gemm_kernel<2>, map_a, map_b, map_d, p) != cudaSuccess) {
+            cudaGetLastError();
+            return LQ_ERR_CUDA;
+        }
+        ++lq_launches_total;
+    } else {
+        lq_tc_gemm_kernel<1><<<active, NUM_THREADS, Cfg<1>::SMEM_BYTES, stream>>>(map_a, map_b, map_d, p);
+        LQ_LAUNCH_CHECK();
+    }
     return LQ_OK;
 }
