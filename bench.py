@@ -36,6 +36,15 @@ WORKLOADS = {
     "c1-512": ("c1", 512, 512, 8192, dict(grid="nonuniform", bits=4, p=4.0, n_iter=20)),
     # a quarter-size layer whose inputs (256 MiB of X) still exceed the L2: the case profiler captures run on
     "q_proj-2k-nu4": ("c2", 2048, 2048, 65536, dict(grid="nonuniform", bits=4, p=4.0, n_iter=20)),
+    # the other benchmark configurations (parity-test cases; timed on request with --no-e2e --no-cpu-baseline)
+    "llama3-8b-q_proj-nu3": ("c2", 4096, 4096, 262144, dict(grid="nonuniform", bits=3, p=4.0, n_iter=20)),
+    "llama3-8b-down_proj-aff4g128": ("c3", 4096, 14336, 131072, dict(grid="affine", bits=4, p=4.0, group=128, T=45, t=9)),
+    "llama3-8b-down_proj-nu3": ("c3", 4096, 14336, 131072, dict(grid="nonuniform", bits=3, p=4.0, n_iter=20)),
+    "llama3-8b-gate_proj-nu3": ("c2", 14336, 4096, 131072, dict(grid="nonuniform", bits=3, p=4.0, n_iter=20)),
+    "llama31-405b-up_proj-nu2": ("c3", 53248, 16384, 65536, dict(grid="nonuniform", bits=2, p=4.0, n_iter=20)),
+    "llama31-405b-up_proj-aff4g128": ("c3", 53248, 16384, 65536, dict(grid="affine", bits=4, p=4.0, group=128, T=45, t=9)),
+    "llama31-405b-down_proj-nu2": ("c3", 16384, 53248, 65536, dict(grid="nonuniform", bits=2, p=4.0, n_iter=20)),
+    "llama31-405b-down_proj-aff4g128": ("c3", 16384, 53248, 65536, dict(grid="affine", bits=4, p=4.0, group=128, T=45, t=9)),
 }
 L2_BYTES = 126 * 1024 * 1024
 
@@ -198,7 +207,8 @@ def run_ours(args):
     h = lq.lq_create(local)
     layer = synth.make_layer(recipe, r, c, n, seed=layer_seed(rank), device=dev)
     W, X = layer.W, layer.X
-    P = lq.LayerPass(h, r, c, cfg, w_dtype=W.dtype, x_dtype=X.dtype, n_chunk=n, device=dev)
+    chunk = n if args.chunk <= 0 else min(n, args.chunk)       # tokens per lq_hessian_accumulate call
+    P = lq.LayerPass(h, r, c, cfg, w_dtype=W.dtype, x_dtype=X.dtype, n_chunk=chunk, device=dev)
     stream = torch.cuda.current_stream()
 
     def barrier():
@@ -210,7 +220,8 @@ def run_ours(args):
         ev = events
         P.H.zero_()
         if ev: ev[0].record(stream)
-        lq.lq_hessian_accumulate(h, X, P.H, 2.0, P.ws)
+        for j in range(0, n, chunk):
+            lq.lq_hessian_accumulate(h, X[:, j:j + chunk], P.H, 2.0, P.ws)
         if ev: ev[1].record(stream)
         lq.lq_hessian_finalize(h, P.H)
         lq.lq_prepare_hinv(h, P.H, P.U, P.dinv, P.ws, 0.01, W)
@@ -246,35 +257,36 @@ def run_ours(args):
     stage_ms = np.array([[e[i].elapsed_time(e[i + 1]) for i in range(4)] for e in evs]).mean(axis=0)
 
     # ---- end to end through the public API with host buffers -------------------------------
-    e2e_steps = max(1, min(args.steps, 3))
-    Xh = torch.empty(X.shape, dtype=X.dtype, pin_memory=True)
-    Wh = torch.empty(W.shape, dtype=W.dtype, pin_memory=True)
-    Xh.copy_(X)
-    Wh.copy_(W)
-    codes_h = torch.empty(P.codes.shape, dtype=torch.uint8, pin_memory=True)
-    grid_h = torch.empty(P.grid.shape, dtype=torch.float32, pin_memory=True)
-    loss_h = torch.empty((1,), dtype=torch.float64, pin_memory=True)
-    Xd, Wd = torch.empty_like(X), torch.empty_like(W)
-    barrier()
-    b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    b0.record(stream)
-    for _ in range(e2e_steps):
-        Xd.copy_(Xh, non_blocking=True)
-        Wd.copy_(Wh, non_blocking=True)
-        P.H.zero_()
-        lq.lq_hessian_accumulate(h, Xd, P.H, 2.0, P.ws)
-        lq.lq_hessian_finalize(h, P.H)
-        lq.lq_prepare_hinv(h, P.H, P.U, P.dinv, P.ws, 0.01, Wd)
-        lq.lq_fit_grid(h, cfg, Wd, P.dinv, P.ws, P.grid, P.scale, P.zero)
-        lq.lq_quantize_layer(h, cfg, Wd, P.U, P.codes, P.ws, P.grid, P.scale, P.zero, None, P.loss)
-        codes_h.copy_(P.codes, non_blocking=True)
-        grid_h.copy_(P.grid, non_blocking=True)
-        loss_h.copy_(P.loss, non_blocking=True)
-    b1.record(stream)
-    barrier()
-    e2e_ms = b0.elapsed_time(b1) / e2e_steps
-    h2d = Xh.numel() * Xh.element_size() + Wh.numel() * Wh.element_size()
-    d2h = codes_h.numel() + grid_h.numel() * 4 + 8
+    e2e_ms, h2d, d2h = float("nan"), 0, 0
+    if not args.no_e2e:
+        e2e_steps = max(1, min(args.steps, 3))
+        Xh = torch.empty(X.shape, dtype=X.dtype, pin_memory=True)
+        Wh = torch.empty(W.shape, dtype=W.dtype, pin_memory=True)
+        Xh.copy_(X)
+        Wh.copy_(W)
+        outs = [t for t in (P.codes, P.grid, P.scale, P.zero, P.loss) if t is not None]
+        outs_h = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
+        Xd, Wd = torch.empty_like(X), torch.empty_like(W)
+        barrier()
+        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        b0.record(stream)
+        for _ in range(e2e_steps):
+            Xd.copy_(Xh, non_blocking=True)
+            Wd.copy_(Wh, non_blocking=True)
+            P.H.zero_()
+            for j in range(0, n, chunk):
+                lq.lq_hessian_accumulate(h, Xd[:, j:j + chunk], P.H, 2.0, P.ws)
+            lq.lq_hessian_finalize(h, P.H)
+            lq.lq_prepare_hinv(h, P.H, P.U, P.dinv, P.ws, 0.01, Wd)
+            lq.lq_fit_grid(h, cfg, Wd, P.dinv, P.ws, P.grid, P.scale, P.zero)
+            lq.lq_quantize_layer(h, cfg, Wd, P.U, P.codes, P.ws, P.grid, P.scale, P.zero, None, P.loss)
+            for th, td in zip(outs_h, outs):
+                th.copy_(td, non_blocking=True)
+        b1.record(stream)
+        barrier()
+        e2e_ms = b0.elapsed_time(b1) / e2e_steps
+        h2d = Xh.numel() * Xh.element_size() + Wh.numel() * Wh.element_size()
+        d2h = sum(t.numel() * t.element_size() for t in outs_h)
 
     t = max_over_ranks(torch.tensor([total_ms, e2e_ms], device=dev, dtype=torch.float64), world)
     total_ms, e2e_ms = float(t[0]), float(t[1])
@@ -306,7 +318,11 @@ def run_ours(args):
         lane_peak = 148 * 128 * sm_ghz / 1e3
         K = 1 << st["bits"]
         s2 = (2.0 / 3.0) * float(c) ** 3 / (stage_ms[1] * 1e-3) / 1e12
-        s3_ops = float(r) * c * st.get("n_iter", 1) * (np.log2(K) + 3) / (stage_ms[2] * 1e-3) / 1e12
+        if st["grid"] == "affine":       # (t + 1)^2 candidates per group, 9 lane-operations per weight and candidate
+            s3_work = float(r) * c * (st["t"] + 1) ** 2 * 9
+        else:
+            s3_work = float(r) * c * st["n_iter"] * (np.log2(K) + 3)
+        s3_ops = s3_work / (stage_ms[2] * 1e-3) / 1e12
         s3_gbs = float(r) * c * W.element_size() / (stage_ms[2] * 1e-3) / 1e9
         s4 = float(r) * c * c / (stage_ms[3] * 1e-3) / 1e12
         stage_roof = {
@@ -317,7 +333,7 @@ def run_ours(args):
                                "executed_frac": 6 * s4 / peak},
         }
         cpu = None
-        if world == 1 and not args.no_cpu_baseline:
+        if world == 1 and not args.no_cpu_baseline and st["grid"] == "nonuniform" and c <= 4096:
             sec, desc, cores = oracle_sample(args.workload, n_tokens=args.ref_tokens, n_rows=args.ref_rows, layer=layer)
             cpu = {"value": r * c / sec, "unit": "weights/s", "cores": cores, "kind": "oracle", "sample": desc}
         line = {
@@ -325,14 +341,15 @@ def run_ours(args):
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
             "data": "synthetic",
-            "config": {"workload": args.workload, "r": r, "c": c, "n_tokens": n, **st, "block": 128, "damp": 0.01,
+            "config": {"workload": args.workload, "r": r, "c": c, "n_tokens": n, "tokens_per_call": chunk, **st, "block": 128,
+                       "damp": 0.01,
                        "l2": f"inputs per step ({(X.numel() * X.element_size()) >> 20} MiB X) exceed the 126 MiB L2",
                        "parallelism": "one layer per GPU, no collective"},
             "stage_ms": {"hessian": float(stage_ms[0]), "prepare_hinv": float(stage_ms[1]),
                          "fit_grid": float(stage_ms[2]), "quantize_layer": float(stage_ms[3])},
             "roofline": roof, "stage_roofline": stage_roof, "cpu_baseline": cpu,
-            "e2e": {"value": weights / (e2e_ms * 1e-3), "unit": "weights/s", "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+            "e2e": None if args.no_e2e else {"value": weights / (e2e_ms * 1e-3), "unit": "weights/s",
+                                             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": int(launches), "clocks": clocks,
         }
         print(json.dumps(line))
@@ -350,6 +367,8 @@ def main():
     ap.add_argument("--workload", default="llama3-8b-q_proj-nu4", choices=sorted(WORKLOADS))
     ap.add_argument("--ref-tokens", type=int, default=32768)
     ap.add_argument("--ref-rows", type=int, default=512)
+    ap.add_argument("--chunk", type=int, default=0, help="tokens per Hessian call (0 = all at once)")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (e2e is then null)")
     ap.add_argument("--no-cpu-baseline", action="store_true",
                     help="skip the oracle timing leg (profiler captures only; cpu_baseline is then null)")
     args = ap.parse_args()

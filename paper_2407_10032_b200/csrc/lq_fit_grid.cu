@@ -7,9 +7,10 @@
 // fall on the same side as in a float64 evaluation, or the centroids drift apart by far more
 // than rounding.
 //
-// Affine (Eq. 7): one CTA per (row, group); every thread evaluates whole candidates
-// (t_min, t_max) over the group's weights held in shared memory, then the CTA takes the
-// arg-min (first minimum in t_min-major order).  Also fp64, for the same reason.
+// Affine (Eq. 7): every (row, group) enumerates the candidates (t_min, t_max) over its weights
+// held in shared memory and takes the arg-min (first minimum in t_min-major order) of the fp64
+// losses.  Groups of up to 1024 weights: one warp per group with an fp32 pre-score (see
+// affine_search_warp_kernel); longer groups: one CTA per group, all candidates in fp64.
 #include <math.h>
 
 #include <mutex>
@@ -555,6 +556,172 @@ affine_search_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, int group,
     }
 }
 
+// ------------------------------------------------------ affine search, warp per group --
+// Groups up to AFW_MAX_GROUP weights: one warp per (row, group), lanes over the candidates
+// (t_min, t_max), the group's (w, s) pairs broadcast out of shared memory.  Every candidate is
+// first scored in fp32 (eight operations per weight); only the candidates whose fp32 loss lies
+// within 0.1 % of the best fp32 loss of the group are then evaluated in fp64 with exactly the
+// arithmetic of Eq. 7, and the arg-min (first minimum in t_min-major order) is taken over
+// those fp64 losses.  A candidate that is skipped has an fp32 loss at least 0.1 % above that of
+// an evaluated one, far outside the fp32 error of such a sum, so it cannot be the fp64 minimum:
+// the result is that of the all-fp64 search.
+constexpr int AFW_WARPS = 8;
+constexpr int AFW_MAX_GROUP = 1024;
+
+template <typename T>
+__global__ void __launch_bounds__(AFW_WARPS * 32)
+affine_search_warp_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_groups, int64_t total_groups,
+                          const double* __restrict__ s64, int K, int Tparts, int t_count,
+                          float* __restrict__ scale, int32_t* __restrict__ zero) {
+    extern __shared__ __align__(16) unsigned char afw_smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float2* ws = reinterpret_cast<float2*>(afw_smem) + static_cast<size_t>(warp) * group;      // (w, s / max s)
+    const int64_t gid = static_cast<int64_t>(blockIdx.x) * AFW_WARPS + warp;
+    if (gid >= total_groups) return;                       // whole warps leave; no block-wide barrier below
+    const int64_t row = gid / n_groups;
+    const int gi = static_cast<int>(gid - row * n_groups);
+    const T* wp = W + row * ldw + static_cast<int64_t>(gi) * group;
+    const double* sp = s64 + static_cast<int64_t>(gi) * group;
+
+    float mn = INFINITY, mx = -INFINITY;
+    double smax = 0.0;
+    for (int j = lane; j < group; j += 32) {
+        const float w = load_w(wp + j);
+        mn = fminf(mn, w);
+        mx = fmaxf(mx, w);
+        smax = fmax(smax, sp[j]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        smax = fmax(smax, __shfl_xor_sync(0xffffffffu, smax, o));
+    }
+    const double sinv = smax > 0.0 ? 1.0 / smax : 1.0;
+    for (int j = lane; j < group; j += 32) ws[j] = make_float2(load_w(wp + j), static_cast<float>(sp[j] * sinv));
+    __syncwarp();
+
+    const double dmn = mn, dmx = mx, R = dmx - dmn;
+    const double Km1 = static_cast<double>(K - 1);
+    if (R == 0.0) {                                // constant group
+        if (lane == 0) {
+            double lo = fmin(dmn, 0.0), hi = fmax(dmx, 0.0);
+            double S = 1.0, Z = 0.0;
+            if (hi != lo) { S = (hi - lo) / Km1; Z = -rint(lo / S); }
+            scale[gid] = static_cast<float>(S);
+            zero[gid] = static_cast<int32_t>(Z);
+        }
+        return;
+    }
+
+    const int side = t_count + 1;
+    const int n_cand = side * side;
+    const float Km1f = static_cast<float>(K - 1);
+    // (S, Z) of a candidate exactly as Eq. 7 gives them; false when the candidate is void
+    auto params = [&](int cand, double& S, double& Z) {
+        const int t_min = cand / side, t_max = cand - t_min * side;
+        const double lo = dmn + static_cast<double>(t_min) * R / static_cast<double>(Tparts);
+        const double hi = dmx - static_cast<double>(t_max) * R / static_cast<double>(Tparts);
+        S = (hi - lo) / Km1;
+        if (!(S > 0.0)) return false;
+        Z = -rint(lo / S);
+        return true;
+    };
+    // fp32 score: with u = w / S + Z the error of a weight is S (q - u), q = clamp(round(u))
+    auto score32 = [&](double S, double Z) {
+        const float rS = static_cast<float>(1.0 / S), Zf = static_cast<float>(Z), Sf = static_cast<float>(S);
+        float a0 = 0.0f, a1 = 0.0f;
+        for (int j = 0; j < group; j += 2) {
+            const float4 p2 = *reinterpret_cast<const float4*>(ws + j);          // two (w, s) pairs
+            const float u0 = fmaf(p2.x, rS, Zf), u1 = fmaf(p2.z, rS, Zf);
+            const float e0 = fminf(fmaxf(rintf(u0), 0.0f), Km1f) - u0;
+            const float e1 = fminf(fmaxf(rintf(u1), 0.0f), Km1f) - u1;
+            a0 = fmaf(p2.y * e0, e0, a0);
+            a1 = fmaf(p2.w * e1, e1, a1);
+        }
+        return (a0 + a1) * Sf * Sf;
+    };
+    // fp64 loss of one candidate, computed by the whole warp (lane l takes weights l, l + 32, ...)
+    auto loss64 = [&](double S, double Z) {
+        double loss = 0.0;
+        for (int j = lane; j < group; j += 32) {
+            const double w = static_cast<double>(ws[j].x);
+            double q = rint(w / S) + Z;
+            q = fmin(fmax(q, 0.0), Km1);
+            const double d = (q - Z) * S - w;
+            loss += sp[j] * (d * d);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
+        return loss;
+    };
+
+    // pass 1: fp32 scores of all candidates and their minimum over the warp
+    constexpr int KEEP = 8;                        // scores kept in registers when there are at most 32 * KEEP candidates
+    const bool keep = n_cand <= 32 * KEEP;
+    float sc[KEEP];
+    float best32 = INFINITY;
+    if (keep) {
+#pragma unroll
+        for (int rd = 0; rd < KEEP; ++rd) {
+            const int cand = lane + 32 * rd;
+            double S, Z;
+            sc[rd] = (cand < n_cand && params(cand, S, Z)) ? score32(S, Z) : INFINITY;
+            if (sc[rd] != sc[rd]) sc[rd] = -INFINITY;          // a NaN score is always re-examined in fp64
+            best32 = fminf(best32, sc[rd] == -INFINITY ? INFINITY : sc[rd]);
+        }
+    } else {
+        for (int cand = lane; cand < n_cand; cand += 32) {
+            double S, Z;
+            if (!params(cand, S, Z)) continue;
+            best32 = fminf(best32, score32(S, Z));             // fminf ignores a NaN
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) best32 = fminf(best32, __shfl_xor_sync(0xffffffffu, best32, o));
+    const float bar32 = best32 * 1.001f;
+
+    // pass 2: candidates within 0.1 % of the best fp32 score are evaluated in fp64, one at a time
+    // in candidate order by the whole warp, so the first minimum wins and every lane holds the result
+    double my_loss = INFINITY;
+    int my_idx = 0x7fffffff;
+    const int rounds = (n_cand + 31) / 32;
+    for (int rd = 0; rd < rounds; ++rd) {
+        const int cand = lane + 32 * rd;
+        bool want = false;
+        if (keep) {
+            float v = INFINITY;
+#pragma unroll
+            for (int k = 0; k < KEEP; ++k) v = (k == rd) ? sc[k] : v;
+            want = cand < n_cand && v <= bar32;
+        } else {
+            double S, Z;
+            if (cand < n_cand && params(cand, S, Z)) want = !(score32(S, Z) > bar32);      // true for a NaN score
+        }
+        uint32_t todo = __ballot_sync(0xffffffffu, want);
+        while (todo) {
+            const int src = __ffs(todo) - 1;
+            todo &= todo - 1;
+            double S, Z;
+            if (!params(src + 32 * rd, S, Z)) continue;
+            const double loss = loss64(S, Z);
+            if (loss < my_loss) { my_loss = loss; my_idx = src + 32 * rd; }
+        }
+    }
+    if (lane == 0) {
+        double S = 1.0, Z = 0.0;
+        if (my_idx != 0x7fffffff) {
+            const int t_min = my_idx / side, t_max = my_idx - t_min * side;
+            const double lo = dmn + static_cast<double>(t_min) * R / static_cast<double>(Tparts);
+            const double hi = dmx - static_cast<double>(t_max) * R / static_cast<double>(Tparts);
+            S = (hi - lo) / Km1;
+            Z = -rint(lo / S);
+        }
+        scale[gid] = static_cast<float>(S);
+        zero[gid] = static_cast<int32_t>(Z);
+    }
+}
+
 int check_cfg(const lq_config* cfg) {
     if (!cfg) return LQ_ERR_INVALID_ARG;
     if (cfg->bits < 2 || cfg->bits > 4) return LQ_ERR_INVALID_ARG;
@@ -620,9 +787,29 @@ extern "C" int lq_fit_grid(lq_handle* h, void* stream, const lq_config* cfg, con
 
     const int64_t g = cfg->group_size == 0 ? c : cfg->group_size;
     const int n_groups = static_cast<int>(c / g);
+    const int K = 1 << cfg->bits;
+    if (g <= AFW_MAX_GROUP && g % 2 == 0) {
+        const int64_t total = r * n_groups;
+        const size_t smem_w = static_cast<size_t>(AFW_WARPS) * g * sizeof(float2);
+        static bool attr_w = false;
+        if (!attr_w) {
+            LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_warp_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, AFW_WARPS * AFW_MAX_GROUP * 8));
+            LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_warp_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, AFW_WARPS * AFW_MAX_GROUP * 8));
+            attr_w = true;
+        }
+        const unsigned nb = static_cast<unsigned>(lq_ceil_div(total, AFW_WARPS));
+        if (w_dtype == LQ_F32)
+            affine_search_warp_kernel<float><<<nb, AFW_WARPS * 32, smem_w, st>>>(static_cast<const float*>(W), ldw, (int)g, n_groups, total,
+                                                                              s64, K, cfg->T, cfg->t_count, scale, zero);
+        else
+            affine_search_warp_kernel<__nv_bfloat16><<<nb, AFW_WARPS * 32, smem_w, st>>>(static_cast<const __nv_bfloat16*>(W), ldw, (int)g,
+                                                                                      n_groups, total, s64, K, cfg->T, cfg->t_count,
+                                                                                      scale, zero);
+        LQ_LAUNCH_CHECK();
+        return LQ_OK;
+    }
     const size_t smem = static_cast<size_t>(g) * sizeof(float);
     const unsigned blocks = static_cast<unsigned>(r * n_groups);
-    const int K = 1 << cfg->bits;
     static bool attr_set = false;
     if (!attr_set) {
         LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
