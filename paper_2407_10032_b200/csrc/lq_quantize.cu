@@ -4,7 +4,8 @@
 //   in-block kernel  : one warp per output row, four block columns per lane, walks the columns
 //                      in order (quantise, E = (w - q)/U_jj, w[k] -= E * U[j][k]); the
 //                      128 x 128 diagonal block of U sits in shared memory.
-//   trailing update  : W[:, i+B:] -= E U[i:i+B, i+B:] on the tensor cores (lq_tc_gemm), fp32
+//   trailing update  : W[:, i+B:] -= E U[i:i+B, i+B:] on the tensor cores (lq_tc_gemm), in two
+//                      levels (see the host loop), fp32
 //                      operands fed as three bf16 terms each (six products), accumulated into
 //                      the fp32 working copy by the copy engine's reduce-add.
 #include <math.h>
@@ -14,6 +15,7 @@
 namespace {
 
 constexpr int B = 128;      // block width of the column loop
+constexpr int OB = 1024;    // outer block: the lazy update of columns beyond it waits until it is complete
 
 template <typename T>
 __global__ void to_f32_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, float* __restrict__ Wc, int64_t ldc) {
@@ -56,7 +58,9 @@ struct QuantOut {
     void* what;              // r x ldwh or null
     int what_bf16;
     int64_t ldwh;
-    __nv_bfloat16* esplit;   // 3 x r x B
+    __nv_bfloat16* esplit;   // 3 x r x e_ld: the errors of one outer block; this launch fills columns e_col ..
+    int64_t e_ld;
+    int e_col;
     double* loss_rows;       // r
 };
 
@@ -200,9 +204,9 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
             pm[t / 2] = static_cast<uint32_t>(__bfloat16_as_ushort(m0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(m1)) << 16);
             pl[t / 2] = static_cast<uint32_t>(__bfloat16_as_ushort(l0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(l1)) << 16);
         }
-        __nv_bfloat16* e0 = out.esplit + row * B + col0;
-        __nv_bfloat16* e1 = e0 + r * B;
-        __nv_bfloat16* e2 = e1 + r * B;
+        __nv_bfloat16* e0 = out.esplit + row * out.e_ld + out.e_col + col0;
+        __nv_bfloat16* e1 = e0 + r * out.e_ld;
+        __nv_bfloat16* e2 = e1 + r * out.e_ld;
         *reinterpret_cast<uint2*>(e0) = make_uint2(ph[0], ph[1]);
         *reinterpret_cast<uint2*>(e1) = make_uint2(pm[0], pm[1]);
         *reinterpret_cast<uint2*>(e2) = make_uint2(pl[0], pl[1]);
@@ -240,7 +244,7 @@ WsLayout ws_layout(int64_t r, int64_t c) {
     size_t off = 0;
     L.wc = off; off += lq_align_up(static_cast<size_t>(r) * L.ldc * sizeof(float), 256);
     L.ut = off; off += lq_align_up(static_cast<size_t>(3) * c * L.ldt * sizeof(__nv_bfloat16), 256);
-    L.es = off; off += lq_align_up(static_cast<size_t>(3) * r * B * sizeof(__nv_bfloat16), 256);
+    L.es = off; off += lq_align_up(static_cast<size_t>(3) * r * OB * sizeof(__nv_bfloat16), 256);
     L.loss = off; off += lq_align_up(static_cast<size_t>(r) * sizeof(double), 256);
     L.total = off;
     return L;
@@ -332,10 +336,14 @@ extern "C" int lq_quantize_layer(lq_handle* h, void* stream, const lq_config* cf
     out.what_bf16 = (what_dtype == LQ_BF16);
     out.ldwh = ldwh;
     out.esplit = ES;
+    out.e_ld = OB;
+    out.e_col = 0;
     out.loss_rows = loss_rows;
 
     for (int64_t i0 = 0; i0 < c; i0 += B) {
         int rc;
+        const int64_t o0 = i0 / OB * OB;          // start of the outer block
+        out.e_col = static_cast<int>(i0 - o0);
         if (affine) {
             switch (cfg->bits) {
                 case 2: rc = launch_inblock<4, true>(st, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
@@ -350,18 +358,37 @@ extern "C" int lq_quantize_layer(lq_handle* h, void* stream, const lq_config* cf
             }
         }
         if (rc) return rc;
-        const int64_t rest = c - (i0 + B);
-        if (rest > 0) {
+        // Lazy update (Algorithm 1 line 20) in two levels.  The columns that the next blocks of
+        // this outer block are about to quantise get this block's errors now (K = 128); the columns
+        // beyond the outer block get the errors of all its blocks in one product once it is complete
+        // (K = 1024), which cuts the read-modify-write traffic on the working copy eightfold.  The
+        // result is the same sum in a different order.
+        const int64_t ob_end = (o0 + OB < c) ? o0 + OB : c;
+        const int64_t ao[6] = {0, 0, r, 0, 2 * r, r};
+        const int64_t bo[6] = {0, c, 0, 2 * c, 0, c};
+        const int64_t near = ob_end - (i0 + B);
+        if (near > 0) {
             lq_tc_gemm_args g = {};
-            g.A_all = ES; g.a_rows = 3 * r; g.lda = B;
+            g.A_all = ES + (i0 - o0); g.a_rows = 3 * r; g.lda = OB;
             g.B_all = UT + (i0 + B) * L.ldt + i0; g.b_rows = 3 * c - (i0 + B); g.ldb = L.ldt;
             g.D = Wc + (i0 + B); g.ldd = L.ldc;
-            g.M = r; g.N = rest; g.K = B;
+            g.M = r; g.N = near; g.K = B;
             g.n_pass = 6;
-            const int64_t ao[6] = {0, 0, r, 0, 2 * r, r};
-            const int64_t bo[6] = {0, c, 0, 2 * c, 0, c};
             for (int i = 0; i < 6; ++i) { g.a_row_off[i] = ao[i]; g.b_row_off[i] = bo[i]; }
             g.alpha = -1.0f; g.accumulate = 1; g.upper_only = 0;
+            rc = lq_tc_gemm(h, st, g);
+            if (rc) return rc;
+        }
+        if (i0 + B >= ob_end && ob_end < c) {
+            lq_tc_gemm_args g = {};
+            g.A_all = ES; g.a_rows = 3 * r; g.lda = OB;
+            g.B_all = UT + ob_end * L.ldt + o0; g.b_rows = 3 * c - ob_end; g.ldb = L.ldt;
+            g.D = Wc + ob_end; g.ldd = L.ldc;
+            g.M = r; g.N = c - ob_end; g.K = ob_end - o0;
+            g.n_pass = 6;
+            for (int i = 0; i < 6; ++i) { g.a_row_off[i] = ao[i]; g.b_row_off[i] = bo[i]; }
+            g.alpha = -1.0f; g.accumulate = 1; g.upper_only = 0;
+            g.seg_iters = 12;          // partial sums leave the tensor core's truncating accumulator every 128 columns
             rc = lq_tc_gemm(h, st, g);
             if (rc) return rc;
         }
