@@ -461,16 +461,21 @@ diag_block_kernel(double* __restrict__ A, int64_t cp, int64_t blk, int64_t c_rea
     }
 }
 
-// U (fp32, c x c, upper, zeros below) and dinv[j] = sum_k U64[k][j]^2: one CTA per 32 columns.
+// U (fp32, c x c, upper, zeros below) and dinv[j] = sum_k U64[k][j]^2.  A CTA converts 256 rows of 32
+// columns and leaves the sum of squares of its piece of every column in part[row chunk][column];
+// dinv_kernel adds the pieces of a column in row order (a fixed order: the result is reproducible).
+constexpr int FIN_ROWS = 256;
 __global__ void __launch_bounds__(256)
 finalize_kernel(const double* __restrict__ A, int64_t cp, int64_t c, float* __restrict__ U, int64_t ldu,
-                float* __restrict__ dinv) {
+                double* __restrict__ part) {
     __shared__ double red[8][33];
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
     const int64_t j = (int64_t)blockIdx.x * 32 + tx;
+    const int64_t i0 = (int64_t)blockIdx.y * FIN_ROWS;
+    const int64_t i1 = i0 + FIN_ROWS < c ? i0 + FIN_ROWS : c;
     double s = 0.0;
     if (j < c) {
-        for (int64_t i = ty; i < c; i += 8) {
+        for (int64_t i = i0 + ty; i < i1; i += 8) {
             double u = 0.0;
             if (i <= j) {
                 u = A[i * cp + j];
@@ -485,8 +490,15 @@ finalize_kernel(const double* __restrict__ A, int64_t cp, int64_t c, float* __re
         double t = 0.0;
 #pragma unroll
         for (int w = 0; w < 8; ++w) t += red[w][tx];
-        dinv[j] = static_cast<float>(t);
+        part[(int64_t)blockIdx.y * c + j] = t;
     }
+}
+__global__ void dinv_kernel(const double* __restrict__ part, int64_t c, int n_chunks, float* __restrict__ dinv) {
+    const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= c) return;
+    double t = 0.0;
+    for (int q = 0; q * (int64_t)FIN_ROWS <= j && q < n_chunks; ++q) t += part[(int64_t)q * c + j];
+    dinv[j] = static_cast<float>(t);
 }
 
 struct PrepLayout {
@@ -523,7 +535,7 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
     const PrepLayout L = prep_layout(c);
     if (!ws || ws_bytes < L.total) return LQ_ERR_WORKSPACE_TOO_SMALL;
     if (reinterpret_cast<uintptr_t>(ws) & 255) return LQ_ERR_INVALID_ARG;
-    if (L.nblk > 32767) return LQ_ERR_UNSUPPORTED;            // grid.y of the update launch
+    if (L.nblk > 32767 || c > 65536) return LQ_ERR_UNSUPPORTED;   // grid.y of the update launch; room for the column sums
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
     const int64_t nblk = L.nblk, cp = L.cp;
@@ -596,7 +608,15 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
         }
     }
     if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_rest, 0));
-    finalize_kernel<<<static_cast<unsigned>(lq_ceil_div(c, 32)), 256, 0, st>>>(A, cp, c, U, ldu, dinv);
-    LQ_LAUNCH_CHECK();
+    {
+        // the panel buffers are free now: they hold the per-chunk column sums (c / 256 x c doubles <= 2 panels for c <= 65536)
+        double* part = reinterpret_cast<double*>(wsp + L.pbuf);
+        const int n_chunks = static_cast<int>(lq_ceil_div(c, FIN_ROWS));
+        dim3 g(static_cast<unsigned>(lq_ceil_div(c, 32)), static_cast<unsigned>(n_chunks));
+        finalize_kernel<<<g, 256, 0, st>>>(A, cp, c, U, ldu, part);
+        LQ_LAUNCH_CHECK();
+        dinv_kernel<<<static_cast<unsigned>(lq_ceil_div(c, 256)), 256, 0, st>>>(part, c, n_chunks, dinv);
+        LQ_LAUNCH_CHECK();
+    }
     return LQ_OK;
 }

@@ -84,11 +84,14 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bw = (c - i0) < B ? static_cast<int>(c - i0) : B;
 
+    // The block of U goes to shared memory with asynchronous copies (plain loads for a ragged
+    // last block); the row's weights and grid are fetched while those copies are in flight.
+    const bool whole = bw == B && (ldu % 4 == 0);
     for (int idx = tid; idx < B * B / 4; idx += IB_THREADS) {
         const int jj = idx / (B / 4), k4 = (idx % (B / 4)) * 4;
-        float4 v;
-        if (jj < bw && k4 + 3 < bw && (ldu % 4 == 0)) {
-            v = *reinterpret_cast<const float4*>(U + (i0 + jj) * ldu + i0 + k4);
+        if (whole) {
+            const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(Us + jj * B + k4));
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(U + (i0 + jj) * ldu + i0 + k4) : "memory");
         } else {
             float t[4];
 #pragma unroll
@@ -96,20 +99,16 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
                 const int kk = k4 + u;
                 t[u] = (jj < bw && kk < bw) ? U[(i0 + jj) * ldu + i0 + kk] : (jj == kk ? 1.0f : 0.0f);
             }
-            v = make_float4(t[0], t[1], t[2], t[3]);
+            *reinterpret_cast<float4*>(Us + jj * B + k4) = make_float4(t[0], t[1], t[2], t[3]);
         }
-        *reinterpret_cast<float4*>(Us + jj * B + k4) = v;
     }
-    __syncthreads();
-    if (tid < B) invd[tid] = 1.0f / Us[tid * B + tid];
-    __syncthreads();
+    asm volatile("cp.async.commit_group;" ::: "memory");
 
     const int64_t row = (int64_t)blockIdx.x * IB_WARPS + warp;
-    if (row >= r) return;
-
+    const bool valid = row < r;
     const int col0 = 4 * lane;             // first of this lane's columns inside the block
-    float w[4];
-    {
+    float w[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    if (valid) {
         const float* wp = Wc + row * ldc + i0 + col0;
         if (col0 + 3 < bw) {
             const float4 v = *reinterpret_cast<const float4*>(wp);
@@ -122,15 +121,20 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
     float gl = 0.0f, ml = INFINITY;        // this lane's grid point and the midpoint above it
     float S_mine = 1.0f, Z_mine = 0.0f;    // affine parameters of this lane's columns
     if (!AFFINE) {
-        if (lane < K) gl = grid[row * K + lane];
+        if (valid && lane < K) gl = grid[row * K + lane];
         const float gn = __shfl_down_sync(0xffffffffu, gl, 1);
         if (lane < K - 1) ml = 0.5f * (gl + gn);
-    } else if (col0 < bw) {
+    } else if (valid && col0 < bw) {
         const int64_t gi = (i0 + col0) / group;
         const int64_t gidx = row * n_groups + (gi < n_groups ? gi : n_groups - 1);
         S_mine = scale[gidx];
         Z_mine = static_cast<float>(zero[gidx]);
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+    if (tid < B) invd[tid] = 1.0f / Us[tid * B + tid];
+    __syncthreads();
+    if (!valid) return;
 
     float qkeep[4] = {0.0f, 0.0f, 0.0f, 0.0f}, ekeep[4] = {0.0f, 0.0f, 0.0f, 0.0f};
     uint32_t cpack = 0;
