@@ -44,7 +44,11 @@ typedef enum {
 typedef enum { LQ_F32 = 0, LQ_BF16 = 1 } lq_dtype;
 typedef enum { LQ_FEATURE_MAJOR = 0 /* X is c x n, tokens contiguous */ } lq_layout;
 typedef enum { LQ_GRID_NONUNIFORM = 0, LQ_GRID_AFFINE = 1 } lq_grid_type;
-typedef enum { LQ_INIT_UNIFORM = 0 /* Eq. 6 */ } lq_init;
+typedef enum {
+    LQ_INIT_UNIFORM = 0,           /* Eq. 6: evenly spaced between the row's minimum and maximum (the paper's choice) */
+    LQ_INIT_WEIGHTED_QUANTILE = 1  /* the sorted weight at the first position whose cumulative sample weight
+                                      reaches (k + 1/2) / K of the row's total; rows of at most 16384 weights */
+} lq_init;
 
 typedef struct lq_handle lq_handle;
 

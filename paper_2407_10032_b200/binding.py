@@ -35,11 +35,11 @@ class Config(C.Structure):
                 ("block", C.c_int32), ("reserved", C.c_int32)]
 
     @classmethod
-    def make(cls, grid="nonuniform", bits=4, p=4.0, n_iter=20, group=0, T=2048, t=None, block=128, **_):
+    def make(cls, grid="nonuniform", bits=4, p=4.0, n_iter=20, group=0, T=2048, t=None, block=128, init="uniform", **_):
         if t is None:
             t = int({4: 0.2, 3: 0.3, 2: 0.4}.get(bits, 0.2) * T)
         gt = LQ_GRID_NONUNIFORM if grid == "nonuniform" else LQ_GRID_AFFINE
-        return cls(bits, gt, float(p), n_iter, 0, group or 0, T, t, block, 0)
+        return cls(bits, gt, float(p), n_iter, {"uniform": 0, "weighted_quantile": 1}[init], group or 0, T, t, block, 0)
 
 
 def library_path() -> str:

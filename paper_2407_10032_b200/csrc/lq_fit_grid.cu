@@ -211,7 +211,7 @@ __device__ __forceinline__ void bitonic_sort(KeyT* keys, int n, int tid) {
 template <int K, typename T>
 __global__ void __launch_bounds__(KS_THREADS, 4)
 kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int n, const double* __restrict__ s64,
-                     float* __restrict__ grid, int n_iter) {
+                     float* __restrict__ grid, int n_iter, int init) {
     typedef typename KeyOf<T>::type KeyT;
     extern __shared__ __align__(16) unsigned char ks_smem[];
     dd2* coarse = reinterpret_cast<dd2*>(ks_smem);            // n / 8 + 1 coarse prefixes, then the n keys (padded slots)
@@ -297,7 +297,24 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
         if (warp == 0) {
             const double lo = static_cast<double>(key_weight(keys[ks_slot(0)]));
             const double hi = static_cast<double>(key_weight(keys[ks_slot(c - 1)]));
-            if (lane < K) g[lane] = lo + (hi - lo) * static_cast<double>(lane) / static_cast<double>(K - 1);   // Eq. 6
+            if (init == LQ_INIT_UNIFORM) {
+                if (lane < K) g[lane] = lo + (hi - lo) * static_cast<double>(lane) / static_cast<double>(K - 1);   // Eq. 6
+            } else if (lane < K) {
+                // weighted quantiles: the sorted weight at the first position whose cumulative sample
+                // weight reaches (k + 1/2) / K of the total
+                const dd total = coarse[nch].s;
+                const double target = (static_cast<double>(lane) + 0.5) / static_cast<double>(K) * (total.hi + total.lo);
+                int p0 = 0, p1 = c - 1;                        // answer in [p0, p1]
+                while (p0 < p1) {
+                    const int mid = (p0 + p1) >> 1;
+                    const int b = mid + 1;                     // cumulative weight of positions 0 .. mid
+                    const int q = b / KS_CHUNK, rem = b % KS_CHUNK;
+                    dd f = coarse[q].s;
+                    for (int e = 0; e < rem; ++e) f = dd_add_d(f, s64[key_index(keys[ks_slot(q * KS_CHUNK + e)])]);
+                    if (f.hi + f.lo >= target) p1 = mid; else p0 = mid + 1;
+                }
+                g[lane] = static_cast<double>(key_weight(keys[ks_slot(p0)]));
+            }
             if (lane == 0) {
                 F[0].s.hi = F[0].s.lo = F[0].sw.hi = F[0].sw.lo = 0.0;
                 F[K] = coarse[nch];
@@ -430,7 +447,7 @@ kmeans_rows_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int64_t c, c
 
 template <int K, typename T>
 int launch_kmeans(cudaStream_t st, int sms, const T* W, int64_t ldw, int64_t r, int64_t c, const double* s64, float* grid,
-                  int n_iter) {
+                  int n_iter, int init) {
     if (c <= KS_MAX_N) {
         int n = 64;
         while (n < c) n <<= 1;
@@ -445,8 +462,9 @@ int launch_kmeans(cudaStream_t st, int sms, const T* W, int64_t ldw, int64_t r, 
         per_sm = per_sm < 1 ? 1 : (per_sm > 4 ? 4 : per_sm);                    // 64 registers x 256 threads: four CTAs per SM
         const int64_t cap = static_cast<int64_t>(sms) * per_sm;
         kmeans_sorted_kernel<K, T><<<static_cast<unsigned>(r < cap ? r : cap), KS_THREADS, smem, st>>>(
-            W, ldw, r, static_cast<int>(c), n, s64, grid, n_iter);
+            W, ldw, r, static_cast<int>(c), n, s64, grid, n_iter, init);
     } else {
+        if (init != LQ_INIT_UNIFORM) return LQ_ERR_UNSUPPORTED;     // rows this long only start from Eq. 6
         const size_t smem = static_cast<size_t>(c) * sizeof(T);
         if (smem > 200 * 1024) return LQ_ERR_UNSUPPORTED;
         static bool attr_set = false;
@@ -726,7 +744,8 @@ int check_cfg(const lq_config* cfg) {
     if (!cfg) return LQ_ERR_INVALID_ARG;
     if (cfg->bits < 2 || cfg->bits > 4) return LQ_ERR_INVALID_ARG;
     if (cfg->grid_type != LQ_GRID_NONUNIFORM && cfg->grid_type != LQ_GRID_AFFINE) return LQ_ERR_INVALID_ARG;
-    if (cfg->grid_type == LQ_GRID_NONUNIFORM && (cfg->n_iter < 0 || cfg->init != LQ_INIT_UNIFORM)) return LQ_ERR_INVALID_ARG;
+    if (cfg->grid_type == LQ_GRID_NONUNIFORM && (cfg->n_iter < 0 || (cfg->init != LQ_INIT_UNIFORM && cfg->init != LQ_INIT_WEIGHTED_QUANTILE)))
+        return LQ_ERR_INVALID_ARG;
     if (cfg->grid_type == LQ_GRID_AFFINE &&
         (cfg->T <= 0 || cfg->t_count < 0 || 2 * (int64_t)cfg->t_count > cfg->T || cfg->group_size < 0 || cfg->t_count > 4095))
         return LQ_ERR_INVALID_ARG;
@@ -775,8 +794,8 @@ extern "C" int lq_fit_grid(lq_handle* h, void* stream, const lq_config* cfg, con
 
     if (cfg->grid_type == LQ_GRID_NONUNIFORM) {
 #define LQ_KM(KK)                                                                                                     \
-    (w_dtype == LQ_F32 ? launch_kmeans<KK, float>(st, h->sm_count, static_cast<const float*>(W), ldw, r, c, s64, grid, cfg->n_iter) \
-                       : launch_kmeans<KK, __nv_bfloat16>(st, h->sm_count, static_cast<const __nv_bfloat16*>(W), ldw, r, c, s64, grid, cfg->n_iter))
+    (w_dtype == LQ_F32 ? launch_kmeans<KK, float>(st, h->sm_count, static_cast<const float*>(W), ldw, r, c, s64, grid, cfg->n_iter, cfg->init) \
+                       : launch_kmeans<KK, __nv_bfloat16>(st, h->sm_count, static_cast<const __nv_bfloat16*>(W), ldw, r, c, s64, grid, cfg->n_iter, cfg->init))
         switch (cfg->bits) {
             case 2: return LQ_KM(4);
             case 3: return LQ_KM(8);

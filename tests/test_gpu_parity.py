@@ -216,6 +216,25 @@ def test_stage3_nonuniform(lq, h, recipe, r, c, bits, p):
     assert centroid_ok(G, Gref, f64(L.W))
 
 
+@pytest.mark.parametrize("recipe,r,c,bits,p", [("c2", 96, 1024, 4, 1.0), ("c2", 64, 520, 3, 2.0), ("c1", 48, 512, 2, 0.0)])
+def test_stage3_weighted_quantile_start(lq, h, recipe, r, c, bits, p):
+    """The second deterministic start (weighted quantiles) against the oracle's; p is kept moderate
+    here: at p = 4 several quantiles fall on one heavy weight and the start degenerates."""
+    L = synth.make_layer(recipe, r, c, 2 * c, seed=3 * bits + c)
+    _, dinv, _, _ = O.prepare_hinv(O.hessian(f64(L.X)), 0.01)
+    dinv32 = torch.from_numpy(dinv).float()
+    for n_iter in (0, 12):
+        Gref = O.fit_grid_nonuniform(f64(L.W), f64(dinv32), bits, p, n_iter, init="weighted_quantile")
+        cfg = lq.Config.make(grid="nonuniform", bits=bits, p=p, n_iter=n_iter, init="weighted_quantile")
+        grid = torch.empty(r, 1 << bits, device="cuda")
+        ws = ws_for(lq, lq.lq_fit_grid_workspace(cfg, r, c))
+        lq.lq_fit_grid(h, cfg, L.W.cuda(), dinv32.cuda(), ws, grid=grid)
+        lq.lq_sync_status(h)
+        G = f64(grid)
+        ok = np.all(np.abs(G - Gref) <= CENT_TOL * np.maximum(np.abs(Gref), (f64(L.W).max(1) - f64(L.W).min(1))[:, None] / G.shape[1]), axis=1)
+        assert ok.mean() >= 0.98        # a quantile that falls between two sums equal to rounding may pick the neighbour
+
+
 def test_stage3_degenerate_rows(lq, h):
     r, c = 4, 256
     W = torch.randn(r, c) * 0.02
