@@ -42,7 +42,11 @@ typedef enum {
 } lq_status;
 
 typedef enum { LQ_F32 = 0, LQ_BF16 = 1 } lq_dtype;
-typedef enum { LQ_FEATURE_MAJOR = 0 /* X is c x n, tokens contiguous */ } lq_layout;
+typedef enum {
+    LQ_FEATURE_MAJOR = 0,  /* X is c x n_chunk, tokens contiguous (what the contraction reads directly) */
+    LQ_TOKEN_MAJOR = 1     /* X is n_chunk x c, features contiguous (activations as a model produces them);
+                              transposed into the workspace first */
+} lq_layout;
 typedef enum { LQ_GRID_NONUNIFORM = 0, LQ_GRID_AFFINE = 1 } lq_grid_type;
 typedef enum {
     LQ_INIT_UNIFORM = 0,           /* Eq. 6: evenly spaced between the row's minimum and maximum (the paper's choice) */
@@ -86,11 +90,13 @@ int lq_sync_status(lq_handle* h, void* stream, int32_t* status, int64_t* info);
  * fp32, ldh >= c, ldh % 4 == 0, 16-byte aligned) is the in/out accumulator and must be
  * zeroed by the caller before the first chunk.  Only tiles touching the upper triangle are
  * updated: entries strictly below the diagonal are unspecified until lq_hessian_finalize.
- * X: device, c x n_chunk, feature-major (ldx >= n_chunk elements; ldx*sizeof(x) % 16 == 0,
- * 16-byte aligned), bf16 or fp32.  bf16 products are exact in the fp32 accumulator; fp32
- * input is split into three bf16 terms (workspace needed) and keeps fp32-level accuracy.
- * workspace: lq_hessian_workspace bytes (0 for bf16 input; ws may then be NULL). */
-int lq_hessian_workspace(int32_t x_dtype, int64_t c, int64_t n_chunk, size_t* bytes);
+ * X: device, 16-byte aligned, bf16 or fp32; feature-major c x n_chunk (ldx >= n_chunk elements,
+ * ldx * sizeof(x) % 16 == 0) or token-major n_chunk x c (ldx >= c, ldx even for bf16).
+ * bf16 products are exact in the fp32 accumulator; fp32 input is split into three bf16 terms
+ * and keeps fp32-level accuracy.
+ * workspace: lq_hessian_workspace bytes (0 for feature-major bf16 input; ws may then be NULL):
+ * the staged copy of the chunk (transposed and / or split). */
+int lq_hessian_workspace(int32_t x_dtype, int32_t layout, int64_t c, int64_t n_chunk, size_t* bytes);
 int lq_hessian_accumulate(lq_handle* h, void* stream, const void* X, int32_t x_dtype,
                           int32_t layout, int64_t c, int64_t n_chunk, int64_t ldx,
                           float* H, int64_t ldh, float alpha, void* ws, size_t ws_bytes);

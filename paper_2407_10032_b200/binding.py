@@ -59,7 +59,7 @@ def LQ():
             "lq_create": [P(vp), C.c_int],
             "lq_destroy": [vp],
             "lq_sync_status": [vp, vp, P(i32), P(i64)],
-            "lq_hessian_workspace": [i32, i64, i64, P(sz)],
+            "lq_hessian_workspace": [i32, i32, i64, i64, P(sz)],
             "lq_hessian_accumulate": [vp, vp, vp, i32, i32, i64, i64, i64, vp, i64, f32, vp, sz],
             "lq_hessian_finalize": [vp, vp, vp, i64, i64],
             "lq_prepare_hinv_workspace": [i64, P(sz)],
@@ -136,16 +136,17 @@ def lq_sync_status(h, stream=None, raise_on_error=True):
     return st.value, info.value
 
 
-def lq_hessian_workspace(x_dtype, c, n_chunk) -> int:
+def lq_hessian_workspace(x_dtype, c, n_chunk, token_major=False) -> int:
     b = C.c_size_t(0)
     dt = x_dtype if isinstance(x_dtype, int) else (LQ_F32 if x_dtype == torch.float32 else LQ_BF16)
-    _check(LQ().lq_hessian_workspace(dt, c, n_chunk, C.byref(b)), "lq_hessian_workspace")
+    _check(LQ().lq_hessian_workspace(dt, 1 if token_major else 0, c, n_chunk, C.byref(b)), "lq_hessian_workspace")
     return b.value
 
 
-def lq_hessian_accumulate(h, X, H, alpha=2.0, ws=None, stream=None):
-    c, n = X.shape
-    _check(LQ().lq_hessian_accumulate(h, _stream(stream), _ptr(X), _dt(X), 0, c, n, _rowmajor(X), _ptr(H),
+def lq_hessian_accumulate(h, X, H, alpha=2.0, ws=None, stream=None, token_major=False):
+    """X is c x n (feature-major) or, with token_major, n x c."""
+    c, n = (X.shape[1], X.shape[0]) if token_major else X.shape
+    _check(LQ().lq_hessian_accumulate(h, _stream(stream), _ptr(X), _dt(X), 1 if token_major else 0, c, n, _rowmajor(X), _ptr(H),
                                       _rowmajor(H), alpha, _ptr(ws), 0 if ws is None else ws.numel() * ws.element_size()),
            "lq_hessian_accumulate")
 

@@ -40,6 +40,7 @@ def test_workspace_queries(lib):
     import torch
     assert lib.lq_hessian_workspace(torch.bfloat16, 4096, 1 << 18) == 0
     assert lib.lq_hessian_workspace(torch.float32, 512, 8192) >= 3 * 512 * 8192 * 2
+    assert lib.lq_hessian_workspace(torch.bfloat16, 512, 8192, token_major=True) >= 512 * 8192 * 2
     assert lib.lq_prepare_hinv_workspace(200) >= 256 * 256 * 8          # padded to the 128-wide panel
     cfg = lib.Config.make(grid="nonuniform", bits=4)
     assert lib.lq_fit_grid_workspace(cfg, 16, 4096) >= 4096 * 8

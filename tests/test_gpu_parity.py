@@ -124,6 +124,24 @@ def test_stage1_hessian(lq, h, c, n, dtype):
     assert np.max(np.abs(H - Href) / scale) < 5e-6
 
 
+@pytest.mark.parametrize("c,n,dtype", [(384, 1000, torch.bfloat16), (520, 4104, torch.bfloat16), (200, 1336, torch.float32),
+                                       (66, 70, torch.bfloat16)])
+def test_stage1_token_major(lq, h, c, n, dtype):
+    """Activations as a model produces them (tokens x features) give the same Hessian."""
+    g = torch.Generator().manual_seed(c * 3 + n)
+    Xt = (torch.randn(n, c, generator=g) * torch.exp(torch.randn(1, c, generator=g))).to(dtype)
+    Href = O.hessian(f64(Xt).T.copy())
+    H = torch.zeros(c, c + (-c) % 4, device="cuda")[:, :c] if c % 4 else torch.zeros(c, c, device="cuda")
+    ws = ws_for(lq, lq.lq_hessian_workspace(dtype, c, n, token_major=True))
+    lq.lq_hessian_accumulate(h, Xt.cuda(), H, 2.0, ws, token_major=True)
+    lq.lq_hessian_finalize(h, H)
+    lq.lq_sync_status(h)
+    Hg = f64(H)
+    assert np.array_equal(Hg, Hg.T)
+    scale = np.sqrt(np.outer(np.diag(Href), np.diag(Href)))
+    assert np.max(np.abs(Hg - Href) / scale) < 5e-6
+
+
 def test_stage1_chunks_add_up(lq, h):
     g = torch.Generator().manual_seed(5)
     X = torch.randn(256, 4096, generator=g).bfloat16().cuda()
