@@ -181,6 +181,16 @@ int lq_quantize_layer(lq_handle* h, void* stream, const lq_config* cfg, const vo
                       uint8_t* codes, void* W_hat, int32_t what_dtype, int64_t ldwh,
                       double* loss_out, void* ws, size_t ws_bytes);
 
+/* ---- storage format: the bit columns of the paper's result tables --------------------- */
+
+/* Packs the codes of lq_quantize_layer (one per byte) into the b-bit form that the paper's bit
+ * accounting assumes (b bits per weight plus a 2^b-entry table per row for non-uniform grids, or
+ * (S, Z) per group for affine ones): row i of `packed` (device, ldp >= ceil(c * bits / 8) bytes per
+ * row) is the little-endian bit stream of row i's codes, code j in bits [j * bits, (j + 1) * bits).
+ * Unused high bits of a row's last byte are zero. */
+int lq_pack_codes(lq_handle* h, void* stream, const uint8_t* codes, int64_t r, int64_t c,
+                  int32_t bits, uint8_t* packed, int64_t ldp);
+
 /* Number of CUDA kernels this library has launched in this process so far (host counter,
  * not thread-safe; for benchmarks and tests that want to see that the kernels ran). */
 uint64_t lq_launch_count(void);

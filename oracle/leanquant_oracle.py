@@ -301,6 +301,23 @@ def quantize_layer(W, U, *, grid=None, scale=None, zero=None, bits: int = 4,
     return codes, What, loss
 
 
+def pack_codes(codes, bits: int) -> np.ndarray:
+    """Storage format behind the paper's bit columns: every row's b-bit codes as one little-endian
+    bit stream (code j in bits [j b, (j+1) b) of the row), padded with zero bits to whole bytes."""
+    codes = np.asarray(codes, dtype=np.uint8)
+    r, c = codes.shape
+    bit_planes = (codes[:, :, None] >> np.arange(bits, dtype=np.uint8)) & 1       # least significant bit first
+    stream = bit_planes.reshape(r, c * bits)
+    return np.packbits(stream, axis=1, bitorder="little")
+
+
+def unpack_codes(packed, bits: int, c: int) -> np.ndarray:
+    """Inverse of pack_codes."""
+    stream = np.unpackbits(np.asarray(packed, dtype=np.uint8), axis=1, bitorder="little")[:, :c * bits]
+    planes = stream.reshape(stream.shape[0], c, bits).astype(np.int64)
+    return (planes << np.arange(bits)).sum(axis=2)
+
+
 def proxy_loss(W, What, H) -> float:
     """tr((W - What) H (W - What)^T); with the undamped H = 2XX^T this is
     2 * ||W X - What X||_F^2, the layer objective of Eq. 1 up to the factor 2."""

@@ -67,6 +67,7 @@ def LQ():
             "lq_fit_grid_workspace": [P(Config), i64, i64, P(sz)],
             "lq_fit_grid": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, sz],
             "lq_fit_grid_noalloc": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, vp, vp, vp],
+            "lq_pack_codes": [vp, vp, vp, i64, i64, i32, vp, i64],
             "lq_quantize_layer_workspace": [P(Config), i64, i64, P(sz)],
             "lq_quantize_layer": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, i64, vp, vp, vp, vp, vp, i32, i64,
                                   vp, vp, sz],
@@ -203,6 +204,16 @@ def lq_quantize_layer(h, cfg, W, U, codes, ws, grid=None, scale=None, zero=None,
                                   _rowmajor(U), _ptr(grid), _ptr(scale), _ptr(zero), _ptr(codes), _ptr(W_hat), whdt,
                                   ldwh, _ptr(loss_out), _ptr(ws), ws.numel() * ws.element_size()),
            "lq_quantize_layer")
+
+
+def lq_pack_codes(h, codes, bits, packed=None, stream=None):
+    """b-bit little-endian packing of the one-code-per-byte output; returns the packed tensor."""
+    r, c = codes.shape
+    nbytes = (c * bits + 7) // 8
+    if packed is None:
+        packed = torch.empty((r, nbytes), dtype=torch.uint8, device=codes.device)
+    _check(LQ().lq_pack_codes(h, _stream(stream), _ptr(codes), r, c, bits, _ptr(packed), _rowmajor(packed)), "lq_pack_codes")
+    return packed
 
 
 class LayerPass:

@@ -218,6 +218,25 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
     if (lane == 0) out.loss_rows[row] += static_cast<double>(loss);
 }
 
+// Packed output: the b-bit codes of a row as one little-endian bit stream (code j in bits
+// [j b, (j + 1) b) of the row), one thread per output byte.
+__global__ void pack_codes_kernel(const uint8_t* __restrict__ codes, int64_t r, int64_t c, int bits,
+                                  uint8_t* __restrict__ packed, int64_t ldp) {
+    const int64_t row = blockIdx.y;
+    const int64_t nbytes = (c * bits + 7) / 8;
+    for (int64_t b = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; b < nbytes; b += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t bit0 = 8 * b;
+        const int64_t j0 = bit0 / bits, j1 = (bit0 + 7) / bits;
+        uint32_t acc = 0;
+        for (int64_t j = j0; j <= j1 && j < c; ++j) {
+            const int64_t sh = j * bits - bit0;                 // position of code j relative to this byte
+            const uint32_t v = codes[row * c + j] & ((1u << bits) - 1u);
+            acc |= sh >= 0 ? (v << sh) : (v >> (-sh));
+        }
+        packed[row * ldp + b] = static_cast<uint8_t>(acc & 0xffu);
+    }
+}
+
 __global__ void zero_doubles_kernel(double* p, int64_t n) {
     const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (i < n) p[i] = 0.0;
@@ -401,5 +420,25 @@ extern "C" int lq_quantize_layer(lq_handle* h, void* stream, const lq_config* cf
         loss_reduce_kernel<<<1, 1024, 0, st>>>(loss_rows, r, loss_out);
         LQ_LAUNCH_CHECK();
     }
+    return LQ_OK;
+}
+
+extern "C" int lq_pack_codes(lq_handle* h, void* stream, const uint8_t* codes, int64_t r, int64_t c, int32_t bits,
+                             uint8_t* packed, int64_t ldp) {
+    if (!h || !codes || !packed || r <= 0 || c <= 0 || bits < 1 || bits > 8) return LQ_ERR_INVALID_ARG;
+    const int64_t nbytes = (c * bits + 7) / 8;
+    if (ldp < nbytes) return LQ_ERR_INVALID_ARG;
+    if (r > 65535) {                       // grid.y limit: rows in slabs
+        for (int64_t r0 = 0; r0 < r; r0 += 65535) {
+            const int64_t rr = r - r0 < 65535 ? r - r0 : 65535;
+            int rc = lq_pack_codes(h, stream, codes + r0 * c, rr, c, bits, packed + r0 * ldp, ldp);
+            if (rc) return rc;
+        }
+        return LQ_OK;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    dim3 g(static_cast<unsigned>(lq_ceil_div(nbytes, 256) < 64 ? lq_ceil_div(nbytes, 256) : 64), static_cast<unsigned>(r));
+    pack_codes_kernel<<<g, 256, 0, st>>>(codes, r, c, bits, packed, ldp);
+    LQ_LAUNCH_CHECK();
     return LQ_OK;
 }

@@ -387,6 +387,21 @@ def test_chained_nonuniform(lq, h, recipe, r, c, n, bits, p):
     assert abs(proxy / ref["proxy"] - 1) <= LOSS_TOL
 
 
+@pytest.mark.parametrize("r,c,n,bits", [(1, 8, 64, 2), (3, 132, 520, 3), (17, 136, 1000, 4), (130, 4, 40, 2)])
+def test_chained_tiny_and_ragged_shapes(lq, h, r, c, n, bits):
+    """Shapes far below one tile in every dimension (a single row, four columns, widths that are not
+    multiples of the 128-column block or of a warp) go through the same four calls."""
+    L = synth.make_layer("c1", r, c, n, seed=r + c)
+    W, X = f64(L.W), f64(L.X)
+    ref = O.run_pass(W, X, bits=bits, p=2.0, block=128, n_iter=10)
+    P = chained(lq, h, L, dict(grid="nonuniform", bits=bits, p=2.0, n_iter=10), what_dtype=torch.float32)
+    assert centroid_ok(f64(P.grid), ref["grid"], W)
+    codes = P.codes.cpu().numpy().astype(np.int64)
+    assert (codes != ref["codes"]).any(axis=1).sum() <= max(1, r // 20)
+    if np.array_equal(codes, ref["codes"]):
+        assert abs(P.loss.item() / ref["loss"] - 1) <= LOSS_TOL
+
+
 def test_chained_affine(lq, h):
     L = synth.make_layer("c3", 128, 1792, 8192, seed=21)
     W, X = f64(L.W), f64(L.X)
@@ -414,3 +429,12 @@ def test_invalid_arguments(lq, h):
     with pytest.raises(lq.LQError) as e:
         lq.lq_prepare_hinv(h, H, torch.empty_like(H), torch.empty(64, device="cuda"), small)
     assert e.value.code == 3
+
+
+@pytest.mark.parametrize("r,c,bits", [(5, 37, 3), (64, 4096, 4), (33, 130, 2), (2, 8, 3)])
+def test_pack_codes_bit_exact(lq, h, r, c, bits):
+    g = torch.Generator().manual_seed(r * c + bits)
+    codes = torch.randint(0, 1 << bits, (r, c), generator=g, dtype=torch.uint8)
+    packed = lq.lq_pack_codes(h, codes.cuda(), bits)
+    lq.lq_sync_status(h)
+    assert np.array_equal(packed.cpu().numpy(), O.pack_codes(codes.numpy(), bits))

@@ -393,3 +393,18 @@ def test_sample_weights_definition():
     raw = dinv ** -2.0
     np.testing.assert_allclose(s / s[0], raw / raw[0], rtol=1e-13)
     np.testing.assert_allclose(np.prod(s), 1.0, rtol=1e-12)
+
+
+# ------------------------------------------------------------- packed codes ---- #
+def test_pack_codes_by_hand_and_round_trip():
+    """2-bit codes 1, 2, 3, 0, 3 -> bits 01 10 11 00 | 11 -> bytes 0b00111001, 0b00000011 (worked by hand);
+    3-bit codes straddle bytes; packing then unpacking gives the codes back for every width."""
+    assert O.pack_codes(np.array([[1, 2, 3, 0, 3]]), 2).tolist() == [[0b00111001, 0b00000011]]
+    # 3-bit codes 5, 7, 1: bits (low first) 1,0,1, 1,1,1, 1,0,0 -> byte 0 = 0b01111101, byte 1 = 0
+    assert O.pack_codes(np.array([[5, 7, 1]]), 3).tolist() == [[0b01111101, 0b00000000]]
+    g = rng(11)
+    for bits in (2, 3, 4):
+        codes = g.integers(0, 1 << bits, size=(7, 37))
+        packed = O.pack_codes(codes, bits)
+        assert packed.shape == (7, (37 * bits + 7) // 8)
+        assert np.array_equal(O.unpack_codes(packed, bits, 37), codes)
