@@ -41,6 +41,11 @@ WORKLOADS = {
     "wide-8k-nu4": ("c2", 512, 8192, 16384, dict(grid="nonuniform", bits=4, p=4.0, n_iter=20)),
     # the other benchmark configurations (parity-test cases; timed on request with --no-e2e --no-cpu-baseline)
     "llama3-8b-q_proj-nu3": ("c2", 4096, 4096, 262144, dict(grid="nonuniform", bits=3, p=4.0, n_iter=20)),
+    # Eq. 7 at the paper's granularity (Appendix B: T = 2048, t = 0.2 T at 4 bits): 168100 candidates per group
+    "aff-2k-g128-T2048": ("c3", 2048, 2048, 65536, dict(grid="affine", bits=4, p=4.0, group=128, T=2048, t=409)),
+    "llama3-8b-q_proj-aff4row-T2048": ("c3", 4096, 4096, 262144, dict(grid="affine", bits=4, p=4.0, group=0, T=2048, t=409)),
+    "llama3-8b-down_proj-aff4g128-T2048": ("c3", 4096, 14336, 131072,
+                                           dict(grid="affine", bits=4, p=4.0, group=128, T=2048, t=409)),
     "llama3-8b-down_proj-aff4g128": ("c3", 4096, 14336, 131072, dict(grid="affine", bits=4, p=4.0, group=128, T=45, t=9)),
     "llama3-8b-down_proj-nu3": ("c3", 4096, 14336, 131072, dict(grid="nonuniform", bits=3, p=4.0, n_iter=20)),
     "llama3-8b-gate_proj-nu3": ("c2", 14336, 4096, 131072, dict(grid="nonuniform", bits=3, p=4.0, n_iter=20)),
@@ -326,12 +331,19 @@ def run_ours(args):
         else:
             s3_work = float(r) * c * st["n_iter"] * (np.log2(K) + 3)
         s3_ops = s3_work / (stage_ms[2] * 1e-3) / 1e12
+        s3_exec = None
+        if st["grid"] == "affine" and (st["t"] + 1) ** 2 >= 256 and st["T"] - 2 * st["t"] > 2 * (K - 1):
+            # Fine partitions: the library scores one representative per class of candidates that give the same
+            # grid (same t_min + t_max, same Z), ten lane-operations per weight; about this many per group:
+            classes = sum((min(st["t"], u) - max(0, u - st["t"])) * (K - 1) / (st["T"] - u) + 1 for u in range(2 * st["t"] + 1))
+            s3_exec = float(r) * c * classes * 10 / (stage_ms[2] * 1e-3) / 1e12
         s3_gbs = float(r) * c * W.element_size() / (stage_ms[2] * 1e-3) / 1e9
         s4 = float(r) * c * c / (stage_ms[3] * 1e-3) / 1e12
         stage_roof = {
             "prepare_hinv": {"bound": "fp64 tensor", "achieved": s2, "peak": fp64_peak, "unit": "TFLOP/s", "frac": s2 / fp64_peak},
             "fit_grid": {"bound": "alu", "achieved": s3_ops, "peak": lane_peak, "unit": "T lane-op/s", "frac": s3_ops / lane_peak,
-                         "hbm_gbs": s3_gbs, "hbm_frac": s3_gbs / pk["hbm"]},
+                         "hbm_gbs": s3_gbs, "hbm_frac": s3_gbs / pk["hbm"],
+                         "executed": s3_exec, "executed_frac": None if s3_exec is None else s3_exec / lane_peak},
             "quantize_layer": {"bound": "tensor", "achieved": s4, "peak": peak, "unit": "TFLOP/s", "frac": s4 / peak,
                                "executed_frac": 6 * s4 / peak},
         }

@@ -574,15 +574,59 @@ affine_search_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, int group,
     }
 }
 
+// ------------------------------------------------------- fp32 screening of candidates --
+// Both searches below score a candidate (S, Z) in fp32 first and evaluate in fp64 only those whose
+// score cannot be told from the best one.  With x = w - min:  w / S + Z = x / S + c0,  c0 = min / S + Z,
+// and the error of a weight is d = q S - x - beta,  beta = min + Z S  (S as a two-float sum).
+struct AffScore { float rS, c0, Sh, Sl, beta; };
+
+__device__ __forceinline__ AffScore aff_score_setup(double S, double Z, double dmn) {
+    AffScore a;
+    const double rS = 1.0 / S;
+    a.rS = static_cast<float>(rS);
+    a.c0 = static_cast<float>(dmn * rS + Z);
+    a.Sh = static_cast<float>(S);
+    a.Sl = static_cast<float>(S - static_cast<double>(a.Sh));
+    a.beta = static_cast<float>(dmn + Z * S);
+    return a;
+}
+
+// sum_j s_j d_j^2 over the (x, s) pairs of a group (group even)
+__device__ __forceinline__ float aff_score32(const float2* __restrict__ ws, int group, const AffScore& a, float Km1f) {
+    float a0 = 0.0f, a1 = 0.0f;
+    for (int j = 0; j < group; j += 2) {
+        const float4 p2 = *reinterpret_cast<const float4*>(ws + j);          // two (x, s) pairs
+        const float q0 = fminf(fmaxf(rintf(fmaf(p2.x, a.rS, a.c0)), 0.0f), Km1f);
+        const float q1 = fminf(fmaxf(rintf(fmaf(p2.z, a.rS, a.c0)), 0.0f), Km1f);
+        const float d0 = fmaf(q0, a.Sl, fmaf(q0, a.Sh, -p2.x)) - a.beta;
+        const float d1 = fmaf(q1, a.Sl, fmaf(q1, a.Sh, -p2.z)) - a.beta;
+        a0 = fmaf(p2.y * d0, d0, a0);
+        a1 = fmaf(p2.w * d1, d1, a1);
+    }
+    return a0 + a1;
+}
+
+// Scores up to this bar are re-examined in fp64.  The fp32 value of d carries an absolute error of at most
+// delta = 1.5e-7 R (roundings of x, of beta and of the intermediate q S - x, each below 2^-25 of a quantity
+// bounded by R or 1.5 R), hence |score - loss| <= 2 delta sqrt(sum_s loss) + delta^2 sum_s (Cauchy-Schwarz);
+// the 0.1 % on top covers the rounding of the sum itself.  When the loss is far above delta^2 sum_s, as it
+// is unless a few heavy weights are met almost exactly, the bar is 0.1 % above the best score.
+__device__ __forceinline__ float aff_bar32(float best, float R, float sum_s) {
+    const float delta = 1.5e-7f * R;
+    const float A = delta * delta * sum_s;
+    const float E = 2.0f * sqrtf(A * best) + A;
+    return best * 1.001f + 2.5f * E;
+}
+
 // ------------------------------------------------------ affine search, warp per group --
 // Groups up to AFW_MAX_GROUP weights: one warp per (row, group), lanes over the candidates
 // (t_min, t_max), the group's (w, s) pairs broadcast out of shared memory.  Every candidate is
-// first scored in fp32 (eight operations per weight); only the candidates whose fp32 loss lies
-// within 0.1 % of the best fp32 loss of the group are then evaluated in fp64 with exactly the
+// first scored in fp32 (ten operations per weight); only the candidates whose score lies below
+// aff_bar32 of the best score of the group are then evaluated in fp64 with exactly the
 // arithmetic of Eq. 7, and the arg-min (first minimum in t_min-major order) is taken over
-// those fp64 losses.  A candidate that is skipped has an fp32 loss at least 0.1 % above that of
-// an evaluated one, far outside the fp32 error of such a sum, so it cannot be the fp64 minimum:
-// the result is that of the all-fp64 search.
+// those fp64 losses.  A candidate that is skipped has a score above that of an evaluated one
+// by more than the fp32 error of both, so it cannot be the fp64 minimum: the result is that of
+// the all-fp64 search.
 constexpr int AFW_WARPS = 8;
 constexpr int AFW_MAX_GROUP = 1024;
 
@@ -593,7 +637,7 @@ affine_search_warp_kernel(const T* __restrict__ W, int64_t ldw, int group, int n
                           float* __restrict__ scale, int32_t* __restrict__ zero) {
     extern __shared__ __align__(16) unsigned char afw_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float2* ws = reinterpret_cast<float2*>(afw_smem) + static_cast<size_t>(warp) * group;      // (w, s / max s)
+    float2* ws = reinterpret_cast<float2*>(afw_smem) + static_cast<size_t>(warp) * group;      // (w - min, s / max s)
     const int64_t gid = static_cast<int64_t>(blockIdx.x) * AFW_WARPS + warp;
     if (gid >= total_groups) return;                       // whole warps leave; no block-wide barrier below
     const int64_t row = gid / n_groups;
@@ -602,21 +646,24 @@ affine_search_warp_kernel(const T* __restrict__ W, int64_t ldw, int group, int n
     const double* sp = s64 + static_cast<int64_t>(gi) * group;
 
     float mn = INFINITY, mx = -INFINITY;
-    double smax = 0.0;
+    double smax = 0.0, ssum = 0.0;
     for (int j = lane; j < group; j += 32) {
         const float w = load_w(wp + j);
         mn = fminf(mn, w);
         mx = fmaxf(mx, w);
         smax = fmax(smax, sp[j]);
+        ssum += sp[j];
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         smax = fmax(smax, __shfl_xor_sync(0xffffffffu, smax, o));
+        ssum += __shfl_xor_sync(0xffffffffu, ssum, o);
     }
     const double sinv = smax > 0.0 ? 1.0 / smax : 1.0;
-    for (int j = lane; j < group; j += 32) ws[j] = make_float2(load_w(wp + j), static_cast<float>(sp[j] * sinv));
+    const float sum_s = static_cast<float>(ssum * sinv);
+    for (int j = lane; j < group; j += 32) ws[j] = make_float2(load_w(wp + j) - mn, static_cast<float>(sp[j] * sinv));
     __syncwarp();
 
     const double dmn = mn, dmx = mx, R = dmx - dmn;
@@ -645,25 +692,12 @@ affine_search_warp_kernel(const T* __restrict__ W, int64_t ldw, int group, int n
         Z = -rint(lo / S);
         return true;
     };
-    // fp32 score: with u = w / S + Z the error of a weight is S (q - u), q = clamp(round(u))
-    auto score32 = [&](double S, double Z) {
-        const float rS = static_cast<float>(1.0 / S), Zf = static_cast<float>(Z), Sf = static_cast<float>(S);
-        float a0 = 0.0f, a1 = 0.0f;
-        for (int j = 0; j < group; j += 2) {
-            const float4 p2 = *reinterpret_cast<const float4*>(ws + j);          // two (w, s) pairs
-            const float u0 = fmaf(p2.x, rS, Zf), u1 = fmaf(p2.z, rS, Zf);
-            const float e0 = fminf(fmaxf(rintf(u0), 0.0f), Km1f) - u0;
-            const float e1 = fminf(fmaxf(rintf(u1), 0.0f), Km1f) - u1;
-            a0 = fmaf(p2.y * e0, e0, a0);
-            a1 = fmaf(p2.w * e1, e1, a1);
-        }
-        return (a0 + a1) * Sf * Sf;
-    };
+    auto score32 = [&](double S, double Z) { return aff_score32(ws, group, aff_score_setup(S, Z, dmn), Km1f); };
     // fp64 loss of one candidate, computed by the whole warp (lane l takes weights l, l + 32, ...)
     auto loss64 = [&](double S, double Z) {
         double loss = 0.0;
         for (int j = lane; j < group; j += 32) {
-            const double w = static_cast<double>(ws[j].x);
+            const double w = static_cast<double>(load_w(wp + j));
             double q = rint(w / S) + Z;
             q = fmin(fmax(q, 0.0), Km1);
             const double d = (q - Z) * S - w;
@@ -697,9 +731,9 @@ affine_search_warp_kernel(const T* __restrict__ W, int64_t ldw, int group, int n
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) best32 = fminf(best32, __shfl_xor_sync(0xffffffffu, best32, o));
-    const float bar32 = best32 * 1.001f;
+    const float bar32 = aff_bar32(best32, static_cast<float>(R), sum_s);
 
-    // pass 2: candidates within 0.1 % of the best fp32 score are evaluated in fp64, one at a time
+    // pass 2: candidates whose score is below the bar are evaluated in fp64, one at a time
     // in candidate order by the whole warp, so the first minimum wins and every lane holds the result
     double my_loss = INFINITY;
     int my_idx = 0x7fffffff;
@@ -738,6 +772,238 @@ affine_search_warp_kernel(const T* __restrict__ W, int64_t ldw, int group, int n
         scale[gid] = static_cast<float>(S);
         zero[gid] = static_cast<int32_t>(Z);
     }
+}
+
+// ------------------------------------------- affine search over classes of candidates --
+// A candidate (t_min, t_max) of Eq. 7 acts on the weights only through (S, Z).  S depends on
+// u = t_min + t_max alone (up to the last bits of its fp64 evaluation), and along a line of
+// constant u the ratio lo / S grows by (K - 1) / (T - u) per step of t_min, so Z = -rint(lo / S)
+// keeps one integer value over a run of about (T - u) / (K - 1) consecutive candidates: at the
+// paper's T = 2048 the (t + 1)^2 = 168100 candidates of the 4-bit search give only ~2400
+// different grids.  This kernel scores each class (u, Z) once, in fp32, and evaluates in fp64,
+// with the arithmetic of Eq. 7, only the first member (in t_min-major order) of every class whose
+// score lies within 0.1 % of the best; the arg-min is the lexicographic minimum of (fp64 loss,
+// candidate index) over those.  The members of a class have fp64 losses that differ by rounding
+// noise only, so this is the all-candidate search up to which member of the winning class is
+// named (same Z, S equal to ~1e-16).
+// One CTA per group.  Requires (K - 1) / (T - 2t) < 1/2: then every integer between the Z of the
+// two ends of a line is taken by some candidate on it.
+constexpr int AC_MAX_U = 2048;           // lines of constant u: 2t + 1 of them
+constexpr int AC_MAX_THREADS = 512;
+
+template <typename T>
+__global__ void __launch_bounds__(AC_MAX_THREADS)
+affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_groups, const double* __restrict__ s64, int K,
+                    int Tparts, int t_count, int p_max, float* __restrict__ scale, int32_t* __restrict__ zero,
+                    lq_dev_status* __restrict__ dstatus) {
+    extern __shared__ __align__(16) unsigned char ac_smem[];
+    const int nu = 2 * t_count + 1;
+    float2* ws = reinterpret_cast<float2*>(ac_smem);                          // (w - min, s / max s) of the group
+    int* off = reinterpret_cast<int*>(ws + group);                             // nu + 1: first class of each line
+    int* za = off + nu + 1;                                                    // nu: Z at the first candidate of the line
+    float* score = reinterpret_cast<float*>(za + nu);                          // p_max
+    int* list = reinterpret_cast<int*>(score + p_max);                         // p_max: classes to evaluate in fp64
+    __shared__ double red_d[AC_MAX_THREADS / 32], red_s[AC_MAX_THREADS / 32];
+    __shared__ float red_f[2][AC_MAX_THREADS / 32];
+    __shared__ int red_i[AC_MAX_THREADS / 32];
+    __shared__ int n_list;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x, nwarp = nthr >> 5;
+    const int64_t gid = blockIdx.x;
+    const int64_t row = gid / n_groups;
+    const int gi = static_cast<int>(gid - row * n_groups);
+    const T* wp = W + row * ldw + static_cast<int64_t>(gi) * group;
+    const double* sp = s64 + static_cast<int64_t>(gi) * group;
+
+    float mn = INFINITY, mx = -INFINITY;
+    double smax = 0.0, ssum = 0.0;
+    for (int j = tid; j < group; j += nthr) {
+        const float w = load_w(wp + j);
+        mn = fminf(mn, w);
+        mx = fmaxf(mx, w);
+        smax = fmax(smax, sp[j]);
+        ssum += sp[j];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+        mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        smax = fmax(smax, __shfl_xor_sync(0xffffffffu, smax, o));
+        ssum += __shfl_xor_sync(0xffffffffu, ssum, o);
+    }
+    if (lane == 0) { red_f[0][warp] = mn; red_f[1][warp] = mx; red_d[warp] = smax; red_s[warp] = ssum; }
+    if (tid == 0) n_list = 0;
+    __syncthreads();
+    ssum = 0.0;
+    for (int w = 0; w < nwarp; ++w) {
+        mn = fminf(mn, red_f[0][w]); mx = fmaxf(mx, red_f[1][w]); smax = fmax(smax, red_d[w]); ssum += red_s[w];
+    }
+    __syncthreads();                                  // the scratch is reused below
+    const double sinv = smax > 0.0 ? 1.0 / smax : 1.0;
+    const float sum_s = static_cast<float>(ssum * sinv);
+    for (int j = tid; j < group; j += nthr) ws[j] = make_float2(load_w(wp + j) - mn, static_cast<float>(sp[j] * sinv));
+
+    const double dmn = mn, dmx = mx, R = dmx - dmn;
+    const double Km1 = static_cast<double>(K - 1);
+    const double dT = static_cast<double>(Tparts);
+    if (R == 0.0) {                                // constant group
+        if (tid == 0) {
+            double lo = fmin(dmn, 0.0), hi = fmax(dmx, 0.0);
+            double S = 1.0, Z = 0.0;
+            if (hi != lo) { S = (hi - lo) / Km1; Z = -rint(lo / S); }
+            scale[gid] = static_cast<float>(S);
+            zero[gid] = static_cast<int32_t>(Z);
+        }
+        return;
+    }
+    const int side = t_count + 1;
+    // (S, Z) of a candidate exactly as Eq. 7 gives them; false when the candidate is void
+    auto params = [&](int t_min, int t_max, double& S, double& Z) {
+        const double lo = dmn + static_cast<double>(t_min) * R / dT;
+        const double hi = dmx - static_cast<double>(t_max) * R / dT;
+        S = (hi - lo) / Km1;
+        if (!(S > 0.0)) return false;
+        Z = -rint(lo / S);
+        return true;
+    };
+
+    // classes per line of constant u, then their exclusive prefix sum
+    for (int u = tid; u < nu; u += nthr) {
+        const int a = max(0, u - t_count), b = min(t_count, u);
+        double Sa, Za, Sb, Zb;
+        int cnt = 0, z0 = 0;
+        if (params(a, u - a, Sa, Za) && params(b, u - b, Sb, Zb) && fabs(Za) < 1e9 && fabs(Zb) < 1e9) {
+            z0 = static_cast<int>(Za);
+            cnt = max(z0 - static_cast<int>(Zb), 0) + 1;
+        }
+        za[u] = z0;
+        off[u] = cnt;
+    }
+    __syncthreads();
+    {
+        const int per = (nu + nthr - 1) / nthr;
+        const int lo_u = min(tid * per, nu), hi_u = min(lo_u + per, nu);
+        int sum = 0;
+        for (int u = lo_u; u < hi_u; ++u) sum += off[u];
+        int incl = sum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
+        }
+        if (lane == 31) red_i[warp] = incl;
+        __syncthreads();
+        int base = incl - sum;
+        for (int w = 0; w < warp; ++w) base += red_i[w];
+        for (int u = lo_u; u < hi_u; ++u) { const int cnt = off[u]; off[u] = base; base += cnt; }
+        if (tid == nthr - 1) off[nu] = base;
+    }
+    __syncthreads();
+    int P = off[nu];
+    if (P > p_max) {                                // cannot happen with the host's bound; never write past the arrays
+        if (tid == 0) lq_report(dstatus, LQ_ERR_UNSUPPORTED, gid);
+        P = p_max;
+    }
+    // line and Z of class p
+    auto class_of = [&](int p, int& u, int& Z) {
+        int lo_u = 0, hi_u = nu - 1;
+        while (lo_u < hi_u) {                        // the last line whose first class is <= p
+            const int mid = (lo_u + hi_u + 1) >> 1;
+            if (off[mid] <= p) lo_u = mid; else hi_u = mid - 1;
+        }
+        u = lo_u;
+        Z = za[u] - (p - off[u]);
+    };
+    const double c_s = R / (dT * Km1);               // S of line u = c_s (T - u)
+    const float Km1f = static_cast<float>(K - 1);
+
+    // fp32 score of every class
+    float best32 = INFINITY;
+    for (int p = tid; p < P; p += nthr) {
+        int u, Zi;
+        class_of(p, u, Zi);
+        const AffScore as = aff_score_setup(c_s * static_cast<double>(Tparts - u), static_cast<double>(Zi), dmn);
+        float sc = aff_score32(ws, group, as, Km1f);
+        if (sc != sc) sc = -INFINITY;                // a NaN score is always re-examined in fp64
+        score[p] = sc;
+        best32 = fminf(best32, sc == -INFINITY ? INFINITY : sc);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) best32 = fminf(best32, __shfl_xor_sync(0xffffffffu, best32, o));
+    if (lane == 0) red_f[0][warp] = best32;
+    __syncthreads();
+    for (int w = 0; w < nwarp; ++w) best32 = fminf(best32, red_f[0][w]);
+    const float bar32 = aff_bar32(best32, static_cast<float>(R), sum_s);
+    for (int p = tid; p < P; p += nthr)
+        if (score[p] <= bar32) list[atomicAdd(&n_list, 1)] = p;
+    __syncthreads();
+    const int n_eval = n_list;
+
+    // fp64 loss of the first member of each listed class, one class per warp at a time
+    double my_loss = INFINITY;
+    int my_idx = 0x7fffffff;
+    for (int i = warp; i < n_eval; i += nwarp) {
+        int u, Zi;
+        class_of(list[i], u, Zi);
+        const int a = max(0, u - t_count), b = min(t_count, u);
+        const double Zd = static_cast<double>(Zi);
+        // first t_min on the line with rint(lo / S) >= -Z, i.e. with Z(t_min) <= Z: estimate, then settle exactly
+        const double S_u = c_s * static_cast<double>(Tparts - u);
+        double est = ceil(((-Zd - 0.5) * S_u - dmn) * dT / R);
+        int tm = static_cast<int>(fmin(fmax(est, static_cast<double>(a)), static_cast<double>(b)));
+        double S, Z;
+        for (int it = 0; it < 8 && tm > a; ++it) {
+            if (params(tm - 1, u - tm + 1, S, Z) && Z <= Zd) --tm; else break;
+        }
+        for (int it = 0; it < 8 && tm < b; ++it) {
+            if (params(tm, u - tm, S, Z) && Z > Zd) ++tm; else break;
+        }
+        if (!params(tm, u - tm, S, Z) || Z != Zd) continue;       // no candidate of the line has this Z
+        double loss = 0.0;
+        for (int j = lane; j < group; j += 32) {
+            const double w = static_cast<double>(load_w(wp + j));
+            double q = rint(w / S) + Z;
+            q = fmin(fmax(q, 0.0), Km1);
+            const double d = (q - Z) * S - w;
+            loss += sp[j] * (d * d);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
+        const int idx = tm * side + (u - tm);
+        if (loss < my_loss || (loss == my_loss && idx < my_idx)) { my_loss = loss; my_idx = idx; }
+    }
+    if (lane == 0) { red_d[warp] = my_loss; red_i[warp] = my_idx; }
+    __syncthreads();
+    if (tid == 0) {
+        for (int w = 1; w < nwarp; ++w)
+            if (red_d[w] < my_loss || (red_d[w] == my_loss && red_i[w] < my_idx)) { my_loss = red_d[w]; my_idx = red_i[w]; }
+        double S = 1.0, Z = 0.0;
+        if (my_idx != 0x7fffffff) {
+            const int t_min = my_idx / side;
+            params(t_min, my_idx - t_min * side, S, Z);
+        }
+        scale[gid] = static_cast<float>(S);
+        zero[gid] = static_cast<int32_t>(Z);
+    }
+}
+
+// Whether the class kernel applies, and an upper bound of the classes of one group: a line whose lo / S spans
+// a width d takes at most floor(d) + 2 integer values of Z.
+bool affine_class_plan(int K, int Tparts, int t_count, int64_t g, int* p_max, size_t* smem) {
+    const int nu = 2 * t_count + 1;
+    if (nu > AC_MAX_U || g % 2 != 0 || Tparts - 2 * t_count <= 2 * (K - 1)) return false;
+    if (static_cast<int64_t>(t_count + 1) * (t_count + 1) < 256) return false;       // few candidates: score them all
+    int64_t total = 0;
+    for (int u = 0; u < nu; ++u) {
+        const int a = u > t_count ? u - t_count : 0, b = u < t_count ? u : t_count;
+        total += static_cast<int64_t>(static_cast<double>(b - a) * (K - 1) / static_cast<double>(Tparts - u)) + 2;
+    }
+    const size_t bytes = static_cast<size_t>(g) * sizeof(float2) + static_cast<size_t>(2 * nu + 1) * sizeof(int) +
+                         static_cast<size_t>(total) * (sizeof(float) + sizeof(int));
+    if (bytes > 200 * 1024) return false;
+    *p_max = static_cast<int>(total);
+    *smem = bytes;
+    return true;
 }
 
 int check_cfg(const lq_config* cfg) {
@@ -807,6 +1073,26 @@ extern "C" int lq_fit_grid(lq_handle* h, void* stream, const lq_config* cfg, con
     const int64_t g = cfg->group_size == 0 ? c : cfg->group_size;
     const int n_groups = static_cast<int>(c / g);
     const int K = 1 << cfg->bits;
+    int p_max = 0;
+    size_t smem_c = 0;
+    if (affine_class_plan(K, cfg->T, cfg->t_count, g, &p_max, &smem_c)) {
+        static bool attr_c = false;
+        if (!attr_c) {
+            LQ_CUDA_TRY(cudaFuncSetAttribute(affine_class_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+            LQ_CUDA_TRY(cudaFuncSetAttribute(affine_class_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+            attr_c = true;
+        }
+        const unsigned nb = static_cast<unsigned>(r * n_groups);
+        const int threads = g > 8192 ? 512 : 256;
+        if (w_dtype == LQ_F32)
+            affine_class_kernel<float><<<nb, threads, smem_c, st>>>(static_cast<const float*>(W), ldw, (int)g, n_groups, s64, K, cfg->T,
+                                                                   cfg->t_count, p_max, scale, zero, h->dstatus);
+        else
+            affine_class_kernel<__nv_bfloat16><<<nb, threads, smem_c, st>>>(static_cast<const __nv_bfloat16*>(W), ldw, (int)g, n_groups,
+                                                                           s64, K, cfg->T, cfg->t_count, p_max, scale, zero, h->dstatus);
+        LQ_LAUNCH_CHECK();
+        return LQ_OK;
+    }
     if (g <= AFW_MAX_GROUP && g % 2 == 0) {
         const int64_t total = r * n_groups;
         const size_t smem_w = static_cast<size_t>(AFW_WARPS) * g * sizeof(float2);

@@ -288,6 +288,60 @@ def test_stage3_affine(lq, h, r, c, bits, group, T, t):
     assert same.mean() >= 0.995       # a different pick only where two candidates tie to rounding
 
 
+def _check_affine_picks(W, dinv, bits, group, T, t, scale, zero, So, Zo, p=4.0):
+    """Pairs (S, Z) that differ from the oracle's must be candidates of the search whose loss, evaluated
+    by the oracle's arithmetic, equals the oracle's minimum up to rounding (several candidates give one
+    grid: Z is an integer and S depends on t_min + t_max only)."""
+    K = 1 << bits
+    r, c = W.shape
+    g = c if group == 0 else group
+    s = O.sample_weights(dinv, p)
+    same = (zero == Zo) & (np.abs(scale / So - 1) < 1e-6)
+    for i, gi in np.argwhere(~same):
+        w, sg = W[i, gi * g:(gi + 1) * g], s[gi * g:(gi + 1) * g]
+        mn, mx = w.min(), w.max()
+        R = mx - mn
+        found = None
+        for t_min in range(t + 1):
+            lo = mn + t_min * R / T
+            hi = mx - np.arange(t + 1) * R / T
+            S = (hi - lo) / (K - 1)
+            ok = S > 0
+            Z = -np.rint(lo / np.where(ok, S, 1.0))
+            hit = ok & (Z == zero[i, gi]) & (S.astype(np.float32) == np.float32(scale[i, gi]))
+            if hit.any():
+                found = S[np.argmax(hit)]
+                break
+        assert found is not None, "the pair is no candidate of Eq. 7"
+        loss_gpu = (sg * (O.quant_aff(w, found, float(zero[i, gi]), K) - w) ** 2).sum()
+        loss_ref = (sg * (O.quant_aff(w, So[i, gi], Zo[i, gi], K) - w) ** 2).sum()
+        assert loss_gpu <= loss_ref * (1 + 1e-9)
+    return same.mean()
+
+
+# fine partitions of the range (many candidates share one grid: the search over classes of candidates) and
+# heavy-tailed sample weights (a few weights met almost exactly: the fp32 screening must not drop the winner)
+@pytest.mark.parametrize("r,c,bits,group,T,t,recipe", [(12, 256, 4, 128, 256, 51, "c3"), (8, 512, 3, 64, 512, 153, "c2"),
+                                                      (6, 512, 4, 0, 256, 51, "c3"), (4, 256, 2, 128, 256, 102, "c2"),
+                                                      (5, 384, 4, 128, 100, 30, "c1"), (6, 384, 4, 128, 45, 9, "c1"),
+                                                      (8, 512, 3, 128, 45, 13, "c2"),
+                                                      (3, 256, 4, 128, 2048, 409, "c3")])
+def test_stage3_affine_fine_partition(lq, h, r, c, bits, group, T, t, recipe):
+    L = synth.make_layer(recipe, r, c, 2 * c, seed=T + bits)
+    _, dinv, _, _ = O.prepare_hinv(O.hessian(f64(L.X)), 0.01)
+    dinv32 = torch.from_numpy(dinv).float()
+    So, Zo = O.fit_grid_affine(f64(L.W), f64(dinv32), bits, 4.0, group, T, t)
+    cfg = lq.Config.make(grid="affine", bits=bits, p=4.0, group=group, T=T, t=t)
+    ng = 1 if group == 0 else c // group
+    scale = torch.empty(r, ng, device="cuda")
+    zero = torch.empty(r, ng, dtype=torch.int32, device="cuda")
+    ws = ws_for(lq, lq.lq_fit_grid_workspace(cfg, r, c))
+    lq.lq_fit_grid(h, cfg, L.W.cuda(), dinv32.cuda(), ws, scale=scale, zero=zero)
+    lq.lq_sync_status(h)
+    frac = _check_affine_picks(f64(L.W), f64(dinv32), bits, group, T, t, f64(scale), zero.cpu().numpy(), So, Zo)
+    assert frac >= 0.98
+
+
 def test_stage3_affine_constant_group(lq, h):
     W = torch.full((2, 128), 0.25)
     W[1] = 0.0
