@@ -373,13 +373,113 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------- a whole decoder block ----
+# Benchmark config 4: the seven linear layers of one Llama-3-8B-shaped decoder block, 3-bit non-uniform,
+# n = 131072 tokens.  Layers that read the same activations share stages 1-2 (one Hessian for q/k/v, one for o,
+# one for gate/up, one for down), which is how a model-level driver would call the library.
+BLOCKS = {
+    "llama3-8b-block-nu3": dict(
+        n=131072, settings=dict(grid="nonuniform", bits=3, p=4.0, n_iter=20),
+        inputs=[("attn_in", 4096, "c2", [("q_proj", 4096), ("k_proj", 1024), ("v_proj", 1024)]),
+                ("o_in", 4096, "c2", [("o_proj", 4096)]),
+                ("mlp_in", 4096, "c2", [("gate_proj", 14336), ("up_proj", 14336)]),
+                ("down_in", 14336, "c3", [("down_proj", 4096)])]),
+}
+
+
+def run_block(args):
+    import paper_2407_10032_b200 as lq
+    rank, world, local = dist_env()
+    if world > 1:
+        raise SystemExit("bench.py: the block workload runs on one GPU")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    spec = BLOCKS[args.workload]
+    n, st = spec["n"], spec["settings"]
+    cfg = lq.Config.make(**st)
+    h = lq.lq_create(local)
+    stream = torch.cuda.current_stream()
+    groups = []
+    for gi, (name, c, recipe, layers) in enumerate(spec["inputs"]):
+        Ws, passes, X = [], [], None
+        for li, (lname, r) in enumerate(layers):
+            layer = synth.make_layer(recipe, r, c, n if li == 0 else 256, seed=layer_seed(rank) + 16 * gi + li, device=dev)
+            if li == 0:
+                X = layer.X
+            Ws.append(layer.W)
+            passes.append(lq.LayerPass(h, r, c, cfg, w_dtype=layer.W.dtype, x_dtype=X.dtype, n_chunk=n, device=dev,
+                                       want_w_hat=False))
+            del layer
+        groups.append((name, c, X, [l[0] for l in layers], Ws, passes))
+
+    def one_step(events=None):
+        k = 0
+        for name, c, X, lnames, Ws, passes in groups:
+            P0 = passes[0]
+            P0.H.zero_()
+            lq.lq_hessian_accumulate(h, X, P0.H, 2.0, P0.ws)
+            lq.lq_hessian_finalize(h, P0.H)
+            lq.lq_prepare_hinv(h, P0.H, P0.U, P0.dinv, P0.ws, 0.01, Ws[0])
+            if events: events[k].record(stream)
+            k += 1
+            for W, P in zip(Ws, passes):
+                lq.lq_fit_grid(h, cfg, W, P0.dinv, P.ws, P.grid, P.scale, P.zero)
+                lq.lq_quantize_layer(h, cfg, W, P0.U, P.codes, P.ws, P.grid, P.scale, P.zero, None, P.loss)
+                if events: events[k].record(stream)
+                k += 1
+
+    n_ev = sum(1 + len(g[3]) for g in groups)
+    for _ in range(args.warmup):
+        one_step()
+    lq.lq_sync_status(h)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(n_ev)] for _ in range(args.steps)]
+    e_beg, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = lq.lq_launch_count()
+    torch.cuda.synchronize()
+    e_beg.record(stream)
+    for i in range(args.steps):
+        one_step(evs[i])
+    e_end.record(stream)
+    torch.cuda.synchronize()
+    launches = lq.lq_launch_count() - launches0
+    total_ms = e_beg.elapsed_time(e_end)
+    clocks = sampler.stop()
+    lq.lq_sync_status(h)
+    names = []
+    for name, c, X, lnames, Ws, passes in groups:
+        names.append("hessian+prepare:" + name)
+        names.extend(lnames)
+    parts = {}
+    for j, nm in enumerate(names):
+        beg = [e_beg if (i == 0 and j == 0) else (evs[i - 1][-1] if j == 0 else evs[i][j - 1]) for i in range(args.steps)]
+        parts[nm] = float(np.mean([beg[i].elapsed_time(evs[i][j]) for i in range(args.steps)]))
+    weights = sum(W.numel() for g in groups for W in g[4])
+    ms_per_step = total_ms / args.steps
+    print(json.dumps({
+        "metric": "weights quantized/sec per linear layer", "value": weights / (ms_per_step * 1e-3), "unit": "weights/s",
+        "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": args.workload, "weights": weights, "n_tokens": n, **st, "block": 128, "damp": 0.01,
+                   "sharing": "stages 1-2 once per distinct input (4 Hessians for 7 layers)",
+                   "l2": "each Hessian input (1 to 3.8 GB) exceeds the 126 MiB L2"},
+        "part_ms": parts, "roofline": None, "cpu_baseline": None, "e2e": None, "gpu_launches": int(launches),
+        "clocks": clocks}))
+    lq.lq_destroy(h)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="llama3-8b-q_proj-nu4", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="llama3-8b-q_proj-nu4", choices=sorted(WORKLOADS) + sorted(BLOCKS))
     ap.add_argument("--ref-tokens", type=int, default=32768)
     ap.add_argument("--ref-rows", type=int, default=512)
     ap.add_argument("--chunk", type=int, default=0, help="tokens per Hessian call (0 = all at once)")
@@ -387,7 +487,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true",
                     help="skip the oracle timing leg (profiler captures only; cpu_baseline is then null)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.workload in BLOCKS:
+        if args.impl == "reference":
+            raise SystemExit("bench.py: the block workload has no reference arm; use a single-layer workload")
+        run_block(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

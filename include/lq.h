@@ -120,6 +120,14 @@ int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64_t c, int64
                     void* W, int32_t w_dtype, int64_t r, int64_t ldw,
                     void* ws, size_t ws_bytes);
 
+/* d[j] = U[j][j]: the diagonal of the factor written by lq_prepare_hinv.  Algorithm 1 keeps the
+ * symbol H^-1 for the Cholesky factor after line 4, so its lines 6 and 8, read to the letter,
+ * weight the grid objective by the diagonal of the factor, diag(U)^-p, instead of the diagonal of
+ * the inverse that Eq. 5 / Eq. 7 name.  Passing d to lq_fit_grid in place of dinv gives that
+ * variant (U_jj^2 is the inverse-Hessian diagonal of weight j at the moment the column loop
+ * reaches it).  U: device fp32 c x c, ldu >= c; d: device fp32[c]. */
+int lq_chol_diag(lq_handle* h, void* stream, const float* U, int64_t c, int64_t ldu, float* d);
+
 /* ---- stage 3: loss-error-aware grid, Eq. 5 (non-uniform) / Eq. 7 (affine) ------------ */
 
 /* Non-uniform: for every row k, K = 2^bits centroids by weighted 1-D k-means with sample

@@ -17,7 +17,9 @@ explicit inverse-Hessian downdate (column loop), the trace identity of the dampe
 proxy loss, H = I giving round-to-nearest, dynamic-programming optimal weighted
 1-D k-means, an independently written plain Lloyd for p = 0, the worked 2-bit grid
 example of Appendix A, a triple-loop affine search, textbook library inverses and
-Cholesky factors, and scale / permutation / row-subset invariances.  The numbers
+Cholesky factors, and scale / permutation / row-subset invariances; Algorithm 2
+(quantize_exact) against principal-submatrix inverses recomputed at every step, the
+identity sum of loss errors = 1/2 dw H dw^T, H = I, and Algorithm 1 in natural order.  The numbers
 it produces on the benchmark configurations themselves are not printed anywhere in
 the paper: for those, parity is "unpinned" beyond these properties.
 """
@@ -301,6 +303,91 @@ def quantize_layer(W, U, *, grid=None, scale=None, zero=None, bits: int = 4,
     return codes, What, loss
 
 
+# --------------------------------------------------------------------------- #
+# Algorithm 2 (Appendix, "LeanQuant-Exact"): greedy order, full inverse-Hessian downdate per row
+# --------------------------------------------------------------------------- #
+def quantize_exact(W, Hinv, *, grid=None, scale=None, zero=None, bits: int = 4, group: int = 0,
+                   order: str = "greedy", return_order: bool = False):
+    """Algorithm 2, rows independent.  For a row w with its own copy of the inverse Hessian:
+    repeat c times { among the weights not yet quantised pick i with the least
+    (quant(w_i) - w_i)^2 / (2 Hinv_ii) (the loss error of Eq. 3; ties: lowest index);
+    w_hat_i = quant(w_i);  w <- w - Hinv[:, i] / Hinv_ii * (w_i - w_hat_i)  (Eq. 3's update);
+    Hinv <- Hinv - Hinv[:, i] Hinv[i, :] / Hinv_ii  (Eq. 9, removes i) }.
+
+    The grid (non-uniform ``grid`` r x K, or ``scale`` / ``zero`` r x n_groups) is fitted beforehand on
+    the original row, as lines 3-7 of the algorithm say.  ``Hinv`` is the c x c inverse the caller
+    chose (Algorithm 2 writes (2 X X^T)^-1; the dampening of Algorithm 1 is the caller's decision).
+    ``order="natural"`` replaces the greedy choice by i = 0, 1, 2, ... (OBQ in fixed order, which is
+    what Algorithm 1 computes through the Cholesky factor); used by the pins.
+
+    Returns codes (r x c int64), W_hat (r x c), loss = sum of the chosen loss errors, and with
+    ``return_order`` the r x c array of indices in the order they were quantised."""
+    W = np.asarray(W, dtype=F64)
+    Hinv0 = np.asarray(Hinv, dtype=F64)
+    r, c = W.shape
+    K = 1 << bits
+    g = c if group in (0, None) else group
+    codes = np.zeros((r, c), dtype=np.int64)
+    What = np.zeros((r, c), dtype=F64)
+    orders = np.zeros((r, c), dtype=np.int64)
+    loss = 0.0
+    cols = np.arange(c)
+    for row in range(r):
+        w = W[row].copy()
+        Hi = Hinv0.copy()
+        todo = np.ones(c, dtype=bool)
+        for step in range(c):
+            if grid is not None:
+                a = assign_nu(w[None, :], grid[row:row + 1])[0]
+                q = grid[row][a]
+            else:
+                S = scale[row, cols // g]
+                Z = zero[row, cols // g]
+                a = affine_codes(w, S, Z, K)
+                q = (a - Z) * S
+            if order == "greedy":
+                score = np.full(c, np.inf)
+                score[todo] = (q[todo] - w[todo]) ** 2 / (2.0 * np.diag(Hi)[todo])
+                i = int(np.argmin(score))                       # first minimum
+            else:
+                i = step
+            dii = Hi[i, i]
+            err = w[i] - q[i]
+            loss += err * err / (2.0 * dii)
+            codes[row, i] = a[i]
+            What[row, i] = q[i]
+            orders[row, step] = i
+            col = Hi[:, i].copy()
+            w -= col / dii * err
+            w[i] = q[i]
+            Hi -= np.outer(col, col) / dii
+            Hi[i, :] = 0.0
+            Hi[:, i] = 0.0
+            todo[i] = False
+    if return_order:
+        return codes, What, loss, orders
+    return codes, What, loss
+
+
+def run_exact(W, X, *, grid_type="nonuniform", bits=4, p=4.0, damp=0.01, n_iter=20, init="uniform",
+              group=0, T=2048, t=None, alpha=2.0):
+    """Algorithm 2 end to end with the dampening of Algorithm 1 (damp = 0 gives (2 X X^T)^-1 to the letter)."""
+    H = hessian(X, alpha)
+    U, dinv, H_d, Wf = prepare_hinv(H, damp, W)
+    Hinv = U.T @ U
+    out = dict(H=H, U=U, dinv=dinv, H_d=H_d, Hinv=Hinv)
+    if grid_type == "nonuniform":
+        G = fit_grid_nonuniform(Wf, dinv, bits, p, n_iter, init)
+        codes, What, loss = quantize_exact(Wf, Hinv, grid=G, bits=bits)
+        out.update(grid=G)
+    else:
+        S, Z = fit_grid_affine(Wf, dinv, bits, p, group, T, t)
+        codes, What, loss = quantize_exact(Wf, Hinv, scale=S, zero=Z, bits=bits, group=group)
+        out.update(scale=S, zero=Z)
+    out.update(codes=codes, W_hat=What, loss=loss, proxy=proxy_loss(Wf, What, H), proxy_d=proxy_loss(Wf, What, H_d))
+    return out
+
+
 def pack_codes(codes, bits: int) -> np.ndarray:
     """Storage format behind the paper's bit columns: every row's b-bit codes as one little-endian
     bit stream (code j in bits [j b, (j+1) b) of the row), padded with zero bits to whole bytes."""
@@ -346,11 +433,18 @@ def minmax_affine_params(W, bits: int, group: int = 0):
 
 
 def run_pass(W, X, *, grid_type="nonuniform", bits=4, p=4.0, block=128, damp=0.01,
-             n_iter=20, init="uniform", group=0, T=2048, t=None, alpha=2.0):
-    """Algorithm 1 end to end; returns a dict with every intermediate."""
+             n_iter=20, init="uniform", group=0, T=2048, t=None, alpha=2.0, weight_src="inv_diag"):
+    """Algorithm 1 end to end; returns a dict with every intermediate.
+    ``weight_src``: "inv_diag" weights the grid objective by diag(H_d^-1)^-p as Eq. 5 / Eq. 7 say;
+    "chol_diag" by diag(U)^-p, Algorithm 1 lines 6 and 8 read to the letter (the symbol H^-1 holds
+    the Cholesky factor from line 4 on)."""
     H = hessian(X, alpha)
     U, dinv, H_d, Wf = prepare_hinv(H, damp, W)
     out = dict(H=H, U=U, dinv=dinv, H_d=H_d)
+    if weight_src == "chol_diag":
+        dinv = np.diag(U).copy()
+    elif weight_src != "inv_diag":
+        raise ValueError("weight_src")
     if grid_type == "nonuniform":
         G = fit_grid_nonuniform(Wf, dinv, bits, p, n_iter, init)
         codes, What, loss = quantize_layer(Wf, U, grid=G, bits=bits, block=block)

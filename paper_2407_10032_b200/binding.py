@@ -64,6 +64,7 @@ def LQ():
             "lq_hessian_finalize": [vp, vp, vp, i64, i64],
             "lq_prepare_hinv_workspace": [i64, P(sz)],
             "lq_prepare_hinv": [vp, vp, vp, i64, i64, f32, vp, i64, vp, vp, i32, i64, i64, vp, sz],
+            "lq_chol_diag": [vp, vp, vp, i64, i64, vp],
             "lq_fit_grid_workspace": [P(Config), i64, i64, P(sz)],
             "lq_fit_grid": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, sz],
             "lq_fit_grid_noalloc": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, vp, vp, vp],
@@ -170,6 +171,15 @@ def lq_prepare_hinv(h, H, U, dinv, ws, damp_frac=0.01, W=None, stream=None):
            "lq_prepare_hinv")
 
 
+def lq_chol_diag(h, U, d=None, stream=None):
+    """Diagonal of the factor U, for the variant of the grid objective weighted by diag(U)^-p."""
+    c = U.shape[0]
+    if d is None:
+        d = torch.empty((c,), dtype=torch.float32, device=U.device)
+    _check(LQ().lq_chol_diag(h, _stream(stream), _ptr(U), c, _rowmajor(U), _ptr(d)), "lq_chol_diag")
+    return d
+
+
 def lq_fit_grid_workspace(cfg, r, c) -> int:
     b = C.c_size_t(0)
     _check(LQ().lq_fit_grid_workspace(C.byref(cfg), r, c, C.byref(b)), "lq_fit_grid_workspace")
@@ -222,7 +232,10 @@ class LayerPass:
     Allocation only (through torch's allocator); all arithmetic is in liblq."""
 
     def __init__(self, handle, r, c, cfg: Config, w_dtype=torch.bfloat16, x_dtype=torch.bfloat16, n_chunk=0,
-                 device="cuda", want_w_hat=True):
+                 device="cuda", want_w_hat=True, weight_src="inv_diag"):
+        if weight_src not in ("inv_diag", "chol_diag"):
+            raise ValueError("weight_src: 'inv_diag' (Eq. 5 / Eq. 7) or 'chol_diag' (Algorithm 1 to the letter)")
+        self.weight_src = weight_src
         self.h, self.r, self.c, self.cfg = handle, r, c, cfg
         dev = torch.device(device)
         K = 1 << cfg.bits
@@ -249,6 +262,8 @@ class LayerPass:
         """Stages 2-4 after all chunks were accumulated."""
         lq_hessian_finalize(self.h, self.H)
         lq_prepare_hinv(self.h, self.H, self.U, self.dinv, self.ws, damp_frac, W)
+        if self.weight_src == "chol_diag":
+            lq_chol_diag(self.h, self.U, self.dinv)
         lq_fit_grid(self.h, self.cfg, W, self.dinv, self.ws, self.grid, self.scale, self.zero)
         lq_quantize_layer(self.h, self.cfg, W, self.U, self.codes, self.ws, self.grid, self.scale, self.zero,
                           self.W_hat, self.loss)

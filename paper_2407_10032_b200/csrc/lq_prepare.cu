@@ -620,3 +620,18 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
     }
     return LQ_OK;
 }
+
+// ------------------------------------------------------------ diagonal of the factor --
+namespace {
+__global__ void chol_diag_kernel(const float* __restrict__ U, int64_t c, int64_t ldu, float* __restrict__ d) {
+    const int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (j < c) d[j] = U[j * ldu + j];
+}
+}  // namespace
+
+extern "C" int lq_chol_diag(lq_handle* h, void* stream, const float* U, int64_t c, int64_t ldu, float* d) {
+    if (!h || !U || !d || c <= 0 || ldu < c) return LQ_ERR_INVALID_ARG;
+    chol_diag_kernel<<<static_cast<unsigned>(lq_ceil_div(c, 256)), 256, 0, static_cast<cudaStream_t>(stream)>>>(U, c, ldu, d);
+    LQ_LAUNCH_CHECK();
+    return LQ_OK;
+}

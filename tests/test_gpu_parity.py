@@ -417,10 +417,11 @@ def test_stage4_identity_hessian_is_round_to_nearest(lq, h):
 
 
 # ------------------------------------------------------------------ chained -------- #
-def chained(lq, h, L, cfg_kw, what_dtype=None):
+def chained(lq, h, L, cfg_kw, what_dtype=None, weight_src="inv_diag"):
     r, c, n = L.r, L.c, L.n
     cfg = lq.Config.make(**cfg_kw)
-    P = lq.LayerPass(h, r, c, cfg, w_dtype=what_dtype or L.W.dtype, x_dtype=L.X.dtype, n_chunk=n, device="cuda")
+    P = lq.LayerPass(h, r, c, cfg, w_dtype=what_dtype or L.W.dtype, x_dtype=L.X.dtype, n_chunk=n, device="cuda",
+                     weight_src=weight_src)
     P.run(L.W.cuda(), L.X.cuda())
     lq.lq_sync_status(h)
     return P
@@ -454,6 +455,20 @@ def test_chained_tiny_and_ragged_shapes(lq, h, r, c, n, bits):
     assert (codes != ref["codes"]).any(axis=1).sum() <= max(1, r // 20)
     if np.array_equal(codes, ref["codes"]):
         assert abs(P.loss.item() / ref["loss"] - 1) <= LOSS_TOL
+
+
+def test_chained_weighted_by_factor_diagonal(lq, h):
+    """Algorithm 1 to the letter: the grid objective weighted by diag(U)^-p (lq_chol_diag feeds lq_fit_grid)."""
+    L = synth.make_layer("c2", 192, 768, 8192, seed=31)
+    W, X = f64(L.W), f64(L.X)
+    ref = O.run_pass(W, X, bits=4, p=4.0, block=128, n_iter=20, weight_src="chol_diag")
+    plain = O.run_pass(W, X, bits=4, p=4.0, block=128, n_iter=20)
+    assert np.abs(ref["grid"] - plain["grid"]).max() > 1e-4 * np.abs(plain["grid"]).max()     # the variant is another grid
+    P = chained(lq, h, L, dict(grid="nonuniform", bits=4, p=4.0, n_iter=20), what_dtype=torch.float32, weight_src="chol_diag")
+    np.testing.assert_allclose(f64(P.dinv), np.diag(ref["U"]), rtol=2e-5)
+    assert centroid_ok(f64(P.grid), ref["grid"], W)
+    assert codes_budget(P.codes.cpu().numpy().astype(np.int64), ref["codes"])
+    assert abs(P.loss.item() / ref["loss"] - 1) <= LOSS_TOL
 
 
 def test_chained_affine(lq, h):

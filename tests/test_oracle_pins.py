@@ -408,3 +408,92 @@ def test_pack_codes_by_hand_and_round_trip():
         packed = O.pack_codes(codes, bits)
         assert packed.shape == (7, (37 * bits + 7) // 8)
         assert np.array_equal(O.unpack_codes(packed, bits, 37), codes)
+
+
+# ---------------------------------------------------- Algorithm 2 (LeanQuant-Exact) ---- #
+def exact_by_submatrix_inverses(w, H, quant):
+    """Algorithm 2 for one row without the Eq. 9 downdate: the inverse of the remaining problem is
+    recomputed at every step as the inverse of the principal submatrix of H over the weights not yet
+    quantised (what removing a row and a column from the inverse stands for), and Eq. 3 is applied
+    with it."""
+    w = w.copy()
+    c = w.size
+    todo = list(range(c))
+    what = np.zeros(c)
+    order = []
+    eps = 0.0
+    while todo:
+        Hi = np.linalg.inv(H[np.ix_(todo, todo)])
+        q = np.array([quant(w[j]) for j in todo])
+        score = (q - w[todo]) ** 2 / (2.0 * np.diag(Hi))
+        k = int(np.argmin(score))
+        i = todo[k]
+        eps += score[k]
+        delta = -(w[i] - q[k]) / Hi[k, k] * Hi[:, k]
+        for m, j in enumerate(todo):
+            w[j] += delta[m]
+        w[i] = q[k]
+        what[i] = q[k]
+        order.append(i)
+        todo.pop(k)
+    return what, eps, order
+
+
+@pytest.mark.parametrize("c,seed", [(5, 0), (9, 1), (14, 2)])
+def test_e1_exact_equals_submatrix_inverse_recomputation(c, seed):
+    g = rng(100 + seed)
+    r = 4
+    W = g.standard_normal((r, c)) * 0.05
+    H = spd(c, 50 + seed, 1e2)
+    grid = np.sort(g.standard_normal((r, 4)) * 0.05, axis=1)
+    codes, What, loss, orders = O.quantize_exact(W, np.linalg.inv(H), grid=grid, bits=2, return_order=True)
+    total = 0.0
+    for k in range(r):
+        what, eps, order = exact_by_submatrix_inverses(W[k], H, lambda x: grid[k, np.argmin(np.abs(grid[k] - x))])
+        assert order == list(orders[k])
+        np.testing.assert_allclose(What[k], what, rtol=0, atol=1e-12)
+        total += eps
+    np.testing.assert_allclose(loss, total, rtol=1e-9)
+    assert np.array_equal(np.take_along_axis(grid, codes, 1), What)
+
+
+def test_e2_exact_sum_of_loss_errors_is_the_quadratic_loss():
+    """Every step's loss error is the exact increase of 1/2 dw H dw^T under the constraint it adds, so the
+    sum over the row is the quadratic loss of the final row, whatever the order."""
+    g = rng(7)
+    r, c = 6, 20
+    W = g.standard_normal((r, c)) * 0.05
+    H = spd(c, 3, 1e3)
+    grid = np.sort(g.standard_normal((r, 8)) * 0.06, axis=1)
+    for order in ("greedy", "natural"):
+        codes, What, loss = O.quantize_exact(W, np.linalg.inv(H), grid=grid, bits=3, order=order)
+        D = W - What
+        np.testing.assert_allclose(loss, 0.5 * np.einsum("ri,ij,rj->", D, H, D), rtol=1e-9)
+
+
+def test_e3_exact_with_identity_hessian_is_round_to_nearest():
+    g = rng(8)
+    r, c = 5, 33
+    W = g.standard_normal((r, c))
+    S = np.full((r, 1), 0.25)
+    Z = np.full((r, 1), 8.0)
+    codes, What, loss = O.quantize_exact(W, np.eye(c), scale=S, zero=Z, bits=4)
+    ref = (np.clip(np.rint(W / 0.25) + 8, 0, 15) - 8) * 0.25
+    assert np.array_equal(What, ref)
+    np.testing.assert_allclose(loss, 0.5 * ((W - ref) ** 2).sum(), rtol=1e-12)
+
+
+def test_e4_exact_in_natural_order_is_algorithm_1():
+    """With the greedy choice replaced by i = 0, 1, 2, ... Algorithm 2 is OBQ in fixed order, which the
+    column loop of Algorithm 1 computes through the Cholesky factor."""
+    g = rng(9)
+    r, c = 7, 40
+    W = g.standard_normal((r, c)) * 0.05
+    H = spd(c, 11, 1e2)
+    U, dinv, H_d, _ = O.prepare_hinv(H, 0.01)
+    grid = O.fit_grid_nonuniform(W, dinv, 3, 4.0, 10)
+    c1, w1, l1 = O.quantize_layer(W, U, grid=grid, bits=3, block=16)
+    c2, w2, l2 = O.quantize_exact(W, np.linalg.inv(H_d), grid=grid, bits=3, order="natural")
+    assert np.array_equal(c1, c2)
+    np.testing.assert_allclose(w1, w2, rtol=0, atol=1e-12)
+    np.testing.assert_allclose(l1, l2, rtol=1e-9)
