@@ -199,6 +199,26 @@ int lq_quantize_layer(lq_handle* h, void* stream, const lq_config* cfg, const vo
 int lq_pack_codes(lq_handle* h, void* stream, const uint8_t* codes, int64_t r, int64_t c,
                   int32_t bits, uint8_t* packed, int64_t ldp);
 
+/* ---- Algorithm 2 (Appendix, "LeanQuant-Exact"): greedy order, full downdate per row ---- */
+
+/* For every row, with the grid fitted beforehand by lq_fit_grid (lines 3-7 of Algorithm 2) and the row's own
+ * copy of the inverse Hessian Hinv = U^T U: c times, among the weights not yet quantised take the one with
+ * the least loss error (quant(w_i) - w_i)^2 / (2 Hinv_ii) (ties: lowest index), quantise it, spread its
+ * error over the others by Eq. 3 and remove it from the inverse by Eq. 9.  O(c^3) operations per row: meant
+ * for layers of up to a few thousand input features.  Arithmetic in fp64.
+ * U is the factor written by lq_prepare_hinv (so the inverse is the damped one; damp_frac = 0 there gives
+ * (2 X X^T)^-1 to the letter).  Arguments, layouts and outputs as for lq_quantize_layer, except that `loss`
+ * is the sum over all weights of the loss error at the moment each was quantised (equal to
+ * 1/2 sum_rows (w - w_hat) H_d (w - w_hat)^T), cfg->block is ignored and any group size dividing c is
+ * accepted.  c <= 8192.  Workspace: lq_quantize_exact_workspace bytes, 256-byte aligned (the fp64 inverse
+ * plus one copy of it per resident CTA).  A non-positive pivot records LQ_ERR_NOT_POSITIVE_DEFINITE
+ * (info = row * c + index). */
+int lq_quantize_exact_workspace(const lq_config* cfg, int64_t r, int64_t c, size_t* bytes);
+int lq_quantize_exact(lq_handle* h, void* stream, const lq_config* cfg, const void* W, int32_t w_dtype,
+                      int64_t r, int64_t c, int64_t ldw, const float* U, int64_t ldu, const float* grid,
+                      const float* scale, const int32_t* zero, uint8_t* codes, void* W_hat,
+                      int32_t what_dtype, int64_t ldwh, double* loss, void* ws, size_t ws_bytes);
+
 /* Number of CUDA kernels this library has launched in this process so far (host counter,
  * not thread-safe; for benchmarks and tests that want to see that the kernels ran). */
 uint64_t lq_launch_count(void);
