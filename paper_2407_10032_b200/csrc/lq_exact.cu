@@ -14,7 +14,7 @@
 
 namespace {
 
-constexpr int EX_THREADS = 512;
+constexpr int EX_THREADS = 256;
 constexpr int EX_WARPS = EX_THREADS / 32;
 constexpr int EX_MAX_NB = 32;
 
@@ -74,25 +74,24 @@ __device__ __forceinline__ void ex_quant(double w, const double* __restrict__ gp
     }
 }
 
+constexpr int EX_PER = 32;      // weights per thread at most (c <= EX_THREADS * EX_PER)
+
 template <typename T, bool AFFINE>
-__global__ void __launch_bounds__(EX_THREADS) exact_row_kernel(ExactArgs A) {
+__global__ void __launch_bounds__(EX_THREADS, 2) exact_row_kernel(ExactArgs A) {
     extern __shared__ __align__(16) unsigned char ex_smem[];
     const int c = A.c, nb = A.nb, K = A.K;
     double* w = reinterpret_cast<double*>(ex_smem);          // c: the row, error-compensated as it goes
     double* d = w + c;                                       // c: diagonal of the current inverse
-    double* v = d + c;                                       // c: the column taken out by this step
-    double* V = v + c;                                       // nb x c: the columns of the current batch
-    double* piv = V + static_cast<size_t>(nb) * c;           // nb: their pivots
-    double* coef = piv + EX_MAX_NB;                          // nb
-    double* arow = coef + EX_MAX_NB;                         // EX_WARPS x 2 x nb: row coefficients of the batch update
-    double* gpts = arow + EX_WARPS * 2 * EX_MAX_NB;          // 16
-    double* red_s = gpts + 16;                               // EX_WARPS
-    int* red_i = reinterpret_cast<int*>(red_s + EX_WARPS);   // EX_WARPS
-    int* rows = red_i + EX_WARPS;                            // c: rows still to do (for the batch update)
+    double* V = d + c;                                       // nb x c: the columns taken out by the steps of the current batch
+    double* rpiv = V + static_cast<size_t>(nb) * c;          // nb: reciprocals of their pivots
+    double* arow = rpiv + EX_MAX_NB;                         // EX_WARPS x 4 x nb: row coefficients of the batch update
+    double* gpts = arow + EX_WARPS * 4 * EX_MAX_NB;          // 16
+    double* red_s = gpts + 16;                               // 2 x EX_WARPS (alternating between steps)
+    int* red_i = reinterpret_cast<int*>(red_s + 2 * EX_WARPS);      // 2 x EX_WARPS
+    int* rows = red_i + 2 * EX_WARPS;                        // c: rows still to do, ascending (for the batch update)
     unsigned char* todo = reinterpret_cast<unsigned char*>(rows + c);      // c
-    __shared__ int n_rows, sh_i;
-    __shared__ double sh_q, sh_loss;
-    __shared__ int sh_code;
+    __shared__ double sh_dii[2];
+    __shared__ int sh_cnt[EX_WARPS];
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     double* Hi = A.slots + static_cast<size_t>(blockIdx.x) * A.slot_stride;
@@ -105,8 +104,7 @@ __global__ void __launch_bounds__(EX_THREADS) exact_row_kernel(ExactArgs A) {
             todo[j] = 1;
         }
         if (!AFFINE && tid < K) gpts[tid] = static_cast<double>(A.grid[row * K + tid]);
-        if (tid == 0) sh_loss = 0.0;
-        {   // this row's own copy of the inverse
+        {   // this row's own copy of the inverse (only its upper triangle is kept up to date below)
             const double2* src = reinterpret_cast<const double2*>(A.Hinv0);
             double2* dst = reinterpret_cast<double2*>(Hi);
             const size_t n2 = static_cast<size_t>(c) * c / 2;
@@ -115,8 +113,10 @@ __global__ void __launch_bounds__(EX_THREADS) exact_row_kernel(ExactArgs A) {
         }
         __syncthreads();
 
+        double loss = 0.0;          // kept by every thread alike
         int kb = 0;
         for (int step = 0; step < c; ++step) {
+            const int par = step & 1;
             // (a) the weight with the least loss error (q - w)^2 / (2 Hinv_ii) among those still to do
             double best = INFINITY;
             int bi = 0x7fffffff;
@@ -141,114 +141,144 @@ __global__ void __launch_bounds__(EX_THREADS) exact_row_kernel(ExactArgs A) {
                 const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
                 if (ob < best || (ob == best && oi < bi)) { best = ob; bi = oi; }
             }
-            if (lane == 0) { red_s[warp] = best; red_i[warp] = bi; }
+            if (lane == 0) { red_s[par * EX_WARPS + warp] = best; red_i[par * EX_WARPS + warp] = bi; }
             __syncthreads();
-            if (tid == 0) {
-                for (int x = 1; x < EX_WARPS; ++x)
-                    if (red_s[x] < best || (red_s[x] == best && red_i[x] < bi)) { best = red_s[x]; bi = red_i[x]; }
-                if (bi == 0x7fffffff) {                         // every score was NaN: take the first weight left
-                    for (int j = 0; j < c; ++j) if (todo[j]) { bi = j; break; }
-                }
-                sh_i = bi;
+            best = red_s[par * EX_WARPS];
+            bi = red_i[par * EX_WARPS];
+#pragma unroll
+            for (int x = 1; x < EX_WARPS; ++x) {
+                const double ob = red_s[par * EX_WARPS + x];
+                const int oi = red_i[par * EX_WARPS + x];
+                if (ob < best || (ob == best && oi < bi)) { best = ob; bi = oi; }
             }
-            __syncthreads();
-            const int i = sh_i;
-            // (b) column i of the current inverse: the row of the stored matrix minus the batch's downdates
-            if (tid < kb) coef[tid] = V[static_cast<size_t>(tid) * c + i] / piv[tid];
-            __syncthreads();
-            const double* hrow = Hi + static_cast<size_t>(i) * c;
-            for (int j = tid; j < c; j += EX_THREADS) {
-                double x = 0.0;
-                if (todo[j]) {
-                    x = hrow[j];
-                    for (int m = 0; m < kb; ++m) x = fma(-coef[m], V[static_cast<size_t>(m) * c + j], x);
-                }
-                v[j] = x;
+            if (bi == 0x7fffffff) {                             // every score was NaN: take the first weight left
+                for (int j = 0; j < c; ++j) if (todo[j]) { bi = j; break; }
             }
-            __syncthreads();
-            // (c) quantise weight i, spread its error (Eq. 3), downdate the diagonal (Eq. 9)
-            const double dii = v[i];
-            if (tid == 0) {
+            const int i = bi;
+            // its grid point (every thread computes it: cheaper than a broadcast)
+            double qi;
+            int code_i;
+            {
                 double S = 1.0, Z = 0.0;
                 if (AFFINE) {
                     const int64_t gi = row * A.n_groups + i / A.group;
                     S = static_cast<double>(A.scale[gi]);
                     Z = static_cast<double>(A.zero[gi]);
                 }
-                int code;
-                double q;
-                ex_quant<AFFINE>(w[i], gpts, K, S, Z, code, q);
-                const double err = w[i] - q;
-                sh_loss += __ddiv_rn(__dmul_rn(err, err), 2.0 * dii);
-                sh_q = q;
-                sh_code = code;
-                A.codes[row * c + i] = static_cast<uint8_t>(code);
-                if (A.what) {
-                    if (A.what_bf16) static_cast<__nv_bfloat16*>(A.what)[row * A.ldwh + i] = __float2bfloat16_rn(static_cast<float>(q));
-                    else static_cast<float*>(A.what)[row * A.ldwh + i] = static_cast<float>(q);
+                ex_quant<AFFINE>(w[i], gpts, K, S, Z, code_i, qi);
+            }
+            const double err = w[i] - qi;
+            // (b) column i of the current inverse: the stored upper triangle as of the start of the batch, minus the
+            //     batch's downdates  sum_m v_m[j] v_m[i] / pivot_m
+            double vj[EX_PER];
+#pragma unroll 4
+            for (int t = 0; t < EX_PER; ++t) {
+                const int j = tid + t * EX_THREADS;
+                if (j >= c) break;
+                double x = 0.0;
+                if (todo[j]) {
+                    x = j <= i ? Hi[static_cast<size_t>(j) * c + i] : Hi[static_cast<size_t>(i) * c + j];
+                    for (int m = 0; m < kb; ++m)
+                        x = fma(-(V[static_cast<size_t>(m) * c + i] * rpiv[m]), V[static_cast<size_t>(m) * c + j], x);
                 }
-                if (!(dii > 0.0)) lq_report(A.dstatus, LQ_ERR_NOT_POSITIVE_DEFINITE, row * c + i);
+                vj[t] = x;
+                if (j == i) sh_dii[par] = x;
             }
             __syncthreads();
-            {
-                const double err = w[i] - sh_q;
-                for (int j = tid; j < c; j += EX_THREADS) {
-                    const double x = v[j];
-                    V[static_cast<size_t>(kb) * c + j] = x;
-                    if (todo[j] && j != i) {
-                        w[j] = __dsub_rn(w[j], __dmul_rn(__ddiv_rn(x, dii), err));
-                        d[j] = __dsub_rn(d[j], __ddiv_rn(__dmul_rn(x, x), dii));
+            // (c) quantise weight i, spread its error (Eq. 3), downdate the diagonal (Eq. 9)
+            const double dii = sh_dii[par];
+            loss += __ddiv_rn(__dmul_rn(err, err), 2.0 * dii);
+#pragma unroll 4
+            for (int t = 0; t < EX_PER; ++t) {
+                const int j = tid + t * EX_THREADS;
+                if (j >= c) break;
+                const double x = vj[t];
+                V[static_cast<size_t>(kb) * c + j] = x;
+                if (j == i) {
+                    w[i] = qi;
+                    todo[i] = 0;
+                    rpiv[kb] = 1.0 / dii;
+                    A.codes[row * c + i] = static_cast<uint8_t>(code_i);
+                    if (A.what) {
+                        if (A.what_bf16) static_cast<__nv_bfloat16*>(A.what)[row * A.ldwh + i] = __float2bfloat16_rn(static_cast<float>(qi));
+                        else static_cast<float*>(A.what)[row * A.ldwh + i] = static_cast<float>(qi);
                     }
+                    if (!(dii > 0.0)) lq_report(A.dstatus, LQ_ERR_NOT_POSITIVE_DEFINITE, row * c + i);
+                } else if (todo[j]) {
+                    w[j] = __dsub_rn(w[j], __dmul_rn(__ddiv_rn(x, dii), err));
+                    d[j] = __dsub_rn(d[j], __ddiv_rn(__dmul_rn(x, x), dii));
                 }
             }
-            __syncthreads();
-            if (tid == 0) { w[i] = sh_q; todo[i] = 0; piv[kb] = dii; n_rows = 0; }
             ++kb;
             __syncthreads();
-            // (d) end of a batch: Hinv[j][l] -= sum_m v_m[j] v_m[l] / pivot_m for the rows still to do
+            // (d) end of a batch: Hinv[j][l] -= sum_m v_m[j] v_m[l] / pivot_m for the rows j still to do, l >= j
             if (kb == nb && step + 1 < c) {
-                for (int j = tid; j < c; j += EX_THREADS)
-                    if (todo[j]) rows[atomicAdd(&n_rows, 1)] = j;
+                // ascending list of the rows still to do
+                const int per = (c + EX_THREADS - 1) / EX_THREADS;
+                const int j_lo = min(tid * per, c), j_hi = min(j_lo + per, c);
+                int cnt = 0;
+                for (int j = j_lo; j < j_hi; ++j) cnt += todo[j];
+                int incl = cnt;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int y = __shfl_up_sync(0xffffffffu, incl, o);
+                    if (lane >= o) incl += y;
+                }
+                if (lane == 31) sh_cnt[warp] = incl;
                 __syncthreads();
-                const int nr = n_rows;
-                double* a0 = arow + (warp * 2) * EX_MAX_NB;
-                double* a1 = a0 + EX_MAX_NB;
-                for (int p = warp * 2; p < nr; p += EX_WARPS * 2) {
-                    const int j0 = rows[p], j1 = rows[min(p + 1, nr - 1)];
-                    const bool two = p + 1 < nr;
+                int base = incl - cnt, nr = 0;
+                for (int x = 0; x < EX_WARPS; ++x) {
+                    if (x < warp) base += sh_cnt[x];
+                    nr += sh_cnt[x];
+                }
+                for (int j = j_lo; j < j_hi; ++j)
+                    if (todo[j]) rows[base++] = j;
+                __syncthreads();
+                // each warp takes four rows at a time and walks them in strips of 128 columns (four per lane),
+                // starting at the strip that holds the diagonal of the first of them
+                double* aw = arow + (warp * 4) * EX_MAX_NB;
+                for (int p = warp * 4; p < nr; p += EX_WARPS * 4) {
+                    int jr[4];
+                    double* hr[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        jr[q] = rows[min(p + q, nr - 1)];
+                        hr[q] = Hi + static_cast<size_t>(jr[q]) * c;
+                    }
+                    const int live = min(4, nr - p);
                     if (lane < kb) {
-                        a0[lane] = V[static_cast<size_t>(lane) * c + j0] / piv[lane];
-                        a1[lane] = V[static_cast<size_t>(lane) * c + j1] / piv[lane];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) aw[q * EX_MAX_NB + lane] = V[static_cast<size_t>(lane) * c + jr[q]] * rpiv[lane];
                     }
                     __syncwarp();
-                    double* h0 = Hi + static_cast<size_t>(j0) * c;
-                    double* h1 = Hi + static_cast<size_t>(j1) * c;
-                    for (int l0 = 0; l0 < c; l0 += 128) {
-                        double x0[4], x1[4];
+                    for (int l0 = jr[0] & ~127; l0 < c; l0 += 128) {
+                        double x[4][4];
 #pragma unroll
-                        for (int t = 0; t < 4; ++t) {
-                            const int l = l0 + lane + 32 * t;
-                            x0[t] = l < c ? h0[l] : 0.0;
-                            x1[t] = (l < c && two) ? h1[l] : 0.0;
-                        }
-                        for (int m = 0; m < kb; ++m) {
-                            const double c0 = a0[m], c1 = a1[m];
-                            const double* vm = V + static_cast<size_t>(m) * c + l0 + lane;
+                        for (int q = 0; q < 4; ++q)
 #pragma unroll
                             for (int t = 0; t < 4; ++t) {
-                                const double y = (l0 + lane + 32 * t < c) ? vm[32 * t] : 0.0;
-                                x0[t] = fma(-c0, y, x0[t]);
-                                x1[t] = fma(-c1, y, x1[t]);
+                                const int l = l0 + lane + 32 * t;
+                                x[q][t] = (l < c && q < live) ? hr[q][l] : 0.0;
+                            }
+                        for (int m = 0; m < kb; ++m) {
+                            const double* vm = V + static_cast<size_t>(m) * c + l0 + lane;
+                            double y[4];
+#pragma unroll
+                            for (int t = 0; t < 4; ++t) y[t] = (l0 + lane + 32 * t < c) ? vm[32 * t] : 0.0;
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const double cq = aw[q * EX_MAX_NB + m];
+#pragma unroll
+                                for (int t = 0; t < 4; ++t) x[q][t] = fma(-cq, y[t], x[q][t]);
                             }
                         }
 #pragma unroll
-                        for (int t = 0; t < 4; ++t) {
-                            const int l = l0 + lane + 32 * t;
-                            if (l < c) {
-                                h0[l] = x0[t];
-                                if (two) h1[l] = x1[t];
+                        for (int q = 0; q < 4; ++q)
+#pragma unroll
+                            for (int t = 0; t < 4; ++t) {
+                                const int l = l0 + lane + 32 * t;
+                                if (l < c && q < live) hr[q][l] = x[q][t];
                             }
-                        }
                     }
                     __syncwarp();
                 }
@@ -256,7 +286,7 @@ __global__ void __launch_bounds__(EX_THREADS) exact_row_kernel(ExactArgs A) {
                 __syncthreads();
             }
         }
-        if (tid == 0) A.loss_rows[row] = sh_loss;
+        if (tid == 0) A.loss_rows[row] = loss;
         __syncthreads();
     }
 }
@@ -282,13 +312,13 @@ struct ExactPlan {
 };
 
 size_t exact_smem(int c, int nb) {
-    return static_cast<size_t>(3 + nb) * c * sizeof(double) + (2 * EX_MAX_NB + EX_WARPS * 2 * EX_MAX_NB + 16 + EX_WARPS) * sizeof(double) +
-           (EX_WARPS + c) * sizeof(int) + static_cast<size_t>(c) + 16;
+    return static_cast<size_t>(2 + nb) * c * sizeof(double) + (EX_MAX_NB + EX_WARPS * 4 * EX_MAX_NB + 16 + 2 * EX_WARPS) * sizeof(double) +
+           (2 * EX_WARPS + c) * sizeof(int) + static_cast<size_t>(c) + 16;
 }
 
 // Batch length: as long as two CTAs still fit on an SM if that leaves at least 8 steps per batch, else one CTA per SM.
 int exact_plan(int64_t r, int64_t c, int sm_count, ExactPlan* P) {
-    if (c > 8192) return LQ_ERR_UNSUPPORTED;
+    if (c > EX_THREADS * EX_PER) return LQ_ERR_UNSUPPORTED;
     int nb = 0, per_sm = 2;
     for (int cand = EX_MAX_NB; cand >= 1; --cand)
         if (exact_smem(static_cast<int>(c), cand) <= 110 * 1024) { nb = cand; break; }
