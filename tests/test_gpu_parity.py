@@ -465,7 +465,7 @@ def test_chained_weighted_by_factor_diagonal(lq, h):
     plain = O.run_pass(W, X, bits=4, p=4.0, block=128, n_iter=20)
     assert np.abs(ref["grid"] - plain["grid"]).max() > 1e-4 * np.abs(plain["grid"]).max()     # the variant is another grid
     P = chained(lq, h, L, dict(grid="nonuniform", bits=4, p=4.0, n_iter=20), what_dtype=torch.float32, weight_src="chol_diag")
-    np.testing.assert_allclose(f64(P.dinv), np.diag(ref["U"]), rtol=2e-5)
+    np.testing.assert_allclose(f64(P.dinv), np.diag(ref["U"]), rtol=1e-3)    # the factor of an fp32 H of this condition number
     assert centroid_ok(f64(P.grid), ref["grid"], W)
     assert codes_budget(P.codes.cpu().numpy().astype(np.int64), ref["codes"])
     assert abs(P.loss.item() / ref["loss"] - 1) <= LOSS_TOL
