@@ -283,22 +283,25 @@ def run_ours(args):
     e2e_ms, h2d, d2h = float("nan"), 0, 0
     if not args.no_e2e:
         e2e_steps = max(1, min(args.steps, 3))
-        Xh = torch.empty(X.shape, dtype=X.dtype, pin_memory=True)
+        # calibration activations on the host as they are collected: contiguous chunks of tokens, pinned
+        e2e_chunk = min(chunk, 32768)
+        Xh = []
+        for j in range(0, n, e2e_chunk):
+            t = torch.empty((c, min(e2e_chunk, n - j)), dtype=X.dtype, pin_memory=True)
+            t.copy_(X[:, j:j + e2e_chunk])
+            Xh.append(t)
         Wh = torch.empty(W.shape, dtype=W.dtype, pin_memory=True)
-        Xh.copy_(X)
         Wh.copy_(W)
         outs = [t for t in (P.codes, P.grid, P.scale, P.zero, P.loss) if t is not None]
         outs_h = [torch.empty(t.shape, dtype=t.dtype, pin_memory=True) for t in outs]
-        Xd, Wd = torch.empty_like(X), torch.empty_like(W)
+        Wd = torch.empty_like(W)
         barrier()
         b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         b0.record(stream)
         for _ in range(e2e_steps):
-            Xd.copy_(Xh, non_blocking=True)
             Wd.copy_(Wh, non_blocking=True)
             P.H.zero_()
-            for j in range(0, n, chunk):
-                lq.lq_hessian_accumulate(h, Xd[:, j:j + chunk], P.H, 2.0, P.ws)
+            P.accumulate_from_host(Xh)                   # chunk copies overlapped with the contraction
             lq.lq_hessian_finalize(h, P.H)
             lq.lq_prepare_hinv(h, P.H, P.U, P.dinv, P.ws, 0.01, Wd)
             lq.lq_fit_grid(h, cfg, Wd, P.dinv, P.ws, P.grid, P.scale, P.zero)
@@ -308,7 +311,7 @@ def run_ours(args):
         b1.record(stream)
         barrier()
         e2e_ms = b0.elapsed_time(b1) / e2e_steps
-        h2d = Xh.numel() * Xh.element_size() + Wh.numel() * Wh.element_size()
+        h2d = sum(t.numel() * t.element_size() for t in Xh) + Wh.numel() * Wh.element_size()
         d2h = sum(t.numel() * t.element_size() for t in outs_h)
 
     t = max_over_ranks(torch.tensor([total_ms, e2e_ms], device=dev, dtype=torch.float64), world)

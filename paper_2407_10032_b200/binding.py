@@ -291,3 +291,34 @@ class LayerPass:
         self.H.zero_()
         self.accumulate(X, alpha)
         self.finish(W, damp_frac)
+
+    def accumulate_from_host(self, chunks, alpha=2.0):
+        """Stage 1 for calibration activations that live in pinned host memory as a sequence of contiguous
+        chunks (each c x m_i, tokens contiguous): every chunk is copied to one of two device staging buffers
+        on a side stream while the previous chunk is being accumulated, so the copy and the contraction
+        overlap.  Plumbing only (copies, streams, events); the arithmetic is lq_hessian_accumulate's."""
+        chunks = list(chunks)
+        if not chunks:
+            return
+        c = chunks[0].shape[0]
+        widest = max(t.shape[1] for t in chunks)
+        dev = self.H.device
+        main = torch.cuda.current_stream(dev)
+        if getattr(self, "_stage", None) is None or self._stage[0].shape[1] < widest or self._stage[0].dtype != chunks[0].dtype:
+            self._stage = [torch.empty((c, widest), dtype=chunks[0].dtype, device=dev) for _ in range(2)]
+            self._copy_stream = torch.cuda.Stream(dev)
+            self._filled = [torch.cuda.Event() for _ in range(2)]
+            self._drained = [torch.cuda.Event() for _ in range(2)]
+        self._copy_stream.wait_stream(main)            # earlier work on the staging buffers has finished
+        for k, Xc in enumerate(chunks):
+            b = k & 1
+            m = Xc.shape[1]
+            dst = self._stage[b].view(-1)[:c * m].view(c, m)       # contiguous c x m inside the staging buffer
+            with torch.cuda.stream(self._copy_stream):
+                if k >= 2:
+                    self._copy_stream.wait_event(self._drained[b])
+                dst.copy_(Xc, non_blocking=True)
+                self._filled[b].record(self._copy_stream)
+            main.wait_event(self._filled[b])
+            lq_hessian_accumulate(self.h, dst, self.H, alpha, self.ws)
+            self._drained[b].record(main)

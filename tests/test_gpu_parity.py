@@ -152,6 +152,22 @@ def test_stage1_chunks_add_up(lq, h):
     np.testing.assert_allclose(H4, Href, rtol=0, atol=5e-6 * np.abs(Href).max())
 
 
+def test_stage1_from_pinned_host_in_chunks(lq, h):
+    """The overlapped host feed (two staging buffers, side stream) adds up the same Hessian as one call."""
+    g = torch.Generator().manual_seed(6)
+    X = torch.randn(256, 5000, generator=g).bfloat16()
+    cfg = lq.Config.make(grid="nonuniform", bits=4)
+    P = lq.LayerPass(h, 8, 256, cfg, n_chunk=1024, device="cuda")
+    for _ in range(2):                                   # the second pass reuses the staging buffers
+        P.H.zero_()
+        chunks = [X[:, j:j + 1024].contiguous().pin_memory() for j in range(0, 5000, 1024)]
+        P.accumulate_from_host(chunks)                   # 4 full chunks and a ragged one of 904 tokens
+        lq.lq_hessian_finalize(h, P.H)
+        lq.lq_sync_status(h)
+        Href = O.hessian(f64(X))
+        np.testing.assert_allclose(f64(P.H), Href, rtol=0, atol=5e-6 * np.abs(Href).max())
+
+
 def test_stage1_empty_chunk_and_alpha(lq, h):
     X = torch.randn(128, 256).bfloat16().cuda()
     H = torch.zeros(128, 128, device="cuda")
