@@ -199,6 +199,20 @@ int lq_quantize_layer(lq_handle* h, void* stream, const lq_config* cfg, const vo
 int lq_pack_codes(lq_handle* h, void* stream, const uint8_t* codes, int64_t r, int64_t c,
                   int32_t bits, uint8_t* packed, int64_t ldp);
 
+/* Variant of lq_quantize_layer for affine grids in which the (S, Z) of a group are not fitted beforehand on the
+ * original weights (Algorithm 1 lines 5-9) but when the column loop reaches the group's first column, on that
+ * group's columns as they stand then, i.e. with the errors of all earlier columns already fed back into them
+ * (the usual practice of GPTQ implementations; the paper's pseudocode fits all grids first).  The search is that
+ * of lq_fit_grid (Eq. 7 with cfg->T, cfg->t_count, cfg->p and the sample weights from dinv); scale / zero
+ * (r x c / group_size) are outputs.  Supported group sizes: multiples of 128 that divide 1024, multiples of
+ * 1024, and one group per row (which is the same as fitting beforehand).  Other arguments as lq_quantize_layer;
+ * workspace: lq_quantize_layer_lazy_workspace bytes. */
+int lq_quantize_layer_lazy_workspace(const lq_config* cfg, int64_t r, int64_t c, size_t* bytes);
+int lq_quantize_layer_lazy(lq_handle* h, void* stream, const lq_config* cfg, const void* W, int32_t w_dtype,
+                           int64_t r, int64_t c, int64_t ldw, const float* U, int64_t ldu, const float* dinv,
+                           float* scale, int32_t* zero, uint8_t* codes, void* W_hat, int32_t what_dtype,
+                           int64_t ldwh, double* loss, void* ws, size_t ws_bytes);
+
 /* ---- Algorithm 2 (Appendix, "LeanQuant-Exact"): greedy order, full downdate per row ---- */
 
 /* For every row, with the grid fitted beforehand by lq_fit_grid (lines 3-7 of Algorithm 2) and the row's own

@@ -194,6 +194,43 @@ def affine_candidate(mn: float, mx: float, t_min: int, t_max: int, T: int, K: in
     return S, -np.rint(lo / S)
 
 
+def affine_search_group(w, sg, K: int, T: int, t: int):
+    """Eq. 7 for one group of columns, all rows at once: w is r x g, sg the g sample weights.
+    Returns (S, Z), each of length r."""
+    w = np.asarray(w, dtype=F64)
+    r = w.shape[0]
+    mn = w.min(axis=1)
+    mx = w.max(axis=1)
+    R = mx - mn
+    bS = np.ones(r)
+    bZ = np.zeros(r)
+    flat = R == 0.0
+    for i in np.nonzero(flat)[0]:
+        bS[i], bZ[i] = affine_candidate(mn[i], mx[i], 0, 0, T, K)
+    live = ~flat
+    if live.any():
+        wl, mnl, mxl, Rl = w[live], mn[live], mx[live], R[live]
+        bl = np.full(wl.shape[0], np.inf)
+        Sl = np.ones(wl.shape[0])
+        Zl = np.zeros(wl.shape[0])
+        for t_min in range(t + 1):
+            lo = mnl + t_min * Rl / T
+            for t_max in range(t + 1):
+                hi = mxl - t_max * Rl / T
+                S = (hi - lo) / (K - 1)
+                valid = S > 0.0
+                Ssafe = np.where(valid, S, 1.0)
+                Z = -np.rint(lo / Ssafe)
+                q = quant_aff(wl, Ssafe[:, None], Z[:, None], K)
+                loss = (sg * (q - wl) ** 2).sum(axis=1)
+                better = valid & (loss < bl)
+                bl[better] = loss[better]
+                Sl[better] = S[better]
+                Zl[better] = Z[better]
+        bS[live], bZ[live] = Sl, Zl
+    return bS, bZ
+
+
 def fit_grid_affine(W, dinv, bits: int, p: float = 4.0, group: int = 0,
                     T: int = 2048, t: int | None = None):
     """Eq. 7: enumerate (t_min, t_max) in {0..t}^2 per (row, group) and keep the pair
@@ -214,39 +251,7 @@ def fit_grid_affine(W, dinv, bits: int, p: float = 4.0, group: int = 0,
     scale = np.empty((r, ng), dtype=F64)
     zero = np.empty((r, ng), dtype=F64)
     for gi in range(ng):
-        w = W[:, gi * g:(gi + 1) * g]
-        sg = s[gi * g:(gi + 1) * g]
-        mn = w.min(axis=1)
-        mx = w.max(axis=1)
-        R = mx - mn
-        best = np.full(r, np.inf)
-        bS = np.ones(r)
-        bZ = np.zeros(r)
-        flat = R == 0.0
-        for i in np.nonzero(flat)[0]:
-            bS[i], bZ[i] = affine_candidate(mn[i], mx[i], 0, 0, T, K)
-        live = ~flat
-        if live.any():
-            wl, mnl, mxl, Rl = w[live], mn[live], mx[live], R[live]
-            bl = np.full(wl.shape[0], np.inf)
-            Sl = np.ones(wl.shape[0])
-            Zl = np.zeros(wl.shape[0])
-            for t_min in range(t + 1):
-                lo = mnl + t_min * Rl / T
-                for t_max in range(t + 1):
-                    hi = mxl - t_max * Rl / T
-                    S = (hi - lo) / (K - 1)
-                    valid = S > 0.0
-                    Ssafe = np.where(valid, S, 1.0)
-                    Z = -np.rint(lo / Ssafe)
-                    q = quant_aff(wl, Ssafe[:, None], Z[:, None], K)
-                    loss = (sg * (q - wl) ** 2).sum(axis=1)
-                    better = valid & (loss < bl)
-                    bl[better] = loss[better]
-                    Sl[better] = S[better]
-                    Zl[better] = Z[better]
-            bS[live], bZ[live] = Sl, Zl
-        scale[:, gi], zero[:, gi] = bS, bZ
+        scale[:, gi], zero[:, gi] = affine_search_group(W[:, gi * g:(gi + 1) * g], s[gi * g:(gi + 1) * g], K, T, t)
     return scale, zero
 
 
@@ -254,7 +259,7 @@ def fit_grid_affine(W, dinv, bits: int, p: float = 4.0, group: int = 0,
 # Stage 4 -- Algorithm 1 lines 10-21: block-wise column loop with error feedback
 # --------------------------------------------------------------------------- #
 def quantize_layer(W, U, *, grid=None, scale=None, zero=None, bits: int = 4,
-                   group: int = 0, block: int = 128, return_pre: bool = False):
+                   group: int = 0, block: int = 128, return_pre: bool = False, lazy=None):
     """The iterative loss-error-based loop on a learned grid.
 
     For each block of ``block`` columns, for each column j in it: quantise W[:, j] for
@@ -265,7 +270,12 @@ def quantize_layer(W, U, *, grid=None, scale=None, zero=None, bits: int = 4,
 
     Returns codes (r x c, int64), W_hat (r x c) and loss = 1/2 * sum(E^2), the summed
     loss error of Eq. 3 with the damped inverse.  With ``return_pre`` a fourth array holds
-    every weight as it stood at the moment it was quantised (for tie analysis in tests)."""
+    every weight as it stood at the moment it was quantised (for tie analysis in tests).
+
+    ``lazy`` = dict(s=sample weights (c), T=, t=) selects the variant in which the (S, Z) of an affine group are
+    fitted by Eq. 7 when the loop reaches the group's first column, on the group's columns as they stand then
+    (all earlier errors fed back), instead of beforehand; ``scale`` / ``zero`` are then filled in and returned
+    at the end of the tuple."""
     Wc = np.array(W, dtype=F64, copy=True)
     U = np.asarray(U, dtype=F64)
     r, c = Wc.shape
@@ -275,10 +285,21 @@ def quantize_layer(W, U, *, grid=None, scale=None, zero=None, bits: int = 4,
     Wpre = np.zeros((r, c), dtype=F64) if return_pre else None
     loss = 0.0
     g = c if group in (0, None) else group
+    if lazy is not None:
+        scale = np.zeros((r, c // g), dtype=F64)
+        zero = np.zeros((r, c // g), dtype=F64)
     for i in range(0, c, block):
         e_end = min(i + block, c)
         E = np.zeros((r, e_end - i), dtype=F64)
         for j in range(i, e_end):
+            if lazy is not None and j % g == 0:
+                if g > block and g % block:
+                    raise ValueError("lazy refit: a group longer than a block must be made of whole blocks")
+                if j + g > e_end and j != i:
+                    raise ValueError("lazy refit: a group must start on a block boundary or lie inside one block")
+                # columns beyond this block have not received this block's earlier errors yet: only allowed when the
+                # group starts the block (then there are none)
+                scale[:, j // g], zero[:, j // g] = affine_search_group(Wc[:, j:j + g], lazy["s"][j:j + g], K, lazy["T"], lazy["t"])
             w = Wc[:, j]
             if return_pre:
                 Wpre[:, j] = w
@@ -298,9 +319,10 @@ def quantize_layer(W, U, *, grid=None, scale=None, zero=None, bits: int = 4,
         loss += 0.5 * float((E * E).sum())
         if e_end < c:
             Wc[:, e_end:] -= E @ U[i:e_end, e_end:]
+    extra = (scale, zero) if lazy is not None else ()
     if return_pre:
-        return codes, What, loss, Wpre
-    return codes, What, loss
+        return (codes, What, loss, Wpre) + extra
+    return (codes, What, loss) + extra
 
 
 # --------------------------------------------------------------------------- #
@@ -433,7 +455,7 @@ def minmax_affine_params(W, bits: int, group: int = 0):
 
 
 def run_pass(W, X, *, grid_type="nonuniform", bits=4, p=4.0, block=128, damp=0.01,
-             n_iter=20, init="uniform", group=0, T=2048, t=None, alpha=2.0, weight_src="inv_diag"):
+             n_iter=20, init="uniform", group=0, T=2048, t=None, alpha=2.0, weight_src="inv_diag", lazy_refit=False):
     """Algorithm 1 end to end; returns a dict with every intermediate.
     ``weight_src``: "inv_diag" weights the grid objective by diag(H_d^-1)^-p as Eq. 5 / Eq. 7 say;
     "chol_diag" by diag(U)^-p, Algorithm 1 lines 6 and 8 read to the letter (the symbol H^-1 holds
@@ -449,6 +471,12 @@ def run_pass(W, X, *, grid_type="nonuniform", bits=4, p=4.0, block=128, damp=0.0
         G = fit_grid_nonuniform(Wf, dinv, bits, p, n_iter, init)
         codes, What, loss = quantize_layer(Wf, U, grid=G, bits=bits, block=block)
         out.update(grid=G)
+    elif lazy_refit:
+        if t is None:
+            t = int(np.floor({4: 0.2, 3: 0.3, 2: 0.4}[bits] * T))
+        codes, What, loss, S, Z = quantize_layer(Wf, U, bits=bits, group=group, block=block,
+                                                 lazy=dict(s=sample_weights(dinv, p), T=T, t=t))
+        out.update(scale=S, zero=Z)
     else:
         S, Z = fit_grid_affine(Wf, dinv, bits, p, group, T, t)
         codes, What, loss = quantize_layer(Wf, U, scale=S, zero=Z, bits=bits, group=group, block=block)

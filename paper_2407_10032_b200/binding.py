@@ -69,6 +69,9 @@ def LQ():
             "lq_fit_grid": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, sz],
             "lq_fit_grid_noalloc": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, vp, vp, vp],
             "lq_pack_codes": [vp, vp, vp, i64, i64, i32, vp, i64],
+            "lq_quantize_layer_lazy_workspace": [P(Config), i64, i64, P(sz)],
+            "lq_quantize_layer_lazy": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, i64, vp, vp, vp, vp, vp, i32, i64,
+                                       vp, vp, sz],
             "lq_quantize_exact_workspace": [P(Config), i64, i64, P(sz)],
             "lq_quantize_exact": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, i64, vp, vp, vp, vp, vp, i32, i64,
                                   vp, vp, sz],
@@ -217,6 +220,22 @@ def lq_quantize_layer(h, cfg, W, U, codes, ws, grid=None, scale=None, zero=None,
                                   _rowmajor(U), _ptr(grid), _ptr(scale), _ptr(zero), _ptr(codes), _ptr(W_hat), whdt,
                                   ldwh, _ptr(loss_out), _ptr(ws), ws.numel() * ws.element_size()),
            "lq_quantize_layer")
+
+
+def lq_quantize_layer_lazy_workspace(cfg, r, c) -> int:
+    b = C.c_size_t(0)
+    _check(LQ().lq_quantize_layer_lazy_workspace(C.byref(cfg), r, c, C.byref(b)), "lq_quantize_layer_lazy_workspace")
+    return b.value
+
+
+def lq_quantize_layer_lazy(h, cfg, W, U, dinv, scale, zero, codes, ws, W_hat=None, loss_out=None, stream=None):
+    """lq_quantize_layer with each group's (S, Z) fitted when the column loop reaches the group (outputs scale, zero)."""
+    r, c = W.shape
+    whdt, ldwh = (0, 0) if W_hat is None else (_dt(W_hat), _rowmajor(W_hat))
+    _check(LQ().lq_quantize_layer_lazy(h, _stream(stream), C.byref(cfg), _ptr(W), _dt(W), r, c, _rowmajor(W), _ptr(U),
+                                       _rowmajor(U), _ptr(dinv), _ptr(scale), _ptr(zero), _ptr(codes), _ptr(W_hat), whdt,
+                                       ldwh, _ptr(loss_out), _ptr(ws), ws.numel() * ws.element_size()),
+           "lq_quantize_layer_lazy")
 
 
 def lq_quantize_exact_workspace(cfg, r, c) -> int:

@@ -72,6 +72,14 @@ struct lq_tc_gemm_args {
 };
 int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a);
 
+// ---- pieces of stage 3 that other stages reuse (lq_fit_grid.cu) ------------------------
+// Sample weights s_j = exp(-p (ln dinv_j - mean ln dinv)) into s64 (c doubles); scal: 256 bytes of scratch.
+int lq_sample_weights(lq_handle* h, cudaStream_t st, const float* dinv, int64_t c, double p, double* scal, double* s64);
+// The search of Eq. 7 over r x n_groups groups of g weights starting at W (row stride ldw); s64 holds the sample
+// weights of those n_groups * g columns; (S, Z) of group gi of row i goes to scale / zero [i * out_ld + gi].
+int lq_affine_search(lq_handle* h, cudaStream_t st, const void* W, int32_t w_dtype, int64_t r, int64_t ldw, int64_t g,
+                     int n_groups, const double* s64, int K, int T, int t_count, float* scale, int32_t* zero, int64_t out_ld);
+
 // Split fp32 into three bf16 terms hi + mid + lo (each the bf16 rounding of what is left).
 __device__ __forceinline__ void lq_split3(float x, __nv_bfloat16& hi, __nv_bfloat16& mid, __nv_bfloat16& lo) {
     hi = __float2bfloat16_rn(x);

@@ -485,7 +485,7 @@ template <typename T>
 __global__ void __launch_bounds__(AF_THREADS)
 affine_search_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, int group, int n_groups,
                      const double* __restrict__ s64, int K, int Tparts, int t_count,
-                     float* __restrict__ scale, int32_t* __restrict__ zero) {
+                     float* __restrict__ scale, int32_t* __restrict__ zero, int64_t out_ld) {
     extern __shared__ float wg[];                 // group weights
     __shared__ float redf[2][AF_THREADS / 32];
     __shared__ double best_loss[AF_THREADS / 32];
@@ -514,7 +514,7 @@ affine_search_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, int group,
     for (int w = 1; w < AF_THREADS / 32; ++w) { mn = fminf(mn, redf[0][w]); mx = fmaxf(mx, redf[1][w]); }
     const double dmn = mn, dmx = mx, R = dmx - dmn;
     const double Km1 = static_cast<double>(K - 1);
-    const int64_t out = row * n_groups + gi;
+    const int64_t out = row * out_ld + gi;
 
     if (R == 0.0) {                                // constant group
         if (tid == 0) {
@@ -634,7 +634,7 @@ template <typename T>
 __global__ void __launch_bounds__(AFW_WARPS * 32)
 affine_search_warp_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_groups, int64_t total_groups,
                           const double* __restrict__ s64, int K, int Tparts, int t_count,
-                          float* __restrict__ scale, int32_t* __restrict__ zero) {
+                          float* __restrict__ scale, int32_t* __restrict__ zero, int64_t out_ld) {
     extern __shared__ __align__(16) unsigned char afw_smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float2* ws = reinterpret_cast<float2*>(afw_smem) + static_cast<size_t>(warp) * group;      // (w - min, s / max s)
@@ -642,6 +642,7 @@ affine_search_warp_kernel(const T* __restrict__ W, int64_t ldw, int group, int n
     if (gid >= total_groups) return;                       // whole warps leave; no block-wide barrier below
     const int64_t row = gid / n_groups;
     const int gi = static_cast<int>(gid - row * n_groups);
+    const int64_t oidx = row * out_ld + gi;
     const T* wp = W + row * ldw + static_cast<int64_t>(gi) * group;
     const double* sp = s64 + static_cast<int64_t>(gi) * group;
 
@@ -673,8 +674,8 @@ affine_search_warp_kernel(const T* __restrict__ W, int64_t ldw, int group, int n
             double lo = fmin(dmn, 0.0), hi = fmax(dmx, 0.0);
             double S = 1.0, Z = 0.0;
             if (hi != lo) { S = (hi - lo) / Km1; Z = -rint(lo / S); }
-            scale[gid] = static_cast<float>(S);
-            zero[gid] = static_cast<int32_t>(Z);
+            scale[oidx] = static_cast<float>(S);
+            zero[oidx] = static_cast<int32_t>(Z);
         }
         return;
     }
@@ -769,8 +770,8 @@ affine_search_warp_kernel(const T* __restrict__ W, int64_t ldw, int group, int n
             S = (hi - lo) / Km1;
             Z = -rint(lo / S);
         }
-        scale[gid] = static_cast<float>(S);
-        zero[gid] = static_cast<int32_t>(Z);
+        scale[oidx] = static_cast<float>(S);
+        zero[oidx] = static_cast<int32_t>(Z);
     }
 }
 
@@ -794,7 +795,7 @@ constexpr int AC_MAX_THREADS = 512;
 template <typename T>
 __global__ void __launch_bounds__(AC_MAX_THREADS)
 affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_groups, const double* __restrict__ s64, int K,
-                    int Tparts, int t_count, int p_max, float* __restrict__ scale, int32_t* __restrict__ zero,
+                    int Tparts, int t_count, int p_max, float* __restrict__ scale, int32_t* __restrict__ zero, int64_t out_ld,
                     lq_dev_status* __restrict__ dstatus) {
     extern __shared__ __align__(16) unsigned char ac_smem[];
     const int nu = 2 * t_count + 1;
@@ -812,6 +813,7 @@ affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_group
     const int64_t gid = blockIdx.x;
     const int64_t row = gid / n_groups;
     const int gi = static_cast<int>(gid - row * n_groups);
+    const int64_t oidx = row * out_ld + gi;
     const T* wp = W + row * ldw + static_cast<int64_t>(gi) * group;
     const double* sp = s64 + static_cast<int64_t>(gi) * group;
 
@@ -851,8 +853,8 @@ affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_group
             double lo = fmin(dmn, 0.0), hi = fmax(dmx, 0.0);
             double S = 1.0, Z = 0.0;
             if (hi != lo) { S = (hi - lo) / Km1; Z = -rint(lo / S); }
-            scale[gid] = static_cast<float>(S);
-            zero[gid] = static_cast<int32_t>(Z);
+            scale[oidx] = static_cast<float>(S);
+            zero[oidx] = static_cast<int32_t>(Z);
         }
         return;
     }
@@ -982,8 +984,8 @@ affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_group
             const int t_min = my_idx / side;
             params(t_min, my_idx - t_min * side, S, Z);
         }
-        scale[gid] = static_cast<float>(S);
-        zero[gid] = static_cast<int32_t>(Z);
+        scale[oidx] = static_cast<float>(S);
+        zero[oidx] = static_cast<int32_t>(Z);
     }
 }
 
@@ -1020,6 +1022,77 @@ int check_cfg(const lq_config* cfg) {
 
 }  // namespace
 
+// Sample weights s_j = exp(-p (ln dinv_j - mean ln dinv)) into s64 (c doubles); scal: 256 bytes of scratch.
+int lq_sample_weights(lq_handle* h, cudaStream_t st, const float* dinv, int64_t c, double p, double* scal, double* s64) {
+    log_mean_kernel<<<1, 1024, 0, st>>>(dinv, c, scal, h->dstatus);
+    LQ_LAUNCH_CHECK();
+    sample_weights_kernel<<<static_cast<unsigned>(lq_ceil_div(c, 256)), 256, 0, st>>>(dinv, c, p, scal, s64);
+    LQ_LAUNCH_CHECK();
+    return LQ_OK;
+}
+
+// The search of Eq. 7 over r x n_groups groups of g weights starting at W (row stride ldw); s64 holds the sample
+// weights of the n_groups * g columns; (S, Z) of group gi of row i goes to scale / zero [i * out_ld + gi].
+int lq_affine_search(lq_handle* h, cudaStream_t st, const void* W, int32_t w_dtype, int64_t r, int64_t ldw, int64_t g,
+                     int n_groups, const double* s64, int K, int T, int t_count, float* scale, int32_t* zero, int64_t out_ld) {
+    int p_max = 0;
+    size_t smem_c = 0;
+    if (affine_class_plan(K, T, t_count, g, &p_max, &smem_c)) {
+        static bool attr_c = false;
+        if (!attr_c) {
+            LQ_CUDA_TRY(cudaFuncSetAttribute(affine_class_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+            LQ_CUDA_TRY(cudaFuncSetAttribute(affine_class_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+            attr_c = true;
+        }
+        const unsigned nb = static_cast<unsigned>(r * n_groups);
+        const int threads = g > 8192 ? 512 : 256;
+        if (w_dtype == LQ_F32)
+            affine_class_kernel<float><<<nb, threads, smem_c, st>>>(static_cast<const float*>(W), ldw, (int)g, n_groups, s64, K, T,
+                                                                   t_count, p_max, scale, zero, out_ld, h->dstatus);
+        else
+            affine_class_kernel<__nv_bfloat16><<<nb, threads, smem_c, st>>>(static_cast<const __nv_bfloat16*>(W), ldw, (int)g, n_groups,
+                                                                           s64, K, T, t_count, p_max, scale, zero, out_ld, h->dstatus);
+        LQ_LAUNCH_CHECK();
+        return LQ_OK;
+    }
+    if (g <= AFW_MAX_GROUP && g % 2 == 0) {
+        const int64_t total = r * n_groups;
+        const size_t smem_w = static_cast<size_t>(AFW_WARPS) * g * sizeof(float2);
+        static bool attr_w = false;
+        if (!attr_w) {
+            LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_warp_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, AFW_WARPS * AFW_MAX_GROUP * 8));
+            LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_warp_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, AFW_WARPS * AFW_MAX_GROUP * 8));
+            attr_w = true;
+        }
+        const unsigned nb = static_cast<unsigned>(lq_ceil_div(total, AFW_WARPS));
+        if (w_dtype == LQ_F32)
+            affine_search_warp_kernel<float><<<nb, AFW_WARPS * 32, smem_w, st>>>(static_cast<const float*>(W), ldw, (int)g, n_groups, total,
+                                                                              s64, K, T, t_count, scale, zero, out_ld);
+        else
+            affine_search_warp_kernel<__nv_bfloat16><<<nb, AFW_WARPS * 32, smem_w, st>>>(static_cast<const __nv_bfloat16*>(W), ldw, (int)g,
+                                                                                      n_groups, total, s64, K, T, t_count, scale, zero,
+                                                                                      out_ld);
+        LQ_LAUNCH_CHECK();
+        return LQ_OK;
+    }
+    const size_t smem = static_cast<size_t>(g) * sizeof(float);
+    const unsigned blocks = static_cast<unsigned>(r * n_groups);
+    static bool attr_set = false;
+    if (!attr_set) {
+        LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+        attr_set = true;
+    }
+    if (w_dtype == LQ_F32)
+        affine_search_kernel<float><<<blocks, AF_THREADS, smem, st>>>(static_cast<const float*>(W), ldw, 0, (int)g, n_groups, s64, K, T,
+                                                                       t_count, scale, zero, out_ld);
+    else
+        affine_search_kernel<__nv_bfloat16><<<blocks, AF_THREADS, smem, st>>>(static_cast<const __nv_bfloat16*>(W), ldw, 0, (int)g,
+                                                                               n_groups, s64, K, T, t_count, scale, zero, out_ld);
+    LQ_LAUNCH_CHECK();
+    return LQ_OK;
+}
+
 extern "C" int lq_fit_grid_workspace(const lq_config* cfg, int64_t r, int64_t c, size_t* bytes) {
     int e = check_cfg(cfg);
     if (e) return e;
@@ -1053,10 +1126,8 @@ extern "C" int lq_fit_grid(lq_handle* h, void* stream, const lq_config* cfg, con
         if (r * (c / g) > 0x7fffffffLL) return LQ_ERR_UNSUPPORTED;
     }
 
-    log_mean_kernel<<<1, 1024, 0, st>>>(dinv, c, scal, h->dstatus);
-    LQ_LAUNCH_CHECK();
-    sample_weights_kernel<<<static_cast<unsigned>(lq_ceil_div(c, 256)), 256, 0, st>>>(dinv, c, static_cast<double>(cfg->p), scal, s64);
-    LQ_LAUNCH_CHECK();
+    e = lq_sample_weights(h, st, dinv, c, static_cast<double>(cfg->p), scal, s64);
+    if (e) return e;
 
     if (cfg->grid_type == LQ_GRID_NONUNIFORM) {
 #define LQ_KM(KK)                                                                                                     \
@@ -1072,63 +1143,7 @@ extern "C" int lq_fit_grid(lq_handle* h, void* stream, const lq_config* cfg, con
 
     const int64_t g = cfg->group_size == 0 ? c : cfg->group_size;
     const int n_groups = static_cast<int>(c / g);
-    const int K = 1 << cfg->bits;
-    int p_max = 0;
-    size_t smem_c = 0;
-    if (affine_class_plan(K, cfg->T, cfg->t_count, g, &p_max, &smem_c)) {
-        static bool attr_c = false;
-        if (!attr_c) {
-            LQ_CUDA_TRY(cudaFuncSetAttribute(affine_class_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-            LQ_CUDA_TRY(cudaFuncSetAttribute(affine_class_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-            attr_c = true;
-        }
-        const unsigned nb = static_cast<unsigned>(r * n_groups);
-        const int threads = g > 8192 ? 512 : 256;
-        if (w_dtype == LQ_F32)
-            affine_class_kernel<float><<<nb, threads, smem_c, st>>>(static_cast<const float*>(W), ldw, (int)g, n_groups, s64, K, cfg->T,
-                                                                   cfg->t_count, p_max, scale, zero, h->dstatus);
-        else
-            affine_class_kernel<__nv_bfloat16><<<nb, threads, smem_c, st>>>(static_cast<const __nv_bfloat16*>(W), ldw, (int)g, n_groups,
-                                                                           s64, K, cfg->T, cfg->t_count, p_max, scale, zero, h->dstatus);
-        LQ_LAUNCH_CHECK();
-        return LQ_OK;
-    }
-    if (g <= AFW_MAX_GROUP && g % 2 == 0) {
-        const int64_t total = r * n_groups;
-        const size_t smem_w = static_cast<size_t>(AFW_WARPS) * g * sizeof(float2);
-        static bool attr_w = false;
-        if (!attr_w) {
-            LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_warp_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, AFW_WARPS * AFW_MAX_GROUP * 8));
-            LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_warp_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, AFW_WARPS * AFW_MAX_GROUP * 8));
-            attr_w = true;
-        }
-        const unsigned nb = static_cast<unsigned>(lq_ceil_div(total, AFW_WARPS));
-        if (w_dtype == LQ_F32)
-            affine_search_warp_kernel<float><<<nb, AFW_WARPS * 32, smem_w, st>>>(static_cast<const float*>(W), ldw, (int)g, n_groups, total,
-                                                                              s64, K, cfg->T, cfg->t_count, scale, zero);
-        else
-            affine_search_warp_kernel<__nv_bfloat16><<<nb, AFW_WARPS * 32, smem_w, st>>>(static_cast<const __nv_bfloat16*>(W), ldw, (int)g,
-                                                                                      n_groups, total, s64, K, cfg->T, cfg->t_count,
-                                                                                      scale, zero);
-        LQ_LAUNCH_CHECK();
-        return LQ_OK;
-    }
-    const size_t smem = static_cast<size_t>(g) * sizeof(float);
-    const unsigned blocks = static_cast<unsigned>(r * n_groups);
-    static bool attr_set = false;
-    if (!attr_set) {
-        LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-        LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-        attr_set = true;
-    }
-    if (w_dtype == LQ_F32)
-        affine_search_kernel<float><<<blocks, AF_THREADS, smem, st>>>(static_cast<const float*>(W), ldw, c, (int)g, n_groups, s64, K,
-                                                                       cfg->T, cfg->t_count, scale, zero);
-    else
-        affine_search_kernel<__nv_bfloat16><<<blocks, AF_THREADS, smem, st>>>(static_cast<const __nv_bfloat16*>(W), ldw, c, (int)g,
-                                                                               n_groups, s64, K, cfg->T, cfg->t_count, scale, zero);
-    LQ_LAUNCH_CHECK();
-    return LQ_OK;
+    return lq_affine_search(h, st, W, w_dtype, r, ldw, g, n_groups, s64, 1 << cfg->bits, cfg->T, cfg->t_count, scale, zero, n_groups);
 }
 
 // ---------------------------------------------------- entry point without allocation --

@@ -306,10 +306,21 @@ extern "C" int lq_quantize_layer_workspace(const lq_config* cfg, int64_t r, int6
     return LQ_OK;
 }
 
-extern "C" int lq_quantize_layer(lq_handle* h, void* stream, const lq_config* cfg, const void* W, int32_t w_dtype,
-                                 int64_t r, int64_t c, int64_t ldw, const float* U, int64_t ldu, const float* grid,
-                                 const float* scale, const int32_t* zero, uint8_t* codes, void* W_hat,
-                                 int32_t what_dtype, int64_t ldwh, double* loss_out, void* ws, size_t ws_bytes) {
+namespace {
+// Whether the (S, Z) of a group can be refitted when the column loop reaches it: by then every earlier block's errors
+// must have reached all of the group's columns, which the two-level update guarantees for groups that tile a
+// 1024-column outer block, for groups made of whole outer blocks, and trivially for one group per row.
+bool lazy_group_ok(int64_t g, int64_t c) {
+    if (g == c) return true;
+    if (g % B) return false;
+    return (g <= OB && OB % g == 0) || (g % OB == 0);
+}
+
+// dinv != nullptr selects the lazy refit: scale / zero are then outputs, filled group by group as the loop goes.
+int quantize_impl(lq_handle* h, void* stream, const lq_config* cfg, const void* W, int32_t w_dtype,
+                  int64_t r, int64_t c, int64_t ldw, const float* U, int64_t ldu, const float* grid,
+                  float* scale, int32_t* zero, const float* dinv, uint8_t* codes, void* W_hat,
+                  int32_t what_dtype, int64_t ldwh, double* loss_out, void* ws, size_t ws_bytes) {
     int e = check_cfg4(cfg);
     if (e) return e;
     if (!h || !W || !U || !codes || r <= 0 || c <= 0 || ldw < c || ldu < c) return LQ_ERR_INVALID_ARG;
@@ -330,10 +341,21 @@ extern "C" int lq_quantize_layer(lq_handle* h, void* stream, const lq_config* cf
         return LQ_ERR_INVALID_ARG;
     }
     const WsLayout L = ws_layout(r, c);
-    if (!ws || ws_bytes < L.total) return LQ_ERR_WORKSPACE_TOO_SMALL;
+    const bool lazy = dinv != nullptr;
+    const size_t lazy_bytes = lazy ? 256 + lq_align_up(static_cast<size_t>(c) * sizeof(double), 256) : 0;
+    if (!ws || ws_bytes < L.total + lazy_bytes) return LQ_ERR_WORKSPACE_TOO_SMALL;
     if (reinterpret_cast<uintptr_t>(ws) & 255) return LQ_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char* wsp = static_cast<char*>(ws);
+    double* s64 = nullptr;
+    if (lazy) {
+        if (!affine) return LQ_ERR_INVALID_ARG;
+        if (cfg->T <= 0 || cfg->t_count < 0 || 2 * static_cast<int64_t>(cfg->t_count) > cfg->T || cfg->t_count > 4095) return LQ_ERR_INVALID_ARG;
+        if (!lazy_group_ok(group, c) || static_cast<size_t>(group) * sizeof(float) > 200 * 1024) return LQ_ERR_UNSUPPORTED;
+        s64 = reinterpret_cast<double*>(wsp + L.total + 256);
+        e = lq_sample_weights(h, st, dinv, c, static_cast<double>(cfg->p), reinterpret_cast<double*>(wsp + L.total), s64);
+        if (e) return e;
+    }
     float* Wc = reinterpret_cast<float*>(wsp + L.wc);
     __nv_bfloat16* UT = reinterpret_cast<__nv_bfloat16*>(wsp + L.ut);
     __nv_bfloat16* ES = reinterpret_cast<__nv_bfloat16*>(wsp + L.es);
@@ -367,6 +389,11 @@ extern "C" int lq_quantize_layer(lq_handle* h, void* stream, const lq_config* cf
         int rc;
         const int64_t o0 = i0 / OB * OB;          // start of the outer block
         out.e_col = static_cast<int>(i0 - o0);
+        if (lazy && i0 % group == 0) {             // (S, Z) of the group that starts here, on the columns as they stand now
+            rc = lq_affine_search(h, st, Wc + i0, LQ_F32, r, L.ldc, group, 1, s64 + i0, 1 << cfg->bits, cfg->T, cfg->t_count,
+                                  scale + i0 / group, zero + i0 / group, n_groups);
+            if (rc) return rc;
+        }
         if (affine) {
             switch (cfg->bits) {
                 case 2: rc = launch_inblock<4, true>(st, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
@@ -421,6 +448,31 @@ extern "C" int lq_quantize_layer(lq_handle* h, void* stream, const lq_config* cf
         LQ_LAUNCH_CHECK();
     }
     return LQ_OK;
+}
+}  // namespace
+
+extern "C" int lq_quantize_layer(lq_handle* h, void* stream, const lq_config* cfg, const void* W, int32_t w_dtype,
+                                 int64_t r, int64_t c, int64_t ldw, const float* U, int64_t ldu, const float* grid,
+                                 const float* scale, const int32_t* zero, uint8_t* codes, void* W_hat,
+                                 int32_t what_dtype, int64_t ldwh, double* loss_out, void* ws, size_t ws_bytes) {
+    return quantize_impl(h, stream, cfg, W, w_dtype, r, c, ldw, U, ldu, grid, const_cast<float*>(scale), const_cast<int32_t*>(zero),
+                         nullptr, codes, W_hat, what_dtype, ldwh, loss_out, ws, ws_bytes);
+}
+
+extern "C" int lq_quantize_layer_lazy_workspace(const lq_config* cfg, int64_t r, int64_t c, size_t* bytes) {
+    int e = lq_quantize_layer_workspace(cfg, r, c, bytes);
+    if (e) return e;
+    *bytes += 256 + lq_align_up(static_cast<size_t>(c) * sizeof(double), 256);
+    return LQ_OK;
+}
+
+extern "C" int lq_quantize_layer_lazy(lq_handle* h, void* stream, const lq_config* cfg, const void* W, int32_t w_dtype,
+                                      int64_t r, int64_t c, int64_t ldw, const float* U, int64_t ldu, const float* dinv,
+                                      float* scale, int32_t* zero, uint8_t* codes, void* W_hat, int32_t what_dtype,
+                                      int64_t ldwh, double* loss_out, void* ws, size_t ws_bytes) {
+    if (!dinv || !cfg || cfg->grid_type != LQ_GRID_AFFINE) return LQ_ERR_INVALID_ARG;
+    return quantize_impl(h, stream, cfg, W, w_dtype, r, c, ldw, U, ldu, nullptr, scale, zero, dinv, codes, W_hat, what_dtype, ldwh,
+                         loss_out, ws, ws_bytes);
 }
 
 extern "C" int lq_pack_codes(lq_handle* h, void* stream, const uint8_t* codes, int64_t r, int64_t c, int32_t bits,

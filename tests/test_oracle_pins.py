@@ -497,3 +497,52 @@ def test_e4_exact_in_natural_order_is_algorithm_1():
     assert np.array_equal(c1, c2)
     np.testing.assert_allclose(w1, w2, rtol=0, atol=1e-12)
     np.testing.assert_allclose(l1, l2, rtol=1e-9)
+
+
+# ------------------------------------------ lazy per-group refit of the affine grid ---- #
+def test_l1_lazy_refit_without_feedback_is_the_upfront_fit():
+    """With H = I nothing is fed back, the columns never change, and fitting a group when the loop reaches it
+    is fitting it beforehand."""
+    g = rng(21)
+    r, c = 6, 64
+    W = g.standard_normal((r, c)) * 0.05
+    dinv = np.exp(g.standard_normal(c))
+    s = O.sample_weights(dinv, 4.0)
+    S, Z = O.fit_grid_affine(W, dinv, 3, 4.0, 16, 30, 6)
+    c0, w0, l0 = O.quantize_layer(W, np.eye(c), scale=S, zero=Z, bits=3, group=16, block=32)
+    c1, w1, l1, S1, Z1 = O.quantize_layer(W, np.eye(c), bits=3, group=16, block=32, lazy=dict(s=s, T=30, t=6))
+    assert np.array_equal(S, S1) and np.array_equal(Z, Z1)
+    assert np.array_equal(c0, c1) and np.array_equal(w0, w1)
+
+
+def test_l2_lazy_refit_sees_the_fed_back_columns():
+    """First group: nothing has been fed back yet, so its (S, Z) are the up-front ones.  A later group: its (S, Z)
+    are the Eq. 7 fit of the columns as the up-front loop with the lazy grids leaves them at that moment, which a
+    second run with those grids given up front reproduces (same grids in, same trajectory)."""
+    g = rng(22)
+    r, c, grp = 5, 48, 16
+    W = g.standard_normal((r, c)) * 0.05
+    H = spd(c, 23, 1e2)
+    U, dinv, H_d, _ = O.prepare_hinv(H, 0.01)
+    s = O.sample_weights(dinv, 4.0)
+    S0, Z0 = O.fit_grid_affine(W, dinv, 4, 4.0, grp, 20, 4)
+    codes, What, loss, S, Z = O.quantize_layer(W, U, bits=4, group=grp, block=16, lazy=dict(s=s, T=20, t=4))
+    assert np.array_equal(S[:, 0], S0[:, 0]) and np.array_equal(Z[:, 0], Z0[:, 0])
+    assert not np.array_equal(S[:, 1:], S0[:, 1:])                      # feedback moved the later groups
+    c2, w2, l2 = O.quantize_layer(W, U, scale=S, zero=Z, bits=4, group=grp, block=16)
+    assert np.array_equal(codes, c2) and np.array_equal(What, w2)
+    for k in range(1, c // grp):                                        # and each later pair is the fit of what stood there
+        Sk, Zk = O.affine_search_group(_columns_at_group_start(W, U, S, Z, grp, k), s[k * grp:(k + 1) * grp], 16, 20, 4)
+        np.testing.assert_allclose(Sk, S[:, k], rtol=1e-9)               # the unblocked loop sums in another order
+        assert np.array_equal(Zk, Z[:, k])
+
+
+def _columns_at_group_start(W, U, S, Z, grp, k):
+    """Columns of group k after the columns of groups < k were quantised with the given grids (unblocked loop)."""
+    Wc = W.copy()
+    c = W.shape[1]
+    for j in range(k * grp):
+        q = O.quant_aff(Wc[:, j], S[:, j // grp], Z[:, j // grp], 16)
+        e = (Wc[:, j] - q) / U[j, j]
+        Wc[:, j:] -= np.outer(e, U[j, j:])
+    return Wc[:, k * grp:(k + 1) * grp]
