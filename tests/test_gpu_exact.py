@@ -65,6 +65,7 @@ def run_exact_gpu(lq, h, cfg, W, P):
     ("c2", 40, 300, 2048, dict(grid="nonuniform", bits=3, p=4.0, n_iter=10)),
     ("c3", 16, 256, 1024, dict(grid="affine", bits=4, p=4.0, group=32, T=40, t=8)),
     ("c3", 6, 132, 1024, dict(grid="affine", bits=3, p=4.0, group=0, T=40, t=8)),   # ragged width, one group per row
+    ("c2", 700, 64, 512, dict(grid="nonuniform", bits=3, p=4.0, n_iter=5)),         # more rows than resident CTAs: each CTA takes several
 ])
 def test_exact_loop_isolated(lq, h, recipe, r, c, n, kw):
     L = synth.make_layer(recipe, r, c, n, seed=r + c)
