@@ -71,11 +71,10 @@ struct QuantOut {
 // lane `code`; then E = (w - q) / U_jj and every lane feeds it into its four weights with one
 // 16-byte read of row j of the block of U held in shared memory.  Entries of that row left of
 // the diagonal are zero, so no lane needs a predicate.
-constexpr int IB_WARPS = 16;
-constexpr int IB_THREADS = IB_WARPS * 32;
+constexpr int IB_MAX_THREADS = 1024;   // warps (= rows) per CTA are chosen at launch so that the rows spread evenly over the SMs
 
 template <int K, bool AFFINE>
-__global__ void __launch_bounds__(IB_THREADS)
+__global__ void __launch_bounds__(IB_MAX_THREADS)
 inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, int64_t i0, const float* __restrict__ U,
                int64_t ldu, const float* __restrict__ grid, const float* __restrict__ scale,
                const int32_t* __restrict__ zero, int group, int n_groups, QuantOut out) {
@@ -87,7 +86,8 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
     // The block of U goes to shared memory with asynchronous copies (plain loads for a ragged
     // last block); the row's weights and grid are fetched while those copies are in flight.
     const bool whole = bw == B && (ldu % 4 == 0);
-    for (int idx = tid; idx < B * B / 4; idx += IB_THREADS) {
+    const int nthr = blockDim.x;
+    for (int idx = tid; idx < B * B / 4; idx += nthr) {
         const int jj = idx / (B / 4), k4 = (idx % (B / 4)) * 4;
         if (whole) {
             const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(Us + jj * B + k4));
@@ -104,7 +104,7 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
 
-    const int64_t row = (int64_t)blockIdx.x * IB_WARPS + warp;
+    const int64_t row = (int64_t)blockIdx.x * (nthr >> 5) + warp;
     const bool valid = row < r;
     const int col0 = 4 * lane;             // first of this lane's columns inside the block
     float w[4] = {0.0f, 0.0f, 0.0f, 0.0f};
@@ -282,7 +282,7 @@ int check_cfg4(const lq_config* cfg) {
 }
 
 template <int K, bool AFFINE>
-int launch_inblock(cudaStream_t st, float* Wc, int64_t ldc, int64_t r, int64_t c, int64_t i0, const float* U, int64_t ldu,
+int launch_inblock(cudaStream_t st, int sm_count, float* Wc, int64_t ldc, int64_t r, int64_t c, int64_t i0, const float* U, int64_t ldu,
                    const float* grid, const float* scale, const int32_t* zero, int group, int n_groups, const QuantOut& out) {
     const int smem = (B * B + B) * sizeof(float);
     static bool attr_set = false;
@@ -290,7 +290,14 @@ int launch_inblock(cudaStream_t st, float* Wc, int64_t ldc, int64_t r, int64_t c
         LQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel<K, AFFINE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
         attr_set = true;
     }
-    inblock_kernel<K, AFFINE><<<static_cast<unsigned>(lq_ceil_div(r, IB_WARPS)), IB_THREADS, smem, st>>>(
+    // One warp per row.  The kernel is bound by instruction issue, so what matters is the largest number of rows
+    // on one SM: up to 32 rows per SM one CTA per SM takes an even share; beyond that, CTAs of 16 rows fill the SMs.
+    int warps = 16;
+    if (r <= 32 * static_cast<int64_t>(sm_count)) {
+        warps = static_cast<int>(lq_ceil_div(r, sm_count));
+        if (warps < 4) warps = 4;                  // the 128 reciprocals of the diagonal are computed by the first 128 threads
+    }
+    inblock_kernel<K, AFFINE><<<static_cast<unsigned>(lq_ceil_div(r, warps)), warps * 32, smem, st>>>(
         Wc, ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out);
     LQ_LAUNCH_CHECK();
     return LQ_OK;
@@ -396,15 +403,15 @@ int quantize_impl(lq_handle* h, void* stream, const lq_config* cfg, const void* 
         }
         if (affine) {
             switch (cfg->bits) {
-                case 2: rc = launch_inblock<4, true>(st, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
-                case 3: rc = launch_inblock<8, true>(st, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
-                default: rc = launch_inblock<16, true>(st, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
+                case 2: rc = launch_inblock<4, true>(st, h->sm_count, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
+                case 3: rc = launch_inblock<8, true>(st, h->sm_count, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
+                default: rc = launch_inblock<16, true>(st, h->sm_count, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
             }
         } else {
             switch (cfg->bits) {
-                case 2: rc = launch_inblock<4, false>(st, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
-                case 3: rc = launch_inblock<8, false>(st, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
-                default: rc = launch_inblock<16, false>(st, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
+                case 2: rc = launch_inblock<4, false>(st, h->sm_count, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
+                case 3: rc = launch_inblock<8, false>(st, h->sm_count, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
+                default: rc = launch_inblock<16, false>(st, h->sm_count, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
             }
         }
         if (rc) return rc;
