@@ -18,8 +18,40 @@ constexpr int B = 128;      // block width of the column loop
 constexpr int OB = 1024;    // outer block: the lazy update of columns beyond it waits until it is complete
 
 template <typename T>
-__global__ void to_f32_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, float* __restrict__ Wc, int64_t ldc) {
+__global__ void to_f32_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, float* __restrict__ Wc, int64_t ldc, int vec) {
     const int64_t row = blockIdx.y;
+    if (vec) {      // eight weights per thread: one 16-byte (bf16) or two 16-byte (fp32) loads, two 16-byte stores
+        const int64_t n8 = c / 8;
+        for (int64_t j8 = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j8 < n8; j8 += (int64_t)gridDim.x * blockDim.x) {
+            float v[8];
+            if (sizeof(T) == 4) {
+                const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(W) + row * ldw + 8 * j8);
+                const float4 x = p[0], y = p[1];
+                v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w; v[4] = y.x; v[5] = y.y; v[6] = y.z; v[7] = y.w;
+            } else {
+                const uint4 x = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(W) + row * ldw + 8 * j8);
+                const uint32_t u[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    v[2 * e] = __uint_as_float(u[e] << 16);
+                    v[2 * e + 1] = __uint_as_float(u[e] & 0xffff0000u);
+                }
+            }
+            float4* q = reinterpret_cast<float4*>(Wc + row * ldc + 8 * j8);
+            q[0] = make_float4(v[0], v[1], v[2], v[3]);
+            q[1] = make_float4(v[4], v[5], v[6], v[7]);
+        }
+        // the ragged end of the row, if any
+        for (int64_t j = n8 * 8 + blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < ldc; j += (int64_t)gridDim.x * blockDim.x) {
+            float v = 0.0f;
+            if (j < c) {
+                if (sizeof(T) == 4) v = reinterpret_cast<const float*>(W)[row * ldw + j];
+                else v = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(W)[row * ldw + j]);
+            }
+            Wc[row * ldc + j] = v;
+        }
+        return;
+    }
     for (int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < ldc; j += (int64_t)gridDim.x * blockDim.x) {
         float v = 0.0f;
         if (j < c) {
@@ -30,26 +62,48 @@ __global__ void to_f32_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, f
     }
 }
 
-// UT[s][n][k] = s-th bf16 term of U[k][n]   (three stacked c x ldt matrices)
-__global__ void split_transpose_kernel(const float* __restrict__ U, int64_t ldu, int64_t c,
-                                       __nv_bfloat16* __restrict__ UT, int64_t ldt) {
-    __shared__ float tile[32][33];
-    const int64_t k0 = (int64_t)blockIdx.y * 32, n0 = (int64_t)blockIdx.x * 32;
-    const int tx = threadIdx.x, ty = threadIdx.y;       // 32 x 8
-    for (int a = ty; a < 32; a += 8) {
-        const int64_t k = k0 + a, n = n0 + tx;
-        tile[a][tx] = (k < c && n < c) ? U[k * ldu + n] : 0.0f;
+// UT[s][n][k] = s-th bf16 term of U[k][n]   (three stacked c x ldt matrices).  64 x 64 tiles: 16-byte reads along n,
+// 16-byte writes (eight bf16) along k.
+__global__ void __launch_bounds__(256)
+split_transpose_kernel(const float* __restrict__ U, int64_t ldu, int64_t c, __nv_bfloat16* __restrict__ UT, int64_t ldt) {
+    __shared__ float tile[64][65];
+    const int64_t k0 = (int64_t)blockIdx.y * 64, n0 = (int64_t)blockIdx.x * 64;
+    const int tid = threadIdx.x;
+    const bool vec_in = (ldu % 4 == 0) && ((reinterpret_cast<uintptr_t>(U) & 15) == 0);
+    for (int idx = tid; idx < 64 * 16; idx += 256) {
+        const int a = idx >> 4, n4 = (idx & 15) * 4;
+        const int64_t k = k0 + a, n = n0 + n4;
+        float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+        if (k < c) {
+            if (vec_in && n + 3 < c) v = *reinterpret_cast<const float4*>(U + k * ldu + n);
+            else {
+                if (n < c) v.x = U[k * ldu + n];
+                if (n + 1 < c) v.y = U[k * ldu + n + 1];
+                if (n + 2 < c) v.z = U[k * ldu + n + 2];
+                if (n + 3 < c) v.w = U[k * ldu + n + 3];
+            }
+        }
+        tile[a][n4] = v.x; tile[a][n4 + 1] = v.y; tile[a][n4 + 2] = v.z; tile[a][n4 + 3] = v.w;
     }
     __syncthreads();
-    for (int a = ty; a < 32; a += 8) {
-        const int64_t n = n0 + a, k = k0 + tx;
-        if (n < c && k < ldt) {
-            __nv_bfloat16 h, m, l;
-            lq_split3(k < c ? tile[tx][a] : 0.0f, h, m, l);
-            UT[n * ldt + k] = h;
-            UT[(c + n) * ldt + k] = m;
-            UT[(2 * c + n) * ldt + k] = l;
+    for (int idx = tid; idx < 64 * 8; idx += 256) {
+        const int a = idx >> 3, k8 = (idx & 7) * 8;        // output row n0 + a, eight consecutive k
+        const int64_t n = n0 + a, k = k0 + k8;
+        if (n >= c || k >= ldt) continue;
+        uint32_t ph[4], pm[4], pl[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            __nv_bfloat16 h0, m0, l0, h1, m1, l1;
+            lq_split3(tile[k8 + 2 * e][a], h0, m0, l0);            // rows k >= c of the tile are zero
+            lq_split3(tile[k8 + 2 * e + 1][a], h1, m1, l1);
+            ph[e] = static_cast<uint32_t>(__bfloat16_as_ushort(h0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(h1)) << 16);
+            pm[e] = static_cast<uint32_t>(__bfloat16_as_ushort(m0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(m1)) << 16);
+            pl[e] = static_cast<uint32_t>(__bfloat16_as_ushort(l0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(l1)) << 16);
         }
+        // ldt is a multiple of 8 and k a multiple of 8: the eight entries are inside the row and 16-byte aligned
+        *reinterpret_cast<uint4*>(UT + n * ldt + k) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
+        *reinterpret_cast<uint4*>(UT + (c + n) * ldt + k) = make_uint4(pm[0], pm[1], pm[2], pm[3]);
+        *reinterpret_cast<uint4*>(UT + (2 * c + n) * ldt + k) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
     }
 }
 
@@ -370,13 +424,15 @@ int quantize_impl(lq_handle* h, void* stream, const lq_config* cfg, const void* 
 
     {
         dim3 g(static_cast<unsigned>(lq_ceil_div(L.ldc, 256) < 32 ? lq_ceil_div(L.ldc, 256) : 32), static_cast<unsigned>(r));
-        if (w_dtype == LQ_F32) to_f32_kernel<float><<<g, 256, 0, st>>>(static_cast<const float*>(W), ldw, c, Wc, L.ldc);
-        else to_f32_kernel<__nv_bfloat16><<<g, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(W), ldw, c, Wc, L.ldc);
+        // 16-byte accesses when rows of W start on 16-byte boundaries (the working copy's always do)
+        const int vec = ((reinterpret_cast<uintptr_t>(W) & 15) == 0 && (ldw * (w_dtype == LQ_F32 ? 4 : 2)) % 16 == 0) ? 1 : 0;
+        if (w_dtype == LQ_F32) to_f32_kernel<float><<<g, 256, 0, st>>>(static_cast<const float*>(W), ldw, c, Wc, L.ldc, vec);
+        else to_f32_kernel<__nv_bfloat16><<<g, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(W), ldw, c, Wc, L.ldc, vec);
         LQ_LAUNCH_CHECK();
     }
     if (c > B) {
-        dim3 g(static_cast<unsigned>(lq_ceil_div(c, 32)), static_cast<unsigned>(lq_ceil_div(L.ldt, 32)));
-        split_transpose_kernel<<<g, dim3(32, 8), 0, st>>>(U, ldu, c, UT, L.ldt);
+        dim3 g(static_cast<unsigned>(lq_ceil_div(c, 64)), static_cast<unsigned>(lq_ceil_div(L.ldt, 64)));
+        split_transpose_kernel<<<g, 256, 0, st>>>(U, ldu, c, UT, L.ldt);
         LQ_LAUNCH_CHECK();
     }
     zero_doubles_kernel<<<static_cast<unsigned>(lq_ceil_div(r, 256)), 256, 0, st>>>(loss_rows, r);
