@@ -63,19 +63,34 @@ __global__ void load_damped_kernel(const float* __restrict__ H, int64_t c, int64
                                    double* __restrict__ A, int64_t cp, lq_dev_status* st) {
     const int64_t i = blockIdx.y;
     const double damp = scal[0];
-    for (int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < cp; j += (int64_t)gridDim.x * blockDim.x) {
-        double v = 0.0;
-        if (i < c && j < c) {
-            if (j >= i) {
-                float hv = H[i * ldh + j];
-                if (!isfinite(hv)) lq_report(st, LQ_ERR_NONFINITE, i * c + j);
-                v = static_cast<double>(hv);
-                if (i == j) v = (hv == 0.0f ? 1.0 : v) + damp;
+    // four entries per thread: one 16-byte read where the row of H allows it, two 16-byte writes
+    const bool vec = (ldh % 4 == 0) && ((reinterpret_cast<uintptr_t>(H) & 15) == 0);
+    for (int64_t j0 = 4 * (blockIdx.x * (int64_t)blockDim.x + threadIdx.x); j0 < cp; j0 += 4 * (int64_t)gridDim.x * blockDim.x) {
+        double v[4] = {0.0, 0.0, 0.0, 0.0};
+        if (i < c && j0 + 3 >= i && j0 < c) {
+            float hv[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+            if (vec && j0 + 3 < c) {
+                const float4 x = *reinterpret_cast<const float4*>(H + i * ldh + j0);
+                hv[0] = x.x; hv[1] = x.y; hv[2] = x.z; hv[3] = x.w;
+            } else {
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (j0 + e < c) hv[e] = H[i * ldh + j0 + e];
             }
-        } else if (i == j) {
-            v = 1.0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int64_t j = j0 + e;
+                if (j < c && j >= i) {
+                    if (!isfinite(hv[e])) lq_report(st, LQ_ERR_NONFINITE, i * c + j);
+                    v[e] = static_cast<double>(hv[e]);
+                    if (i == j) v[e] = (hv[e] == 0.0f ? 1.0 : v[e]) + damp;
+                }
+            }
         }
-        A[i * cp + j] = v;
+        if (i >= c && i >= j0 && i < j0 + 4) v[i - j0] = 1.0;        // identity on the padding
+        double2* out = reinterpret_cast<double2*>(A + i * cp + j0);  // cp is a multiple of 128
+        out[0] = make_double2(v[0], v[1]);
+        out[1] = make_double2(v[2], v[3]);
     }
 }
 
@@ -535,7 +550,7 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
     const PrepLayout L = prep_layout(c);
     if (!ws || ws_bytes < L.total) return LQ_ERR_WORKSPACE_TOO_SMALL;
     if (reinterpret_cast<uintptr_t>(ws) & 255) return LQ_ERR_INVALID_ARG;
-    if (L.nblk > 32767 || c > 65536) return LQ_ERR_UNSUPPORTED;   // grid.y of the update launch; room for the column sums
+    if (L.nblk > 32767 || L.cp > 65535) return LQ_ERR_UNSUPPORTED;   // grid.y of the set-up and update launches; room for the column sums
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
     const int64_t nblk = L.nblk, cp = L.cp;
@@ -562,7 +577,7 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
         LQ_LAUNCH_CHECK();
     }
     {
-        dim3 g(static_cast<unsigned>(lq_ceil_div(cp, 256) < 32 ? lq_ceil_div(cp, 256) : 32), static_cast<unsigned>(cp));
+        dim3 g(static_cast<unsigned>(lq_ceil_div(cp, 1024) < 32 ? lq_ceil_div(cp, 1024) : 32), static_cast<unsigned>(cp));
         load_damped_kernel<<<g, 256, 0, st>>>(H, c, ldh, scal, A, cp, h->dstatus);
         LQ_LAUNCH_CHECK();
     }
