@@ -64,6 +64,7 @@ struct KParams {
     int upper_only;
     int tile_m;               // rows of a tile: 128 or 256
     int tiles_m, tiles_n;
+    int band;                 // upper_only: tile rows per band of the schedule
     int num_tiles;
     int seg_iters;            // k-iterations accumulated in TMEM before the partial sum is flushed to D
     int segs_per_tile;        // ceil(k_iters / seg_iters)
@@ -233,20 +234,38 @@ __device__ __forceinline__ uint64_t make_desc_sw128(uint32_t saddr) {
 }
 
 // Map the idx-th scheduled tile to (tile row, tile column).  With upper_only, row tm keeps
-// the columns tn with (tn + 1) * BN > tm * tile_m.
+// the columns tn with (tn + 1) * BN > tm * tile_m, and the tiles are ordered in bands of `band`
+// tile rows, column by column inside a band: the CTAs of one scheduling round then work on a
+// roughly square patch of the output and share a few panels of each operand through the L2
+// (in plain row-major order a round shares one panel of A and reads as many panels of B as it
+// has tiles, which makes wide symmetric products HBM-bound).
 __device__ __forceinline__ void tile_coords(const KParams& p, int idx, int& tm, int& tn) {
     if (!p.upper_only) {
         tm = idx / p.tiles_n;
         tn = idx - tm * p.tiles_n;
         return;
     }
-    int m = 0;
-    for (;; ++m) {
-        int first = (m * p.tile_m) / BN;
-        int cnt = p.tiles_n - first;
-        if (cnt < 0) cnt = 0;
-        if (idx < cnt) { tm = m; tn = first + idx; return; }
-        idx -= cnt;
+    const int G = p.band;
+    for (int m0 = 0;; m0 += G) {
+        const int m1 = (m0 + G < p.tiles_m) ? m0 + G : p.tiles_m;
+        int band_cnt = 0;
+        for (int m = m0; m < m1; ++m) {
+            const int cnt = p.tiles_n - (m * p.tile_m) / BN;
+            band_cnt += cnt > 0 ? cnt : 0;
+        }
+        if (idx >= band_cnt && m1 < p.tiles_m) { idx -= band_cnt; continue; }
+        // inside the band: the first columns are met by some of its rows only (first column of a row never decreases)
+        const int rows_all = m1 - m0;
+        const int full_from = ((m1 - 1) * p.tile_m) / BN;            // from this column on every row of the band is present
+        for (int c = (m0 * p.tile_m) / BN; c < full_from && c < p.tiles_n; ++c) {
+            int rows = 0;
+            for (int m = m0; m < m1; ++m) rows += ((m * p.tile_m) / BN <= c) ? 1 : 0;
+            if (idx < rows) { tm = m0 + idx; tn = c; return; }
+            idx -= rows;
+        }
+        tn = full_from + idx / rows_all;
+        tm = m0 + idx % rows_all;
+        return;
     }
 }
 
@@ -589,6 +608,7 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
     p.alpha = a.alpha;
     p.accumulate = a.accumulate;
     p.upper_only = a.upper_only;
+    p.band = 8;
     p.tile_m = BM * ctas_per_tile;
     p.tiles_m = static_cast<int>(lq_ceil_div(a.M, p.tile_m));
     p.tiles_n = static_cast<int>(lq_ceil_div(a.N, BN));
