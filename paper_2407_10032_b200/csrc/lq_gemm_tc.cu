@@ -64,7 +64,7 @@ struct KParams {
     int upper_only;
     int tile_m;               // rows of a tile: 128 or 256
     int tiles_m, tiles_n;
-    int band;                 // upper_only: tile rows per band of the schedule
+    int band;                 // tile rows per band of the schedule (see tile_coords)
     int num_tiles;
     int seg_iters;            // k-iterations accumulated in TMEM before the partial sum is flushed to D
     int segs_per_tile;        // ceil(k_iters / seg_iters)
@@ -234,18 +234,22 @@ __device__ __forceinline__ uint64_t make_desc_sw128(uint32_t saddr) {
 }
 
 // Map the idx-th scheduled tile to (tile row, tile column).  With upper_only, row tm keeps
-// the columns tn with (tn + 1) * BN > tm * tile_m, and the tiles are ordered in bands of `band`
+// the columns tn with (tn + 1) * BN > tm * tile_m.  The tiles are ordered in bands of `band`
 // tile rows, column by column inside a band: the CTAs of one scheduling round then work on a
 // roughly square patch of the output and share a few panels of each operand through the L2
 // (in plain row-major order a round shares one panel of A and reads as many panels of B as it
 // has tiles, which makes wide symmetric products HBM-bound).
 __device__ __forceinline__ void tile_coords(const KParams& p, int idx, int& tm, int& tn) {
+    const int G = p.band;
     if (!p.upper_only) {
-        tm = idx / p.tiles_n;
-        tn = idx - tm * p.tiles_n;
+        const int per_band = G * p.tiles_n;
+        const int m0 = (idx / per_band) * G;
+        const int rows = (m0 + G < p.tiles_m) ? G : p.tiles_m - m0;      // the last band may be lower
+        const int in_band = idx - (m0 / G) * per_band;
+        tn = in_band / rows;
+        tm = m0 + in_band - tn * rows;
         return;
     }
-    const int G = p.band;
     for (int m0 = 0;; m0 += G) {
         const int m1 = (m0 + G < p.tiles_m) ? m0 + G : p.tiles_m;
         int band_cnt = 0;
