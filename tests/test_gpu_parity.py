@@ -1,5 +1,5 @@
 """Parity of the CUDA path (through the C ABI) with the float64 oracle, stage by stage and
-chained, on seeded synthetic layers.  Tolerances (from the benchmark spec): centroids within
+chained, on seeded synthetic layers.  Tolerances: centroids within
 1e-4 relative, at most 0.1 % of integer codes differing, layer loss within 1e-3 relative."""
 import numpy as np
 import pytest
