@@ -250,8 +250,24 @@ __global__ void __launch_bounds__(EX_THREADS, 2) exact_row_kernel(ExactArgs A) {
 #pragma unroll
                         for (int q = 0; q < 4; ++q) aw[q * EX_MAX_NB + lane] = V[static_cast<size_t>(lane) * c + jr[q]] * rpiv[lane];
                     }
+                    {   // the first strip of the four rows this warp takes next is asked for now
+                        const int pn = p + EX_WARPS * 4 + (lane >> 3);
+                        if (pn < nr) {
+                            const int jn = rows[pn];
+                            const int ln = (rows[min(p + EX_WARPS * 4, nr - 1)] & ~127) + (lane & 7) * 16;
+                            if (ln < c) asm volatile("prefetch.global.L2 [%0];" ::"l"(Hi + static_cast<size_t>(jn) * c + ln));
+                        }
+                    }
                     __syncwarp();
                     for (int l0 = jr[0] & ~127; l0 < c; l0 += 128) {
+                        {   // the strip after the next of the four rows is asked for now (32 lines of 128 bytes, one per lane)
+                            const int ln = l0 + 256 + (lane & 7) * 16;
+                            if (ln < c) asm volatile("prefetch.global.L2 [%0];" ::"l"(hr[lane >> 3] + ln));
+                            if (l0 == (jr[0] & ~127)) {          // and at the start of a group also the next one
+                                const int l1 = l0 + 128 + (lane & 7) * 16;
+                                if (l1 < c) asm volatile("prefetch.global.L2 [%0];" ::"l"(hr[lane >> 3] + l1));
+                            }
+                        }
                         double x[4][4];
 #pragma unroll
                         for (int q = 0; q < 4; ++q)
