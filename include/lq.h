@@ -225,7 +225,7 @@ int lq_quantize_layer_lazy(lq_handle* h, void* stream, const lq_config* cfg, con
  * is the sum over all weights of the loss error at the moment each was quantised (equal to
  * 1/2 sum_rows (w - w_hat) H_d (w - w_hat)^T), cfg->block is ignored and any group size dividing c is
  * accepted.  c <= 8192.  Workspace: lq_quantize_exact_workspace bytes, 256-byte aligned (the fp64 inverse
- * plus one copy of it per resident CTA).  A non-positive pivot records LQ_ERR_NOT_POSITIVE_DEFINITE
+ * plus one copy of it per resident CTA, 16 GiB of copies at most).  A non-positive pivot records LQ_ERR_NOT_POSITIVE_DEFINITE
  * (info = row * c + index). */
 int lq_quantize_exact_workspace(const lq_config* cfg, int64_t r, int64_t c, size_t* bytes);
 int lq_quantize_exact(lq_handle* h, void* stream, const lq_config* cfg, const void* W, int32_t w_dtype,

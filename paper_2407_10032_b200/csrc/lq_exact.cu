@@ -347,10 +347,12 @@ int exact_plan(int64_t r, int64_t c, int sm_count, ExactPlan* P) {
     }
     P->nb = nb;
     P->smem = exact_smem(static_cast<int>(c), nb);
+    const size_t mat = lq_align_up(static_cast<size_t>(c) * c * sizeof(double), 256);
     int64_t slots = static_cast<int64_t>(sm_count) * per_sm;
     if (slots > r) slots = r;
+    const int64_t fit = static_cast<int64_t>((static_cast<size_t>(16) << 30) / mat);     // copies of the inverse: at most 16 GiB
+    if (slots > fit) slots = fit < 1 ? 1 : fit;
     P->slots = static_cast<int>(slots);
-    const size_t mat = lq_align_up(static_cast<size_t>(c) * c * sizeof(double), 256);
     P->off_hinv = 0;
     P->off_slots = mat;
     P->off_loss = mat + static_cast<size_t>(P->slots) * mat;
