@@ -45,6 +45,19 @@ extern unsigned long long lq_launches_total;
         if (cudaGetLastError() != cudaSuccess) return LQ_ERR_CUDA; \
     } while (0)
 
+// Kernel attributes (opt-in shared memory sizes) are per device: each set-up site keeps one of these and runs its
+// set-up once per device of the process.  Setting an attribute twice is harmless, so no lock is taken.
+struct lq_once_per_device {
+    bool done[64] = {};
+    bool first() {
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
+        if (done[dev]) return false;
+        done[dev] = true;
+        return true;
+    }
+};
+
 static inline size_t lq_align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline int64_t lq_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 

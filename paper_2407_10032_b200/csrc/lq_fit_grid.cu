@@ -453,10 +453,9 @@ int launch_kmeans(cudaStream_t st, int sms, const T* W, int64_t ldw, int64_t r, 
         while (n < c) n <<= 1;
         const size_t smem = (static_cast<size_t>(n) / KS_CHUNK + 1) * sizeof(dd2) +
                             static_cast<size_t>(n + n / 32) * sizeof(typename KeyOf<T>::type);
-        static bool attr_set = false;
-        if (!attr_set) {
+        static lq_once_per_device attr_set;
+        if (attr_set.first()) {
             LQ_CUDA_TRY(cudaFuncSetAttribute(kmeans_sorted_kernel<K, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-            attr_set = true;
         }
         int per_sm = static_cast<int>((228 * 1024) / (smem + 10 * 1024));      // static shared memory and the per-CTA reserve
         per_sm = per_sm < 1 ? 1 : (per_sm > 4 ? 4 : per_sm);                    // 64 registers x 256 threads: four CTAs per SM
@@ -467,10 +466,9 @@ int launch_kmeans(cudaStream_t st, int sms, const T* W, int64_t ldw, int64_t r, 
         if (init != LQ_INIT_UNIFORM) return LQ_ERR_UNSUPPORTED;     // rows this long only start from Eq. 6
         const size_t smem = static_cast<size_t>(c) * sizeof(T);
         if (smem > 200 * 1024) return LQ_ERR_UNSUPPORTED;
-        static bool attr_set = false;
-        if (!attr_set) {
+        static lq_once_per_device attr_set;
+        if (attr_set.first()) {
             LQ_CUDA_TRY(cudaFuncSetAttribute(kmeans_rows_kernel<K, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-            attr_set = true;
         }
         kmeans_rows_kernel<K, T><<<static_cast<unsigned>(r < sms ? r : sms), KM_THREADS, smem, st>>>(W, ldw, r, c, s64, grid, n_iter);
     }
@@ -1038,11 +1036,10 @@ int lq_affine_search(lq_handle* h, cudaStream_t st, const void* W, int32_t w_dty
     int p_max = 0;
     size_t smem_c = 0;
     if (affine_class_plan(K, T, t_count, g, &p_max, &smem_c)) {
-        static bool attr_c = false;
-        if (!attr_c) {
+        static lq_once_per_device attr_c;
+        if (attr_c.first()) {
             LQ_CUDA_TRY(cudaFuncSetAttribute(affine_class_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
             LQ_CUDA_TRY(cudaFuncSetAttribute(affine_class_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-            attr_c = true;
         }
         const unsigned nb = static_cast<unsigned>(r * n_groups);
         const int threads = g > 8192 ? 512 : 256;
@@ -1058,11 +1055,10 @@ int lq_affine_search(lq_handle* h, cudaStream_t st, const void* W, int32_t w_dty
     if (g <= AFW_MAX_GROUP && g % 2 == 0) {
         const int64_t total = r * n_groups;
         const size_t smem_w = static_cast<size_t>(AFW_WARPS) * g * sizeof(float2);
-        static bool attr_w = false;
-        if (!attr_w) {
+        static lq_once_per_device attr_w;
+        if (attr_w.first()) {
             LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_warp_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, AFW_WARPS * AFW_MAX_GROUP * 8));
             LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_warp_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, AFW_WARPS * AFW_MAX_GROUP * 8));
-            attr_w = true;
         }
         const unsigned nb = static_cast<unsigned>(lq_ceil_div(total, AFW_WARPS));
         if (w_dtype == LQ_F32)
@@ -1077,11 +1073,10 @@ int lq_affine_search(lq_handle* h, cudaStream_t st, const void* W, int32_t w_dty
     }
     const size_t smem = static_cast<size_t>(g) * sizeof(float);
     const unsigned blocks = static_cast<unsigned>(r * n_groups);
-    static bool attr_set = false;
-    if (!attr_set) {
+    static lq_once_per_device attr_set;
+    if (attr_set.first()) {
         LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
         LQ_CUDA_TRY(cudaFuncSetAttribute(affine_search_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
-        attr_set = true;
     }
     if (w_dtype == LQ_F32)
         affine_search_kernel<float><<<blocks, AF_THREADS, smem, st>>>(static_cast<const float*>(W), ldw, 0, (int)g, n_groups, s64, K, T,

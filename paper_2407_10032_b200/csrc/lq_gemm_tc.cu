@@ -546,8 +546,12 @@ bool make_map_2d(CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const
 
 // Number of CTA pairs that can be resident at once (0 when the pair form cannot be launched).
 int max_pairs(int sm_count) {
-    static int cached = -1;
-    if (cached >= 0) return cached;
+    static int cached_per_device[64];
+    static lq_once_per_device once;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+    int& cached = cached_per_device[dev];
+    if (!once.first()) return cached;
     cached = 0;
     if (cudaFuncSetAttribute(lq_tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::SMEM_BYTES) != cudaSuccess) {
         cudaGetLastError();
@@ -584,10 +588,9 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
         a.N > 0x7fffffffLL)
         return LQ_ERR_UNSUPPORTED;
 
-    static bool attr_set = false;
-    if (!attr_set) {
+    static lq_once_per_device attr_set;
+    if (attr_set.first()) {
         LQ_CUDA_TRY(cudaFuncSetAttribute(lq_tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<1>::SMEM_BYTES));
-        attr_set = true;
     }
     // The pair form pays off once there are at least a few 256-row tiles; below that one CTA per tile.
     const int pairs = (a.M > BM) ? max_pairs(h->sm_count) : 0;

@@ -558,12 +558,11 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
     double* scal = reinterpret_cast<double*>(wsp + L.scal);
     double* A = reinterpret_cast<double*>(wsp + L.a);
 
-    static bool attr_set = false;
-    if (!attr_set) {
+    static lq_once_per_device attr_set;
+    if (attr_set.first()) {
         LQ_CUDA_TRY(cudaFuncSetAttribute(diag_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DIAG_SMEM));
         LQ_CUDA_TRY(cudaFuncSetAttribute(panel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
         LQ_CUDA_TRY(cudaFuncSetAttribute(update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
-        attr_set = true;
     }
 
     diag_mean_kernel<<<1, 1024, 0, st>>>(H, c, ldh, static_cast<double>(damp_frac), scal);

@@ -339,10 +339,9 @@ template <int K, bool AFFINE>
 int launch_inblock(cudaStream_t st, int sm_count, float* Wc, int64_t ldc, int64_t r, int64_t c, int64_t i0, const float* U, int64_t ldu,
                    const float* grid, const float* scale, const int32_t* zero, int group, int n_groups, const QuantOut& out) {
     const int smem = (B * B + B) * sizeof(float);
-    static bool attr_set = false;
-    if (!attr_set) {
+    static lq_once_per_device attr_set;
+    if (attr_set.first()) {
         LQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel<K, AFFINE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        attr_set = true;
     }
     // One warp per row.  The kernel is bound by instruction issue, so what matters is the largest number of rows
     // on one SM: up to 32 rows per SM one CTA per SM takes an even share; beyond that, CTAs of 16 rows fill the SMs.
