@@ -546,3 +546,28 @@ def _columns_at_group_start(W, U, S, Z, grp, k):
         e = (Wc[:, j] - q) / U[j, j]
         Wc[:, j:] -= np.outer(e, U[j, j:])
     return Wc[:, k * grp:(k + 1) * grp]
+
+
+def test_p7b_candidates_with_one_grid_have_one_loss():
+    """Eq. 7 on a fine partition: S depends on t_min + t_max only and Z = -rint(lo / S) is an integer, so many
+    candidates give the same grid.  Their float64 losses agree to rounding noise, there are far fewer distinct
+    grids than candidates, and the search's answer is a member of the class with the least loss."""
+    g = rng(31)
+    w = g.standard_normal(64) * 0.05
+    s = np.exp(g.standard_normal(64))
+    K, T, t = 16, 512, 102
+    mn, mx = w.min(), w.max()
+    classes = {}
+    for t_min in range(t + 1):
+        for t_max in range(t + 1):
+            S, Z = O.affine_candidate(mn, mx, t_min, t_max, T, K)
+            loss = (s * (O.quant_aff(w, S, Z, K) - w) ** 2).sum()
+            classes.setdefault((t_min + t_max, Z), []).append(loss)
+    assert len(classes) < (t + 1) ** 2 / 10
+    for losses in classes.values():
+        assert max(losses) <= min(losses) * (1 + 1e-10)
+    So, Zo = O.affine_search_group(w[None, :], s, K, T, t)
+    best_class = min(classes, key=lambda k: min(classes[k]))
+    assert Zo[0] == best_class[1]
+    R = mx - mn
+    assert abs(So[0] / (R * (T - best_class[0]) / (T * (K - 1))) - 1) < 1e-12
