@@ -196,10 +196,11 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
     const int n_owner = (bw + 3) / 4;
 #pragma unroll 1
     for (int jj = 0; jj < n_owner; ++jj) {
-        float S = 1.0f, Zf = 0.0f;
+        float S = 1.0f, Zf = 0.0f, rS = 1.0f;
         if (AFFINE) {
             S = __shfl_sync(0xffffffffu, S_mine, jj);
             Zf = __shfl_sync(0xffffffffu, Z_mine, jj);
+            rS = __fdiv_rn(1.0f, S);               // one division per four columns; w / S below is w * (1 / S)
         }
         const bool mine = lane == jj;
 #pragma unroll
@@ -209,7 +210,7 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
             int code;
             float q;
             if (AFFINE) {
-                float qi = rintf(__fdiv_rn(wj, S)) + Zf;
+                float qi = rintf(wj * rS) + Zf;
                 qi = fminf(fmaxf(qi, 0.0f), static_cast<float>(K - 1));
                 code = static_cast<int>(qi);
                 q = (qi - Zf) * S;
