@@ -188,11 +188,21 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
     __syncthreads();
     if (tid < B) invd[tid] = 1.0f / Us[tid * B + tid];
     __syncthreads();
+    // rows of the block scaled by the reciprocal of their diagonal entry: the column loop then feeds w - q straight
+    // into the other columns, and only the lane that owns a column turns it into E = (w - q) / U_jj afterwards
+    for (int idx = tid; idx < B * B / 4; idx += nthr) {
+        const int jj = idx / (B / 4);
+        float4* p4 = reinterpret_cast<float4*>(Us) + idx;
+        float4 v = *p4;
+        const float sc = invd[jj];
+        v.x *= sc; v.y *= sc; v.z *= sc; v.w *= sc;
+        *p4 = v;
+    }
+    __syncthreads();
     if (!valid) return;
 
-    float qkeep[4] = {0.0f, 0.0f, 0.0f, 0.0f}, ekeep[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    float dkeep[4] = {0.0f, 0.0f, 0.0f, 0.0f};
     uint32_t cpack = 0;
-    float loss = 0.0f;
     const int n_owner = (bw + 3) / 4;
 #pragma unroll 1
     for (int jj = 0; jj < n_owner; ++jj) {
@@ -218,21 +228,32 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
                 code = __popc(__ballot_sync(0xffffffffu, wj > ml));
                 q = __shfl_sync(0xffffffffu, gl, code);
             }
-            const float e = (j < bw) ? (wj - q) * invd[j] : 0.0f;
-            loss = fmaf(e, e, loss);
+            const float d = wj - q;
             if (mine) {
-                qkeep[u] = q;
-                ekeep[u] = e;
+                dkeep[u] = d;
                 cpack |= static_cast<uint32_t>(code) << (8 * u);
             }
             const float4 uv = *reinterpret_cast<const float4*>(Us + j * B + col0);
-            w[0] = fmaf(-e, uv.x, w[0]);
-            w[1] = fmaf(-e, uv.y, w[1]);
-            w[2] = fmaf(-e, uv.z, w[2]);
-            w[3] = fmaf(-e, uv.w, w[3]);
+            w[0] = fmaf(-d, uv.x, w[0]);
+            w[1] = fmaf(-d, uv.y, w[1]);
+            w[2] = fmaf(-d, uv.z, w[2]);
+            w[3] = fmaf(-d, uv.w, w[3]);
         }
     }
 
+    // this lane's four columns: grid values from the codes, E from w - q, and the row's share of the loss
+    float qkeep[4], ekeep[4];
+    float loss = 0.0f;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int code = static_cast<int>((cpack >> (8 * u)) & 0xffu);
+        if (AFFINE) qkeep[u] = (static_cast<float>(code) - Z_mine) * S_mine;
+        else qkeep[u] = __shfl_sync(0xffffffffu, gl, code);
+        ekeep[u] = (col0 + u < bw) ? dkeep[u] * invd[col0 + u] : 0.0f;
+        loss = fmaf(ekeep[u], ekeep[u], loss);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
     // outputs of this lane's four columns
     if (col0 < bw) {
         const int64_t gcol = i0 + col0;
