@@ -575,8 +575,8 @@ affine_search_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, int group,
 // ------------------------------------------------------- fp32 screening of candidates --
 // Both searches below score a candidate (S, Z) in fp32 first and evaluate in fp64 only those whose
 // score cannot be told from the best one.  With x = w - min:  w / S + Z = x / S + c0,  c0 = min / S + Z,
-// and the error of a weight is d = q S - x - beta,  beta = min + Z S  (S as a two-float sum).
-struct AffScore { float rS, c0, Sh, Sl, beta; };
+// and the error of a weight is d = q S - x - beta,  beta = min + Z S.
+struct AffScore { float rS, c0, Sh, beta; };
 
 __device__ __forceinline__ AffScore aff_score_setup(double S, double Z, double dmn) {
     AffScore a;
@@ -584,7 +584,6 @@ __device__ __forceinline__ AffScore aff_score_setup(double S, double Z, double d
     a.rS = static_cast<float>(rS);
     a.c0 = static_cast<float>(dmn * rS + Z);
     a.Sh = static_cast<float>(S);
-    a.Sl = static_cast<float>(S - static_cast<double>(a.Sh));
     a.beta = static_cast<float>(dmn + Z * S);
     return a;
 }
@@ -596,8 +595,8 @@ __device__ __forceinline__ float aff_score32(const float2* __restrict__ ws, int 
         const float4 p2 = *reinterpret_cast<const float4*>(ws + j);          // two (x, s) pairs
         const float q0 = fminf(fmaxf(rintf(fmaf(p2.x, a.rS, a.c0)), 0.0f), Km1f);
         const float q1 = fminf(fmaxf(rintf(fmaf(p2.z, a.rS, a.c0)), 0.0f), Km1f);
-        const float d0 = fmaf(q0, a.Sl, fmaf(q0, a.Sh, -p2.x)) - a.beta;
-        const float d1 = fmaf(q1, a.Sl, fmaf(q1, a.Sh, -p2.z)) - a.beta;
+        const float d0 = fmaf(q0, a.Sh, -p2.x) - a.beta;
+        const float d1 = fmaf(q1, a.Sh, -p2.z) - a.beta;
         a0 = fmaf(p2.y * d0, d0, a0);
         a1 = fmaf(p2.w * d1, d1, a1);
     }
@@ -605,12 +604,13 @@ __device__ __forceinline__ float aff_score32(const float2* __restrict__ ws, int 
 }
 
 // Scores up to this bar are re-examined in fp64.  The fp32 value of d carries an absolute error of at most
-// delta = 1.5e-7 R (roundings of x, of beta and of the intermediate q S - x, each below 2^-25 of a quantity
-// bounded by R or 1.5 R), hence |score - loss| <= 2 delta sqrt(sum_s loss) + delta^2 sum_s (Cauchy-Schwarz);
-// the 0.1 % on top covers the rounding of the sum itself.  When the loss is far above delta^2 sum_s, as it
-// is unless a few heavy weights are met almost exactly, the bar is 0.1 % above the best score.
+// delta = 2.2e-7 R: roundings of x, of beta and of the intermediate q S - x, each below 2^-25 of a quantity
+// bounded by R or 1.5 R, plus q times the rounding of S to fp32 (q <= K - 1, S <= R / (K - 1): below 2^-24 R).
+// Hence |score - loss| <= 2 delta sqrt(sum_s loss) + delta^2 sum_s (Cauchy-Schwarz); the 0.1 % on top covers the
+// rounding of the sum itself.  When the loss is far above delta^2 sum_s, as it is unless a few heavy weights are
+// met almost exactly, the bar is 0.1 % above the best score.
 __device__ __forceinline__ float aff_bar32(float best, float R, float sum_s) {
-    const float delta = 1.5e-7f * R;
+    const float delta = 2.2e-7f * R;
     const float A = delta * delta * sum_s;
     const float E = 2.0f * sqrtf(A * best) + A;
     return best * 1.001f + 2.5f * E;
