@@ -369,9 +369,9 @@ def run_ours(args):
         s3_exec = None
         if st["grid"] == "affine" and (st["t"] + 1) ** 2 >= 256 and st["T"] - 2 * st["t"] > 2 * (K - 1):
             # Fine partitions: the library scores one representative per class of candidates that give the same
-            # grid (same t_min + t_max, same Z), nine lane-operations per weight; about this many per group:
+            # grid (same t_min + t_max, same Z), eight lane-operations per weight; about this many per group:
             classes = sum((min(st["t"], u) - max(0, u - st["t"])) * (K - 1) / (st["T"] - u) + 1 for u in range(2 * st["t"] + 1))
-            s3_exec = float(r) * c * classes * 9 / (stage_ms[2] * 1e-3) / 1e12
+            s3_exec = float(r) * c * classes * 8 / (stage_ms[2] * 1e-3) / 1e12
         s3_gbs = float(r) * c * W.element_size() / (stage_ms[2] * 1e-3) / 1e9
         s4 = float(r) * c * c / (stage_ms[3] * 1e-3) / 1e12
         # Algorithm 2: r rows x c steps x a c x c downdate = r c^3 fp64 FMAs on the plain FP64 pipe (same peak as the

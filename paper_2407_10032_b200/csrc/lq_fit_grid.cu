@@ -574,15 +574,16 @@ affine_search_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, int group,
 
 // ------------------------------------------------------- fp32 screening of candidates --
 // Both searches below score a candidate (S, Z) in fp32 first and evaluate in fp64 only those whose
-// score cannot be told from the best one.  With x = w - min:  w / S + Z = x / S + c0,  c0 = min / S + Z,
+// score cannot be told from the best one.  With x = w - min:  w / S + Z = x / S + c0,  c0 = min / S + Z
+// (both divided by K - 1 in AffScore, so that the clamp to [0, K - 1] is a saturation),
 // and the error of a weight is d = q S - x - beta,  beta = min + Z S.
 struct AffScore { float rS, c0, Sh, beta; };
 
-__device__ __forceinline__ AffScore aff_score_setup(double S, double Z, double dmn) {
+__device__ __forceinline__ AffScore aff_score_setup(double S, double Z, double dmn, double Km1) {
     AffScore a;
     const double rS = 1.0 / S;
-    a.rS = static_cast<float>(rS);
-    a.c0 = static_cast<float>(dmn * rS + Z);
+    a.rS = static_cast<float>(rS / Km1);                 // u / (K - 1) = x rS + c0, saturated to [0, 1] in aff_score32
+    a.c0 = static_cast<float>((dmn * rS + Z) / Km1);
     a.Sh = static_cast<float>(S);
     a.beta = static_cast<float>(dmn + Z * S);
     return a;
@@ -593,8 +594,10 @@ __device__ __forceinline__ float aff_score32(const float2* __restrict__ ws, int 
     float a0 = 0.0f, a1 = 0.0f;
     for (int j = 0; j < group; j += 2) {
         const float4 p2 = *reinterpret_cast<const float4*>(ws + j);          // two (x, s) pairs
-        const float q0 = fminf(fmaxf(rintf(fmaf(p2.x, a.rS, a.c0)), 0.0f), Km1f);
-        const float q1 = fminf(fmaxf(rintf(fmaf(p2.z, a.rS, a.c0)), 0.0f), Km1f);
+        // clamp to [0, K - 1] and round: the clamp rides on the multiply-add as a saturation of u / (K - 1) to [0, 1]
+        // (a weight within rounding of a tie may take the other neighbour, which leaves its error where it was)
+        const float q0 = rintf(__saturatef(fmaf(p2.x, a.rS, a.c0)) * Km1f);
+        const float q1 = rintf(__saturatef(fmaf(p2.z, a.rS, a.c0)) * Km1f);
         const float d0 = fmaf(q0, a.Sh, -p2.x) - a.beta;
         const float d1 = fmaf(q1, a.Sh, -p2.z) - a.beta;
         a0 = fmaf(p2.y * d0, d0, a0);
@@ -608,7 +611,8 @@ __device__ __forceinline__ float aff_score32(const float2* __restrict__ ws, int 
 // bounded by R or 1.5 R, plus q times the rounding of S to fp32 (q <= K - 1, S <= R / (K - 1): below 2^-24 R).
 // Hence |score - loss| <= 2 delta sqrt(sum_s loss) + delta^2 sum_s (Cauchy-Schwarz); the 0.1 % on top covers the
 // rounding of the sum itself.  When the loss is far above delta^2 sum_s, as it is unless a few heavy weights are
-// met almost exactly, the bar is 0.1 % above the best score.
+// met almost exactly, the bar is 0.1 % above the best score.  (A weight within the fp32 error of u of a rounding tie,
+// ~1e-5, may be given the other neighbour: its error is then S / 2 either way, up to that 1e-5 relative.)
 __device__ __forceinline__ float aff_bar32(float best, float R, float sum_s) {
     const float delta = 2.2e-7f * R;
     const float A = delta * delta * sum_s;
@@ -691,7 +695,7 @@ affine_search_warp_kernel(const T* __restrict__ W, int64_t ldw, int group, int n
         Z = -rint(lo / S);
         return true;
     };
-    auto score32 = [&](double S, double Z) { return aff_score32(ws, group, aff_score_setup(S, Z, dmn), Km1f); };
+    auto score32 = [&](double S, double Z) { return aff_score32(ws, group, aff_score_setup(S, Z, dmn, Km1), Km1f); };
     // fp64 loss of one candidate, computed by the whole warp (lane l takes weights l, l + 32, ...)
     auto loss64 = [&](double S, double Z) {
         double loss = 0.0;
@@ -922,7 +926,7 @@ affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_group
     for (int p = tid; p < P; p += nthr) {
         int u, Zi;
         class_of(p, u, Zi);
-        const AffScore as = aff_score_setup(c_s * static_cast<double>(Tparts - u), static_cast<double>(Zi), dmn);
+        const AffScore as = aff_score_setup(c_s * static_cast<double>(Tparts - u), static_cast<double>(Zi), dmn, Km1);
         float sc = aff_score32(ws, group, as, Km1f);
         if (sc != sc) sc = -INFINITY;                // a NaN score is always re-examined in fp64
         score[p] = sc;
