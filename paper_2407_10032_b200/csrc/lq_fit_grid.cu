@@ -192,16 +192,18 @@ __device__ __forceinline__ void bitonic_sort(KeyT* keys, int n, int tid) {
             const int nst = bhi - lo + 1;
             for (int vt = tid; vt < (n >> 4); vt += KS_THREADS) {
                 const int base = ((vt >> lo) << (lo + 4)) | (vt & ((1 << lo) - 1));
-                const bool up = ((base >> L) & 1) == 0;
+                // a descending block is sorted ascending on the complemented keys: one flip on the way in and one on
+                // the way out instead of a direction select in every compare-exchange
+                const KeyT flip = ((base >> L) & 1) == 0 ? static_cast<KeyT>(0) : ~static_cast<KeyT>(0);
                 KeyT e[16];
 #pragma unroll
-                for (int m = 0; m < 16; ++m) e[m] = keys[ks_slot(base | (m << lo))];
-                if (nst == 4) ce_stages<KeyT, 4>(e, up);
-                else if (nst == 3) ce_stages<KeyT, 3>(e, up);
-                else if (nst == 2) ce_stages<KeyT, 2>(e, up);
-                else ce_stages<KeyT, 1>(e, up);
+                for (int m = 0; m < 16; ++m) e[m] = keys[ks_slot(base | (m << lo))] ^ flip;
+                if (nst == 4) ce_stages<KeyT, 4>(e, true);
+                else if (nst == 3) ce_stages<KeyT, 3>(e, true);
+                else if (nst == 2) ce_stages<KeyT, 2>(e, true);
+                else ce_stages<KeyT, 1>(e, true);
 #pragma unroll
-                for (int m = 0; m < 16; ++m) keys[ks_slot(base | (m << lo))] = e[m];
+                for (int m = 0; m < 16; ++m) keys[ks_slot(base | (m << lo))] = e[m] ^ flip;
             }
             __syncthreads();
         }
