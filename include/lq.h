@@ -159,8 +159,10 @@ int lq_fit_grid(lq_handle* h, void* stream, const lq_config* cfg, const void* W,
  *   - c > LQ_FIT_GRID_NOALLOC_MAX_C (or any future setting whose scratch need exceeds the
  *     array) fails with LQ_ERR_STATIC_SCRATCH_TOO_SMALL before anything is launched.
  *   - The first call on each device looks up the array's device address (one-time set-up,
- *     guarded by a mutex) with that device current; make that first call before any stream
- *     capture begins.  Later calls only launch kernels.
+ *     guarded by a mutex) with that device current, and the first call of each configuration
+ *     (bit width, weight type, grid type and search path) on a device opts its kernel in to the
+ *     shared memory it needs; make the first call of each configuration you use before any
+ *     stream capture begins.  Later calls only launch kernels.
  *   - All calls on one device share the one array.  It keeps whatever the previous call left
  *     there; nothing has to be cleared because every word a call reads it has written first.
  *     Two calls whose kernels may overlap on the GPU (different streams, no ordering between
@@ -233,8 +235,19 @@ int lq_quantize_exact(lq_handle* h, void* stream, const lq_config* cfg, const vo
                       const float* scale, const int32_t* zero, uint8_t* codes, void* W_hat,
                       int32_t what_dtype, int64_t ldwh, double* loss, void* ws, size_t ws_bytes);
 
-/* Number of CUDA kernels this library has launched in this process so far (host counter,
- * not thread-safe; for benchmarks and tests that want to see that the kernels ran). */
+/* ---- measurement aid (no counterpart in the paper) ------------------------------------- */
+
+/* Launches one dependent-free arithmetic loop that fills the device (2048 threads per SM, eight
+ * independent chains per thread, `iters` iterations) and returns in *ops (host) the number of operations
+ * it executes: fp32 lane-operations (one FMA each) for LQ_PROBE_F32_FMA, flops for the two fp64 kinds.
+ * A benchmark times the launch with events on `stream`; ops / time is the rate of that pipe on this
+ * machine at its clocks, the denominator for the stages that are bound by it (grid fitting: fp32
+ * lanes; dampen / invert / factor and Algorithm 2: fp64). */
+typedef enum { LQ_PROBE_F32_FMA = 0, LQ_PROBE_F64_FMA = 1, LQ_PROBE_F64_MMA = 2 } lq_probe_kind;
+int lq_peak_probe(lq_handle* h, void* stream, int32_t kind, int64_t iters, double* ops);
+
+/* Number of CUDA kernels this library has launched in this process so far (an atomic host counter;
+ * for benchmarks and tests that want to see that the kernels ran). */
 uint64_t lq_launch_count(void);
 
 /* Library version string (static storage). */

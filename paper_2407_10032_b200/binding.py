@@ -69,6 +69,8 @@ def LQ():
             "lq_fit_grid": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, vp, vp, vp, vp, sz],
             "lq_fit_grid_noalloc": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, vp, vp, vp],
             "lq_pack_codes": [vp, vp, vp, i64, i64, i32, vp, i64],
+            "lq_peak_probe": [vp, vp, i32, i64, P(C.c_double)],
+            "lq_testing_set_wait_limit_ns": [vp, C.c_uint64],
             "lq_quantize_layer_lazy_workspace": [P(Config), i64, i64, P(sz)],
             "lq_quantize_layer_lazy": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, i64, vp, vp, vp, vp, vp, i32, i64,
                                        vp, vp, sz],
@@ -252,6 +254,19 @@ def lq_quantize_exact(h, cfg, W, U, codes, ws, grid=None, scale=None, zero=None,
                                   _rowmajor(U), _ptr(grid), _ptr(scale), _ptr(zero), _ptr(codes), _ptr(W_hat), whdt,
                                   ldwh, _ptr(loss_out), _ptr(ws), ws.numel() * ws.element_size()),
            "lq_quantize_exact")
+
+
+def lq_peak_probe(h, kind, iters, stream=None) -> float:
+    """Launches the dependent-free loop `kind` ("f32_fma", "f64_fma" or "f64_mma"); returns the operations it executes."""
+    ops = C.c_double(0.0)
+    k = {"f32_fma": 0, "f64_fma": 1, "f64_mma": 2}[kind]
+    _check(LQ().lq_peak_probe(h, _stream(stream), k, iters, C.byref(ops)), "lq_peak_probe")
+    return ops.value
+
+
+def lq_testing_set_wait_limit_ns(h, ns):
+    """Test hook (include/lq_testing.h): time limit of the bounded waits inside kernels; 0 restores the default."""
+    _check(LQ().lq_testing_set_wait_limit_ns(h, ns), "lq_testing_set_wait_limit_ns")
 
 
 def lq_pack_codes(h, codes, bits, packed=None, stream=None):

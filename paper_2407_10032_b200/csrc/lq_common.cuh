@@ -6,6 +6,8 @@
 #include <stdint.h>
 #include <stddef.h>
 
+#include <atomic>
+
 #include "lq.h"
 
 struct lq_dev_status {
@@ -23,7 +25,10 @@ struct lq_handle {
     // (everything then runs on the caller's stream).
     cudaStream_t aux;
     cudaEvent_t ev_fork, ev_next, ev_rest;
+    // Time limit of every bounded wait inside a kernel launched through this handle (nanoseconds).
+    unsigned long long wait_limit_ns;
 };
+constexpr unsigned long long LQ_DEFAULT_WAIT_LIMIT_NS = 5ull * 1000ull * 1000ull * 1000ull;
 
 // Record the first device-side failure; later ones are dropped.
 __device__ __forceinline__ void lq_report(lq_dev_status* st, int code, long long info) {
@@ -38,23 +43,23 @@ __device__ __forceinline__ void lq_report(lq_dev_status* st, int code, long long
 
 // Every kernel launch of the library goes through this: it counts the launch (see
 // lq_launch_count) and turns a launch failure into LQ_ERR_CUDA.
-extern unsigned long long lq_launches_total;
+extern std::atomic<unsigned long long> lq_launches_total;
 #define LQ_LAUNCH_CHECK()                                   \
     do {                                                    \
-        ++lq_launches_total;                                \
+        lq_launches_total.fetch_add(1, std::memory_order_relaxed); \
         if (cudaGetLastError() != cudaSuccess) return LQ_ERR_CUDA; \
     } while (0)
 
 // Kernel attributes (opt-in shared memory sizes) are per device: each set-up site keeps one of these and runs its
-// set-up once per device of the process.  Setting an attribute twice is harmless, so no lock is taken.
+// set-up once per device of the process.  The flags are atomic; two host threads that race on the first use of a
+// device may both run the set-up, which is harmless (setting an attribute twice gives the same state).
 struct lq_once_per_device {
-    bool done[64] = {};
+    std::atomic<bool> done[64];
+    lq_once_per_device() { for (auto& d : done) d.store(false, std::memory_order_relaxed); }
     bool first() {
         int dev = -1;
         if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return true;
-        if (done[dev]) return false;
-        done[dev] = true;
-        return true;
+        return !done[dev].exchange(true, std::memory_order_acq_rel);
     }
 };
 

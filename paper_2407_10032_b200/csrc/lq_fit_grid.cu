@@ -1127,6 +1127,12 @@ extern "C" int lq_fit_grid(lq_handle* h, void* stream, const lq_config* cfg, con
         if (r * (c / g) > 0x7fffffffLL) return LQ_ERR_UNSUPPORTED;
     }
 
+    if (cfg->grid_type == LQ_GRID_NONUNIFORM && c > KS_MAX_N) {
+        // rows too long for the sorted path: what the direct path cannot do is refused before anything is enqueued
+        if (cfg->init != LQ_INIT_UNIFORM) return LQ_ERR_UNSUPPORTED;
+        if (static_cast<size_t>(c) * (w_dtype == LQ_F32 ? 4 : 2) > 200 * 1024) return LQ_ERR_UNSUPPORTED;
+    }
+
     e = lq_sample_weights(h, st, dinv, c, static_cast<double>(cfg->p), scal, s64);
     if (e) return e;
 
@@ -1213,6 +1219,7 @@ extern "C" int lq_fit_grid_noalloc(lq_handle* h, void* stream, const lq_config* 
     local.dstatus = d.status;
     local.aux = nullptr;
     local.ev_fork = local.ev_next = local.ev_rest = nullptr;
+    local.wait_limit_ns = LQ_DEFAULT_WAIT_LIMIT_NS;
     return lq_fit_grid(h ? h : &local, stream, cfg, W, w_dtype, r, c, ldw, dinv, grid, scale, zero, d.scratch,
                        kNoAllocScratchBytes);
 }

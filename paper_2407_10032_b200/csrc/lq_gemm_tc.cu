@@ -107,7 +107,6 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t bar, uint32_t rank) 
     asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(bar), "r"(rank));
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(remote) : "memory");
 }
-template <bool CLUSTER>
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -118,14 +117,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // Bounded wait.  Returns false when the CTA is aborting (this wait or another one ran out).
-template <bool CLUSTER>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           const KParams& p, int where) {
-    if (mbar_try_wait<CLUSTER>(bar, parity)) return true;
+    if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = global_timer();
     uint32_t spins = 0;
     for (;;) {
-        if (mbar_try_wait<CLUSTER>(bar, parity)) return true;
+        if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 63u) == 0u) {
             if (*abort_flag) return false;
             if (global_timer() - t0 > p.timeout_ns) {
@@ -220,6 +218,16 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void group_bar_sync(uint32_t id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
+// Barrier over the 128 threads of an epilogue group that also tells every thread whether any of them passed `v`.
+__device__ __forceinline__ bool group_bar_or(uint32_t id, bool v) {
+    uint32_t out;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %2, 0;\n\t"
+        "bar.red.or.pred p, %1, 128, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(out) : "r"(id), "r"(static_cast<uint32_t>(v)) : "memory");
+    return out != 0;
+}
 
 // Shared-memory matrix descriptor for a K-major bf16 tile stored by TMA with the 128-byte
 // swizzle: rows of 128 bytes, groups of 8 rows 1024 bytes apart.
@@ -358,7 +366,7 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             const int n0 = tn * BN + static_cast<int>(rank) * C::B_ROWS;
             const int kit_end = min(k_iters, pc.s1 * p.seg_iters);
             for (int kit = pc.s0 * p.seg_iters; kit < kit_end; ++kit) {       // segments only matter to the consumers
-                if (!mbar_wait<PAIR>(bar_empty + 8 * stage, phase ^ 1u, abortp, p, 1)) { alive = false; break; }
+                if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abortp, p, 1)) { alive = false; break; }
                 if (lane == 0) {
                     const int pass = kit / k_blocks;
                     const int k0 = (kit - pass * k_blocks) * BK;
@@ -393,11 +401,11 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 const int k_hi = min(k_iters, k_lo + p.seg_iters);
                 const uint32_t acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
-                if (!mbar_wait<PAIR>(bar_tempty + 8 * acc, acc_phase ^ 1u, abortp, p, 2)) { alive = false; break; }
+                if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abortp, p, 2)) { alive = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + acc * BN;
                 for (int kit = k_lo; kit < k_hi; ++kit) {
-                    if (!mbar_wait<PAIR>(bar_full + 8 * stage, phase, abortp, p, 3)) { alive = false; break; }
+                    if (!mbar_wait(bar_full + 8 * stage, phase, abortp, p, 3)) { alive = false; break; }
                     tc_fence_after();
                     if (lane == 0) {
                         const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
@@ -445,7 +453,7 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             for (int k_lo = piece_lo; k_lo < piece_end; k_lo += p.seg_iters, ++it) {
                 const uint32_t acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
-                if (!mbar_wait<PAIR>(bar_tfull + 8 * acc, acc_phase, abortp, p, 4)) { alive = false; break; }
+                if (!mbar_wait(bar_tfull + 8 * acc, acc_phase, abortp, p, 4)) { alive = false; break; }
                 tc_fence_after();
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) {
@@ -467,7 +475,9 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     else mbar_arrive_remote(bar_tempty + 8 * acc, 0);
                 }
             }
-            if (!alive) break;
+            // A wait may have run out in some warps of the group and not in others: the group leaves together, or
+            // the warps that went on would wait at the slab barriers below for warps that never come.
+            if (group_bar_or(1 + hf, !alive)) { alive = false; break; }
 #pragma unroll
             for (int ch = 0; ch < 4; ++ch) {
                 const int col0 = n0 + hf * (BN / 2) + ch * EPI_COLS;
@@ -630,7 +640,7 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
         p.num_tiles = p.tiles_m * p.tiles_n;
     }
     p.status = h->dstatus;
-    p.timeout_ns = 5ull * 1000ull * 1000ull * 1000ull;
+    p.timeout_ns = h->wait_limit_ns;
     if (p.num_tiles == 0) return LQ_OK;
     {
         const int k_iters = static_cast<int>(lq_ceil_div(a.K, BK)) * a.n_pass;
@@ -665,7 +675,7 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
             cudaGetLastError();
             return LQ_ERR_CUDA;
         }
-        ++lq_launches_total;
+        lq_launches_total.fetch_add(1, std::memory_order_relaxed);
     } else {
         lq_tc_gemm_kernel<1><<<active, NUM_THREADS, Cfg<1>::SMEM_BYTES, stream>>>(map_a, map_b, map_d, p);
         LQ_LAUNCH_CHECK();

@@ -152,6 +152,7 @@ extern "C" int lq_hessian_accumulate(lq_handle* h, void* stream, const void* X, 
         g.a_rows = g.b_rows = c;
         g.n_pass = 1;
     } else {
+        if (c > 65535) return LQ_ERR_UNSUPPORTED;        // rows of the split / transpose launches ride on the second grid dimension
         if (!token_major) {
             dim3 grid(static_cast<unsigned>(lq_ceil_div(ld, 256) < 64 ? lq_ceil_div(ld, 256) : 64), static_cast<unsigned>(c));
             split3_kernel<<<grid, 256, 0, st>>>(static_cast<const float*>(X), ldx, c, n_chunk, staged, ld);

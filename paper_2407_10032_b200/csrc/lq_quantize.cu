@@ -443,12 +443,16 @@ int quantize_impl(lq_handle* h, void* stream, const lq_config* cfg, const void* 
     __nv_bfloat16* ES = reinterpret_cast<__nv_bfloat16*>(wsp + L.es);
     double* loss_rows = reinterpret_cast<double*>(wsp + L.loss);
 
-    {
-        dim3 g(static_cast<unsigned>(lq_ceil_div(L.ldc, 256) < 32 ? lq_ceil_div(L.ldc, 256) : 32), static_cast<unsigned>(r));
-        // 16-byte accesses when rows of W start on 16-byte boundaries (the working copy's always do)
-        const int vec = ((reinterpret_cast<uintptr_t>(W) & 15) == 0 && (ldw * (w_dtype == LQ_F32 ? 4 : 2)) % 16 == 0) ? 1 : 0;
-        if (w_dtype == LQ_F32) to_f32_kernel<float><<<g, 256, 0, st>>>(static_cast<const float*>(W), ldw, c, Wc, L.ldc, vec);
-        else to_f32_kernel<__nv_bfloat16><<<g, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(W), ldw, c, Wc, L.ldc, vec);
+    // 16-byte accesses when rows of W start on 16-byte boundaries (the working copy's always do)
+    const int vec = ((reinterpret_cast<uintptr_t>(W) & 15) == 0 && (ldw * (w_dtype == LQ_F32 ? 4 : 2)) % 16 == 0) ? 1 : 0;
+    for (int64_t r0 = 0; r0 < r; r0 += 65535) {          // rows in slabs: the second grid dimension holds 65535 at most
+        const int64_t rr = r - r0 < 65535 ? r - r0 : 65535;
+        dim3 g(static_cast<unsigned>(lq_ceil_div(L.ldc, 256) < 32 ? lq_ceil_div(L.ldc, 256) : 32), static_cast<unsigned>(rr));
+        if (w_dtype == LQ_F32)
+            to_f32_kernel<float><<<g, 256, 0, st>>>(static_cast<const float*>(W) + r0 * ldw, ldw, c, Wc + r0 * L.ldc, L.ldc, vec);
+        else
+            to_f32_kernel<__nv_bfloat16><<<g, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(W) + r0 * ldw, ldw, c, Wc + r0 * L.ldc,
+                                                           L.ldc, vec);
         LQ_LAUNCH_CHECK();
     }
     if (c > B) {

@@ -159,6 +159,9 @@ def run_and_check_layer(lq, h, W, X, kw, seed, n_rows=24, prefix=4096, chunk=Non
     codes = P.codes[rows_t][:, :m].cpu().numpy().astype(np.int64)
     n_diverged = tie_ok(codes, codes_o, Wpre, points)      # every divergence must start at a near-tie ...
     assert n_diverged <= max(1, len(rows) // 12), n_diverged   # ... and only a few of the sampled rows may diverge at all
+    frac = float((codes != codes_o).mean())                # ... and the sampled codes stay inside the 0.1 % budget
+    print(f"{r} x {c} {kw['grid']} {cfg.bits}-bit: {100 * frac:.4f} % of {codes.size} sampled codes differ ({n_diverged} rows)")
+    assert frac <= CODE_TOL, frac
 
     # whole layer: codes in range, W_hat is the grid value of its code, loss identity
     assert int(P.codes.max()) < K

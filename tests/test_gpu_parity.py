@@ -76,6 +76,12 @@ def codes_budget(codes, codes_o):
     return diff.any(axis=1).sum() <= max(2, 0.02 * codes.shape[0])
 
 
+def proxy_rows(W, What, H):
+    """Each row's share of the proxy loss tr((W - What) H (W - What)^T)."""
+    D = np.asarray(W, dtype=np.float64) - np.asarray(What, dtype=np.float64)
+    return np.einsum("ij,ij->i", D @ H, D)
+
+
 def nu_points(G):
     G = np.asarray(G, dtype=np.float64)
     return lambda i, j: 0.5 * (G[i, :-1] + G[i, 1:])
@@ -388,7 +394,9 @@ def run_stage4(lq, h, W, U32, cfg, grid=None, scale=None, zero=None, what_dtype=
 
 
 @pytest.mark.parametrize("recipe,r,c,bits", [("c1", 512, 512, 4), ("c2", 300, 1024, 4), ("c2", 128, 1024, 3),
-                                             ("c2", 100, 200, 2), ("c2", 64, 1160, 4), ("c2", 16, 64, 4)])
+                                             ("c2", 100, 200, 2), ("c2", 64, 1160, 4), ("c2", 16, 64, 4),
+                                             # just over 250000 codes: the 0.1 % budget itself applies, at every bit width
+                                             ("c2", 256, 1024, 3), ("c2", 256, 1024, 2)])
 def test_stage4_nonuniform_isolated(lq, h, recipe, r, c, bits):
     L = synth.make_layer(recipe, r, c, 2 * c, seed=bits * 7 + c)
     W = f64(L.W)
@@ -398,7 +406,8 @@ def test_stage4_nonuniform_isolated(lq, h, recipe, r, c, bits):
     codes_o, What_o, loss_o, Wpre = O.quantize_layer(W, f64(U32), grid=f64(G32), bits=bits, block=128, return_pre=True)
     cfg = lq.Config.make(grid="nonuniform", bits=bits)
     codes, What, loss = run_stage4(lq, h, L.W, U32, cfg, grid=G32)
-    codes_agree(codes, codes_o, Wpre, nu_points(G32))
+    frac, n_rows = codes_agree(codes, codes_o, Wpre, nu_points(G32))
+    print(f"stage 4 isolated {recipe} {r}x{c} {bits}-bit: {100 * frac:.4f} % of codes differ ({n_rows} rows), loss rel err {abs(loss / loss_o - 1):.1e}")
     assert abs(loss / loss_o - 1) <= LOSS_TOL
     assert np.array_equal(What, np.take_along_axis(f64(G32), codes, 1))     # W_hat is the grid value of the code
     assert codes.max() < (1 << bits)
@@ -444,7 +453,8 @@ def chained(lq, h, L, cfg_kw, what_dtype=None, weight_src="inv_diag"):
 
 
 @pytest.mark.parametrize("recipe,r,c,n,bits,p", [("c1", 512, 512, 8192, 4, 4.0), ("c2", 256, 1024, 16384, 4, 4.0),
-                                                 ("c2", 256, 1024, 16384, 3, 2.0), ("c2", 128, 520, 4096, 3, 1.0)])
+                                                 ("c2", 256, 1024, 16384, 3, 2.0), ("c2", 128, 520, 4096, 3, 1.0),
+                                                 ("c2", 256, 1024, 16384, 2, 4.0)])
 def test_chained_nonuniform(lq, h, recipe, r, c, n, bits, p):
     L = synth.make_layer(recipe, r, c, n, seed=11 + bits)
     W, X = f64(L.W), f64(L.X)
@@ -452,9 +462,11 @@ def test_chained_nonuniform(lq, h, recipe, r, c, n, bits, p):
     P = chained(lq, h, L, dict(grid="nonuniform", bits=bits, p=p, n_iter=20), what_dtype=torch.float32)
     codes = P.codes.cpu().numpy().astype(np.int64)
     assert centroid_ok(f64(P.grid), ref["grid"], W)
+    proxy = O.proxy_loss(W, f64(P.W_hat), ref["H"])
+    print(f"chained {recipe} {r}x{c} {bits}-bit: {100 * (codes != ref['codes']).mean():.4f} % of codes differ, "
+          f"loss rel err {abs(P.loss.item() / ref['loss'] - 1):.1e}, proxy rel err {abs(proxy / ref['proxy'] - 1):.1e}")
     assert codes_budget(codes, ref["codes"])
     assert abs(P.loss.item() / ref["loss"] - 1) <= LOSS_TOL
-    proxy = O.proxy_loss(W, f64(P.W_hat), ref["H"])
     assert abs(proxy / ref["proxy"] - 1) <= LOSS_TOL
 
 
@@ -468,9 +480,14 @@ def test_chained_tiny_and_ragged_shapes(lq, h, r, c, n, bits):
     P = chained(lq, h, L, dict(grid="nonuniform", bits=bits, p=2.0, n_iter=10), what_dtype=torch.float32)
     assert centroid_ok(f64(P.grid), ref["grid"], W)
     codes = P.codes.cpu().numpy().astype(np.int64)
-    assert (codes != ref["codes"]).any(axis=1).sum() <= max(1, r // 20)
-    if np.array_equal(codes, ref["codes"]):
+    same = ~(codes != ref["codes"]).any(axis=1)
+    assert (~same).sum() <= max(1, r // 20)
+    if same.all():
         assert abs(P.loss.item() / ref["loss"] - 1) <= LOSS_TOL
+    # the rows that agree carry the oracle's loss: their share of the proxy loss tr(D H D^T), row by row
+    if same.any():
+        mine, theirs = proxy_rows(W, f64(P.W_hat), ref["H"])[same], proxy_rows(W, ref["W_hat"], ref["H"])[same]
+        assert abs(mine.sum() / theirs.sum() - 1) <= LOSS_TOL
 
 
 def test_chained_weighted_by_factor_diagonal(lq, h):
@@ -481,7 +498,15 @@ def test_chained_weighted_by_factor_diagonal(lq, h):
     plain = O.run_pass(W, X, bits=4, p=4.0, block=128, n_iter=20)
     assert np.abs(ref["grid"] - plain["grid"]).max() > 1e-4 * np.abs(plain["grid"]).max()     # the variant is another grid
     P = chained(lq, h, L, dict(grid="nonuniform", bits=4, p=4.0, n_iter=20), what_dtype=torch.float32, weight_src="chol_diag")
-    np.testing.assert_allclose(f64(P.dinv), np.diag(ref["U"]), rtol=1e-3)    # the factor of an fp32 H of this condition number
+    # The library factors the fp32 Hessian it accumulated; the oracle the float64 one.  Rounding H to fp32 perturbs it by
+    # 2^-24 relative, which the inverse amplifies by up to cond(H_d): that, with a factor 4 for the square root of c
+    # roundings that meet in one entry, is the bound the diagonal of U is held to.
+    ev = np.linalg.eigvalsh(ref["H_d"])
+    cond = ev[-1] / ev[0]
+    bound = 4 * cond * 2.0 ** -24
+    err = np.abs(f64(P.dinv) / np.diag(ref["U"]) - 1).max()
+    print(f"diag(U): cond(H_d) = {cond:.2e}, bound {bound:.1e}, measured {err:.1e}")
+    assert err <= bound
     assert centroid_ok(f64(P.grid), ref["grid"], W)
     assert codes_budget(P.codes.cpu().numpy().astype(np.int64), ref["codes"])
     assert abs(P.loss.item() / ref["loss"] - 1) <= LOSS_TOL
@@ -495,10 +520,16 @@ def test_chained_affine(lq, h):
     codes = P.codes.cpu().numpy().astype(np.int64)
     same_grid = (P.zero.cpu().numpy() == ref["zero"]) & (np.abs(f64(P.scale) / ref["scale"] - 1) < 1e-5)
     assert same_grid.mean() >= 0.99
-    proxy = O.proxy_loss(W, f64(P.W_hat), ref["H"])
-    assert abs(proxy / ref["proxy"] - 1) <= 5 * LOSS_TOL
     rows_ok = same_grid.all(axis=1)
     assert codes_budget(codes[rows_ok], ref["codes"][rows_ok])
+    # Proxy loss at the stated 1e-3 on the rows whose every (S, Z) is the oracle's; a row in which one group took
+    # the other of two candidates that tie to rounding is quantised on another grid from there on, so the
+    # whole-layer figure (printed, held to 5e-3) also measures how many such rows there are.
+    mine, theirs = proxy_rows(W, f64(P.W_hat), ref["H"]), proxy_rows(W, ref["W_hat"], ref["H"])
+    print(f"chained affine: {rows_ok.mean():.3f} of rows with the oracle's grids; proxy rel err on them "
+          f"{abs(mine[rows_ok].sum() / theirs[rows_ok].sum() - 1):.1e}, whole layer {abs(mine.sum() / theirs.sum() - 1):.1e}")
+    assert abs(mine[rows_ok].sum() / theirs[rows_ok].sum() - 1) <= LOSS_TOL
+    assert abs(mine.sum() / theirs.sum() - 1) <= 5 * LOSS_TOL
 
 
 @pytest.mark.parametrize("r,c,group", [(96, 1024, 128), (64, 1536, 256), (32, 2048, 1024), (48, 640, 0)])
@@ -526,8 +557,11 @@ def test_chained_affine_lazy_refit(lq, h, r, c, group):
     rows_ok = same_grid.all(axis=1)
     assert rows_ok.mean() >= 0.9
     assert codes_budget(codes[rows_ok], ref["codes"][rows_ok])
-    proxy = O.proxy_loss(W, f64(P.W_hat), ref["H"])
-    assert abs(proxy / ref["proxy"] - 1) <= 5 * LOSS_TOL
+    mine, theirs = proxy_rows(W, f64(P.W_hat), ref["H"]), proxy_rows(W, ref["W_hat"], ref["H"])
+    print(f"lazy refit g={group}: {rows_ok.mean():.3f} of rows with the oracle's grids; proxy rel err on them "
+          f"{abs(mine[rows_ok].sum() / theirs[rows_ok].sum() - 1):.1e}, whole layer {abs(mine.sum() / theirs.sum() - 1):.1e}")
+    assert abs(mine[rows_ok].sum() / theirs[rows_ok].sum() - 1) <= LOSS_TOL
+    assert abs(mine.sum() / theirs.sum() - 1) <= 5 * LOSS_TOL
     if group:                       # the refit is not the up-front fit once errors have been fed back
         up = O.fit_grid_affine(W, ref["dinv"], 4, 4.0, group, 45, 9)
         assert not np.array_equal(up[1][:, 1:], ref["zero"][:, 1:]) or not np.allclose(up[0][:, 1:], ref["scale"][:, 1:])
@@ -546,6 +580,44 @@ def test_lazy_refit_rejects_groups_it_cannot_place(lq, h):
     with pytest.raises(lq.LQError) as e:
         lq.lq_quantize_layer_lazy(h, cfg, W, U, dinv, scale, zero, codes, ws)
     assert e.value.code == 2
+
+
+def test_bounded_wait_runs_out_and_the_handle_recovers(lq):
+    """The only failure path of the tensor-core contraction: a wait on an mbarrier that gives up.  With the limit
+    set to one nanosecond the waits of a healthy launch run out; the call must return, the status must say
+    LQ_ERR_TIMEOUT, and with the default limit back the same handle must accumulate the right Hessian."""
+    hh = lq.lq_create(0)
+    try:
+        g = torch.Generator().manual_seed(77)
+        X = torch.randn(512, 4096, generator=g).bfloat16().cuda()
+        H = torch.zeros(512, 512, device="cuda")
+        lq.lq_testing_set_wait_limit_ns(hh, 1)
+        lq.lq_hessian_accumulate(hh, X, H, 2.0, None)
+        st, info = lq.lq_sync_status(hh, raise_on_error=False)
+        assert st == 7, (st, info)
+        assert 1 <= info <= 4                           # which wait gave up first
+        lq.lq_testing_set_wait_limit_ns(hh, 0)
+        H.zero_()
+        lq.lq_hessian_accumulate(hh, X, H, 2.0, None)
+        lq.lq_hessian_finalize(hh, H)
+        assert lq.lq_sync_status(hh, raise_on_error=False)[0] == 0
+        Href = O.hessian(f64(X))
+        np.testing.assert_allclose(f64(H), Href, rtol=0, atol=5e-6 * np.abs(Href).max())
+    finally:
+        lq.lq_destroy(hh)
+
+
+def test_more_rows_than_one_grid_dimension_holds(lq, h):
+    """r > 65535: the launches that put rows on the second grid dimension go in slabs."""
+    r, c = 65600, 128
+    g = torch.Generator().manual_seed(5)
+    W = (torch.randn(r, c, generator=g) * 0.02).cuda()
+    U32 = torch.eye(c) * 0.5
+    G = torch.sort(torch.randn(1, 4, generator=g) * 0.03, dim=1).values.repeat(r, 1)
+    cfg = lq.Config.make(grid="nonuniform", bits=2)
+    codes, What, loss = run_stage4(lq, h, W.cpu(), U32, cfg, grid=G)
+    nearest = np.abs(f64(W)[:, :, None] - f64(G)[:, None, :]).argmin(-1)
+    assert np.array_equal(codes, nearest)
 
 
 def test_invalid_arguments(lq, h):

@@ -364,6 +364,41 @@ def test_dead_channel_convention():
     assert np.isfinite(U).all() and np.isfinite(dinv).all()
 
 
+def test_dead_channel_is_the_layer_without_it():
+    """What the convention (H_ii = 1, weight column zeroed) must achieve: a channel that never fires is decoupled from
+    the others, so the live columns are quantised exactly as in the layer with that channel deleted.  The two
+    layers' damping terms coincide when the live diagonal averages 1 (the dead entry counts as 1), which a rescaling
+    of X arranges; then the factor and the inverse diagonal restricted to the live channels must be those of the
+    smaller layer, the dead row and column of U must hold nothing but the diagonal entry 1 / sqrt(1 + damp), and the
+    column loop must give the same codes and values on the live columns.  A mistake in the convention (dead entry
+    left at 0, set to the mean, column not zeroed, coupling left in) fails one of these."""
+    g = rng(16)
+    c, dead, r = 40, 13, 6
+    X = g.standard_normal((c, 200)) * np.exp(g.standard_normal((c, 1)))
+    X[dead] = 0.0
+    live = np.delete(np.arange(c), dead)
+    X *= 1.0 / np.sqrt(np.mean(np.diag(O.hessian(X))[live]))           # mean of the live diagonal -> 1
+    W = g.standard_normal((r, c)) * 0.05
+    H = O.hessian(X)
+    U, dinv, H_d, Wf = O.prepare_hinv(H, 0.01, W)
+    Us, dinvs, H_ds, _ = O.prepare_hinv(H[np.ix_(live, live)], 0.01)
+    damp = H_d[0, 0] - H[0, 0]
+    np.testing.assert_allclose(damp, H_ds[0, 0] - H[live[0], live[0]], rtol=1e-12)
+    np.testing.assert_allclose(U[np.ix_(live, live)], Us, rtol=1e-9, atol=1e-12)
+    np.testing.assert_allclose(dinv[live], dinvs, rtol=1e-9)
+    np.testing.assert_allclose(U[dead, dead], 1.0 / np.sqrt(1.0 + damp), rtol=1e-12)
+    assert np.abs(np.delete(U[dead], dead)).max() < 1e-12 and np.abs(np.delete(U[:, dead], dead)).max() < 1e-12
+    grid = O.grid_init_uniform(W.min(1), W.max(1), 8)
+    codes, What, loss = O.quantize_layer(Wf, U, grid=grid, bits=3, block=16)
+    codes_s, What_s, loss_s = O.quantize_layer(W[:, live], Us, grid=grid, bits=3, block=16)
+    assert np.array_equal(codes[:, live], codes_s)
+    np.testing.assert_allclose(What[:, live], What_s, rtol=0, atol=1e-12)
+    # the dead column itself: the value 0 rounded to the grid, its loss error on top of the smaller layer's
+    q0 = np.take_along_axis(grid, O.assign_nu(np.zeros((r, 1)), grid), 1)[:, 0]
+    np.testing.assert_allclose(What[:, dead], q0)
+    np.testing.assert_allclose(loss, loss_s + 0.5 * np.sum(q0 ** 2) * (1.0 + damp), rtol=1e-9)
+
+
 def test_weighted_quantile_init_is_deterministic_and_sorted():
     g = rng(12)
     W = g.standard_normal((3, 64))

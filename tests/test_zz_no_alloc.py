@@ -12,6 +12,7 @@ import pytest
 import torch
 
 import synth
+from oracle import leanquant_oracle as O
 
 pytestmark = pytest.mark.gpu
 
@@ -76,6 +77,15 @@ def test_noalloc_matches_fit_grid_on_two_calls_in_a_row(lq):
                 G, Gw = got[0].double().cpu().numpy(), want[0].double().cpu().numpy()
                 span = (L.W.double().numpy().max(1) - L.W.double().numpy().min(1))[:, None] / G.shape[1]
                 assert np.all(np.abs(G - Gw) <= CENT_TOL * np.maximum(np.abs(Gw), span))
+                # and against the float64 oracle itself, at the same tolerance
+                Go = O.fit_grid_nonuniform(L.W.double().numpy(), dinv.double().cpu().numpy(), kw["bits"], kw["p"], kw["n_iter"])
+                assert np.all(np.abs(G - Go) <= CENT_TOL * np.maximum(np.abs(Go), span))
+            # what the entry point is for: a repeated call (every one-time set-up of this configuration is behind us)
+            # leaves the free device memory where it was
+            free0 = torch.cuda.mem_get_info()[0]
+            _without_allocation(lq, handle, cfg, W, dinv, affine, got)
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free0
     finally:
         lq.lq_destroy(h)
 
