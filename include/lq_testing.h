@@ -21,6 +21,19 @@ extern "C" {
  * whose wait ran out are unspecified. */
 int lq_testing_set_wait_limit_ns(lq_handle* h, uint64_t ns);
 
+/* Makes the failure those waits exist for, from the host: while `on` is nonzero, every load barrier of the
+ * tensor-core contractions launched through `h` expects 16 bytes more than its loads deliver, so it never
+ * completes -- a load that does not arrive.  Every wait in the kernel then runs into its limit (set a short one
+ * first), the kernel records LQ_ERR_TIMEOUT, waits for the copies it has in flight, frees its tensor memory and
+ * returns.  Nothing faults and nothing waits without limit. */
+int lq_testing_inject_stall(lq_handle* h, int32_t on);
+
+/* lq_prepare_hinv sends the updates of far tiles through the bf16 tensor cores (digit slices) only for matrices of
+ * at least 48 blocks of 128 columns; smaller ones stay on the FP64 MMA throughout, which is faster there.  This sets
+ * that threshold for `h` (0: always defer when there is more than one outer block of 1024 columns; negative: the
+ * default), so that tests can run the deferred path on matrices small enough for a float64 check in full. */
+int lq_testing_set_prepare_defer_min_blocks(lq_handle* h, int32_t n_blocks);
+
 #ifdef __cplusplus
 }
 #endif

@@ -71,6 +71,8 @@ def LQ():
             "lq_pack_codes": [vp, vp, vp, i64, i64, i32, vp, i64],
             "lq_peak_probe": [vp, vp, i32, i64, P(C.c_double)],
             "lq_testing_set_wait_limit_ns": [vp, C.c_uint64],
+            "lq_testing_inject_stall": [vp, i32],
+            "lq_testing_set_prepare_defer_min_blocks": [vp, i32],
             "lq_quantize_layer_lazy_workspace": [P(Config), i64, i64, P(sz)],
             "lq_quantize_layer_lazy": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, i64, vp, vp, vp, vp, vp, i32, i64,
                                        vp, vp, sz],
@@ -267,6 +269,16 @@ def lq_peak_probe(h, kind, iters, stream=None) -> float:
 def lq_testing_set_wait_limit_ns(h, ns):
     """Test hook (include/lq_testing.h): time limit of the bounded waits inside kernels; 0 restores the default."""
     _check(LQ().lq_testing_set_wait_limit_ns(h, ns), "lq_testing_set_wait_limit_ns")
+
+
+def lq_testing_inject_stall(h, on):
+    """Test hook (include/lq_testing.h): load barriers of the tensor-core contraction that never complete."""
+    _check(LQ().lq_testing_inject_stall(h, 1 if on else 0), "lq_testing_inject_stall")
+
+
+def lq_testing_set_prepare_defer_min_blocks(h, n_blocks):
+    """Test hook (include/lq_testing.h): matrix size from which stage 2 defers far updates to the bf16 tensor cores."""
+    _check(LQ().lq_testing_set_prepare_defer_min_blocks(h, n_blocks), "lq_testing_set_prepare_defer_min_blocks")
 
 
 def lq_pack_codes(h, codes, bits, packed=None, stream=None):

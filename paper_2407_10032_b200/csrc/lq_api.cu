@@ -13,6 +13,18 @@ extern "C" int lq_testing_set_wait_limit_ns(lq_handle* h, uint64_t ns) {
     return LQ_OK;
 }
 
+extern "C" int lq_testing_inject_stall(lq_handle* h, int32_t on) {
+    if (!h) return LQ_ERR_INVALID_ARG;
+    h->inject_stall = on ? 1 : 0;
+    return LQ_OK;
+}
+
+extern "C" int lq_testing_set_prepare_defer_min_blocks(lq_handle* h, int32_t n_blocks) {
+    if (!h) return LQ_ERR_INVALID_ARG;
+    h->prep_defer_min_blocks = n_blocks < 0 ? LQ_DEFAULT_PREP_DEFER_MIN_BLOCKS : n_blocks;
+    return LQ_OK;
+}
+
 extern "C" const char* lq_version(void) { return "lq 0.1 (sm_100a)"; }
 
 extern "C" int lq_create(lq_handle** out, int device) {
@@ -31,6 +43,8 @@ extern "C" int lq_create(lq_handle** out, int device) {
     h->aux = nullptr;
     h->ev_fork = h->ev_next = h->ev_rest = nullptr;
     h->wait_limit_ns = LQ_DEFAULT_WAIT_LIMIT_NS;
+    h->inject_stall = 0;
+    h->prep_defer_min_blocks = LQ_DEFAULT_PREP_DEFER_MIN_BLOCKS;
     if (cudaStreamCreateWithFlags(&h->aux, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_next, cudaEventDisableTiming) != cudaSuccess ||

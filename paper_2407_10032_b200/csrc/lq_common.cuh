@@ -27,7 +27,14 @@ struct lq_handle {
     cudaEvent_t ev_fork, ev_next, ev_rest;
     // Time limit of every bounded wait inside a kernel launched through this handle (nanoseconds).
     unsigned long long wait_limit_ns;
+    // Test hook: nonzero makes the load barriers of the tensor-core contraction expect bytes that never arrive, so that
+    // its bounded waits run out (see lq_testing.h).
+    int inject_stall;
+    // Stage 2 defers the updates of far tiles to the bf16 tensor cores when the matrix has at least this many
+    // 128-column blocks; below that the whole sweep stays on the FP64 MMA (a test hook can change the threshold).
+    int prep_defer_min_blocks;
 };
+constexpr int LQ_DEFAULT_PREP_DEFER_MIN_BLOCKS = 48;
 constexpr unsigned long long LQ_DEFAULT_WAIT_LIMIT_NS = 5ull * 1000ull * 1000ull * 1000ull;
 
 // Record the first device-side failure; later ones are dropped.
@@ -75,18 +82,29 @@ static inline int64_t lq_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b
 // 128 x 256 tiles that lie strictly below the diagonal (symmetric results).
 // The tensor core adds into its fp32 accumulator with truncation, so a long K is cut into
 // segments whose partial sums are added to D with round-to-nearest (seg_iters).
+constexpr int LQ_TC_MAX_PASS = 16;
+constexpr int LQ_TC_MAX_LVL = 5;
 struct lq_tc_gemm_args {
     const __nv_bfloat16* A_all; int64_t a_rows; int64_t lda;   // a_rows = total rows of A_all
     const __nv_bfloat16* B_all; int64_t b_rows; int64_t ldb;
     float* D; int64_t ldd;
     int64_t M, N, K;
     int n_pass;
-    int64_t a_row_off[6];
-    int64_t b_row_off[6];
+    int64_t a_row_off[LQ_TC_MAX_PASS];
+    int64_t b_row_off[LQ_TC_MAX_PASS];
     float alpha;
     int accumulate;
     int upper_only;
     int seg_iters;   // flush the TMEM partial sum into D every seg_iters 64-wide k-steps (0 = only at the end)
+    // Optional level-major order.  With n_lvl > 0 the passes are taken in n_lvl consecutive groups of lvl_npass[i]
+    // passes ("levels"), and the work of a tile is ordered level by level: for each level, for each chunk of
+    // chunk_kb k-steps of K, all passes of the level over that chunk form one segment (one TMEM partial sum, added to
+    // the running fp32 sum with round-to-nearest).  This is what a product of fixed-point digit slices needs: the
+    // digit products of one level are integers that a short segment sums exactly, and the levels -- least significant
+    // first -- are then combined with one rounding each.  seg_iters is ignored.
+    int n_lvl;
+    int lvl_npass[LQ_TC_MAX_LVL];
+    int chunk_kb;
 };
 int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a);
 

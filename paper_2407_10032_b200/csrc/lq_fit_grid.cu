@@ -1220,6 +1220,8 @@ extern "C" int lq_fit_grid_noalloc(lq_handle* h, void* stream, const lq_config* 
     local.aux = nullptr;
     local.ev_fork = local.ev_next = local.ev_rest = nullptr;
     local.wait_limit_ns = LQ_DEFAULT_WAIT_LIMIT_NS;
+    local.inject_stall = 0;
+    local.prep_defer_min_blocks = LQ_DEFAULT_PREP_DEFER_MIN_BLOCKS;
     return lq_fit_grid(h ? h : &local, stream, cfg, W, w_dtype, r, c, ldw, dinv, grid, scale, zero, d.scratch,
                        kNoAllocScratchBytes);
 }

@@ -57,8 +57,8 @@ template <int CTAS> struct Cfg {
 struct KParams {
     int M, N, K;
     int n_pass;
-    int a_off[6];
-    int b_off[6];
+    int a_off[LQ_TC_MAX_PASS];
+    int b_off[LQ_TC_MAX_PASS];
     float alpha;
     int accumulate;
     int upper_only;
@@ -67,11 +67,19 @@ struct KParams {
     int band;                 // tile rows per band of the schedule (see tile_coords)
     int num_tiles;
     int seg_iters;            // k-iterations accumulated in TMEM before the partial sum is flushed to D
-    int segs_per_tile;        // ceil(k_iters / seg_iters)
+    int segs_per_tile;        // ceil(k_iters / seg_iters), or n_lvl * n_chunks with levels
+    // Level-major order (n_lvl > 0): the passes form groups ("levels"); a segment is one level over one chunk of
+    // chunk_kb 64-wide k-blocks, and the segments run level by level.  See lq_tc_gemm_args::n_lvl.
+    int n_lvl;
+    int lvl_pass0[LQ_TC_MAX_LVL];
+    int lvl_npass[LQ_TC_MAX_LVL];
+    int chunk_kb;
+    int n_chunks;
     int k_parts;              // K is cut into this many parts (<= segs_per_tile)
     long long total_units;    // num_tiles * k_parts work units, dealt round-robin to the CTAs (or CTA pairs)
     lq_dev_status* status;
     unsigned long long timeout_ns;
+    int stall_bytes;          // test hook: bytes a load barrier expects on top of what its loads deliver (0 in normal use)
 };
 
 // ---------------------------------------------------------------- PTX wrappers ----
@@ -298,6 +306,31 @@ __device__ __forceinline__ bool next_piece(const KParams& p, long long& u, long 
     return true;
 }
 
+// Segment s of a tile: how many (pass, k-block) items it has and which they are.
+struct Seg { int len, kit0, pass0, kb0, kbn; };
+__device__ __forceinline__ Seg seg_of(const KParams& p, int k_blocks, int k_iters, int s) {
+    Seg g;
+    if (p.n_lvl == 0) {
+        g.kit0 = s * p.seg_iters;
+        g.len = min(p.seg_iters, k_iters - g.kit0);
+        g.pass0 = 0; g.kb0 = 0; g.kbn = k_blocks;
+    } else {
+        const int lvl = s / p.n_chunks, ch = s - lvl * p.n_chunks;
+        g.kit0 = 0;
+        g.pass0 = p.lvl_pass0[lvl];
+        g.kb0 = ch * p.chunk_kb;
+        g.kbn = min(p.chunk_kb, k_blocks - g.kb0);
+        g.len = p.lvl_npass[lvl] * g.kbn;
+    }
+    return g;
+}
+__device__ __forceinline__ void seg_item(const Seg& g, int q, int& pass, int& kb) {
+    const int kit = g.kit0 + q;
+    const int ps = kit / g.kbn;
+    pass = g.pass0 + ps;
+    kb = g.kb0 + kit - ps * g.kbn;
+}
+
 template <int CTAS>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -364,21 +397,23 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             tile_coords(p, pc.tile, tm, tn);
             const int m0 = tm * C::TILE_M + static_cast<int>(rank) * BM;
             const int n0 = tn * BN + static_cast<int>(rank) * C::B_ROWS;
-            const int kit_end = min(k_iters, pc.s1 * p.seg_iters);
-            for (int kit = pc.s0 * p.seg_iters; kit < kit_end; ++kit) {       // segments only matter to the consumers
+            for (int sg = pc.s0; sg < pc.s1 && alive; ++sg) {
+              const Seg g = seg_of(p, k_blocks, k_iters, sg);
+              for (int q = 0; q < g.len; ++q) {
                 if (!mbar_wait(bar_empty + 8 * stage, phase ^ 1u, abortp, p, 1)) { alive = false; break; }
                 if (lane == 0) {
-                    const int pass = kit / k_blocks;
-                    const int k0 = (kit - pass * k_blocks) * BK;
+                    int pass, kb;
+                    seg_item(g, q, pass, kb);
+                    const int k0 = kb * BK;
                     const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
                     const uint32_t sb = sa + A_STAGE_BYTES;
                     if (!PAIR) {
-                        mbar_arrive_expect_tx(bar_full + 8 * stage, C::STAGE_BYTES);
+                        mbar_arrive_expect_tx(bar_full + 8 * stage, C::STAGE_BYTES + p.stall_bytes);
                         tma_load_2d(sa, &map_a, bar_full + 8 * stage, k0, p.a_off[pass] + m0);
                         tma_load_2d(sb, &map_b, bar_full + 8 * stage, k0, p.b_off[pass] + n0);
                     } else {
                         // both CTAs' loads of a stage complete on the even CTA's barrier, which expects the bytes of both
-                        if (mma_cta) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * C::STAGE_BYTES);
+                        if (mma_cta) mbar_arrive_expect_tx(bar_full + 8 * stage, 2 * C::STAGE_BYTES + p.stall_bytes);
                         const uint32_t full0 = cluster_addr(bar_full + 8 * stage, 0);
                         tma_load_2d_pair(sa, &map_a, full0, k0, p.a_off[pass] + m0);
                         tma_load_2d_pair(sb, &map_b, full0, k0, p.b_off[pass] + n0);
@@ -386,6 +421,7 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 }
                 __syncwarp();
                 if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+              }
             }
         }
     } else if (warp_idx == 1 && mma_cta) {
@@ -396,15 +432,14 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         long long u = u_begin;
         Piece pc;
         while (alive && next_piece(p, u, u_stride, pc)) {
-            const int piece_end = min(k_iters, pc.s1 * p.seg_iters);
-            for (int k_lo = pc.s0 * p.seg_iters; k_lo < piece_end && alive; k_lo += p.seg_iters, ++it) {
-                const int k_hi = min(k_iters, k_lo + p.seg_iters);
+            for (int sg = pc.s0; sg < pc.s1 && alive; ++sg, ++it) {
+                const int seg_len = seg_of(p, k_blocks, k_iters, sg).len;
                 const uint32_t acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abortp, p, 2)) { alive = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + acc * BN;
-                for (int kit = k_lo; kit < k_hi; ++kit) {
+                for (int q = 0; q < seg_len; ++q) {
                     if (!mbar_wait(bar_full + 8 * stage, phase, abortp, p, 3)) { alive = false; break; }
                     tc_fence_after();
                     if (lane == 0) {
@@ -414,7 +449,7 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 #pragma unroll
                         for (int kk = 0; kk < BK / UMMA_K; ++kk) {
                             // advancing 16 bf16 = 32 bytes inside the swizzle row: +2 in the address field
-                            umma_bf16<CTAS>(tmem_d, da + 2 * kk, db + 2 * kk, C::IDESC, (kit > k_lo || kk > 0) ? 1u : 0u);
+                            umma_bf16<CTAS>(tmem_d, da + 2 * kk, db + 2 * kk, C::IDESC, (q > 0 || kk > 0) ? 1u : 0u);
                         }
                         umma_commit<CTAS>(bar_empty + 8 * stage);
                     }
@@ -449,8 +484,7 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             int tm, tn;
             tile_coords(p, pc.tile, tm, tn);
             const int m0 = tm * C::TILE_M + static_cast<int>(rank) * BM, n0 = tn * BN;
-            const int piece_lo = pc.s0 * p.seg_iters, piece_end = min(k_iters, pc.s1 * p.seg_iters);
-            for (int k_lo = piece_lo; k_lo < piece_end; k_lo += p.seg_iters, ++it) {
+            for (int sg = pc.s0; sg < pc.s1; ++sg, ++it) {
                 const uint32_t acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
                 if (!mbar_wait(bar_tfull + 8 * acc, acc_phase, abortp, p, 4)) { alive = false; break; }
@@ -460,7 +494,7 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     uint32_t v[32];
                     tmem_ld32(tmem_base + ((q * 32u) << 16) + acc * BN + hf * (BN / 2) + ch * EPI_COLS, v);
                     tmem_wait_ld();
-                    if (k_lo == piece_lo) {
+                    if (sg == pc.s0) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) accr[ch * 32 + i] = __uint_as_float(v[i]);
                     } else {
@@ -590,7 +624,8 @@ int max_pairs(int sm_count) {
 int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
     if (a.M <= 0 || a.N <= 0) return LQ_OK;
     if (a.K <= 0) return LQ_OK;
-    if (a.n_pass < 1 || a.n_pass > 6) return LQ_ERR_INVALID_ARG;
+    if (a.n_pass < 1 || a.n_pass > LQ_TC_MAX_PASS) return LQ_ERR_INVALID_ARG;
+    if (a.n_lvl < 0 || a.n_lvl > LQ_TC_MAX_LVL || (a.n_lvl > 0 && a.chunk_kb < 1)) return LQ_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(a.A_all) & 15) || (reinterpret_cast<uintptr_t>(a.B_all) & 15) ||
         (reinterpret_cast<uintptr_t>(a.D) & 15) || (a.lda % 8) || (a.ldb % 8) || (a.ldd % 4))
         return LQ_ERR_INVALID_ARG;
@@ -618,7 +653,7 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
     p.N = static_cast<int>(a.N);
     p.K = static_cast<int>(a.K);
     p.n_pass = a.n_pass;
-    for (int i = 0; i < 6; ++i) {
+    for (int i = 0; i < LQ_TC_MAX_PASS; ++i) {
         p.a_off[i] = static_cast<int>(a.a_row_off[i]);
         p.b_off[i] = static_cast<int>(a.b_row_off[i]);
     }
@@ -641,11 +676,28 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
     }
     p.status = h->dstatus;
     p.timeout_ns = h->wait_limit_ns;
+    p.stall_bytes = h->inject_stall ? 16 : 0;
     if (p.num_tiles == 0) return LQ_OK;
     {
-        const int k_iters = static_cast<int>(lq_ceil_div(a.K, BK)) * a.n_pass;
+        const int k_blocks = static_cast<int>(lq_ceil_div(a.K, BK));
+        const int k_iters = k_blocks * a.n_pass;
         p.seg_iters = (a.seg_iters > 0 && a.seg_iters < k_iters) ? a.seg_iters : k_iters;
         p.segs_per_tile = static_cast<int>(lq_ceil_div(k_iters, p.seg_iters));
+        p.n_lvl = a.n_lvl;
+        p.chunk_kb = a.chunk_kb > 0 ? a.chunk_kb : k_blocks;
+        p.n_chunks = static_cast<int>(lq_ceil_div(k_blocks, p.chunk_kb));
+        for (int i = 0; i < LQ_TC_MAX_LVL; ++i) { p.lvl_pass0[i] = 0; p.lvl_npass[i] = 0; }
+        if (a.n_lvl > 0) {
+            int next = 0;
+            for (int i = 0; i < a.n_lvl; ++i) {
+                if (a.lvl_npass[i] < 1) return LQ_ERR_INVALID_ARG;
+                p.lvl_pass0[i] = next;
+                p.lvl_npass[i] = a.lvl_npass[i];
+                next += a.lvl_npass[i];
+            }
+            if (next != a.n_pass) return LQ_ERR_INVALID_ARG;
+            p.segs_per_tile = a.n_lvl * p.n_chunks;
+        }
     }
     // number of K parts: the one that leaves the shortest schedule, ceil(tiles * q / workers) / q
     const int workers = ctas_per_tile == 2 ? pairs : h->sm_count;

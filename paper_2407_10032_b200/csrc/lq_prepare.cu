@@ -19,9 +19,24 @@
 // Every product has inner dimension 128 and all of a step's updates form one launch over the
 // whole width, so the grid stays large from the first step to the last.
 //
-// Everything is fp64 (fp32 factors of an ill-conditioned H move too many quantisation
-// decisions); all products run on the FP64 tensor-core MMA (mma.sync m8n8k4 f64) fed by a
-// cp.async ring.
+// The matrix, the diagonal blocks and the panels are fp64 (fp32 factors of an ill-conditioned H move
+// too many quantisation decisions).  The updates are done in two levels over outer blocks of
+// OBB = 8 block columns (1024 columns):
+//   eager    : the rows and the columns of the current outer block get every step's update at once, on the
+//              FP64 tensor-core MMA (mma.sync m8n8k4 f64) fed by a cp.async ring -- these are the tiles the
+//              outer block's own diagonal and panel kernels read;
+//   deferred : all other tiles (rows above the outer block, columns outside it) get the updates of the outer
+//              block's steps in one product of inner dimension 1024 when the outer block is complete, on the
+//              bf16 tensor cores (tcgen05, lq_tc_gemm).  The fp64 operands are cut into S = 5 slices of 8-bit
+//              integer digits below a per-row power of two; a product of two slices is a sum of integers that
+//              the fp32 accumulator holds exactly, the leading slice pair (s = t = 1) is kept as a result of its
+//              own and the other pairs with s + t <= S + 1 are combined, least significant level first, in fp32;
+//              the two results are added in fp64 and scaled back (15 bf16 products in all).  Worth ~39 bits relative
+//              to the largest entry of a row; entries of one row of a panel differ by the ratio of the channel scales,
+//              several bits, which is why four slices are not enough (U then comes out 1e-7 to 5e-7 of its largest
+//              entry off, measured here and in the CPU emulation alike; five hold it to 1e-8).  An fp32 accumulation
+//              of split floating-point operands keeps ~20 bits whatever the number of terms and moves 0.1 - 0.2 % of
+//              the codes.
 #include "lq_common.cuh"
 
 namespace {
@@ -224,20 +239,20 @@ __device__ __forceinline__ void gemm_tile(const double* __restrict__ A, int64_t 
     }
 }
 
-// Step k, panel.  Blocks [0, 4k): 64 x 64 tiles of P_i = A[i][k] V_k^T (to Pbuf, and transposed
-// into Q's columns of block i).  Blocks [4k, 4(nblk-1)): 128 x 32 tiles of the row scaling
+// Step k, panel.  Blocks [0, 4k): 64 x 64 tiles of P_i = A[i][k] V_k^T (to Pbuf: this step's 128 columns of the
+// outer block's panel buffer, row stride ldp; and transposed into Q's columns of block i).  Blocks [4k, 4(nblk-1)): 128 x 32 tiles of the row scaling
 // A[k][j] <- V_k A[k][j] for j > k (in place: these are final entries of U) with a copy in Q's
 // columns of block j.  Q is 128 x cp: the right-hand operand of the step's update for every
 // block column.
 __global__ void __launch_bounds__(GEMM_THREADS, 2)
-panel_kernel(double* __restrict__ A, int64_t cp, int k, double* __restrict__ Pbuf, double* __restrict__ Q) {
+panel_kernel(double* __restrict__ A, int64_t cp, int k, double* __restrict__ Pbuf, int64_t ldp, double* __restrict__ Q) {
     extern __shared__ double smem[];
     const int t = blockIdx.x >> 2, q = blockIdx.x & 3;
     const double* Vk = A + (int64_t)k * NB * cp + (int64_t)k * NB;
     TileOut o = {};
     if (t < k) {
         const int i = t, mh = q >> 1, h = q & 1;
-        o.C = Pbuf + (int64_t)i * NB * NB + (int64_t)(mh * 64) * NB + h * 64; o.ldc = NB;
+        o.C = Pbuf + ((int64_t)i * NB + mh * 64) * ldp + h * 64; o.ldc = ldp;
         o.Ct = Q + (int64_t)(h * 64) * cp + (int64_t)i * NB + mh * 64; o.ldct = cp;
         gemm_tile<2, 4, true>(A + ((int64_t)i * NB + mh * 64) * cp + (int64_t)k * NB, cp, Vk + (int64_t)(h * 64) * cp, cp, 1.0,
                               0.0, o, smem);
@@ -250,15 +265,15 @@ panel_kernel(double* __restrict__ A, int64_t cp, int k, double* __restrict__ Pbu
     }
 }
 
-// Step k, update of block rows i < k over the whole width.  The tiles of block column k-1 and
-// of block row k-1 are all that step k-1's diagonal and panel kernels read, so they can be
+// Step k, eager update of tiles (i, j), i < k: A[i][j] -= P_i Q[:, j] (A[i][k] = -P_i V_k).  A launch covers the
+// block rows i_base + blockIdx.y and the block columns j_base + (blockIdx.x >> 1) (128 x 64 tiles).  The tiles of
+// block column k-1 and of block row k-1 are all that step k-1's diagonal and panel kernels read, so they can be
 // updated first ("next") and the remainder ("rest") left to run beside step k-1:
-//   part 0: everything, grid 2 nblk x k, 128 x 64 tiles;  part 2: the rest, same grid;
-//   part 1: next only, grid 4 nblk x 1, 64 x 64 tiles -- block tile t < k is (t, k-1),
-//           t >= k is (k-1, t).
+//   part 0: every tile of the launch;  part 2: all but block row and block column k-1;
+//   part 1: next only, grid 4 nblk x 1, 64 x 64 tiles -- block tile t < k is (t, k-1), t >= k is (k-1, t).
 __global__ void __launch_bounds__(GEMM_THREADS, 2)
-update_kernel(double* __restrict__ A, int64_t cp, int k, int part, const double* __restrict__ Pbuf,
-              const double* __restrict__ Q) {
+update_kernel(double* __restrict__ A, int64_t cp, int k, int part, int i_base, int j_base, const double* __restrict__ Pbuf,
+              int64_t ldp, const double* __restrict__ Q) {
     extern __shared__ double smem[];
     int i, j, r0, c0;
     if (part == 1) {
@@ -267,21 +282,134 @@ update_kernel(double* __restrict__ A, int64_t cp, int k, int part, const double*
         r0 = ((blockIdx.x >> 1) & 1) * 64;
         c0 = (blockIdx.x & 1) * 64;
     } else {
-        j = blockIdx.x >> 1;
-        i = blockIdx.y;
+        j = j_base + (blockIdx.x >> 1);
+        i = i_base + blockIdx.y;
         if (part == 2 && (j == k - 1 || i == k - 1)) return;
         r0 = 0;
         c0 = (blockIdx.x & 1) * 64;
     }
     if (j < i) return;                                  // strictly lower tiles of the symmetric part
-    const double* Pi = Pbuf + (int64_t)i * NB * NB + (int64_t)r0 * NB;
+    const double* Pi = Pbuf + ((int64_t)i * NB + r0) * ldp;
     TileOut o = {};
     o.C = A + ((int64_t)i * NB + r0) * cp + (int64_t)j * NB + c0; o.ldc = cp;
     // A[i][k] = -P_i V_k;  A[i][j] -= P_i Q[:, j] otherwise
     const double* Bsrc = (j == k) ? A + (int64_t)k * NB * cp + (int64_t)k * NB + c0 : Q + (int64_t)j * NB + c0;
     const double beta = (j == k) ? 0.0 : 1.0;
-    if (part == 1) gemm_tile<2, 4, false>(Pi, NB, Bsrc, cp, -1.0, beta, o, smem);
-    else gemm_tile<4, 4, false>(Pi, NB, Bsrc, cp, -1.0, beta, o, smem);
+    if (part == 1) gemm_tile<2, 4, false>(Pi, ldp, Bsrc, cp, -1.0, beta, o, smem);
+    else gemm_tile<4, 4, false>(Pi, ldp, Bsrc, cp, -1.0, beta, o, smem);
+}
+
+// ------------------------------------------------ deferred update: operands as digit slices ----
+// x = 2^e (d_1 2^-8 + d_2 2^-16 + ... + d_S 2^-8S) + remainder, with integer digits |d_s| <= 128 and e such that
+// |x| 2^-e <= 1/2 for every entry of the row: slice s holds d_s 2^-8s as bf16 (exact).
+constexpr int OBB = 8;                   // block columns per outer block
+constexpr int LDP = OBB * NB;            // row stride of the panel buffer and of the slices
+constexpr int NSL = 5;                   // slices
+constexpr int64_t BAND = 4096;           // rows of the deferred region handled per product
+
+__device__ __forceinline__ int exp_for(double mx) { return mx > 0.0 ? ilogb(mx) + 2 : 0; }
+
+__device__ __forceinline__ void digits_of(double x, int e, __nv_bfloat16 (&d)[NSL]) {
+    double rest = scalbn(x, 8 - e);                     // |rest| <= 128
+    double w = 0.00390625;                              // 2^-8
+#pragma unroll
+    for (int s = 0; s < NSL; ++s) {
+        const double q = rint(rest);
+        d[s] = __float2bfloat16_rn(static_cast<float>(q * w));     // an integer of at most 8 bits times a power of two
+        rest = (rest - q) * 256.0;
+        w *= 0.00390625;
+    }
+}
+
+// Rows [0, rows) of the panel buffer (K columns each): exponent and slices.  One CTA per row.
+__global__ void __launch_bounds__(256)
+slice_rows_kernel(const double* __restrict__ P, int64_t ldp, int K, int* __restrict__ ex, __nv_bfloat16* __restrict__ SL,
+                  int64_t slice_rows) {
+    __shared__ double red[8];
+    const int64_t row = blockIdx.x;
+    const double* p = P + row * ldp;
+    double v[4];
+    double mx = 0.0;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int kx = threadIdx.x + 256 * u;
+        v[u] = kx < K ? p[kx] : 0.0;
+        mx = fmax(mx, fabs(v[u]));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    mx = red[0];
+#pragma unroll
+    for (int w = 1; w < 8; ++w) mx = fmax(mx, red[w]);
+    const int e = isfinite(mx) ? exp_for(mx) : 0;
+    if (threadIdx.x == 0) ex[row] = e;
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+        const int kx = threadIdx.x + 256 * u;
+        if (kx >= K) continue;
+        __nv_bfloat16 d[NSL];
+        digits_of(isfinite(v[u]) ? v[u] : 0.0, e, d);
+#pragma unroll
+        for (int s = 0; s < NSL; ++s) SL[(s * slice_rows + row) * LDP + kx] = d[s];
+    }
+}
+
+// Exponents of the columns j >= col0 of the K rows of A that start at row0 (the final rows of U of an outer block).
+__global__ void __launch_bounds__(256)
+col_exp_kernel(const double* __restrict__ A, int64_t cp, int64_t row0, int K, int64_t col0, int* __restrict__ ex) {
+    const int64_t j = col0 + blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (j >= cp) return;
+    double mx = 0.0;
+    for (int kx = 0; kx < K; ++kx) mx = fmax(mx, fabs(A[(row0 + kx) * cp + j]));
+    ex[j] = isfinite(mx) ? exp_for(mx) : 0;
+}
+
+// Slices of those columns, transposed: SL[s][j][kx] = digit s of A[row0 + kx][j].  64 x 64 tiles through shared memory.
+__global__ void __launch_bounds__(256)
+slice_cols_kernel(const double* __restrict__ A, int64_t cp, int64_t row0, int K, int64_t col0, const int* __restrict__ ex,
+                  __nv_bfloat16* __restrict__ SL, int64_t slice_rows) {
+    __shared__ double tile[64][65];
+    const int64_t j0 = col0 + (int64_t)blockIdx.x * 64;
+    const int k0 = blockIdx.y * 64;
+    for (int idx = threadIdx.x; idx < 64 * 64; idx += 256) {
+        const int a = idx >> 6, b = idx & 63;            // row k0 + a, column j0 + b
+        const int64_t j = j0 + b;
+        tile[a][b] = (k0 + a < K && j < cp) ? A[(row0 + k0 + a) * cp + j] : 0.0;
+    }
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < 64 * 64; idx += 256) {
+        const int b = idx >> 6, a = idx & 63;            // output row j0 + b, position k0 + a
+        const int64_t j = j0 + b;
+        if (j >= cp || k0 + a >= K) continue;
+        const double x = tile[a][b];
+        __nv_bfloat16 d[NSL];
+        digits_of(isfinite(x) ? x : 0.0, ex[j], d);
+#pragma unroll
+        for (int s = 0; s < NSL; ++s) SL[(s * slice_rows + j) * LDP + k0 + a] = d[s];
+    }
+}
+
+// A[row0 + i][col0 + j] -= 2^(ex[row0 + i] + ex[col0 + j]) (Ta[i][col0 + j] + Tb[i][col0 + j]) over nrows x ncols entries;
+// with `upper`, only the 128 x 128 blocks on or above the diagonal.  Two columns per thread.
+__global__ void __launch_bounds__(256)
+apply_kernel(double* __restrict__ A, int64_t cp, const float* __restrict__ Ta, const float* __restrict__ Tb, int64_t ldt,
+             const int* __restrict__ ex, int64_t row0, int64_t nrows, int64_t col0, int64_t ncols, int upper) {
+    const int64_t i = blockIdx.y;
+    const int64_t row = row0 + i;
+    const int er = ex[row];
+    for (int64_t j2 = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; 2 * j2 < ncols; j2 += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t col = col0 + 2 * j2;
+        if (upper && col / NB < row / NB) continue;
+        const float2 a = *reinterpret_cast<const float2*>(Ta + i * ldt + col);
+        const float2 b = *reinterpret_cast<const float2*>(Tb + i * ldt + col);
+        double2* ap = reinterpret_cast<double2*>(A + row * cp + col);
+        double2 v = *ap;
+        v.x -= scalbn(static_cast<double>(a.x) + static_cast<double>(b.x), er + ex[col]);
+        v.y -= scalbn(static_cast<double>(a.y) + static_cast<double>(b.y), er + ex[col + 1]);
+        *ap = v;
+    }
 }
 
 // --------------------------------------------------------- diagonal block kernel ----
@@ -297,31 +425,55 @@ constexpr int PP = 36;           // pitch of the panel buffer
 constexpr int DIAG_THREADS = 256;
 constexpr int DIAG_SMEM = (NB * DP + (NB - SB) * PP + 2 * SB + SB) * 8;
 
+// 1 / sqrt(d) for a positive finite d: single-precision seed, two Newton steps in fp64 (full precision; shorter
+// dependency chain than the library routine, and this sits on the one serial chain of the whole stage).
+__device__ __forceinline__ double rsqrt_pos(double d) {
+    const float df = static_cast<float>(d);
+    if (!(df > 1e-30f) || !(df < 1e30f)) return rsqrt(d);         // outside the comfortable range of the seed
+    double r = static_cast<double>(rsqrtf(df));
+    const double hd = 0.5 * d;
+    double e = fma(-hd * r, r, 0.5);
+    r = fma(r, e, r);
+    e = fma(-hd * r, r, 0.5);
+    return fma(r, e, r);
+}
+
 // 32 x 32 sub-block at S (pitch DP): upper triangle in, V = R^-1 out (upper, zeros below).
+// One warp, lane i holds row i.  The pivots form a serial chain (pivot -> reciprocal square root -> column ->
+// next pivot); per pivot only the next pivot's column is updated on that chain (one shuffle and one multiply-add),
+// the other columns follow through shared memory beside the next reciprocal square root.
 __device__ __forceinline__ void warp_factor_invert(double* S, double* colbuf, double* rinvb, int lane,
                                                    long long col_global, long long c_real, lq_dev_status* st) {
     double a[SB];
 #pragma unroll
     for (int t = 0; t < SB; ++t) a[t] = (t >= lane) ? S[lane * DP + t] : 0.0;
-    // R R^T factorisation, last column first; lane i holds row i.
+    // R R^T factorisation, last column first.
+    double d = __shfl_sync(0xffffffffu, a[SB - 1], SB - 1);
 #pragma unroll
     for (int j = SB - 1; j >= 0; --j) {
-        double d = __shfl_sync(0xffffffffu, a[j], j);
         if (!(d > 0.0) || !isfinite(d)) {
             if (lane == 0 && col_global + j < c_real) lq_report(st, LQ_ERR_NOT_POSITIVE_DEFINITE, col_global + j);
             d = 1.0;
         }
-        const double rinv = rsqrt(d);
-        const double l = (lane < j) ? a[j] * rinv : ((lane == j) ? d * rinv : 0.0);   // R[i][j]; sqrt(d) on the diagonal
-        a[j] = l;
+        const double rinv = rsqrt_pos(d);
+        const double lu = (lane < j) ? a[j] * rinv : 0.0;                 // R[i][j] above the diagonal
+        a[j] = (lane == j) ? d * rinv : lu;                               // sqrt(d) on the diagonal
         if (lane == j) rinvb[j] = rinv;
         double* cb = colbuf + (j & 1) * SB;
-        cb[lane] = (lane < j) ? l : 0.0;
+        cb[lane] = lu;
+        double dn = 1.0;
+        if (j > 0) {
+            const double ln = __shfl_sync(0xffffffffu, lu, j - 1);        // R[j-1][j]
+            a[j - 1] = fma(-lu, ln, a[j - 1]);
+            dn = __shfl_sync(0xffffffffu, a[j - 1], j - 1);               // the next pivot
+        }
         __syncwarp();
 #pragma unroll
-        for (int t = 0; t < j; ++t) a[t] -= l * cb[t];            // meaningful for lane <= t
+        for (int t = 0; t < j - 1; ++t) a[t] = fma(-lu, cb[t], a[t]);     // meaningful for lane <= t
+        d = dn;
     }
-    // R to shared memory (rows), then V = R^-1 row by row: V[i][j] = (delta_ij - sum_{t<j} V[i][t] R[t][j]) / R[j][j]
+    // R to shared memory (rows), then V = R^-1 row by row: V[i][j] = (delta_ij - sum_{t<j} V[i][t] R[t][j]) / R[j][j];
+    // the newest term enters last, so that only it and the scaling sit between one entry and the next
 #pragma unroll
     for (int t = 0; t < SB; ++t) S[lane * DP + t] = (t >= lane) ? a[t] : 0.0;
     __syncwarp();
@@ -330,14 +482,15 @@ __device__ __forceinline__ void warp_factor_invert(double* S, double* colbuf, do
     for (int j = 0; j < SB; ++j) {
         double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
 #pragma unroll
-        for (int t = 0; t < j; ++t) {
+        for (int t = 0; t < j - 1; ++t) {
             const double rt = S[t * DP + j];
             if ((t & 3) == 0) s0 = fma(v[t], rt, s0);
             else if ((t & 3) == 1) s1 = fma(v[t], rt, s1);
             else if ((t & 3) == 2) s2 = fma(v[t], rt, s2);
             else s3 = fma(v[t], rt, s3);
         }
-        const double rhs = ((lane == j) ? 1.0 : 0.0) - ((s0 + s1) + (s2 + s3));
+        double rhs = ((lane == j) ? 1.0 : 0.0) - ((s0 + s1) + (s2 + s3));
+        if (j > 0) rhs = fma(-v[j - 1], S[(j - 1) * DP + j], rhs);
         v[j] = (lane <= j) ? rhs * rinvb[j] : 0.0;
     }
     __syncwarp();
@@ -517,21 +670,103 @@ __global__ void dinv_kernel(const double* __restrict__ part, int64_t c, int n_ch
 }
 
 struct PrepLayout {
-    int64_t nblk, cp;
-    size_t scal, a, pbuf, q, total, panel_bytes;
+    int64_t nblk, cp, band;
+    size_t scal, a, pbuf, q, ex, sl, ta, tb, total, panel_bytes;
 };
 PrepLayout prep_layout(int64_t c) {
     PrepLayout L;
     L.nblk = lq_ceil_div(c, NB);
     L.cp = L.nblk * NB;
+    L.band = L.cp < BAND ? L.cp : BAND;
     size_t off = 0;
     L.scal = off; off += 256;
     L.a = off;    off += lq_align_up(static_cast<size_t>(L.cp) * L.cp * sizeof(double), 256);
     L.panel_bytes = lq_align_up(static_cast<size_t>(L.cp) * NB * sizeof(double), 256);
-    L.pbuf = off; off += 2 * L.panel_bytes;            // P and Q are double-buffered: one step's
-    L.q = off;    off += 2 * L.panel_bytes;            // update may still read them while the next is written
+    L.pbuf = off; off += lq_align_up(static_cast<size_t>(L.cp) * LDP * sizeof(double), 256);   // the panels of one outer block
+    L.q = off;    off += 2 * L.panel_bytes;            // Q is double-buffered: one step's update may still read it while the next is written
+    L.ex = off;   off += lq_align_up(static_cast<size_t>(L.cp) * sizeof(int), 256);
+    L.sl = off;   off += lq_align_up(static_cast<size_t>(NSL) * L.cp * LDP * sizeof(__nv_bfloat16), 256);
+    L.ta = off;   off += lq_align_up(static_cast<size_t>(L.band) * L.cp * sizeof(float), 256);
+    L.tb = off;   off += lq_align_up(static_cast<size_t>(L.band) * L.cp * sizeof(float), 256);
     L.total = off;
     return L;
+}
+
+// The updates that the steps of outer block [o_lo, o_hi] owe to the tiles outside its rows and columns:
+//   A[i][j] -= sum_k P_i^(k) Q_j^(k)    for block rows i < o_lo and block columns j outside the outer block, j >= i,
+// with Q_j^(k) = P_j^(k)^T left of the outer block (the Cholesky part) and the final row k of U right of it (the
+// Gauss-Jordan part).  Both operands go through the digit slices; row bands of at most `band` rows at a time.
+int deferred_update(lq_handle* h, cudaStream_t st, double* A, int64_t cp, int64_t o_lo, int64_t o_hi, const double* Pob, int* ex,
+                    __nv_bfloat16* SL, float* Ta, float* Tb, int64_t band) {
+    const int K = static_cast<int>((o_hi - o_lo + 1) * NB);
+    const int64_t top = o_lo * NB;                     // rows [0, top) are updated
+    const int64_t right0 = (o_hi + 1) * NB;            // columns [right0, cp) on the right of the outer block
+    const int64_t n_right = cp - right0;
+    slice_rows_kernel<<<static_cast<unsigned>(top), 256, 0, st>>>(Pob, LDP, K, ex, SL, cp);
+    LQ_LAUNCH_CHECK();
+    if (n_right > 0) {
+        col_exp_kernel<<<static_cast<unsigned>(lq_ceil_div(n_right, 256)), 256, 0, st>>>(A, cp, top, K, right0, ex);
+        LQ_LAUNCH_CHECK();
+        dim3 g(static_cast<unsigned>(lq_ceil_div(n_right, 64)), static_cast<unsigned>(lq_ceil_div(K, 64)));
+        slice_cols_kernel<<<g, 256, 0, st>>>(A, cp, top, K, right0, ex, SL, cp);
+        LQ_LAUNCH_CHECK();
+    }
+    // passes: the leading pair alone (exact), then the pairs of levels s + t = NSL + 1 down to 3, least significant first
+    lq_tc_gemm_args lead = {};
+    lead.A_all = lead.B_all = SL;
+    lead.a_rows = lead.b_rows = static_cast<int64_t>(NSL) * cp;
+    lead.lda = lead.ldb = LDP;
+    lead.ldd = cp;
+    lead.K = K;
+    lead.alpha = 1.0f;
+    lead.n_pass = 1;
+    lead.seg_iters = 4;                                // 256 digit products per partial sum: far below 2^24
+    lq_tc_gemm_args tail = lead;
+    tail.seg_iters = 0;
+    tail.n_pass = 0;
+    tail.n_lvl = 0;
+    tail.chunk_kb = 2;                                 // 128 of the inner dimension per segment: at most 5 x 128 x 2^14 < 2^24 per sum
+    int pair_s[LQ_TC_MAX_PASS], pair_t[LQ_TC_MAX_PASS];
+    for (int lvl = NSL + 1; lvl >= 3; --lvl) {
+        int cnt = 0;
+        for (int sdig = 1; sdig <= NSL; ++sdig) {
+            const int tdig = lvl - sdig;
+            if (tdig < 1 || tdig > NSL) continue;
+            pair_s[tail.n_pass] = sdig - 1;
+            pair_t[tail.n_pass] = tdig - 1;
+            ++tail.n_pass;
+            ++cnt;
+        }
+        tail.lvl_npass[tail.n_lvl++] = cnt;
+    }
+    for (int64_t b0 = 0; b0 < top; b0 += band) {
+        const int64_t b1 = b0 + band < top ? b0 + band : top;
+        for (int side = 0; side < 2; ++side) {
+            // side 0: columns [b0, top) with the tiles below the diagonal left out; side 1: columns [right0, cp)
+            const int64_t col0 = side == 0 ? b0 : right0;
+            const int64_t ncols = side == 0 ? top - b0 : n_right;
+            if (ncols <= 0) continue;
+            for (int which = 0; which < 2; ++which) {
+                lq_tc_gemm_args g = which == 0 ? lead : tail;
+                g.D = (which == 0 ? Ta : Tb) + col0;
+                g.M = b1 - b0;
+                g.N = ncols;
+                g.upper_only = side == 0 ? 1 : 0;
+                for (int ps = 0; ps < g.n_pass; ++ps) {
+                    const int sd = which == 0 ? 0 : pair_s[ps], td = which == 0 ? 0 : pair_t[ps];
+                    g.a_row_off[ps] = sd * cp + b0;
+                    g.b_row_off[ps] = td * cp + col0;
+                }
+                int rc = lq_tc_gemm(h, st, g);
+                if (rc) return rc;
+            }
+            const unsigned gx = static_cast<unsigned>(lq_ceil_div(ncols / 2, 256) < 256 ? lq_ceil_div(ncols / 2, 256) : 256);
+            apply_kernel<<<dim3(gx, static_cast<unsigned>(b1 - b0)), 256, 0, st>>>(A, cp, Ta, Tb, cp, ex, b0, b1 - b0, col0, ncols,
+                                                                                 side == 0 ? 1 : 0);
+            LQ_LAUNCH_CHECK();
+        }
+    }
+    return LQ_OK;
 }
 
 }  // namespace
@@ -581,44 +816,88 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
         LQ_LAUNCH_CHECK();
     }
 
-    // The sweep.  With an auxiliary stream: step k's diagonal and panel kernels and the "next"
-    // part of its update stay on the caller's stream; the rest of the update goes to the
-    // auxiliary stream and overlaps step k-1's diagonal and panel kernels.
+    // The sweep, outer block by outer block (last first).  Inside an outer block every step updates the rows and the
+    // columns of the outer block at once (the "eager" tiles).  With an auxiliary stream, step k's diagonal and panel
+    // kernels and the "next" part of its update stay on the caller's stream; the rest of the eager update goes to
+    // the auxiliary stream and overlaps step k-1's diagonal and panel kernels.  When the outer block is complete,
+    // all other tiles get its steps' updates in one product on the bf16 tensor cores (deferred_update).
     cudaStream_t aux = h->aux;
     const bool fork = aux != nullptr && nblk > 2;
     if (fork) {
         LQ_CUDA_TRY(cudaEventRecord(h->ev_fork, st));
         LQ_CUDA_TRY(cudaStreamWaitEvent(aux, h->ev_fork, 0));
     }
+    double* Pob = reinterpret_cast<double*>(wsp + L.pbuf);
+    // Small matrices are bound by the serial chain of diagonal blocks, not by the updates: they stay on the FP64 MMA
+    // throughout (one outer block as wide as the matrix).
+    const bool defer = nblk > OBB && nblk >= h->prep_defer_min_blocks;
+    const int64_t obb = defer ? OBB : nblk;
+    if (defer) LQ_CUDA_TRY(cudaMemsetAsync(wsp + L.sl, 0, static_cast<size_t>(NSL) * cp * LDP * sizeof(__nv_bfloat16), st));
     bool rest_pending = false;
-    for (int64_t k = nblk - 1; k >= 0; --k) {
-        double* Pk = reinterpret_cast<double*>(wsp + L.pbuf + (k & 1) * L.panel_bytes);
-        double* Qk = reinterpret_cast<double*>(wsp + L.q + (k & 1) * L.panel_bytes);
-        diag_block_kernel<<<1, DIAG_THREADS, DIAG_SMEM, st>>>(A, cp, k, c, h->dstatus);
-        LQ_LAUNCH_CHECK();
-        if (nblk > 1) {
-            panel_kernel<<<static_cast<unsigned>(4 * (nblk - 1)), GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, static_cast<int>(k), Pk, Qk);
+    const int64_t n_ob = lq_ceil_div(nblk, obb);
+    for (int64_t m = n_ob - 1; m >= 0; --m) {
+        const int64_t o_lo = m * obb;
+        const int64_t o_hi = (o_lo + obb < nblk ? o_lo + obb : nblk) - 1;
+        const int obw = static_cast<int>(o_hi - o_lo + 1);
+        for (int64_t k = o_hi; k >= o_lo; --k) {
+            // this step's 128 columns of the panel buffer: its place in the outer block, or one of two alternating
+            // slots when nothing is deferred (the previous step's update may still be reading the other one)
+            double* Pk = Pob + (defer ? k - o_lo : (k & 1)) * NB;
+            double* Qk = reinterpret_cast<double*>(wsp + L.q + (k & 1) * L.panel_bytes);
+            const int ki = static_cast<int>(k);
+            diag_block_kernel<<<1, DIAG_THREADS, DIAG_SMEM, st>>>(A, cp, k, c, h->dstatus);
             LQ_LAUNCH_CHECK();
+            if (nblk > 1) {
+                panel_kernel<<<static_cast<unsigned>(4 * (nblk - 1)), GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, ki, Pk, LDP, Qk);
+                LQ_LAUNCH_CHECK();
+            }
+            if (k == 0) break;
+            // eager tiles of step k: block rows [o_lo, k) over the whole width, block rows [0, o_lo) over the
+            // outer block's columns
+            const int rows_in = static_cast<int>(k - o_lo);
+            if (!fork || k == o_lo) {
+                if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_rest, 0));
+                rest_pending = false;
+                if (rows_in > 0) {
+                    dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(rows_in));
+                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, ki, 0, static_cast<int>(o_lo), 0, Pk, LDP, Qk);
+                    LQ_LAUNCH_CHECK();
+                }
+                if (o_lo > 0) {
+                    dim3 g(static_cast<unsigned>(2 * obw), static_cast<unsigned>(o_lo));
+                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, ki, 0, 0, static_cast<int>(o_lo), Pk, LDP, Qk);
+                    LQ_LAUNCH_CHECK();
+                }
+                continue;
+            }
+            if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_rest, 0));     // step k+1's rest touched the same tiles
+            update_kernel<<<static_cast<unsigned>(4 * nblk), GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, ki, 1, 0, 0, Pk, LDP, Qk);
+            LQ_LAUNCH_CHECK();
+            rest_pending = false;
+            if (rows_in > 1 || o_lo > 0) {
+                LQ_CUDA_TRY(cudaEventRecord(h->ev_next, st));
+                LQ_CUDA_TRY(cudaStreamWaitEvent(aux, h->ev_next, 0));
+                if (rows_in > 1) {             // block row k-1 is part of "next"
+                    dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(rows_in - 1));
+                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, aux>>>(A, cp, ki, 2, static_cast<int>(o_lo), 0, Pk, LDP, Qk);
+                    LQ_LAUNCH_CHECK();
+                }
+                if (o_lo > 0) {
+                    dim3 g(static_cast<unsigned>(2 * obw), static_cast<unsigned>(o_lo));
+                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, aux>>>(A, cp, ki, 2, 0, static_cast<int>(o_lo), Pk, LDP, Qk);
+                    LQ_LAUNCH_CHECK();
+                }
+                LQ_CUDA_TRY(cudaEventRecord(h->ev_rest, aux));
+                rest_pending = true;
+            }
         }
-        if (k == 0) break;
-        if (!fork) {
-            dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(k));
-            update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, static_cast<int>(k), 0, Pk, Qk);
-            LQ_LAUNCH_CHECK();
-            continue;
-        }
-        if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_rest, 0));     // step k+1's rest touched the same tiles
-        update_kernel<<<static_cast<unsigned>(4 * nblk), GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, static_cast<int>(k), 1, Pk, Qk);
-        LQ_LAUNCH_CHECK();
-        rest_pending = false;
-        if (k > 1) {
-            LQ_CUDA_TRY(cudaEventRecord(h->ev_next, st));
-            LQ_CUDA_TRY(cudaStreamWaitEvent(aux, h->ev_next, 0));
-            dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(k - 1));
-            update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, aux>>>(A, cp, static_cast<int>(k), 2, Pk, Qk);
-            LQ_LAUNCH_CHECK();
-            LQ_CUDA_TRY(cudaEventRecord(h->ev_rest, aux));
-            rest_pending = true;
+        if (o_lo > 0) {
+            if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_rest, 0));
+            rest_pending = false;
+            int rc = deferred_update(h, st, A, cp, o_lo, o_hi, Pob, reinterpret_cast<int*>(wsp + L.ex),
+                                     reinterpret_cast<__nv_bfloat16*>(wsp + L.sl), reinterpret_cast<float*>(wsp + L.ta),
+                                     reinterpret_cast<float*>(wsp + L.tb), L.band);
+            if (rc) return rc;
         }
     }
     if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_rest, 0));

@@ -122,6 +122,7 @@ def run_and_check_layer(lq, h, W, X, kw, seed, n_rows=24, prefix=4096, chunk=Non
         check_hessian_tiles(X, P.H, rng)
     if full_stage2:
         Uo, dinvo, _, _ = O.prepare_hinv(f64(P.H), 0.01)
+        print(f"stage 2 c={c}: max |dU| / max |U| = {np.abs(f64(P.U) - Uo).max() / np.abs(Uo).max():.2e}")
         assert np.abs(f64(P.U) - Uo).max() <= 3e-7 * np.abs(Uo).max()
         np.testing.assert_allclose(f64(P.dinv), dinvo, rtol=3e-7)
         del Uo

@@ -186,23 +186,33 @@ def test_stage1_empty_chunk_and_alpha(lq, h):
 
 
 # ------------------------------------------------------------------ stage 2 -------- #
-@pytest.mark.parametrize("c", [96, 128, 200, 512, 1024])
-def test_stage2_prepare(lq, h, c):
+@pytest.mark.parametrize("c", [96, 128, 200, 512, 1024, 1100, 1536, 2200, 3000])      # beyond 1024 columns the deferred
+def test_stage2_prepare(lq, h, c):                                                       # tensor-core update takes part
     L = synth.make_layer("c2", 8, c, 4 * c, seed=c)
     H32 = torch.from_numpy(O.hessian(f64(L.X))).float()
     Uo, dinvo, H_d, _ = O.prepare_hinv(f64(H32), 0.01)
     U = torch.empty(c, c, device="cuda")
     dinv = torch.empty(c, device="cuda")
     ws = ws_for(lq, lq.lq_prepare_hinv_workspace(c))
-    lq.lq_prepare_hinv(h, H32.cuda(), U, dinv, ws, 0.01)
-    lq.lq_sync_status(h)
-    Ug, dg = f64(U), f64(dinv)
-    assert np.array_equal(Ug, np.triu(Ug)) and (np.diag(Ug) > 0).all()
-    assert np.abs(Ug - Uo).max() <= 2e-7 * np.abs(Uo).max() + 1e-7 * np.abs(Uo).max()
-    np.testing.assert_allclose(dg, dinvo, rtol=3e-7)
-    # the factor really inverts the damped Hessian
-    resid = Ug.T @ (Ug @ H_d) - np.eye(c)
-    assert np.abs(resid).max() < 1e-4
+    # both forms of the sweep: everything on the FP64 MMA (what matrices of this size get by default), and with the
+    # far tiles' updates deferred to the bf16 tensor cores (what wide layers get; forced here through the test hook)
+    for defer_from in ((-1, 0) if c > 1024 else (-1,)):
+        lq.lq_testing_set_prepare_defer_min_blocks(h, defer_from)
+        try:
+            U.fill_(float("nan"))
+            lq.lq_prepare_hinv(h, H32.cuda(), U, dinv, ws, 0.01)
+            lq.lq_sync_status(h)
+        finally:
+            lq.lq_testing_set_prepare_defer_min_blocks(h, -1)
+        Ug, dg = f64(U), f64(dinv)
+        assert np.array_equal(Ug, np.triu(Ug)) and (np.diag(Ug) > 0).all()
+        print(f"stage 2 c={c} ({'deferred' if defer_from == 0 else 'default'}): max |dU| / max |U| = "
+              f"{np.abs(Ug - Uo).max() / np.abs(Uo).max():.2e}, dinv rel err {np.abs(dg / dinvo - 1).max():.2e}")
+        assert np.abs(Ug - Uo).max() <= 2e-7 * np.abs(Uo).max() + 1e-7 * np.abs(Uo).max()
+        np.testing.assert_allclose(dg, dinvo, rtol=3e-7)
+        # the factor really inverts the damped Hessian
+        resid = Ug.T @ (Ug @ H_d) - np.eye(c)
+        assert np.abs(resid).max() < 1e-4
 
 
 def test_stage2_dead_channel_and_status(lq, h):
@@ -583,26 +593,30 @@ def test_lazy_refit_rejects_groups_it_cannot_place(lq, h):
 
 
 def test_bounded_wait_runs_out_and_the_handle_recovers(lq):
-    """The only failure path of the tensor-core contraction: a wait on an mbarrier that gives up.  With the limit
-    set to one nanosecond the waits of a healthy launch run out; the call must return, the status must say
-    LQ_ERR_TIMEOUT, and with the default limit back the same handle must accumulate the right Hessian."""
+    """The only failure path of the tensor-core contraction: a wait on an mbarrier that gives up.  The failure is made
+    on the host (load barriers that expect bytes which never arrive, the wait limit set to two milliseconds): every
+    wait in the kernel must run into its limit, the call must return, the status must say LQ_ERR_TIMEOUT, and with
+    the hook off and the default limit back the same handle must accumulate the right Hessian."""
     hh = lq.lq_create(0)
     try:
         g = torch.Generator().manual_seed(77)
-        X = torch.randn(512, 4096, generator=g).bfloat16().cuda()
-        H = torch.zeros(512, 512, device="cuda")
-        lq.lq_testing_set_wait_limit_ns(hh, 1)
-        lq.lq_hessian_accumulate(hh, X, H, 2.0, None)
-        st, info = lq.lq_sync_status(hh, raise_on_error=False)
-        assert st == 7, (st, info)
-        assert 1 <= info <= 4                           # which wait gave up first
-        lq.lq_testing_set_wait_limit_ns(hh, 0)
-        H.zero_()
-        lq.lq_hessian_accumulate(hh, X, H, 2.0, None)
-        lq.lq_hessian_finalize(hh, H)
-        assert lq.lq_sync_status(hh, raise_on_error=False)[0] == 0
-        Href = O.hessian(f64(X))
-        np.testing.assert_allclose(f64(H), Href, rtol=0, atol=5e-6 * np.abs(Href).max())
+        for c, n in ((128, 1024), (512, 4096)):          # one CTA per tile, and CTA pairs
+            X = torch.randn(c, n, generator=g).bfloat16().cuda()
+            H = torch.zeros(c, c, device="cuda")
+            lq.lq_testing_set_wait_limit_ns(hh, 2_000_000)
+            lq.lq_testing_inject_stall(hh, True)
+            lq.lq_hessian_accumulate(hh, X, H, 2.0, None)
+            st, info = lq.lq_sync_status(hh, raise_on_error=False)
+            assert st == 7, (st, info)
+            assert 1 <= info <= 4                       # which wait gave up first
+            lq.lq_testing_inject_stall(hh, False)
+            lq.lq_testing_set_wait_limit_ns(hh, 0)
+            H.zero_()
+            lq.lq_hessian_accumulate(hh, X, H, 2.0, None)
+            lq.lq_hessian_finalize(hh, H)
+            assert lq.lq_sync_status(hh, raise_on_error=False)[0] == 0
+            Href = O.hessian(f64(X))
+            np.testing.assert_allclose(f64(H), Href, rtol=0, atol=5e-6 * np.abs(Href).max())
     finally:
         lq.lq_destroy(hh)
 
