@@ -425,29 +425,15 @@ constexpr int PP = 36;           // pitch of the panel buffer
 constexpr int DIAG_THREADS = 256;
 constexpr int DIAG_SMEM = (NB * DP + (NB - SB) * PP + 2 * SB + SB) * 8;
 
-// 1 / sqrt(d) for a positive finite d: single-precision seed, two Newton steps in fp64 (full precision; shorter
-// dependency chain than the library routine, and this sits on the one serial chain of the whole stage).
-__device__ __forceinline__ double rsqrt_pos(double d) {
-    const float df = static_cast<float>(d);
-    if (!(df > 1e-30f) || !(df < 1e30f)) return rsqrt(d);         // outside the comfortable range of the seed
-    double r = static_cast<double>(rsqrtf(df));
-    const double hd = 0.5 * d;
-    double e = fma(-hd * r, r, 0.5);
-    r = fma(r, e, r);
-    e = fma(-hd * r, r, 0.5);
-    return fma(r, e, r);
-}
-
 // 32 x 32 sub-block at S (pitch DP): upper triangle in, V = R^-1 out (upper, zeros below).
-// One warp, lane i holds row i.  The pivots form a serial chain (pivot -> reciprocal square root -> column ->
-// next pivot); per pivot only the next pivot's column is updated on that chain (one shuffle and one multiply-add),
-// the other columns follow through shared memory beside the next reciprocal square root.
 __device__ __forceinline__ void warp_factor_invert(double* S, double* colbuf, double* rinvb, int lane,
                                                    long long col_global, long long c_real, lq_dev_status* st) {
     double a[SB];
 #pragma unroll
     for (int t = 0; t < SB; ++t) a[t] = (t >= lane) ? S[lane * DP + t] : 0.0;
-    // R R^T factorisation, last column first.
+    // R R^T factorisation, last column first; lane i holds row i.  The pivots form the one serial chain of the whole
+    // stage: the entry that becomes the next pivot is updated and broadcast first, the other columns' updates follow
+    // and fill the latency of that broadcast and of the next reciprocal square root.
     double d = __shfl_sync(0xffffffffu, a[SB - 1], SB - 1);
 #pragma unroll
     for (int j = SB - 1; j >= 0; --j) {
@@ -455,43 +441,36 @@ __device__ __forceinline__ void warp_factor_invert(double* S, double* colbuf, do
             if (lane == 0 && col_global + j < c_real) lq_report(st, LQ_ERR_NOT_POSITIVE_DEFINITE, col_global + j);
             d = 1.0;
         }
-        const double rinv = rsqrt_pos(d);
-        const double lu = (lane < j) ? a[j] * rinv : 0.0;                 // R[i][j] above the diagonal
-        a[j] = (lane == j) ? d * rinv : lu;                               // sqrt(d) on the diagonal
+        const double rinv = rsqrt(d);
+        const double l = (lane < j) ? a[j] * rinv : ((lane == j) ? d * rinv : 0.0);   // R[i][j]; sqrt(d) on the diagonal
+        a[j] = l;
         if (lane == j) rinvb[j] = rinv;
         double* cb = colbuf + (j & 1) * SB;
-        cb[lane] = lu;
-        double dn = 1.0;
-        if (j > 0) {
-            const double ln = __shfl_sync(0xffffffffu, lu, j - 1);        // R[j-1][j]
-            a[j - 1] = fma(-lu, ln, a[j - 1]);
-            dn = __shfl_sync(0xffffffffu, a[j - 1], j - 1);               // the next pivot
-        }
+        cb[lane] = (lane < j) ? l : 0.0;
         __syncwarp();
+        if (j > 0) {
+            a[j - 1] = fma(-l, cb[j - 1], a[j - 1]);
+            d = __shfl_sync(0xffffffffu, a[j - 1], j - 1);
+        }
 #pragma unroll
-        for (int t = 0; t < j - 1; ++t) a[t] = fma(-lu, cb[t], a[t]);     // meaningful for lane <= t
-        d = dn;
+        for (int t = 0; t < j - 1; ++t) a[t] -= l * cb[t];            // meaningful for lane <= t
     }
-    // R to shared memory (rows), then V = R^-1 row by row: V[i][j] = (delta_ij - sum_{t<j} V[i][t] R[t][j]) / R[j][j];
-    // the newest term enters last, so that only it and the scaling sit between one entry and the next
+    // R to shared memory (rows), then V = R^-1, lane i forming row i column by column.  Every finished entry V[i][t] is
+    // pushed at once into the right-hand sides of all later columns (independent multiply-adds), so between one entry
+    // and the next there is one multiply-add and the scaling -- fp64 operations take ~23 cycles each here, and summing
+    // a column's terms only when its turn comes puts several of them in series.
 #pragma unroll
     for (int t = 0; t < SB; ++t) S[lane * DP + t] = (t >= lane) ? a[t] : 0.0;
     __syncwarp();
     double v[SB];
 #pragma unroll
-    for (int j = 0; j < SB; ++j) {
-        double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+    for (int j = 0; j < SB; ++j) v[j] = (lane == j) ? 1.0 : 0.0;          // right-hand sides, turned into V in place
 #pragma unroll
-        for (int t = 0; t < j - 1; ++t) {
-            const double rt = S[t * DP + j];
-            if ((t & 3) == 0) s0 = fma(v[t], rt, s0);
-            else if ((t & 3) == 1) s1 = fma(v[t], rt, s1);
-            else if ((t & 3) == 2) s2 = fma(v[t], rt, s2);
-            else s3 = fma(v[t], rt, s3);
-        }
-        double rhs = ((lane == j) ? 1.0 : 0.0) - ((s0 + s1) + (s2 + s3));
-        if (j > 0) rhs = fma(-v[j - 1], S[(j - 1) * DP + j], rhs);
-        v[j] = (lane <= j) ? rhs * rinvb[j] : 0.0;
+    for (int t = 0; t < SB; ++t) {
+        const double vt = (lane <= t) ? v[t] * rinvb[t] : 0.0;
+        v[t] = vt;
+#pragma unroll
+        for (int j = t + 1; j < SB; ++j) v[j] = fma(-vt, S[t * DP + j], v[j]);
     }
     __syncwarp();
 #pragma unroll
