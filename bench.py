@@ -580,41 +580,37 @@ BLOCKS = {
 
 
 def block_measure(lq, h, dev, rank, name, steps, warmup):
-    """Times the decoder-block workload; returns the fields of its report."""
+    """Times the decoder-block workload through the library's stack driver (StackPass: layers in order, stages 1-2 once
+    per distinct input, a packed record per layer); returns the fields of its report."""
     spec = BLOCKS[name]
     n, st = spec["n"], spec["settings"]
     cfg = lq.Config.make(**st)
     stream = torch.cuda.current_stream()
-    groups = []
+    inputs, weights, names = [], [], []
     for gi, (gname, c, recipe, layers) in enumerate(spec["inputs"]):
-        Ws, passes, X = [], [], None
+        Ws = []
         for li, (lname, r) in enumerate(layers):
             layer = synth.make_layer(recipe, r, c, n if li == 0 else 256, seed=layer_seed(rank) + 16 * gi + li, device=dev)
             if li == 0:
-                X = layer.X
+                inputs.append(layer.X)
             Ws.append(layer.W)
-            passes.append(lq.LayerPass(h, r, c, cfg, w_dtype=layer.W.dtype, x_dtype=X.dtype, n_chunk=n, device=dev,
-                                       want_w_hat=False))
             del layer
-        groups.append((gname, c, X, [l[0] for l in layers], Ws, passes))
+        weights.append(Ws)
+        names.append("hessian+prepare:" + gname)
+        names.extend(l[0] for l in layers)
+    S = lq.StackPass(h, [(c, [r for _, r in layers]) for _, c, _, layers in spec["inputs"]], cfg, w_dtype=weights[0][0].dtype,
+                     x_dtype=inputs[0].dtype, n_chunk=n, device=dev, want_w_hat=False, want_records=True)
 
     def one_step(events=None):
-        k = 0
-        for gname, c, X, lnames, Ws, passes in groups:
-            P0 = passes[0]
-            P0.H.zero_()
-            lq.lq_hessian_accumulate(h, X, P0.H, 2.0, P0.ws)
-            lq.lq_hessian_finalize(h, P0.H)
-            lq.lq_prepare_hinv(h, P0.H, P0.U, P0.dinv, P0.ws, 0.01, Ws[0])
-            if events: events[k].record(stream)
-            k += 1
-            for W, P in zip(Ws, passes):
-                lq.lq_fit_grid(h, cfg, W, P0.dinv, P.ws, P.grid, P.scale, P.zero)
-                lq.lq_quantize_layer(h, cfg, W, P0.U, P.codes, P.ws, P.grid, P.scale, P.zero, None, P.loss)
-                if events: events[k].record(stream)
-                k += 1
+        k = [0]
 
-    n_ev = sum(1 + len(g[3]) for g in groups)
+        def mark(g, l):
+            if events:
+                events[k[0]].record(stream)
+                k[0] += 1
+        S.run(inputs, weights, on_layer=mark)
+
+    n_ev = len(names)
     for _ in range(warmup):
         one_step()
     lq.lq_sync_status(h)
@@ -631,19 +627,17 @@ def block_measure(lq, h, dev, rank, name, steps, warmup):
     launches = lq.lq_launch_count() - launches0
     total_ms = e_beg.elapsed_time(e_end)
     lq.lq_sync_status(h)
-    names = []
-    for gname, c, X, lnames, Ws, passes in groups:
-        names.append("hessian+prepare:" + gname)
-        names.extend(lnames)
     parts = {}
     for j, nm in enumerate(names):
         beg = [e_beg if (i == 0 and j == 0) else (evs[i - 1][-1] if j == 0 else evs[i][j - 1]) for i in range(steps)]
         parts[nm] = float(np.mean([beg[i].elapsed_time(evs[i][j]) for i in range(steps)]))
-    weights = sum(W.numel() for g in groups for W in g[4])
+    weights_n = sum(W.numel() for Ws in weights for W in Ws)
+    payload_bits = sum(W.numel() * lq.lq_pack_layer_bytes(cfg, W.shape[0], W.shape[1])[1] for Ws in weights for W in Ws)
     ms_per_step = total_ms / steps
-    return {"weights": weights, "n_tokens": n, **st, "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step,
-            "value": weights / (ms_per_step * 1e-3), "unit": "weights/s",
+    return {"weights": weights_n, "n_tokens": n, **st, "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step,
+            "value": weights_n / (ms_per_step * 1e-3), "unit": "weights/s",
             "sharing": "stages 1-2 once per distinct input (4 Hessians for 7 layers)", "part_ms": parts,
+            "record_bits_per_weight": payload_bits / weights_n,
             "gpu_launches_per_step": int(launches) // steps}
 
 

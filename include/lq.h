@@ -201,6 +201,31 @@ int lq_quantize_layer(lq_handle* h, void* stream, const lq_config* cfg, const vo
 int lq_pack_codes(lq_handle* h, void* stream, const uint8_t* codes, int64_t r, int64_t c,
                   int32_t bits, uint8_t* packed, int64_t ldp);
 
+/* A whole quantised layer in the form the paper's bit accounting assumes (result tables, bit columns; Appendix A):
+ *   non-uniform: b-bit codes plus a 2^b-entry fp16 table per output row      -> b + 16 * 2^b / c bits per weight
+ *                (4.06 / 3.03 / 2.02 at c = 4096; 4.05 / 3.02 / 2.01 averaged over a Llama-3-8B-shaped block);
+ *   affine:      b-bit codes plus an fp16 scale and an int16 zero point per group -> b + 32 / g bits per weight
+ *                (4.25 with groups of 128, 4.00 row-wise at these widths).
+ * record (device, 16-byte aligned, lq_pack_layer_bytes bytes): a 64-byte header {magic "LQP1", bits, grid type, group size,
+ * r, c, byte offsets of the three sections, total bytes}, the packed codes (row i at codes_offset + i * ceil(c * bits / 8),
+ * the bit stream of lq_pack_codes), then the tables (r x 2^b fp16) or the scales (r x c/g fp16) and zero points
+ * (r x c/g int16); sections start on 16-byte boundaries.  grid / scale are rounded to fp16 (round to nearest even); a
+ * zero point outside int16 records LQ_ERR_UNSUPPORTED (info = its index) and is stored saturated.
+ * *bits_per_weight (may be NULL) is the figure above: header and alignment padding are not counted. */
+int lq_pack_layer_bytes(const lq_config* cfg, int64_t r, int64_t c, size_t* bytes, double* bits_per_weight);
+int lq_pack_layer(lq_handle* h, void* stream, const lq_config* cfg, const uint8_t* codes, int64_t r, int64_t c,
+                  const float* grid, const float* scale, const int32_t* zero, void* record, size_t record_bytes);
+/* The weights a record stands for: W_hat[i][j] = table[i][code] or (code - Z) * S with the record's fp16 values
+ * (device, what_dtype, r x c with ldwh).  A header that does not match (cfg, r, c) records LQ_ERR_INVALID_ARG. */
+int lq_unpack_layer(lq_handle* h, void* stream, const lq_config* cfg, const void* record, size_t record_bytes,
+                    int64_t r, int64_t c, void* W_hat, int32_t what_dtype, int64_t ldwh);
+
+/* For layers that share a Hessian (the q / k / v projections of a block read the same activations): lq_prepare_hinv
+ * zeroes the dead input channels' columns of the one W it is given; this does the same for another layer's W.
+ * H: the accumulated Hessian as lq_prepare_hinv read it (so U must not have been written over it). */
+int lq_zero_dead_columns(lq_handle* h, void* stream, const float* H, int64_t c, int64_t ldh, void* W, int32_t w_dtype,
+                         int64_t r, int64_t ldw);
+
 /* Variant of lq_quantize_layer for affine grids in which the (S, Z) of a group are not fitted beforehand on the
  * original weights (Algorithm 1 lines 5-9) but when the column loop reaches the group's first column, on that
  * group's columns as they stand then, i.e. with the errors of all earlier columns already fed back into them

@@ -427,6 +427,88 @@ def unpack_codes(packed, bits: int, c: int) -> np.ndarray:
     return (planes << np.arange(bits)).sum(axis=2)
 
 
+RECORD_MAGIC = 0x3150514C      # "LQP1"
+
+
+def _align16(n: int) -> int:
+    return (n + 15) // 16 * 16
+
+
+def record_bits_per_weight(bits: int, c: int, grid_type: str = "nonuniform", group: int = 0) -> float:
+    """Storage cost per weight behind the bit columns of the paper's result tables: b-bit codes plus, per output
+    row, a 2^b-entry fp16 table (non-uniform), or per group an fp16 scale and a 16-bit zero point (affine)."""
+    if grid_type == "nonuniform":
+        return bits + 16.0 * (1 << bits) / c
+    g = c if group in (0, None) else group
+    return bits + 32.0 / g
+
+
+def pack_layer(codes, bits: int, *, grid=None, scale=None, zero=None, group: int = 0) -> np.ndarray:
+    """One quantised layer as a byte record: 64-byte header (magic "LQP1", bits, grid type 0 / 1, group size as given,
+    r, c, byte offsets of the codes, of the tables or scales, of the zero points, total bytes; int32 x 4 then int64 x 6,
+    little endian), the packed codes (pack_codes), then the fp16 tables (r x 2^b) or the fp16 scales and int16 zero points
+    (r x n_groups each); every section starts on a 16-byte boundary, padding bytes are zero."""
+    codes = np.asarray(codes)
+    r, c = codes.shape
+    packed = pack_codes(codes, bits)
+    row_bytes = packed.shape[1]
+    affine = grid is None
+    off_codes = 64
+    off_table = off_codes + _align16(r * row_bytes)
+    if affine:
+        ng = np.asarray(scale).shape[1]
+        off_zero = off_table + _align16(r * ng * 2)
+        total = off_zero + _align16(r * ng * 2)
+    else:
+        off_zero = off_table + _align16(r * (1 << bits) * 2)
+        total = off_zero
+    rec = np.zeros(total, dtype=np.uint8)
+    rec[:16] = np.array([RECORD_MAGIC, bits, 1 if affine else 0, group or 0], dtype="<u4").view(np.uint8)
+    rec[16:64] = np.array([r, c, off_codes, off_table, off_zero, total], dtype="<i8").view(np.uint8)
+    rec[off_codes:off_codes + r * row_bytes] = packed.reshape(-1)
+    if affine:
+        s16 = np.asarray(scale, dtype=np.float32).astype(np.float16)
+        z16 = np.clip(np.asarray(zero), -32768, 32767).astype("<i2")
+        rec[off_table:off_table + s16.size * 2] = s16.reshape(-1).view(np.uint8)
+        rec[off_zero:off_zero + z16.size * 2] = z16.reshape(-1).view(np.uint8)
+    else:
+        t16 = np.asarray(grid, dtype=np.float32).astype(np.float16)
+        rec[off_table:off_table + t16.size * 2] = t16.reshape(-1).view(np.uint8)
+    return rec
+
+
+def unpack_layer(rec: np.ndarray) -> np.ndarray:
+    """The weights a record stands for, in float64: table[row][code], or (code - Z) * S with the stored fp16 / int16
+    values (the product rounded to float32, as the format's consumers compute it)."""
+    rec = np.asarray(rec, dtype=np.uint8)
+    magic, bits, affine, group = (int(v) for v in rec[:16].view("<u4"))
+    r, c, off_codes, off_table, off_zero, total = (int(v) for v in rec[16:64].view("<i8"))
+    if magic != RECORD_MAGIC or total != rec.size:
+        raise ValueError("not a layer record")
+    row_bytes = (c * bits + 7) // 8
+    codes = unpack_codes(rec[off_codes:off_codes + r * row_bytes].reshape(r, row_bytes), bits, c)
+    if affine:
+        g = c if group == 0 else group
+        ng = c // g
+        S = rec[off_table:off_table + r * ng * 2].view(np.float16).reshape(r, ng).astype(np.float32)
+        Z = rec[off_zero:off_zero + r * ng * 2].view("<i2").reshape(r, ng).astype(np.float32)
+        gi = np.arange(c) // g
+        return ((codes.astype(np.float32) - Z[:, gi]) * S[:, gi]).astype(F64)
+    table = rec[off_table:off_table + r * (1 << bits) * 2].view(np.float16).reshape(r, 1 << bits)
+    return np.take_along_axis(table, codes, 1).astype(F64)
+
+
+def run_stack(groups, **kw):
+    """A stack of layers quantised in order, as a model-level driver calls the pass: `groups` is a list of
+    (X, [W, ...]) -- every W of a group reads the same activations X, so the group shares stages 1-2 (one Hessian,
+    one factor) and each W gets its own grid and column loop.  Returns one run_pass-style dict per layer, in order."""
+    out = []
+    for X, Ws in groups:
+        for W in Ws:
+            out.append(run_pass(W, X, **kw))
+    return out
+
+
 def proxy_loss(W, What, H) -> float:
     """tr((W - What) H (W - What)^T); with the undamped H = 2XX^T this is
     2 * ||W X - What X||_F^2, the layer objective of Eq. 1 up to the factor 2."""

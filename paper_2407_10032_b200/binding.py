@@ -70,6 +70,10 @@ def LQ():
             "lq_fit_grid_noalloc": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, vp, vp, vp],
             "lq_pack_codes": [vp, vp, vp, i64, i64, i32, vp, i64],
             "lq_peak_probe": [vp, vp, i32, i64, P(C.c_double)],
+            "lq_pack_layer_bytes": [P(Config), i64, i64, P(sz), P(C.c_double)],
+            "lq_pack_layer": [vp, vp, P(Config), vp, i64, i64, vp, vp, vp, vp, sz],
+            "lq_unpack_layer": [vp, vp, P(Config), vp, sz, i64, i64, vp, i32, i64],
+            "lq_zero_dead_columns": [vp, vp, vp, i64, i64, vp, i32, i64, i64],
             "lq_testing_set_wait_limit_ns": [vp, C.c_uint64],
             "lq_testing_inject_stall": [vp, i32],
             "lq_testing_set_prepare_defer_min_blocks": [vp, i32],
@@ -291,13 +295,91 @@ def lq_pack_codes(h, codes, bits, packed=None, stream=None):
     return packed
 
 
+def lq_pack_layer_bytes(cfg, r, c):
+    """(bytes of a layer record, bits per weight of the format)."""
+    b, bpw = C.c_size_t(0), C.c_double(0.0)
+    _check(LQ().lq_pack_layer_bytes(C.byref(cfg), r, c, C.byref(b), C.byref(bpw)), "lq_pack_layer_bytes")
+    return b.value, bpw.value
+
+
+def lq_pack_layer(h, cfg, codes, grid=None, scale=None, zero=None, record=None, stream=None):
+    """The layer as one record (packed codes + fp16 tables, or fp16 scales + int16 zero points); returns the record."""
+    r, c = codes.shape
+    nbytes, _ = lq_pack_layer_bytes(cfg, r, c)
+    if record is None:
+        record = torch.zeros((nbytes,), dtype=torch.uint8, device=codes.device)
+    _check(LQ().lq_pack_layer(h, _stream(stream), C.byref(cfg), _ptr(codes), r, c, _ptr(grid), _ptr(scale), _ptr(zero),
+                              _ptr(record), record.numel()), "lq_pack_layer")
+    return record
+
+
+def lq_unpack_layer(h, cfg, record, r, c, W_hat=None, dtype=torch.float32, stream=None):
+    """The weights a record stands for."""
+    if W_hat is None:
+        W_hat = torch.empty((r, c), dtype=dtype, device=record.device)
+    _check(LQ().lq_unpack_layer(h, _stream(stream), C.byref(cfg), _ptr(record), record.numel(), r, c, _ptr(W_hat), _dt(W_hat),
+                                _rowmajor(W_hat)), "lq_unpack_layer")
+    return W_hat
+
+
+def lq_zero_dead_columns(h, H, W, stream=None):
+    """Zeroes the columns of W whose input channel never fired (H_ii = 0): for layers that share a Hessian."""
+    r, c = W.shape
+    _check(LQ().lq_zero_dead_columns(h, _stream(stream), _ptr(H), c, _rowmajor(H), _ptr(W), _dt(W), r, _rowmajor(W)),
+           "lq_zero_dead_columns")
+
+
+class StackPass:
+    """A stack of layers quantised in order, the way a model-level driver walks a decoder block: layers that read the
+    same activations form a group and share stages 1-2 (one Hessian, one factor); every layer then gets its own grid,
+    its column loop and its packed record.  Only buffers and the order of the library calls live here.
+
+    groups: list of (c, [r, ...]) -- input width of the group and the output widths of its layers."""
+
+    def __init__(self, handle, groups, cfg: Config, w_dtype=torch.bfloat16, x_dtype=torch.bfloat16, n_chunk=0,
+                 device="cuda", want_w_hat=False, want_records=True):
+        self.h, self.cfg, self.groups, self.want_records = handle, cfg, groups, want_records
+        self.passes = []
+        for c, rs in groups:
+            ps = []
+            for r in rs:                          # one Hessian, one factor and one inverse diagonal per group
+                ps.append(LayerPass(handle, r, c, cfg, w_dtype=w_dtype, x_dtype=x_dtype, n_chunk=n_chunk, device=device,
+                                    want_w_hat=want_w_hat, share=ps[0] if ps else None))
+            self.passes.append(ps)
+        self.records = [[None] * len(rs) for _, rs in groups]
+
+    def run(self, inputs, weights, damp_frac=0.01, alpha=2.0, n_chunk=0, on_layer=None):
+        """inputs[g]: the group's activations X (c x n); weights[g][l]: that layer's W (r x c, dead columns are zeroed
+        in place).  `on_layer(g, l)` is called after each layer's work has been enqueued (a benchmark records an event)."""
+        for g, (X, Ws, ps) in enumerate(zip(inputs, weights, self.passes)):
+            P0 = ps[0]
+            n = X.shape[1]
+            step = n if n_chunk <= 0 else n_chunk
+            P0.H.zero_()
+            for j in range(0, n, step):
+                lq_hessian_accumulate(self.h, X[:, j:j + step], P0.H, alpha, P0.ws)
+            lq_hessian_finalize(self.h, P0.H)
+            lq_prepare_hinv(self.h, P0.H, P0.U, P0.dinv, P0.ws, damp_frac, Ws[0])
+            for W in Ws[1:]:
+                lq_zero_dead_columns(self.h, P0.H, W)
+            if on_layer:
+                on_layer(g, -1)
+            for l, (W, P) in enumerate(zip(Ws, ps)):
+                lq_fit_grid(self.h, self.cfg, W, P0.dinv, P.ws, P.grid, P.scale, P.zero)
+                lq_quantize_layer(self.h, self.cfg, W, P0.U, P.codes, P.ws, P.grid, P.scale, P.zero, P.W_hat, P.loss)
+                if self.want_records:
+                    self.records[g][l] = lq_pack_layer(self.h, self.cfg, P.codes, P.grid, P.scale, P.zero, self.records[g][l])
+                if on_layer:
+                    on_layer(g, l)
+
+
 class LayerPass:
     """Buffers for one layer shape plus the four calls in Algorithm 1's order.
 
     Allocation only (through torch's allocator); all arithmetic is in liblq."""
 
     def __init__(self, handle, r, c, cfg: Config, w_dtype=torch.bfloat16, x_dtype=torch.bfloat16, n_chunk=0,
-                 device="cuda", want_w_hat=True, weight_src="inv_diag"):
+                 device="cuda", want_w_hat=True, weight_src="inv_diag", share=None):
         if weight_src not in ("inv_diag", "chol_diag"):
             raise ValueError("weight_src: 'inv_diag' (Eq. 5 / Eq. 7) or 'chol_diag' (Algorithm 1 to the letter)")
         self.weight_src = weight_src
@@ -305,9 +387,12 @@ class LayerPass:
         dev = torch.device(device)
         K = 1 << cfg.bits
         f32 = dict(device=dev, dtype=torch.float32)
-        self.H = torch.zeros((c, c), **f32)
-        self.U = torch.empty((c, c), **f32)
-        self.dinv = torch.empty((c,), **f32)
+        if share is not None:                 # a layer that reads the same activations: one Hessian, factor and diagonal
+            self.H, self.U, self.dinv = share.H, share.U, share.dinv
+        else:
+            self.H = torch.zeros((c, c), **f32)
+            self.U = torch.empty((c, c), **f32)
+            self.dinv = torch.empty((c,), **f32)
         self.affine = cfg.grid_type == LQ_GRID_AFFINE
         ng = 1 if cfg.group_size == 0 else c // cfg.group_size
         self.grid = None if self.affine else torch.empty((r, K), **f32)

@@ -26,6 +26,49 @@ def spd(c, seed, cond=1e3):
     return (Q * lam) @ Q.T
 
 
+# Linear layers of one Llama-3-8B-shaped decoder block, (r, c): what the paper's bit widths average over.
+LLAMA3_8B_BLOCK = [(4096, 4096), (1024, 4096), (1024, 4096), (4096, 4096), (14336, 4096), (14336, 4096), (4096, 14336)]
+
+
+def test_record_format_costs_the_bits_the_paper_prints():
+    """Codes plus a 2^b-entry fp16 table per row (non-uniform) or an fp16 scale and a 16-bit zero point per group
+    (affine), averaged over the linear layers of a Llama-3-8B-shaped block, give the bit widths of the paper's tables
+    to the two decimals it prints (4.0505 -> 4.05, 3.0252 -> 3.02, 2.0126 -> 2.01, 4.0063 -> 4.00: the printed figures
+    are the averages cut after two decimals).  A table per 128 columns, fp32 tables, or (S, Z) stored wider would not."""
+    total = sum(r * c for r, c in LLAMA3_8B_BLOCK)
+    for line in open(os.path.join(GOLDEN, "table_bits.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        grid_type, bits, group, printed = line.split()
+        avg = sum(r * c * O.record_bits_per_weight(int(bits), c, grid_type, int(group)) for r, c in LLAMA3_8B_BLOCK) / total
+        assert int(avg * 100 + 1e-9) == round(float(printed) * 100), (line, avg)
+
+
+def test_pack_layer_by_hand_and_round_trip():
+    g = rng(21)
+    # non-uniform, 2 bits, 3 x 5: header fields, section offsets, table bytes and the weights it stands for
+    codes = g.integers(0, 4, size=(3, 5))
+    grid = np.sort(g.standard_normal((3, 4)), axis=1)
+    rec = O.pack_layer(codes, 2, grid=grid)
+    assert rec[:4].tobytes() == b"LQP1" and rec.dtype == np.uint8
+    assert list(rec[4:16].view("<u4")) == [2, 0, 0]
+    r, c, oc, ot, oz, tot = (int(v) for v in rec[16:64].view("<i8"))
+    assert (r, c, oc) == (3, 5, 64) and ot == 64 + 16 and tot == ot + 32 and oz == tot and tot == rec.size
+    assert np.array_equal(rec[oc:oc + 6].reshape(3, 2), O.pack_codes(codes, 2))
+    t16 = rec[ot:ot + 24].view(np.float16).reshape(3, 4)
+    assert np.array_equal(t16, grid.astype(np.float16))
+    np.testing.assert_array_equal(O.unpack_layer(rec), np.take_along_axis(grid.astype(np.float16).astype(np.float64), codes, 1))
+    # affine, 4 bits, groups of 8 in a 2 x 16 layer
+    codes = g.integers(0, 16, size=(2, 16))
+    S = np.abs(g.standard_normal((2, 2))) * 0.01 + 0.001
+    Z = g.integers(-3, 12, size=(2, 2)).astype(np.float64)
+    rec = O.pack_layer(codes, 4, scale=S, zero=Z, group=8)
+    assert list(rec[4:16].view("<u4")) == [4, 1, 8]
+    want = (codes - np.repeat(Z, 8, axis=1)).astype(np.float32) * np.repeat(S.astype(np.float16).astype(np.float32), 8, axis=1)
+    np.testing.assert_array_equal(O.unpack_layer(rec), want.astype(np.float64))
+    assert rec.size == 64 + 16 + 16 + 16
+
+
 # ------------------------------------------------------------------ P1 ---- #
 def obq_fixed_order(W, Hinv, quant_row):
     """Eq. 3 and Eq. 9 taken literally, column by column in fixed order:
