@@ -210,97 +210,7 @@ __device__ __forceinline__ void bitonic_sort(KeyT* keys, int n, int tid) {
     }
 }
 
-// ---------------------------------------------------------------- counting sort ----
-// bf16 rows: the 16-bit order-preserving key has 65536 values, so a row is sorted exactly by two counting passes
-// instead of a comparison network: pass 1 spreads the row over 4096 buckets by the top 12 bits of the key (histogram,
-// prefix sums, scatter with one shared-memory atomic each), pass 2 orders every bucket by the remaining 4 bits (one
-// warp per bucket, 16 ballots per 32 members).  Equal weights end up next to one another in no particular order,
-// which no boundary search can tell.  O(c) shared-memory operations against O(c log^2 c) for the network.
-constexpr int CS_BUCKET_BITS = 12;
-constexpr int CS_BUCKETS = 1 << CS_BUCKET_BITS;
-constexpr int CS_LOW_BITS = 16 - CS_BUCKET_BITS;
-constexpr int CS_LOW = 1 << CS_LOW_BITS;
-
-// keys[0..c): (key16 << 16 | column) unsorted on entry, sorted on return; tmp: c words of scratch; hist: CS_BUCKETS words.
-__device__ __forceinline__ void counting_sort_bf16(uint32_t* keys, uint32_t* tmp, uint32_t* hist, int c, int tid) {
-    const int lane = tid & 31, warp = tid >> 5;
-    __shared__ uint32_t warp_tot[KS_THREADS / 32];
-    for (int b = tid; b < CS_BUCKETS; b += KS_THREADS) hist[b] = 0;
-    __syncthreads();
-    for (int i = tid; i < c; i += KS_THREADS) atomicAdd(&hist[keys[i] >> (32 - CS_BUCKET_BITS)], 1u);
-    __syncthreads();
-    {   // exclusive prefix sums of the bucket counts: CS_BUCKETS / KS_THREADS consecutive buckets per thread
-        constexpr int PER = CS_BUCKETS / KS_THREADS;
-        uint32_t loc[PER];
-        uint32_t sum = 0;
-#pragma unroll
-        for (int e = 0; e < PER; ++e) { loc[e] = sum; sum += hist[tid * PER + e]; }
-        uint32_t incl = sum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const uint32_t v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        if (lane == 31) warp_tot[warp] = incl;
-        __syncthreads();
-        uint32_t base = incl - sum;
-        for (int w = 0; w < warp; ++w) base += warp_tot[w];
-#pragma unroll
-        for (int e = 0; e < PER; ++e) hist[tid * PER + e] = base + loc[e];
-    }
-    __syncthreads();
-    for (int i = tid; i < c; i += KS_THREADS) {
-        const uint32_t v = keys[i];
-        tmp[atomicAdd(&hist[v >> (32 - CS_BUCKET_BITS)], 1u)] = v;
-    }
-    __syncthreads();
-    // now hist[b] is the end of bucket b (the start of bucket b + 1).  Pass 2: a warp takes 32 buckets at a time and
-    // works through the non-empty ones.
-    for (int b0 = warp * 32; b0 < CS_BUCKETS; b0 += KS_THREADS) {
-        const int b = b0 + lane;
-        const uint32_t my_end = hist[b];
-        const uint32_t my_start = b == 0 ? 0u : hist[b - 1];
-        uint32_t todo = __ballot_sync(0xffffffffu, my_end > my_start);
-        while (todo) {
-            const int src = __ffs(todo) - 1;
-            todo &= todo - 1;
-            const uint32_t start = __shfl_sync(0xffffffffu, my_start, src);
-            const uint32_t end = __shfl_sync(0xffffffffu, my_end, src);
-            const uint32_t n = end - start;
-            if (n == 1) {
-                if (lane == 0) keys[start] = tmp[start];
-                continue;
-            }
-            uint32_t cnt[CS_LOW];
-#pragma unroll
-            for (int v = 0; v < CS_LOW; ++v) cnt[v] = 0;
-            for (uint32_t m0 = 0; m0 < n; m0 += 32) {
-                const bool have = m0 + lane < n;
-                const uint32_t low = have ? (tmp[start + m0 + lane] >> 16) & (CS_LOW - 1) : CS_LOW;
-#pragma unroll
-                for (int v = 0; v < CS_LOW; ++v) cnt[v] += __popc(__ballot_sync(0xffffffffu, low == static_cast<uint32_t>(v)));
-            }
-            uint32_t run = start;
-#pragma unroll
-            for (int v = 0; v < CS_LOW; ++v) { const uint32_t t = cnt[v]; cnt[v] = run; run += t; }     // first slot of each value
-            const uint32_t lt = (1u << lane) - 1u;
-            for (uint32_t m0 = 0; m0 < n; m0 += 32) {
-                const bool have = m0 + lane < n;
-                const uint32_t val = have ? tmp[start + m0 + lane] : 0u;
-                const uint32_t low = have ? (val >> 16) & (CS_LOW - 1) : CS_LOW;
-#pragma unroll
-                for (int v = 0; v < CS_LOW; ++v) {
-                    const uint32_t mask = __ballot_sync(0xffffffffu, low == static_cast<uint32_t>(v));
-                    if (low == static_cast<uint32_t>(v)) keys[cnt[v] + __popc(mask & lt)] = val;
-                    cnt[v] += __popc(mask);
-                }
-            }
-        }
-    }
-    __syncthreads();
-}
-
-template <int K, typename T, bool CSORT>
+template <int K, typename T>
 __global__ void __launch_bounds__(KS_THREADS, 4)
 kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int n, const double* __restrict__ s64,
                      float* __restrict__ grid, int n_iter, int init) {
@@ -308,9 +218,6 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
     extern __shared__ __align__(16) unsigned char ks_smem[];
     dd2* coarse = reinterpret_cast<dd2*>(ks_smem);            // n / 8 + 1 coarse prefixes, then the n keys (padded slots)
     KeyT* keys = reinterpret_cast<KeyT*>(coarse + (n / KS_CHUNK + 1));
-    // counting sort (CSORT, bf16 rows): the keys are unpadded, the scratch of the first pass shares the room of the
-    // coarse prefixes (they are formed after the sort), and the bucket counters follow the keys
-    auto slot = [](int i) { return CSORT ? i : ks_slot(i); };
     __shared__ dd2 tot[KS_THREADS];                            // per-thread totals, then their exclusive scan
     __shared__ double g[K];
     __shared__ dd2 F[K + 1];
@@ -320,14 +227,9 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
 
     for (int64_t row = blockIdx.x; row < r; row += gridDim.x) {
         const T* wp = W + row * ldw;
-        for (int i = tid; i < n; i += KS_THREADS) keys[slot(i)] = i < c ? KeyOf<T>::make(wp[i], i) : KeyOf<T>::pad();
+        for (int i = tid; i < n; i += KS_THREADS) keys[ks_slot(i)] = i < c ? KeyOf<T>::make(wp[i], i) : KeyOf<T>::pad();
         __syncthreads();
-        if (CSORT) {
-            counting_sort_bf16(reinterpret_cast<uint32_t*>(keys), reinterpret_cast<uint32_t*>(coarse),
-                               reinterpret_cast<uint32_t*>(keys) + n, c, tid);
-        } else {
-            bitonic_sort<KeyT>(keys, n, tid);
-        }
+        bitonic_sort<KeyT>(keys, n, tid);
         // chunk totals, thread-local exclusive prefixes
         dd2 run;
         run.s.hi = run.s.lo = run.sw.hi = run.sw.lo = 0.0;
@@ -337,7 +239,7 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
             for (int e = 0; e < KS_CHUNK; ++e) {
                 const int i = q * KS_CHUNK + e;
                 if (i < c) {
-                    const KeyT key = keys[slot(i)];
+                    const KeyT key = keys[ks_slot(i)];
                     const double sv = s64[key_index(key)];
                     run.s = dd_add_d(run.s, sv);                 // same order and arithmetic as F(b) below
                     run.sw = dd_add_d(run.sw, __dmul_rn(sv, static_cast<double>(key_weight(key))));
@@ -395,8 +297,8 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
         __syncthreads();
 
         if (warp == 0) {
-            const double lo = static_cast<double>(key_weight(keys[slot(0)]));
-            const double hi = static_cast<double>(key_weight(keys[slot(c - 1)]));
+            const double lo = static_cast<double>(key_weight(keys[ks_slot(0)]));
+            const double hi = static_cast<double>(key_weight(keys[ks_slot(c - 1)]));
             if (init == LQ_INIT_UNIFORM) {
                 if (lane < K) g[lane] = lo + (hi - lo) * static_cast<double>(lane) / static_cast<double>(K - 1);   // Eq. 6
             } else if (lane < K) {
@@ -410,10 +312,10 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
                     const int b = mid + 1;                     // cumulative weight of positions 0 .. mid
                     const int q = b / KS_CHUNK, rem = b % KS_CHUNK;
                     dd f = coarse[q].s;
-                    for (int e = 0; e < rem; ++e) f = dd_add_d(f, s64[key_index(keys[slot(q * KS_CHUNK + e)])]);
+                    for (int e = 0; e < rem; ++e) f = dd_add_d(f, s64[key_index(keys[ks_slot(q * KS_CHUNK + e)])]);
                     if (f.hi + f.lo >= target) p1 = mid; else p0 = mid + 1;
                 }
-                g[lane] = static_cast<double>(key_weight(keys[slot(p0)]));
+                g[lane] = static_cast<double>(key_weight(keys[ks_slot(p0)]));
             }
             if (lane == 0) {
                 F[0].s.hi = F[0].s.lo = F[0].sw.hi = F[0].sw.lo = 0.0;
@@ -428,7 +330,7 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
                     int b1 = c;                                // first position whose weight exceeds m
                     while (b0 < b1) {
                         const int mid = (b0 + b1) >> 1;
-                        if (static_cast<double>(key_weight(keys[slot(mid)])) > m) b1 = mid; else b0 = mid + 1;
+                        if (static_cast<double>(key_weight(keys[ks_slot(mid)])) > m) b1 = mid; else b0 = mid + 1;
                     }
                 }
                 // Unchanged boundaries give back the same centroids, and so would every later
@@ -439,7 +341,7 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
                     const int q = b0 / KS_CHUNK, rem = b0 % KS_CHUNK;
                     dd2 f = coarse[q];
                     for (int e = 0; e < rem; ++e) {
-                        const KeyT key = keys[slot(q * KS_CHUNK + e)];
+                        const KeyT key = keys[ks_slot(q * KS_CHUNK + e)];
                         const double sv = s64[key_index(key)];
                         f.s = dd_add_d(f.s, sv);
                         f.sw = dd_add_d(f.sw, __dmul_rn(sv, static_cast<double>(key_weight(key))));
@@ -545,35 +447,22 @@ kmeans_rows_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int64_t c, c
     }
 }
 
-template <typename T> struct CanCountSort { static constexpr bool value = false; };
-template <> struct CanCountSort<__nv_bfloat16> { static constexpr bool value = true; };
-
 template <int K, typename T>
 int launch_kmeans(cudaStream_t st, int sms, const T* W, int64_t ldw, int64_t r, int64_t c, const double* s64, float* grid,
                   int n_iter, int init) {
     if (c <= KS_MAX_N) {
-        constexpr bool CS = CanCountSort<T>::value;
         int n = 64;
         while (n < c) n <<= 1;
-        size_t smem;
-        if (CS) {
-            // coarse prefixes (which hold the first pass's scratch before), unpadded keys, bucket counters; n is c
-            // rounded up to a multiple of the chunk
-            n = static_cast<int>(lq_ceil_div(c, KS_CHUNK) * KS_CHUNK);
-            smem = (static_cast<size_t>(n) / KS_CHUNK + 1) * sizeof(dd2) + static_cast<size_t>(n) * sizeof(uint32_t) +
-                   static_cast<size_t>(CS_BUCKETS) * sizeof(uint32_t);
-        } else {
-            smem = (static_cast<size_t>(n) / KS_CHUNK + 1) * sizeof(dd2) +
-                   static_cast<size_t>(n + n / 32) * sizeof(typename KeyOf<T>::type);
-        }
+        const size_t smem = (static_cast<size_t>(n) / KS_CHUNK + 1) * sizeof(dd2) +
+                            static_cast<size_t>(n + n / 32) * sizeof(typename KeyOf<T>::type);
         static lq_once_per_device attr_set;
         if (attr_set.first()) {
-            LQ_CUDA_TRY(cudaFuncSetAttribute(kmeans_sorted_kernel<K, T, CS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+            LQ_CUDA_TRY(cudaFuncSetAttribute(kmeans_sorted_kernel<K, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
         }
         int per_sm = static_cast<int>((228 * 1024) / (smem + 10 * 1024));      // static shared memory and the per-CTA reserve
         per_sm = per_sm < 1 ? 1 : (per_sm > 4 ? 4 : per_sm);                    // 64 registers x 256 threads: four CTAs per SM
         const int64_t cap = static_cast<int64_t>(sms) * per_sm;
-        kmeans_sorted_kernel<K, T, CS><<<static_cast<unsigned>(r < cap ? r : cap), KS_THREADS, smem, st>>>(
+        kmeans_sorted_kernel<K, T><<<static_cast<unsigned>(r < cap ? r : cap), KS_THREADS, smem, st>>>(
             W, ldw, r, static_cast<int>(c), n, s64, grid, n_iter, init);
     } else {
         if (init != LQ_INIT_UNIFORM) return LQ_ERR_UNSUPPORTED;     // rows this long only start from Eq. 6
