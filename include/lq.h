@@ -231,8 +231,9 @@ int lq_zero_dead_columns(lq_handle* h, void* stream, const float* H, int64_t c, 
  * group's columns as they stand then, i.e. with the errors of all earlier columns already fed back into them
  * (the usual practice of GPTQ implementations; the paper's pseudocode fits all grids first).  The search is that
  * of lq_fit_grid (Eq. 7 with cfg->T, cfg->t_count, cfg->p and the sample weights from dinv); scale / zero
- * (r x c / group_size) are outputs.  Supported group sizes: multiples of 128 that divide 1024, multiples of
- * 1024, and one group per row (which is the same as fitting beforehand).  Other arguments as lq_quantize_layer;
+ * (r x c / group_size) are outputs.  Supported group sizes: divisors of 128 that are multiples of 4 (refitted inside the
+ * in-block kernel), multiples of 128 that divide 1024, multiples of 1024, and one group per row (which is the same as
+ * fitting beforehand).  Other arguments as lq_quantize_layer;
  * workspace: lq_quantize_layer_lazy_workspace bytes. */
 int lq_quantize_layer_lazy_workspace(const lq_config* cfg, int64_t r, int64_t c, size_t* bytes);
 int lq_quantize_layer_lazy(lq_handle* h, void* stream, const lq_config* cfg, const void* W, int32_t w_dtype,

@@ -11,6 +11,7 @@
 #include <math.h>
 
 #include "lq_common.cuh"
+#include "lq_affine_warp.cuh"
 
 namespace {
 
@@ -127,13 +128,22 @@ struct QuantOut {
 // the diagonal are zero, so no lane needs a predicate.
 constexpr int IB_MAX_THREADS = 1024;   // warps (= rows) per CTA are chosen at launch so that the rows spread evenly over the SMs
 
-template <int K, bool AFFINE>
-__global__ void __launch_bounds__(IB_MAX_THREADS)
+// Refit of groups shorter than a block inside the loop (the lazy variant of the affine grid): what the kernel needs
+// for the search of Eq. 7 when it reaches a group's first column.
+struct RefitArgs {
+    const double* s64;       // sample weights of all c columns
+    float* scale;            // outputs, r x n_groups
+    int32_t* zero;
+    int T, t_count;
+};
+
+template <int K, bool AFFINE, bool REFIT>
+__global__ void __launch_bounds__(REFIT ? IB_MAX_THREADS / 2 : IB_MAX_THREADS)
 inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, int64_t i0, const float* __restrict__ U,
                int64_t ldu, const float* __restrict__ grid, const float* __restrict__ scale,
-               const int32_t* __restrict__ zero, int group, int n_groups, QuantOut out) {
+               const int32_t* __restrict__ zero, int group, int n_groups, QuantOut out, RefitArgs refit) {
     extern __shared__ float Us[];          // B x B block of U, then B reciprocals of its diagonal
-    float* invd = Us + B * B;
+    float* invd = Us + B * B;              // (REFIT: then per warp `group` floats and `group` float2 of search scratch)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int bw = (c - i0) < B ? static_cast<int>(c - i0) : B;
 
@@ -178,7 +188,7 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
         if (valid && lane < K) gl = grid[row * K + lane];
         const float gn = __shfl_down_sync(0xffffffffu, gl, 1);
         if (lane < K - 1) ml = 0.5f * (gl + gn);
-    } else if (valid && col0 < bw) {
+    } else if (!REFIT && valid && col0 < bw) {
         const int64_t gi = (i0 + col0) / group;
         const int64_t gidx = row * n_groups + (gi < n_groups ? gi : n_groups - 1);
         S_mine = scale[gidx];
@@ -207,6 +217,28 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
 #pragma unroll 1
     for (int jj = 0; jj < n_owner; ++jj) {
         float S = 1.0f, Zf = 0.0f, rS = 1.0f;
+        if (REFIT && (i0 + 4 * jj) % group == 0) {
+            // a group starts at this column: fit its (S, Z) by Eq. 7 on the group's weights as they stand now, with the
+            // errors of every earlier column already fed back (the lanes that own the group hand their weights over)
+            float* wtmp = invd + B + static_cast<size_t>(warp) * 3 * group;
+            float2* ws = reinterpret_cast<float2*>(wtmp + group);
+            const int gl = group / 4;                        // lanes per group
+            if (lane >= jj && lane < jj + gl) {
+#pragma unroll
+                for (int u = 0; u < 4; ++u) wtmp[4 * (lane - jj) + u] = w[u];
+            }
+            __syncwarp();
+            double Sd, Zd;
+            lq_affine_warp_search([&](int j) { return wtmp[j]; }, refit.s64 + i0 + 4 * jj, group, ws, K, refit.T, refit.t_count, lane,
+                                  Sd, Zd);
+            if (lane >= jj && lane < jj + gl) { S_mine = static_cast<float>(Sd); Z_mine = static_cast<float>(static_cast<int32_t>(Zd)); }
+            if (lane == jj) {
+                const int64_t gidx = row * n_groups + (i0 + 4 * jj) / group;
+                refit.scale[gidx] = static_cast<float>(Sd);
+                refit.zero[gidx] = static_cast<int32_t>(Zd);
+            }
+            __syncwarp();
+        }
         if (AFFINE) {
             S = __shfl_sync(0xffffffffu, S_mine, jj);
             Zf = __shfl_sync(0xffffffffu, Z_mine, jj);
@@ -357,23 +389,25 @@ int check_cfg4(const lq_config* cfg) {
     return LQ_OK;
 }
 
-template <int K, bool AFFINE>
+template <int K, bool AFFINE, bool REFIT>
 int launch_inblock(cudaStream_t st, int sm_count, float* Wc, int64_t ldc, int64_t r, int64_t c, int64_t i0, const float* U, int64_t ldu,
-                   const float* grid, const float* scale, const int32_t* zero, int group, int n_groups, const QuantOut& out) {
-    const int smem = (B * B + B) * sizeof(float);
-    static lq_once_per_device attr_set;
-    if (attr_set.first()) {
-        LQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel<K, AFFINE>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    }
+                   const float* grid, const float* scale, const int32_t* zero, int group, int n_groups, const QuantOut& out,
+                   const RefitArgs& refit) {
     // One warp per row.  The kernel is bound by instruction issue, so what matters is the largest number of rows
     // on one SM: up to 32 rows per SM one CTA per SM takes an even share; beyond that, CTAs of 16 rows fill the SMs.
     int warps = 16;
-    if (r <= 32 * static_cast<int64_t>(sm_count)) {
+    if (r <= (REFIT ? 16 : 32) * static_cast<int64_t>(sm_count)) {
         warps = static_cast<int>(lq_ceil_div(r, sm_count));
         if (warps < 4) warps = 4;                  // the 128 reciprocals of the diagonal are computed by the first 128 threads
     }
-    inblock_kernel<K, AFFINE><<<static_cast<unsigned>(lq_ceil_div(r, warps)), warps * 32, smem, st>>>(
-        Wc, ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out);
+    const int smem = (B * B + B) * sizeof(float) + (REFIT ? warps * 3 * group * static_cast<int>(sizeof(float)) : 0);
+    static lq_once_per_device attr_set;
+    if (attr_set.first()) {
+        LQ_CUDA_TRY(cudaFuncSetAttribute(inblock_kernel<K, AFFINE, REFIT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (B * B + B) * static_cast<int>(sizeof(float)) + (REFIT ? 16 * 3 * B * static_cast<int>(sizeof(float)) : 0)));
+    }
+    inblock_kernel<K, AFFINE, REFIT><<<static_cast<unsigned>(lq_ceil_div(r, warps)), warps * 32, smem, st>>>(
+        Wc, ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out, refit);
     LQ_LAUNCH_CHECK();
     return LQ_OK;
 }
@@ -394,6 +428,7 @@ namespace {
 // 1024-column outer block, for groups made of whole outer blocks, and trivially for one group per row.
 bool lazy_group_ok(int64_t g, int64_t c) {
     if (g == c) return true;
+    if (g < B) return g % 4 == 0 && B % g == 0;        // inside a block: refitted by the in-block kernel itself
     if (g % B) return false;
     return (g <= OB && OB % g == 0) || (g % OB == 0);
 }
@@ -477,24 +512,35 @@ int quantize_impl(lq_handle* h, void* stream, const lq_config* cfg, const void* 
         int rc;
         const int64_t o0 = i0 / OB * OB;          // start of the outer block
         out.e_col = static_cast<int>(i0 - o0);
-        if (lazy && i0 % group == 0) {             // (S, Z) of the group that starts here, on the columns as they stand now
+        const bool refit_inside = lazy && group < B;     // groups shorter than a block are refitted by the in-block kernel
+        if (lazy && !refit_inside && i0 % group == 0) {  // (S, Z) of the group that starts here, on the columns as they stand now
             rc = lq_affine_search(h, st, Wc + i0, LQ_F32, r, L.ldc, group, 1, s64 + i0, 1 << cfg->bits, cfg->T, cfg->t_count,
                                   scale + i0 / group, zero + i0 / group, n_groups);
             if (rc) return rc;
         }
-        if (affine) {
+        RefitArgs refit = {};
+        if (refit_inside) { refit.s64 = s64; refit.scale = scale; refit.zero = zero; refit.T = cfg->T; refit.t_count = cfg->t_count; }
+#define LQ_IB(KK, AFF, RF) launch_inblock<KK, AFF, RF>(st, h->sm_count, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out, refit)
+        if (refit_inside) {
             switch (cfg->bits) {
-                case 2: rc = launch_inblock<4, true>(st, h->sm_count, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
-                case 3: rc = launch_inblock<8, true>(st, h->sm_count, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
-                default: rc = launch_inblock<16, true>(st, h->sm_count, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
+                case 2: rc = LQ_IB(4, true, true); break;
+                case 3: rc = LQ_IB(8, true, true); break;
+                default: rc = LQ_IB(16, true, true); break;
+            }
+        } else if (affine) {
+            switch (cfg->bits) {
+                case 2: rc = LQ_IB(4, true, false); break;
+                case 3: rc = LQ_IB(8, true, false); break;
+                default: rc = LQ_IB(16, true, false); break;
             }
         } else {
             switch (cfg->bits) {
-                case 2: rc = launch_inblock<4, false>(st, h->sm_count, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
-                case 3: rc = launch_inblock<8, false>(st, h->sm_count, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
-                default: rc = launch_inblock<16, false>(st, h->sm_count, Wc, L.ldc, r, c, i0, U, ldu, grid, scale, zero, group, n_groups, out); break;
+                case 2: rc = LQ_IB(4, false, false); break;
+                case 3: rc = LQ_IB(8, false, false); break;
+                default: rc = LQ_IB(16, false, false); break;
             }
         }
+#undef LQ_IB
         if (rc) return rc;
         // Lazy update (Algorithm 1 line 20) in two levels.  The columns that the next blocks of
         // this outer block are about to quantise get this block's errors now (K = 128); the columns

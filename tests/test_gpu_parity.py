@@ -542,7 +542,8 @@ def test_chained_affine(lq, h):
     assert abs(mine.sum() / theirs.sum() - 1) <= 5 * LOSS_TOL
 
 
-@pytest.mark.parametrize("r,c,group", [(96, 1024, 128), (64, 1536, 256), (32, 2048, 1024), (48, 640, 0)])
+@pytest.mark.parametrize("r,c,group", [(96, 1024, 128), (64, 1536, 256), (32, 2048, 1024), (48, 640, 0),
+                                       (64, 1280, 64), (40, 384, 32)])       # groups shorter than a block: refitted inside the in-block kernel
 def test_chained_affine_lazy_refit(lq, h, r, c, group):
     """(S, Z) of a group fitted when the column loop reaches it (lq_quantize_layer_lazy); c = 1536 and 2048 have a
     second 1024-column outer block, so the far update is in the path of the columns that get refitted."""
@@ -578,14 +579,14 @@ def test_chained_affine_lazy_refit(lq, h, r, c, group):
 
 
 def test_lazy_refit_rejects_groups_it_cannot_place(lq, h):
-    cfg = lq.Config.make(grid="affine", bits=4, p=4.0, group=64, T=45, t=9)       # shorter than a block
-    r, c = 8, 256
+    cfg = lq.Config.make(grid="affine", bits=4, p=4.0, group=192, T=45, t=9)      # neither inside a block nor made of blocks that tile 1024
+    r, c = 8, 384
     W = torch.zeros(r, c, device="cuda")
     U = torch.eye(c, device="cuda")
     dinv = torch.ones(c, device="cuda")
-    scale = torch.empty(r, c // 64, device="cuda")
-    zero = torch.empty(r, c // 64, dtype=torch.int32, device="cuda")
     codes = torch.empty(r, c, dtype=torch.uint8, device="cuda")
+    scale = torch.empty(r, c // 192, device="cuda")
+    zero = torch.empty(r, c // 192, dtype=torch.int32, device="cuda")
     ws = ws_for(lq, lq.lq_quantize_layer_lazy_workspace(cfg, r, c))
     with pytest.raises(lq.LQError) as e:
         lq.lq_quantize_layer_lazy(h, cfg, W, U, dinv, scale, zero, codes, ws)
