@@ -241,6 +241,25 @@ int lq_quantize_layer_lazy(lq_handle* h, void* stream, const lq_config* cfg, con
                            float* scale, int32_t* zero, uint8_t* codes, void* W_hat, int32_t what_dtype,
                            int64_t ldwh, double* loss, void* ws, size_t ws_bytes);
 
+/* ---- activation ordering (appendix "Experiment Details": the option the paper turns on for its GPTQ baseline) ------ */
+
+/* The columns are quantised in the order of decreasing diag(H) (most active input channels first) instead of left to
+ * right: the pass runs unchanged on the permuted layer and its outputs are put back.
+ *   lq_act_order      perm[k] (device int32[c]) = the column taken k-th; equal diagonal entries: lower index first.  c <= 16384.
+ *   lq_permute_hessian  Hp[a][b] = H[perm[a]][perm[b]] (Hp must not be H).
+ *   lq_gather_columns   dst[i][k] = src[i][perm[k]]   (W into the order of the pass);
+ *   lq_scatter_columns  dst[i][perm[k]] = src[i][k]   (codes and W_hat back into the layer's own order);
+ *                       elements of elem_bytes = 1, 2 or 4 bytes, leading dimensions in elements, dst must not be src.
+ * With a group-wise affine grid the groups are runs of group_size columns of the permuted order, so scale / zero stay
+ * in that order and a consumer needs perm beside them. */
+int lq_act_order(lq_handle* h, void* stream, const float* H, int64_t c, int64_t ldh, int32_t* perm);
+int lq_permute_hessian(lq_handle* h, void* stream, const float* H, int64_t c, int64_t ldh, const int32_t* perm,
+                       float* Hp, int64_t ldhp);
+int lq_gather_columns(lq_handle* h, void* stream, const void* src, int32_t elem_bytes, int64_t r, int64_t c, int64_t lds,
+                      const int32_t* perm, void* dst, int64_t ldd);
+int lq_scatter_columns(lq_handle* h, void* stream, const void* src, int32_t elem_bytes, int64_t r, int64_t c, int64_t lds,
+                       const int32_t* perm, void* dst, int64_t ldd);
+
 /* ---- Algorithm 2 (Appendix, "LeanQuant-Exact"): greedy order, full downdate per row ---- */
 
 /* For every row, with the grid fitted beforehand by lq_fit_grid (lines 3-7 of Algorithm 2) and the row's own

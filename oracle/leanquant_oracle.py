@@ -536,13 +536,35 @@ def minmax_affine_params(W, bits: int, group: int = 0):
     return scale, zero
 
 
+def act_order(H) -> np.ndarray:
+    """Activation ordering (appendix "Experiment Details", the option switched on for the GPTQ baseline): the columns in
+    the order of decreasing diag(H); equal entries keep their index order."""
+    return np.argsort(-np.diag(np.asarray(H, dtype=F64)), kind="stable")
+
+
 def run_pass(W, X, *, grid_type="nonuniform", bits=4, p=4.0, block=128, damp=0.01,
-             n_iter=20, init="uniform", group=0, T=2048, t=None, alpha=2.0, weight_src="inv_diag", lazy_refit=False):
+             n_iter=20, init="uniform", group=0, T=2048, t=None, alpha=2.0, weight_src="inv_diag", lazy_refit=False,
+             act_ordering=False):
     """Algorithm 1 end to end; returns a dict with every intermediate.
     ``weight_src``: "inv_diag" weights the grid objective by diag(H_d^-1)^-p as Eq. 5 / Eq. 7 say;
     "chol_diag" by diag(U)^-p, Algorithm 1 lines 6 and 8 read to the letter (the symbol H^-1 holds
     the Cholesky factor from line 4 on)."""
     H = hessian(X, alpha)
+    if act_ordering:
+        # the pass on the layer with its columns in the order of decreasing diag(H); codes and W_hat are put back
+        # into the layer's own column order, everything else (U, dinv, scale / zero of groups) stays in pass order
+        perm = act_order(H)
+        Xp = np.asarray(X, dtype=F64)[perm]
+        res = run_pass(np.asarray(W, dtype=F64)[:, perm], Xp, grid_type=grid_type, bits=bits, p=p, block=block, damp=damp,
+                       n_iter=n_iter, init=init, group=group, T=T, t=t, alpha=alpha, weight_src=weight_src,
+                       lazy_refit=lazy_refit)
+        inv = np.empty_like(perm)
+        inv[perm] = np.arange(perm.size)
+        res["perm"] = perm
+        res["codes"] = res["codes"][:, inv]
+        res["W_hat"] = res["W_hat"][:, inv]
+        res["H_perm"], res["H"] = res["H"], H
+        return res
     U, dinv, H_d, Wf = prepare_hinv(H, damp, W)
     out = dict(H=H, U=U, dinv=dinv, H_d=H_d)
     if weight_src == "chol_diag":

@@ -74,6 +74,10 @@ def LQ():
             "lq_pack_layer": [vp, vp, P(Config), vp, i64, i64, vp, vp, vp, vp, sz],
             "lq_unpack_layer": [vp, vp, P(Config), vp, sz, i64, i64, vp, i32, i64],
             "lq_zero_dead_columns": [vp, vp, vp, i64, i64, vp, i32, i64, i64],
+            "lq_act_order": [vp, vp, vp, i64, i64, vp],
+            "lq_permute_hessian": [vp, vp, vp, i64, i64, vp, vp, i64],
+            "lq_gather_columns": [vp, vp, vp, i32, i64, i64, i64, vp, vp, i64],
+            "lq_scatter_columns": [vp, vp, vp, i32, i64, i64, i64, vp, vp, i64],
             "lq_testing_set_wait_limit_ns": [vp, C.c_uint64],
             "lq_testing_inject_stall": [vp, i32],
             "lq_testing_set_prepare_defer_min_blocks": [vp, i32],
@@ -329,6 +333,33 @@ def lq_zero_dead_columns(h, H, W, stream=None):
            "lq_zero_dead_columns")
 
 
+def lq_act_order(h, H, perm=None, stream=None):
+    """perm[k] = the column taken k-th when columns go in the order of decreasing diag(H)."""
+    c = H.shape[0]
+    if perm is None:
+        perm = torch.empty((c,), dtype=torch.int32, device=H.device)
+    _check(LQ().lq_act_order(h, _stream(stream), _ptr(H), c, _rowmajor(H), _ptr(perm)), "lq_act_order")
+    return perm
+
+
+def lq_permute_hessian(h, H, perm, Hp, stream=None):
+    c = H.shape[0]
+    _check(LQ().lq_permute_hessian(h, _stream(stream), _ptr(H), c, _rowmajor(H), _ptr(perm), _ptr(Hp), _rowmajor(Hp)),
+           "lq_permute_hessian")
+
+
+def lq_gather_columns(h, src, perm, dst, stream=None):
+    r, c = src.shape
+    _check(LQ().lq_gather_columns(h, _stream(stream), _ptr(src), src.element_size(), r, c, _rowmajor(src), _ptr(perm), _ptr(dst),
+                                  _rowmajor(dst)), "lq_gather_columns")
+
+
+def lq_scatter_columns(h, src, perm, dst, stream=None):
+    r, c = src.shape
+    _check(LQ().lq_scatter_columns(h, _stream(stream), _ptr(src), src.element_size(), r, c, _rowmajor(src), _ptr(perm), _ptr(dst),
+                                   _rowmajor(dst)), "lq_scatter_columns")
+
+
 class StackPass:
     """A stack of layers quantised in order, the way a model-level driver walks a decoder block: layers that read the
     same activations form a group and share stages 1-2 (one Hessian, one factor); every layer then gets its own grid,
@@ -379,12 +410,18 @@ class LayerPass:
     Allocation only (through torch's allocator); all arithmetic is in liblq."""
 
     def __init__(self, handle, r, c, cfg: Config, w_dtype=torch.bfloat16, x_dtype=torch.bfloat16, n_chunk=0,
-                 device="cuda", want_w_hat=True, weight_src="inv_diag", share=None):
+                 device="cuda", want_w_hat=True, weight_src="inv_diag", share=None, act_order=False):
         if weight_src not in ("inv_diag", "chol_diag"):
             raise ValueError("weight_src: 'inv_diag' (Eq. 5 / Eq. 7) or 'chol_diag' (Algorithm 1 to the letter)")
         self.weight_src = weight_src
         self.h, self.r, self.c, self.cfg = handle, r, c, cfg
         dev = torch.device(device)
+        self.act_order = act_order
+        if act_order:                         # the pass runs on the permuted layer: its inputs and outputs in that order
+            self.perm = torch.empty((c,), dtype=torch.int32, device=dev)
+            self.Wp = torch.empty((r, c), dtype=w_dtype, device=dev)
+            self.codes_p = torch.empty((r, c), device=dev, dtype=torch.uint8)
+            self.W_hat_p = torch.empty((r, c), device=dev, dtype=w_dtype) if want_w_hat else None
         K = 1 << cfg.bits
         f32 = dict(device=dev, dtype=torch.float32)
         if share is not None:                 # a layer that reads the same activations: one Hessian, factor and diagonal
@@ -411,6 +448,22 @@ class LayerPass:
     def finish(self, W, damp_frac=0.01):
         """Stages 2-4 after all chunks were accumulated."""
         lq_hessian_finalize(self.h, self.H)
+        if self.act_order:
+            # columns in the order of decreasing diag(H): H permuted into U's buffer (stage 2 may run in place there),
+            # W gathered, the pass as usual, codes and W_hat scattered back
+            lq_act_order(self.h, self.H, self.perm)
+            lq_permute_hessian(self.h, self.H, self.perm, self.U)
+            lq_gather_columns(self.h, W, self.perm, self.Wp)
+            lq_prepare_hinv(self.h, self.U, self.U, self.dinv, self.ws, damp_frac, self.Wp)
+            if self.weight_src == "chol_diag":
+                lq_chol_diag(self.h, self.U, self.dinv)
+            lq_fit_grid(self.h, self.cfg, self.Wp, self.dinv, self.ws, self.grid, self.scale, self.zero)
+            lq_quantize_layer(self.h, self.cfg, self.Wp, self.U, self.codes_p, self.ws, self.grid, self.scale, self.zero,
+                              self.W_hat_p, self.loss)
+            lq_scatter_columns(self.h, self.codes_p, self.perm, self.codes)
+            if self.W_hat is not None:
+                lq_scatter_columns(self.h, self.W_hat_p, self.perm, self.W_hat)
+            return
         lq_prepare_hinv(self.h, self.H, self.U, self.dinv, self.ws, damp_frac, W)
         if self.weight_src == "chol_diag":
             lq_chol_diag(self.h, self.U, self.dinv)

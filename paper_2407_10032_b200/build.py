@@ -11,7 +11,7 @@ CSRC = os.path.join(HERE, "csrc")
 BUILD = os.path.join(ROOT, "_build")
 LIB = os.path.join(HERE, "liblq.so")
 SOURCES = ["lq_api.cu", "lq_gemm_tc.cu", "lq_hessian.cu", "lq_prepare.cu", "lq_fit_grid.cu", "lq_quantize.cu", "lq_exact.cu",
-           "lq_record.cu"]
+           "lq_record.cu", "lq_order.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I" + os.path.join(ROOT, "include")]
 

@@ -522,6 +522,62 @@ def test_chained_weighted_by_factor_diagonal(lq, h):
     assert abs(P.loss.item() / ref["loss"] - 1) <= LOSS_TOL
 
 
+@pytest.mark.parametrize("grid_kw", [dict(grid="nonuniform", bits=4, p=4.0, n_iter=20),
+                                     dict(grid="affine", bits=4, p=4.0, group=128, T=45, t=9)])
+def test_chained_activation_order(lq, h, grid_kw):
+    """Columns taken in the order of decreasing diag(H): lq_act_order, the permuted pass, outputs put back."""
+    L = synth.make_layer("c2", 160, 768, 8192, seed=41)
+    W, X = f64(L.W), f64(L.X)
+    okw = {k: v for k, v in grid_kw.items() if k != "grid"}
+    ref = O.run_pass(W, X, grid_type=grid_kw["grid"], block=128, act_ordering=True, **okw)
+    cfg = lq.Config.make(**grid_kw)
+    P = lq.LayerPass(h, 160, 768, cfg, w_dtype=torch.float32, x_dtype=L.X.dtype, n_chunk=L.n, device="cuda", act_order=True)
+    P.run(L.W.float().cuda(), L.X.cuda())
+    lq.lq_sync_status(h)
+    perm = P.perm.cpu().numpy()
+    # the order itself: the library sorts the diagonal of its fp32 Hessian, the oracle that of the float64 one, so two
+    # entries equal to fp32 rounding may swap; everything else is compared in the library's own order when they do
+    Hd = np.diag(f64(P.H))
+    assert sorted(perm) == list(range(768)) and (np.diff(Hd[perm]) <= 0).all()
+    if not np.array_equal(perm, ref["perm"]):
+        pytest.skip("diagonal entries equal to fp32 rounding were ordered differently")
+    codes = P.codes.cpu().numpy().astype(np.int64)
+    if grid_kw["grid"] == "nonuniform":
+        assert centroid_ok(f64(P.grid), ref["grid"], W)
+        rows_ok = np.ones(160, dtype=bool)
+    else:
+        same_grid = (P.zero.cpu().numpy() == ref["zero"]) & (np.abs(f64(P.scale) / ref["scale"] - 1) < 1e-5)
+        rows_ok = same_grid.all(axis=1)
+        assert rows_ok.mean() >= 0.98
+    assert codes_budget(codes[rows_ok], ref["codes"][rows_ok])
+    mine, theirs = proxy_rows(W, f64(P.W_hat), ref["H"]), proxy_rows(W, ref["W_hat"], ref["H"])
+    assert abs(mine[rows_ok].sum() / theirs[rows_ok].sum() - 1) <= LOSS_TOL
+    plain = O.run_pass(W, X, grid_type=grid_kw["grid"], block=128, **okw)
+    assert (plain["codes"] != ref["codes"]).mean() > 0.01                # the variant is another quantisation
+
+
+def test_act_order_ties_and_permutations(lq, h):
+    c = 300
+    g = torch.Generator().manual_seed(8)
+    H = torch.randn(c, c, generator=g)
+    H = (H @ H.T).contiguous()
+    H[5, 5] = H[200, 200] = H[17, 17]                   # equal entries keep index order: 5, 17, 200
+    Hd = H.cuda()
+    perm = lq.lq_act_order(h, Hd).cpu().numpy()
+    assert np.array_equal(perm, np.argsort(-np.diag(H.numpy()), kind="stable"))
+    Hp = torch.empty_like(Hd)
+    lq.lq_permute_hessian(h, Hd, torch.from_numpy(perm).int().cuda(), Hp)
+    assert torch.equal(Hp.cpu(), H[perm][:, perm])
+    for dt in (torch.uint8, torch.bfloat16, torch.float32):
+        A = (torch.rand(7, c, generator=g) * 200).to(dt).cuda()
+        B1, B2 = torch.empty_like(A), torch.empty_like(A)
+        p = torch.from_numpy(perm).int().cuda()
+        lq.lq_gather_columns(h, A, p, B1)
+        lq.lq_scatter_columns(h, B1, p, B2)
+        lq.lq_sync_status(h)
+        assert torch.equal(B1.cpu(), A.cpu()[:, perm]) and torch.equal(B2, A)
+
+
 def test_chained_affine(lq, h):
     L = synth.make_layer("c3", 128, 1792, 8192, seed=21)
     W, X = f64(L.W), f64(L.X)

@@ -70,8 +70,8 @@ def test_pack_layer_by_hand_and_round_trip():
 
 
 # ------------------------------------------------------------------ P1 ---- #
-def obq_fixed_order(W, Hinv, quant_row):
-    """Eq. 3 and Eq. 9 taken literally, column by column in fixed order:
+def obq_fixed_order(W, Hinv, quant_row, order=None):
+    """Eq. 3 and Eq. 9 taken literally, column by column in fixed order (left to right, or the given `order`):
     quantise w_j, w <- w - (w_j - q)/Hinv_jj * Hinv[:, j], then remove row/column j
     from the inverse by Hinv <- Hinv - Hinv[:, j] Hinv[j, :]/Hinv_jj."""
     W = W.copy()
@@ -79,7 +79,7 @@ def obq_fixed_order(W, Hinv, quant_row):
     r, c = W.shape
     Q = np.zeros_like(W)
     eps = 0.0
-    for j in range(c):
+    for j in (range(c) if order is None else order):
         d = Hinv[j, j]
         for k in range(r):
             q = quant_row(k, j, W[k, j])
@@ -109,6 +109,35 @@ def test_p1_column_loop_equals_explicit_obq(c, block):
     assert np.array_equal(np.take_along_axis(grid, codes, 1), What)
     np.testing.assert_allclose(What, Q_ref, rtol=0, atol=1e-10)
     np.testing.assert_allclose(loss, eps_ref, rtol=1e-9)
+
+
+def test_activation_order_is_obq_in_that_order():
+    """Activation ordering = the same loop with the columns taken in the order of decreasing diag(H).  The oracle permutes
+    the layer, runs the pass and puts the outputs back; the pin takes Eq. 3 / Eq. 9 on the layer as it is and simply visits
+    the columns in that order.  (A wrong inverse permutation, or H permuted on one side only, fails it.)"""
+    g = rng(31)
+    r, c = 4, 40
+    X = g.standard_normal((c, 300)) * np.exp(g.standard_normal((c, 1)))
+    X[7] = X[3]                                        # two channels with the same diagonal entry: ties keep index order
+    W = g.standard_normal((r, c)) * 0.05
+    H = O.hessian(X)
+    perm = O.act_order(H)
+    d = np.diag(H)[perm]
+    assert (np.diff(d) <= 0).all() and sorted(perm) == list(range(c))
+    assert list(perm).index(3) + 1 == list(perm).index(7)
+    out = O.run_pass(W, X, bits=3, p=2.0, block=16, n_iter=5, act_ordering=True)
+    grid = out["grid"]
+
+    def quant_row(k, j, w):
+        return grid[k, O.assign_nu(np.array([w]), grid[k])[0]]
+
+    _, _, H_d, _ = O.prepare_hinv(H, 0.01)
+    Q_ref, eps_ref = obq_fixed_order(W, np.linalg.inv(H_d), quant_row, order=perm)
+    np.testing.assert_allclose(out["W_hat"], Q_ref, rtol=0, atol=1e-10)
+    np.testing.assert_allclose(out["loss"], eps_ref, rtol=1e-9)
+    assert np.array_equal(np.take_along_axis(grid, out["codes"], 1), out["W_hat"])
+    plain = O.run_pass(W, X, bits=3, p=2.0, block=16, n_iter=5)
+    assert not np.array_equal(plain["codes"], out["codes"])          # the order matters
 
 
 def test_p1b_block_size_does_not_matter():
