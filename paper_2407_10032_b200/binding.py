@@ -11,7 +11,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_LIB_PATH = os.path.join(_HERE, "liblq.so")
+# LQ_LIBRARY_VARIANT=debug selects the build with address checks in the kernels (liblq_debug.so, see build.py)
+_LIB_PATH = os.path.join(_HERE, "liblq_debug.so" if os.environ.get("LQ_LIBRARY_VARIANT") == "debug" else "liblq.so")
 _lib = None
 
 LQ_F32, LQ_BF16 = 0, 1

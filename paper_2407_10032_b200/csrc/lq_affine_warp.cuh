@@ -27,7 +27,7 @@ __device__ __forceinline__ AffScore aff_score_setup(double S, double Z, double d
 __device__ __forceinline__ float aff_score32(const float2* __restrict__ ws, int group, const AffScore& a, float Km1f) {
     float a0 = 0.0f, a1 = 0.0f;
     for (int j = 0; j < group; j += 2) {
-        const float4 p2 = *reinterpret_cast<const float4*>(ws + j);          // two (x, s) pairs
+        const float4 p2 = LQ_AT(reinterpret_cast<const float4*>(ws + j));    // two (x, s) pairs
         // clamp to [0, K - 1] and round: the clamp rides on the multiply-add as a saturation of u / (K - 1) to [0, 1]
         // (a weight within rounding of a tie may take the other neighbour, which leaves its error where it was)
         const float q0 = rintf(__saturatef(fmaf(p2.x, a.rS, a.c0)) * Km1f);
@@ -69,8 +69,8 @@ __device__ __forceinline__ void lq_affine_warp_search(WAt w_at, const double* __
         const float w = w_at(j);
         mn = fminf(mn, w);
         mx = fmaxf(mx, w);
-        smax = fmax(smax, sp[j]);
-        ssum += sp[j];
+        smax = fmax(smax, LQ_AT(sp + j));
+        ssum += LQ_AT(sp + j);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -81,7 +81,7 @@ __device__ __forceinline__ void lq_affine_warp_search(WAt w_at, const double* __
     }
     const double sinv = smax > 0.0 ? 1.0 / smax : 1.0;
     const float sum_s = static_cast<float>(ssum * sinv);
-    for (int j = lane; j < group; j += 32) ws[j] = make_float2(w_at(j) - mn, static_cast<float>(sp[j] * sinv));
+    for (int j = lane; j < group; j += 32) LQ_AT(ws + j) = make_float2(w_at(j) - mn, static_cast<float>(LQ_AT(sp + j) * sinv));
     __syncwarp();
 
     const double dmn = mn, dmx = mx, R = dmx - dmn;
@@ -116,7 +116,7 @@ __device__ __forceinline__ void lq_affine_warp_search(WAt w_at, const double* __
             double q = rint(w / S) + Z;
             q = fmin(fmax(q, 0.0), Km1);
             const double d = (q - Z) * S - w;
-            loss += sp[j] * (d * d);
+            loss += LQ_AT(sp + j) * (d * d);
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);

@@ -42,6 +42,73 @@ __device__ __forceinline__ void lq_report(lq_dev_status* st, int code, long long
     if (atomicCAS(&st->code, 0, code) == 0) st->info = info;
 }
 
+// ---- debug build with address checks (-DLQ_DEBUG_BOUNDS) ------------------------------------------------------
+// Every entry point registers the byte ranges of the buffers it was given (and of its workspace) in a small device
+// table before it launches anything; the kernels then take each global or shared-memory address whose index derives
+// from r, c, n, a leading dimension, a group or a block offset through LQ_AT(pointer): an address inside a registered
+// range (or inside the CTA's shared-memory window) is used as it is, any other one records LQ_ERR_INVALID_ARG in the
+// handle's status word (info = source line << 40 | low 40 bits of the address) and the access goes to a scratch
+// word instead -- nothing traps and nothing touches memory the caller did not hand over.  In a normal build LQ_AT(p)
+// is *(p) and the registration macros vanish.  The tensor-core contraction needs none of this: its global accesses are
+// TMA copies, which the hardware clips to the tensor map.
+#ifdef LQ_DEBUG_BOUNDS
+constexpr int LQ_DBG_MAX_RANGES = 24;
+struct lq_dbg_table {
+    unsigned long long lo[LQ_DBG_MAX_RANGES], hi[LQ_DBG_MAX_RANGES];
+    int n;
+    lq_dev_status* st;
+};
+// one table and one scratch word per translation unit (the library is built without relocatable device code)
+static __device__ lq_dbg_table lq_dbg_tab;
+static __device__ __align__(16) unsigned char lq_dbg_sink[64];
+
+__device__ __forceinline__ bool lq_dbg_ok(const void* p, size_t bytes, int line) {
+    const unsigned long long a = reinterpret_cast<unsigned long long>(p);
+    if (__isShared(p)) {
+        const unsigned off = static_cast<unsigned>(__cvta_generic_to_shared(p));
+        unsigned total;
+        asm("mov.u32 %0, %%total_smem_size;" : "=r"(total));
+        // the CTA's own shared memory starts behind the kilobyte the system reserves at the front of the window,
+        // which %total_smem_size (static + dynamic) does not count
+        if (off >= 1024u && off - 1024u + bytes <= total) return true;
+    } else if (__isGlobal(p)) {
+        const int n = lq_dbg_tab.n;
+        for (int i = 0; i < n; ++i)
+            if (a >= lq_dbg_tab.lo[i] && a + bytes <= lq_dbg_tab.hi[i]) return true;
+    } else {
+        return true;                       // local memory: the compiler's own
+    }
+    if (lq_dbg_tab.st) lq_report(lq_dbg_tab.st, LQ_ERR_INVALID_ARG, (static_cast<long long>(line) << 40) | static_cast<long long>(a & 0xffffffffffull));
+    return false;
+}
+template <typename T> __device__ __forceinline__ T* lq_dbg_at(T* p, int line) {
+    return lq_dbg_ok(p, sizeof(T), line) ? p : reinterpret_cast<T*>(lq_dbg_sink);
+}
+#define LQ_AT(p) (*lq_dbg_at((p), __LINE__))
+#define LQ_DBG_OK(p, bytes) lq_dbg_ok((p), (bytes), __LINE__)
+
+struct lq_dbg_scope {
+    lq_dbg_table t;
+    cudaStream_t stream;
+    lq_dbg_scope(lq_handle* h, cudaStream_t st) : stream(st) { t.n = 0; t.st = h ? h->dstatus : nullptr; }
+    void reg(const void* p, size_t bytes) {
+        if (!p || !bytes || t.n >= LQ_DBG_MAX_RANGES) return;
+        t.lo[t.n] = reinterpret_cast<unsigned long long>(p);
+        t.hi[t.n] = t.lo[t.n] + bytes;
+        ++t.n;
+    }
+};
+#define LQ_DBG_SCOPE(h, st) lq_dbg_scope lq_dbg_s((h), (st))
+#define LQ_DBG_REG(p, bytes) lq_dbg_s.reg((p), (bytes))
+#define LQ_DBG_COMMIT() cudaMemcpyToSymbolAsync(lq_dbg_tab, &lq_dbg_s.t, sizeof(lq_dbg_table), 0, cudaMemcpyHostToDevice, lq_dbg_s.stream)
+#else
+#define LQ_AT(p) (*(p))
+#define LQ_DBG_OK(p, bytes) (true)
+#define LQ_DBG_SCOPE(h, st) do { } while (0)
+#define LQ_DBG_REG(p, bytes) do { } while (0)
+#define LQ_DBG_COMMIT() do { } while (0)
+#endif
+
 #define LQ_CUDA_TRY(expr)                                   \
     do {                                                    \
         cudaError_t _e = (expr);                            \

@@ -29,7 +29,7 @@ __global__ void log_mean_kernel(const float* __restrict__ dinv, int64_t c, doubl
     __shared__ double red[1024];
     double s = 0.0;
     for (int64_t j = threadIdx.x; j < c; j += blockDim.x) {
-        float d = dinv[j];
+        float d = LQ_AT(dinv + j);
         if (!(d > 0.0f) || !isfinite(d)) { lq_report(st, LQ_ERR_NONFINITE, j); d = 1.0f; }
         s += log(static_cast<double>(d));
     }
@@ -47,13 +47,13 @@ __global__ void sample_weights_kernel(const float* __restrict__ dinv, int64_t c,
                                       double* __restrict__ s) {
     const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (j >= c) return;
-    float d = dinv[j];
+    float d = LQ_AT(dinv + j);
     if (!(d > 0.0f) || !isfinite(d)) d = 1.0f;
-    s[j] = exp(-p * (log(static_cast<double>(d)) - scal[1]));
+    LQ_AT(s + j) = exp(-p * (log(static_cast<double>(d)) - scal[1]));
 }
 
-__device__ __forceinline__ float load_w(const float* p) { return *p; }
-__device__ __forceinline__ float load_w(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+__device__ __forceinline__ float load_w(const float* p) { return LQ_AT(p); }
+__device__ __forceinline__ float load_w(const __nv_bfloat16* p) { return __bfloat162float(LQ_AT(p)); }
 
 // ---------------------------------------------------------------- sorted k-means ----
 // In one dimension the members of a cluster are a contiguous range of the sorted row, so the
@@ -153,20 +153,20 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
 
     for (int64_t row = blockIdx.x; row < r; row += gridDim.x) {
         const T* wp = W + row * ldw;
-        for (int i = tid; i < n; i += KS_THREADS) keys[ks_slot(i)] = i < c ? KeyOf<T>::make(wp[i], i) : KeyOf<T>::pad();
+        for (int i = tid; i < n; i += KS_THREADS) LQ_AT(keys + ks_slot(i)) = i < c ? KeyOf<T>::make(LQ_AT(wp + i), i) : KeyOf<T>::pad();
         __syncthreads();
         bitonic_sort<KeyT>(keys, n, tid);
         // chunk totals, thread-local exclusive prefixes
         dd2 run;
         run.s.hi = run.s.lo = run.sw.hi = run.sw.lo = 0.0;
         for (int q = tid * cpt; q < (tid + 1) * cpt && q < nch; ++q) {
-            coarse[q] = run;
+            LQ_AT(coarse + q) = run;
 #pragma unroll
             for (int e = 0; e < KS_CHUNK; ++e) {
                 const int i = q * KS_CHUNK + e;
                 if (i < c) {
-                    const KeyT key = keys[ks_slot(i)];
-                    const double sv = s64[key_index(key)];
+                    const KeyT key = LQ_AT(keys + ks_slot(i));
+                    const double sv = LQ_AT(s64 + key_index(key));
                     run.s = dd_add_d(run.s, sv);                 // same order and arithmetic as F(b) below
                     run.sw = dd_add_d(run.sw, __dmul_rn(sv, static_cast<double>(key_weight(key))));
                 }
@@ -208,23 +208,23 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
                 v.sw = dd_add(excl.sw, loc[e].sw);
                 tot[lane * (KS_THREADS / 32) + e] = v;
             }
-            if (lane == 31) coarse[nch] = inc;                  // grand total
+            if (lane == 31) LQ_AT(coarse + nch) = inc;          // grand total
         }
         __syncthreads();
         {
             const dd2 off = tot[tid];
             for (int q = tid * cpt; q < (tid + 1) * cpt && q < nch; ++q) {
-                dd2 v = coarse[q];
+                dd2 v = LQ_AT(coarse + q);
                 v.s = dd_add(off.s, v.s);
                 v.sw = dd_add(off.sw, v.sw);
-                coarse[q] = v;
+                LQ_AT(coarse + q) = v;
             }
         }
         __syncthreads();
 
         if (warp == 0) {
             const double lo = static_cast<double>(key_weight(keys[ks_slot(0)]));
-            const double hi = static_cast<double>(key_weight(keys[ks_slot(c - 1)]));
+            const double hi = static_cast<double>(key_weight(LQ_AT(keys + ks_slot(c - 1))));
             if (init == LQ_INIT_UNIFORM) {
                 if (lane < K) g[lane] = lo + (hi - lo) * static_cast<double>(lane) / static_cast<double>(K - 1);   // Eq. 6
             } else if (lane < K) {
@@ -237,11 +237,11 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
                     const int mid = (p0 + p1) >> 1;
                     const int b = mid + 1;                     // cumulative weight of positions 0 .. mid
                     const int q = b / KS_CHUNK, rem = b % KS_CHUNK;
-                    dd f = coarse[q].s;
-                    for (int e = 0; e < rem; ++e) f = dd_add_d(f, s64[key_index(keys[ks_slot(q * KS_CHUNK + e)])]);
+                    dd f = LQ_AT(coarse + q).s;
+                    for (int e = 0; e < rem; ++e) f = dd_add_d(f, LQ_AT(s64 + key_index(LQ_AT(keys + ks_slot(q * KS_CHUNK + e)))));
                     if (f.hi + f.lo >= target) p1 = mid; else p0 = mid + 1;
                 }
-                g[lane] = static_cast<double>(key_weight(keys[ks_slot(p0)]));
+                g[lane] = static_cast<double>(key_weight(LQ_AT(keys + ks_slot(p0))));
             }
             if (lane == 0) {
                 F[0].s.hi = F[0].s.lo = F[0].sw.hi = F[0].sw.lo = 0.0;
@@ -256,7 +256,7 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
                     int b1 = c;                                // first position whose weight exceeds m
                     while (b0 < b1) {
                         const int mid = (b0 + b1) >> 1;
-                        if (static_cast<double>(key_weight(keys[ks_slot(mid)])) > m) b1 = mid; else b0 = mid + 1;
+                        if (static_cast<double>(key_weight(LQ_AT(keys + ks_slot(mid)))) > m) b1 = mid; else b0 = mid + 1;
                     }
                 }
                 // Unchanged boundaries give back the same centroids, and so would every later
@@ -265,10 +265,10 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
                 b_prev = b0;
                 if (lane < K - 1) {
                     const int q = b0 / KS_CHUNK, rem = b0 % KS_CHUNK;
-                    dd2 f = coarse[q];
+                    dd2 f = LQ_AT(coarse + q);
                     for (int e = 0; e < rem; ++e) {
-                        const KeyT key = keys[ks_slot(q * KS_CHUNK + e)];
-                        const double sv = s64[key_index(key)];
+                        const KeyT key = LQ_AT(keys + ks_slot(q * KS_CHUNK + e));
+                        const double sv = LQ_AT(s64 + key_index(key));
                         f.s = dd_add_d(f.s, sv);
                         f.sw = dd_add_d(f.sw, __dmul_rn(sv, static_cast<double>(key_weight(key))));
                     }
@@ -282,7 +282,7 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
                 }
                 __syncwarp();
             }
-            if (lane < K) grid[row * K + lane] = static_cast<float>(g[lane]);
+            if (lane < K) LQ_AT(grid + row * K + lane) = static_cast<float>(g[lane]);
         }
         __syncthreads();
     }
@@ -307,8 +307,8 @@ kmeans_rows_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int64_t c, c
         const T* wp = W + row * ldw;
         float mn = INFINITY, mx = -INFINITY;
         for (int64_t j = tid; j < c; j += KM_THREADS) {
-            const T raw = wp[j];
-            wrow[j] = raw;
+            const T raw = LQ_AT(wp + j);
+            LQ_AT(wrow + j) = raw;
             const float w = load_w(&raw);
             mn = fminf(mn, w);
             mx = fmaxf(mx, w);
@@ -336,7 +336,7 @@ kmeans_rows_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int64_t c, c
             for (int k = 0; k < K; ++k) ns[k] = nsw[k] = 0.0;
             for (int64_t j = tid; j < c; j += KM_THREADS) {
                 const double w = static_cast<double>(load_w(wrow + j));
-                const double sv = s64[j];
+                const double sv = LQ_AT(s64 + j);
                 int a = 0;
 #pragma unroll
                 for (int step = K / 2; step > 0; step >>= 1)
@@ -368,7 +368,7 @@ kmeans_rows_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int64_t c, c
             }
             __syncthreads();
         }
-        if (tid < K) grid[row * K + tid] = static_cast<float>(g[tid]);
+        if (tid < K) LQ_AT(grid + row * K + tid) = static_cast<float>(g[tid]);
         __syncthreads();
     }
 }
@@ -425,7 +425,7 @@ affine_search_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, int group,
     float mn = INFINITY, mx = -INFINITY;
     for (int j = tid; j < group; j += AF_THREADS) {
         float w = load_w(wp + j);
-        wg[j] = w;
+        LQ_AT(wg + j) = w;
         mn = fminf(mn, w);
         mx = fmaxf(mx, w);
     }
@@ -447,8 +447,8 @@ affine_search_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, int group,
             double lo = fmin(dmn, 0.0), hi = fmax(dmx, 0.0);
             double S = 1.0, Z = 0.0;
             if (hi != lo) { S = (hi - lo) / Km1; Z = -rint(lo / S); }
-            scale[out] = static_cast<float>(S);
-            zero[out] = static_cast<int32_t>(Z);
+            LQ_AT(scale + out) = static_cast<float>(S);
+            LQ_AT(zero + out) = static_cast<int32_t>(Z);
         }
         return;
     }
@@ -466,11 +466,11 @@ affine_search_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, int group,
         const double Z = -rint(lo / S);
         double loss = 0.0;
         for (int j = 0; j < group; ++j) {
-            const double w = static_cast<double>(wg[j]);
+            const double w = static_cast<double>(LQ_AT(wg + j));
             double q = rint(w / S) + Z;
             q = fmin(fmax(q, 0.0), Km1);
             const double d = (q - Z) * S - w;
-            loss += sp[j] * (d * d);
+            loss += LQ_AT(sp + j) * (d * d);
         }
         if (loss < my_loss) { my_loss = loss; my_idx = cand; }
     }
@@ -495,8 +495,8 @@ affine_search_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, int group,
             S = (hi - lo) / Km1;
             Z = -rint(lo / S);
         }
-        scale[out] = static_cast<float>(S);
-        zero[out] = static_cast<int32_t>(Z);
+        LQ_AT(scale + out) = static_cast<float>(S);
+        LQ_AT(zero + out) = static_cast<int32_t>(Z);
     }
 }
 
@@ -530,8 +530,8 @@ affine_search_warp_kernel(const T* __restrict__ W, int64_t ldw, int group, int n
     double S, Z;
     lq_affine_warp_search([&](int j) { return load_w(wp + j); }, sp, group, ws, K, Tparts, t_count, lane, S, Z);
     if (lane == 0) {
-        scale[oidx] = static_cast<float>(S);
-        zero[oidx] = static_cast<int32_t>(Z);
+        LQ_AT(scale + oidx) = static_cast<float>(S);
+        LQ_AT(zero + oidx) = static_cast<int32_t>(Z);
     }
 }
 
@@ -583,8 +583,8 @@ affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_group
         const float w = load_w(wp + j);
         mn = fminf(mn, w);
         mx = fmaxf(mx, w);
-        smax = fmax(smax, sp[j]);
-        ssum += sp[j];
+        smax = fmax(smax, LQ_AT(sp + j));
+        ssum += LQ_AT(sp + j);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -603,7 +603,7 @@ affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_group
     __syncthreads();                                  // the scratch is reused below
     const double sinv = smax > 0.0 ? 1.0 / smax : 1.0;
     const float sum_s = static_cast<float>(ssum * sinv);
-    for (int j = tid; j < group; j += nthr) ws[j] = make_float2(load_w(wp + j) - mn, static_cast<float>(sp[j] * sinv));
+    for (int j = tid; j < group; j += nthr) LQ_AT(ws + j) = make_float2(load_w(wp + j) - mn, static_cast<float>(LQ_AT(sp + j) * sinv));
 
     const double dmn = mn, dmx = mx, R = dmx - dmn;
     const double Km1 = static_cast<double>(K - 1);
@@ -613,8 +613,8 @@ affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_group
             double lo = fmin(dmn, 0.0), hi = fmax(dmx, 0.0);
             double S = 1.0, Z = 0.0;
             if (hi != lo) { S = (hi - lo) / Km1; Z = -rint(lo / S); }
-            scale[oidx] = static_cast<float>(S);
-            zero[oidx] = static_cast<int32_t>(Z);
+            LQ_AT(scale + oidx) = static_cast<float>(S);
+            LQ_AT(zero + oidx) = static_cast<int32_t>(Z);
         }
         return;
     }
@@ -638,15 +638,15 @@ affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_group
             z0 = static_cast<int>(Za);
             cnt = max(z0 - static_cast<int>(Zb), 0) + 1;
         }
-        za[u] = z0;
-        off[u] = cnt;
+        LQ_AT(za + u) = z0;
+        LQ_AT(off + u) = cnt;
     }
     __syncthreads();
     {
         const int per = (nu + nthr - 1) / nthr;
         const int lo_u = min(tid * per, nu), hi_u = min(lo_u + per, nu);
         int sum = 0;
-        for (int u = lo_u; u < hi_u; ++u) sum += off[u];
+        for (int u = lo_u; u < hi_u; ++u) sum += LQ_AT(off + u);
         int incl = sum;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -657,11 +657,11 @@ affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_group
         __syncthreads();
         int base = incl - sum;
         for (int w = 0; w < warp; ++w) base += red_i[w];
-        for (int u = lo_u; u < hi_u; ++u) { const int cnt = off[u]; off[u] = base; base += cnt; }
-        if (tid == nthr - 1) off[nu] = base;
+        for (int u = lo_u; u < hi_u; ++u) { const int cnt = LQ_AT(off + u); LQ_AT(off + u) = base; base += cnt; }
+        if (tid == nthr - 1) LQ_AT(off + nu) = base;
     }
     __syncthreads();
-    int P = off[nu];
+    int P = LQ_AT(off + nu);
     if (P > p_max) {                                // cannot happen with the host's bound; never write past the arrays
         if (tid == 0) lq_report(dstatus, LQ_ERR_UNSUPPORTED, gid);
         P = p_max;
@@ -671,10 +671,10 @@ affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_group
         int lo_u = 0, hi_u = nu - 1;
         while (lo_u < hi_u) {                        // the last line whose first class is <= p
             const int mid = (lo_u + hi_u + 1) >> 1;
-            if (off[mid] <= p) lo_u = mid; else hi_u = mid - 1;
+            if (LQ_AT(off + mid) <= p) lo_u = mid; else hi_u = mid - 1;
         }
         u = lo_u;
-        Z = za[u] - (p - off[u]);
+        Z = LQ_AT(za + u) - (p - LQ_AT(off + u));
     };
     const double c_s = R / (dT * Km1);               // S of line u = c_s (T - u)
     const float Km1f = static_cast<float>(K - 1);
@@ -687,7 +687,7 @@ affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_group
         const AffScore as = aff_score_setup(c_s * static_cast<double>(Tparts - u), static_cast<double>(Zi), dmn, Km1);
         float sc = aff_score32(ws, group, as, Km1f);
         if (sc != sc) sc = -INFINITY;                // a NaN score is always re-examined in fp64
-        score[p] = sc;
+        LQ_AT(score + p) = sc;
         best32 = fminf(best32, sc == -INFINITY ? INFINITY : sc);
     }
 #pragma unroll
@@ -697,7 +697,7 @@ affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_group
     for (int w = 0; w < nwarp; ++w) best32 = fminf(best32, red_f[0][w]);
     const float bar32 = aff_bar32(best32, static_cast<float>(R), sum_s);
     for (int p = tid; p < P; p += nthr)
-        if (score[p] <= bar32) list[atomicAdd(&n_list, 1)] = p;
+        if (LQ_AT(score + p) <= bar32) LQ_AT(list + atomicAdd(&n_list, 1)) = p;
     __syncthreads();
     const int n_eval = n_list;
 
@@ -706,7 +706,7 @@ affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_group
     int my_idx = 0x7fffffff;
     for (int i = warp; i < n_eval; i += nwarp) {
         int u, Zi;
-        class_of(list[i], u, Zi);
+        class_of(LQ_AT(list + i), u, Zi);
         const int a = max(0, u - t_count), b = min(t_count, u);
         const double Zd = static_cast<double>(Zi);
         // first t_min on the line with rint(lo / S) >= -Z, i.e. with Z(t_min) <= Z: estimate, then settle exactly
@@ -727,7 +727,7 @@ affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_group
             double q = rint(w / S) + Z;
             q = fmin(fmax(q, 0.0), Km1);
             const double d = (q - Z) * S - w;
-            loss += sp[j] * (d * d);
+            loss += LQ_AT(sp + j) * (d * d);
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
@@ -744,8 +744,8 @@ affine_class_kernel(const T* __restrict__ W, int64_t ldw, int group, int n_group
             const int t_min = my_idx / side;
             params(t_min, my_idx - t_min * side, S, Z);
         }
-        scale[oidx] = static_cast<float>(S);
-        zero[oidx] = static_cast<int32_t>(Z);
+        LQ_AT(scale + oidx) = static_cast<float>(S);
+        LQ_AT(zero + oidx) = static_cast<int32_t>(Z);
     }
 }
 
@@ -784,6 +784,13 @@ int check_cfg(const lq_config* cfg) {
 
 // Sample weights s_j = exp(-p (ln dinv_j - mean ln dinv)) into s64 (c doubles); scal: 256 bytes of scratch.
 int lq_sample_weights(lq_handle* h, cudaStream_t st, const float* dinv, int64_t c, double p, double* scal, double* s64) {
+    {
+        LQ_DBG_SCOPE(h, st);
+        LQ_DBG_REG(dinv, static_cast<size_t>(c) * sizeof(float));
+        LQ_DBG_REG(scal, 256);
+        LQ_DBG_REG(s64, static_cast<size_t>(c) * sizeof(double));
+        LQ_DBG_COMMIT();
+    }
     log_mean_kernel<<<1, 1024, 0, st>>>(dinv, c, scal, h->dstatus);
     LQ_LAUNCH_CHECK();
     sample_weights_kernel<<<static_cast<unsigned>(lq_ceil_div(c, 256)), 256, 0, st>>>(dinv, c, p, scal, s64);
@@ -795,6 +802,14 @@ int lq_sample_weights(lq_handle* h, cudaStream_t st, const float* dinv, int64_t 
 // weights of the n_groups * g columns; (S, Z) of group gi of row i goes to scale / zero [i * out_ld + gi].
 int lq_affine_search(lq_handle* h, cudaStream_t st, const void* W, int32_t w_dtype, int64_t r, int64_t ldw, int64_t g,
                      int n_groups, const double* s64, int K, int T, int t_count, float* scale, int32_t* zero, int64_t out_ld) {
+    {
+        LQ_DBG_SCOPE(h, st);
+        LQ_DBG_REG(W, (static_cast<size_t>(r - 1) * ldw + static_cast<size_t>(g) * n_groups) * (w_dtype == LQ_F32 ? 4 : 2));
+        LQ_DBG_REG(s64, static_cast<size_t>(g) * n_groups * sizeof(double));
+        LQ_DBG_REG(scale, (static_cast<size_t>(r - 1) * out_ld + n_groups) * sizeof(float));
+        LQ_DBG_REG(zero, (static_cast<size_t>(r - 1) * out_ld + n_groups) * sizeof(int32_t));
+        LQ_DBG_COMMIT();
+    }
     int p_max = 0;
     size_t smem_c = 0;
     if (affine_class_plan(K, T, t_count, g, &p_max, &smem_c)) {
@@ -893,6 +908,13 @@ extern "C" int lq_fit_grid(lq_handle* h, void* stream, const lq_config* cfg, con
     if (e) return e;
 
     if (cfg->grid_type == LQ_GRID_NONUNIFORM) {
+        {   // (after lq_sample_weights, which registered its own buffers for its two launches)
+            LQ_DBG_SCOPE(h, st);
+            LQ_DBG_REG(W, (static_cast<size_t>(r - 1) * ldw + c) * (w_dtype == LQ_F32 ? 4 : 2));
+            LQ_DBG_REG(s64, static_cast<size_t>(c) * sizeof(double));
+            LQ_DBG_REG(grid, static_cast<size_t>(r) * (size_t(1) << cfg->bits) * sizeof(float));
+            LQ_DBG_COMMIT();
+        }
 #define LQ_KM(KK)                                                                                                     \
     (w_dtype == LQ_F32 ? launch_kmeans<KK, float>(st, h->sm_count, static_cast<const float*>(W), ldw, r, c, s64, grid, cfg->n_iter, cfg->init) \
                        : launch_kmeans<KK, __nv_bfloat16>(st, h->sm_count, static_cast<const __nv_bfloat16*>(W), ldw, r, c, s64, grid, cfg->n_iter, cfg->init))

@@ -17,10 +17,10 @@ __global__ void split3_kernel(const float* __restrict__ src, int64_t ld, int64_t
     __nv_bfloat16* d1 = d0 + rows * dst_ld;
     __nv_bfloat16* d2 = d1 + rows * dst_ld;
     for (int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < dst_ld; j += (int64_t)gridDim.x * blockDim.x) {
-        float x = j < cols ? s[j] : 0.0f;
+        float x = j < cols ? LQ_AT(s + j) : 0.0f;
         __nv_bfloat16 a, b, c;
         lq_split3(x, a, b, c);
-        d0[j] = a; d1[j] = b; d2[j] = c;
+        LQ_AT(d0 + j) = a; LQ_AT(d1 + j) = b; LQ_AT(d2 + j) = c;
     }
 }
 
@@ -38,11 +38,11 @@ transpose_bf16_kernel(const __nv_bfloat16* __restrict__ src, int64_t lds, int64_
         unsigned short a = 0, b = 0;
         if (tok < n) {
             if (f + 1 < c) {
-                const uint32_t v = *reinterpret_cast<const uint32_t*>(s16 + tok * lds + f);
+                const uint32_t v = LQ_AT(reinterpret_cast<const uint32_t*>(s16 + tok * lds + f));
                 a = static_cast<unsigned short>(v & 0xffffu);
                 b = static_cast<unsigned short>(v >> 16);
             } else if (f < c) {
-                a = s16[tok * lds + f];
+                a = LQ_AT(s16 + tok * lds + f);
             }
         }
         tile[rr][2 * tx] = a;
@@ -54,7 +54,7 @@ transpose_bf16_kernel(const __nv_bfloat16* __restrict__ src, int64_t lds, int64_
         const int64_t f = f0 + ff, tok = t0 + 2 * tx;
         if (f < c && tok < ldd) {          // ldd is even: a pair never straddles the end of a row
             const uint32_t v = static_cast<uint32_t>(tile[2 * tx][ff]) | (static_cast<uint32_t>(tile[2 * tx + 1][ff]) << 16);
-            *reinterpret_cast<uint32_t*>(d16 + f * ldd + tok) = v;
+            LQ_AT(reinterpret_cast<uint32_t*>(d16 + f * ldd + tok)) = v;
         }
     }
 }
@@ -68,7 +68,7 @@ transpose_split3_kernel(const float* __restrict__ src, int64_t lds, int64_t n, i
     const int64_t t0 = (int64_t)blockIdx.x * 32, f0 = (int64_t)blockIdx.y * 32;
     for (int rr = ty; rr < 32; rr += 8) {
         const int64_t tok = t0 + rr, f = f0 + tx;
-        tile[rr][tx] = (tok < n && f < c) ? src[tok * lds + f] : 0.0f;
+        tile[rr][tx] = (tok < n && f < c) ? LQ_AT(src + tok * lds + f) : 0.0f;
     }
     __syncthreads();
     for (int ff = ty; ff < 32; ff += 8) {
@@ -76,9 +76,9 @@ transpose_split3_kernel(const float* __restrict__ src, int64_t lds, int64_t n, i
         if (f < c && tok < ldd) {
             __nv_bfloat16 a, b, cc;
             lq_split3(tile[tx][ff], a, b, cc);
-            dst[f * ldd + tok] = a;
-            dst[(c + f) * ldd + tok] = b;
-            dst[(2 * c + f) * ldd + tok] = cc;
+            LQ_AT(dst + f * ldd + tok) = a;
+            LQ_AT(dst + (c + f) * ldd + tok) = b;
+            LQ_AT(dst + (2 * c + f) * ldd + tok) = cc;
         }
     }
 }
@@ -91,12 +91,12 @@ __global__ void mirror_upper_kernel(float* __restrict__ H, int64_t c, int64_t ld
     const int tx = threadIdx.x, ty = threadIdx.y;   // 32 x 8
     for (int k = ty; k < 32; k += 8) {
         int64_t i = (int64_t)bi * 32 + k, j = (int64_t)bj * 32 + tx;
-        tile[k][tx] = (i < c && j < c) ? H[i * ldh + j] : 0.0f;
+        tile[k][tx] = (i < c && j < c) ? LQ_AT(H + i * ldh + j) : 0.0f;
     }
     __syncthreads();
     for (int k = ty; k < 32; k += 8) {
         int64_t j = (int64_t)bj * 32 + k, i = (int64_t)bi * 32 + tx;   // destination H[j][i]
-        if (j < c && i < c && j > i) H[j * ldh + i] = tile[tx][k];
+        if (j < c && i < c && j > i) LQ_AT(H + j * ldh + i) = tile[tx][k];
     }
 }
 
@@ -136,6 +136,13 @@ extern "C" int lq_hessian_accumulate(lq_handle* h, void* stream, const void* X, 
     if (need && (reinterpret_cast<uintptr_t>(ws) & 15)) return LQ_ERR_INVALID_ARG;
     const int64_t ld = lq_ceil_div(n_chunk, 8) * 8;
     __nv_bfloat16* staged = static_cast<__nv_bfloat16*>(ws);
+    {
+        LQ_DBG_SCOPE(h, st);
+        const size_t xb = x_dtype == LQ_F32 ? 4 : 2;
+        LQ_DBG_REG(X, (static_cast<size_t>((token_major ? n_chunk : c) - 1) * ldx + (token_major ? c : n_chunk)) * xb);
+        LQ_DBG_REG(ws, need);
+        LQ_DBG_COMMIT();
+    }
     if (x_dtype == LQ_BF16) {
         if (!token_major) {
             if (ldx % 8) return LQ_ERR_INVALID_ARG;
@@ -175,6 +182,11 @@ extern "C" int lq_hessian_accumulate(lq_handle* h, void* stream, const void* X, 
 extern "C" int lq_hessian_finalize(lq_handle* h, void* stream, float* H, int64_t c, int64_t ldh) {
     if (!h || !H || c <= 0 || ldh < c) return LQ_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    {
+        LQ_DBG_SCOPE(h, st);
+        LQ_DBG_REG(H, (static_cast<size_t>(c - 1) * ldh + c) * sizeof(float));
+        LQ_DBG_COMMIT();
+    }
     unsigned nb = static_cast<unsigned>(lq_ceil_div(c, 32));
     mirror_upper_kernel<<<dim3(nb, nb), dim3(32, 8), 0, st>>>(H, c, ldh);
     LQ_LAUNCH_CHECK();

@@ -18,23 +18,23 @@ act_order_kernel(const float* __restrict__ H, int c, int64_t ldh, int n, int32_t
     for (int i = tid; i < n; i += KS_THREADS) {
         unsigned long long key = ~0ull;                              // padding sorts last
         if (i < c) {
-            uint32_t u = __float_as_uint(H[static_cast<int64_t>(i) * ldh + i]);
+            uint32_t u = __float_as_uint(LQ_AT(H + static_cast<int64_t>(i) * ldh + i));
             u ^= (u & 0x80000000u) ? 0xffffffffu : 0x80000000u;      // ascending in the value ...
             key = (static_cast<unsigned long long>(~u) << 32) | static_cast<uint32_t>(i);   // ... so descending here
         }
-        keys[ks_slot(i)] = key;
+        LQ_AT(keys + ks_slot(i)) = key;
     }
     __syncthreads();
     bitonic_sort<unsigned long long>(keys, n, tid);
-    for (int i = tid; i < c; i += KS_THREADS) perm[i] = static_cast<int32_t>(keys[ks_slot(i)] & 0xffffffffu);
+    for (int i = tid; i < c; i += KS_THREADS) LQ_AT(perm + i) = static_cast<int32_t>(LQ_AT(keys + ks_slot(i)) & 0xffffffffu);
 }
 
 __global__ void permute_sym_kernel(const float* __restrict__ H, int64_t c, int64_t ldh, const int32_t* __restrict__ perm,
                                    float* __restrict__ Hp, int64_t ldo) {
     const int64_t a = blockIdx.y;
-    const int64_t src_row = perm[a];
+    const int64_t src_row = LQ_AT(perm + a);
     for (int64_t b = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; b < c; b += (int64_t)gridDim.x * blockDim.x)
-        Hp[a * ldo + b] = H[src_row * ldh + perm[b]];
+        LQ_AT(Hp + a * ldo + b) = LQ_AT(H + src_row * ldh + LQ_AT(perm + b));
 }
 
 // gather: dst[i][k] = src[i][perm[k]];  scatter: dst[i][perm[k]] = src[i][k].  Elements of 1, 2 or 4 bytes.
@@ -43,9 +43,9 @@ __global__ void permute_columns_kernel(const E* __restrict__ src, int64_t r, int
                                        E* __restrict__ dst, int64_t ldd) {
     for (int64_t i = blockIdx.y; i < r; i += gridDim.y)
         for (int64_t k = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; k < c; k += (int64_t)gridDim.x * blockDim.x) {
-            const int64_t p = perm[k];
-            if (SCATTER) dst[i * ldd + p] = src[i * lds + k];
-            else dst[i * ldd + k] = src[i * lds + p];
+            const int64_t p = LQ_AT(perm + k);
+            if (SCATTER) LQ_AT(dst + i * ldd + p) = LQ_AT(src + i * lds + k);
+            else LQ_AT(dst + i * ldd + k) = LQ_AT(src + i * lds + p);
         }
 }
 
@@ -55,6 +55,13 @@ int permute_columns(lq_handle* h, void* stream, const void* src, int32_t elem_by
     if (!h || !src || !dst || !perm || r <= 0 || c <= 0 || lds < c || ldd < c || src == dst) return LQ_ERR_INVALID_ARG;
     if (elem_bytes != 1 && elem_bytes != 2 && elem_bytes != 4) return LQ_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    {
+        LQ_DBG_SCOPE(h, st);
+        LQ_DBG_REG(src, (static_cast<size_t>(r - 1) * lds + c) * elem_bytes);
+        LQ_DBG_REG(dst, (static_cast<size_t>(r - 1) * ldd + c) * elem_bytes);
+        LQ_DBG_REG(perm, static_cast<size_t>(c) * sizeof(int32_t));
+        LQ_DBG_COMMIT();
+    }
     dim3 g(static_cast<unsigned>(lq_ceil_div(c, 256) < 64 ? lq_ceil_div(c, 256) : 64), static_cast<unsigned>(r < 65535 ? r : 65535));
     if (elem_bytes == 1)
         permute_columns_kernel<uint8_t, SCATTER><<<g, 256, 0, st>>>(static_cast<const uint8_t*>(src), r, c, lds, perm, static_cast<uint8_t*>(dst), ldd);
@@ -79,6 +86,12 @@ extern "C" int lq_act_order(lq_handle* h, void* stream, const float* H, int64_t 
         LQ_CUDA_TRY(cudaFuncSetAttribute(act_order_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (ORD_MAX_C + ORD_MAX_C / 32) * static_cast<int>(sizeof(unsigned long long))));
     }
+    {
+        LQ_DBG_SCOPE(h, static_cast<cudaStream_t>(stream));
+        LQ_DBG_REG(H, (static_cast<size_t>(c - 1) * ldh + c) * sizeof(float));
+        LQ_DBG_REG(perm, static_cast<size_t>(c) * sizeof(int32_t));
+        LQ_DBG_COMMIT();
+    }
     act_order_kernel<<<1, KS_THREADS, smem, static_cast<cudaStream_t>(stream)>>>(H, static_cast<int>(c), ldh, n, perm);
     LQ_LAUNCH_CHECK();
     return LQ_OK;
@@ -88,6 +101,13 @@ extern "C" int lq_permute_hessian(lq_handle* h, void* stream, const float* H, in
                                   float* Hp, int64_t ldhp) {
     if (!h || !H || !Hp || !perm || c <= 0 || ldh < c || ldhp < c || H == Hp) return LQ_ERR_INVALID_ARG;
     if (c > 65535) return LQ_ERR_UNSUPPORTED;
+    {
+        LQ_DBG_SCOPE(h, static_cast<cudaStream_t>(stream));
+        LQ_DBG_REG(H, (static_cast<size_t>(c - 1) * ldh + c) * sizeof(float));
+        LQ_DBG_REG(Hp, (static_cast<size_t>(c - 1) * ldhp + c) * sizeof(float));
+        LQ_DBG_REG(perm, static_cast<size_t>(c) * sizeof(int32_t));
+        LQ_DBG_COMMIT();
+    }
     dim3 g(static_cast<unsigned>(lq_ceil_div(c, 256) < 64 ? lq_ceil_div(c, 256) : 64), static_cast<unsigned>(c));
     permute_sym_kernel<<<g, 256, 0, static_cast<cudaStream_t>(stream)>>>(H, c, ldh, perm, Hp, ldhp);
     LQ_LAUNCH_CHECK();

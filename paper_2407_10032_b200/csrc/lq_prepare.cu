@@ -50,7 +50,7 @@ __global__ void diag_mean_kernel(const float* __restrict__ H, int64_t c, int64_t
     __shared__ double red[1024];
     double s = 0.0;
     for (int64_t i = threadIdx.x; i < c; i += blockDim.x) {
-        float d = H[i * ldh + i];
+        float d = LQ_AT(H + i * ldh + i);
         s += (d == 0.0f) ? 1.0 : static_cast<double>(d);
     }
     red[threadIdx.x] = s;
@@ -68,8 +68,8 @@ __global__ void zero_dead_columns_kernel(const float* __restrict__ H, int64_t c,
                                          int64_t r, int64_t ldw) {
     const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (j >= c) return;
-    if (H[j * ldh + j] != 0.0f) return;
-    for (int64_t i = blockIdx.y; i < r; i += gridDim.y) W[i * ldw + j] = T(0.0f);
+    if (LQ_AT(H + j * ldh + j) != 0.0f) return;
+    for (int64_t i = blockIdx.y; i < r; i += gridDim.y) LQ_AT(W + i * ldw + j) = T(0.0f);
 }
 
 // A[cp x cp] (fp64): upper triangle of H plus damping; identity on the padding; the strictly
@@ -85,12 +85,12 @@ __global__ void load_damped_kernel(const float* __restrict__ H, int64_t c, int64
         if (i < c && j0 + 3 >= i && j0 < c) {
             float hv[4] = {0.0f, 0.0f, 0.0f, 0.0f};
             if (vec && j0 + 3 < c) {
-                const float4 x = *reinterpret_cast<const float4*>(H + i * ldh + j0);
+                const float4 x = LQ_AT(reinterpret_cast<const float4*>(H + i * ldh + j0));
                 hv[0] = x.x; hv[1] = x.y; hv[2] = x.z; hv[3] = x.w;
             } else {
 #pragma unroll
                 for (int e = 0; e < 4; ++e)
-                    if (j0 + e < c) hv[e] = H[i * ldh + j0 + e];
+                    if (j0 + e < c) hv[e] = LQ_AT(H + i * ldh + j0 + e);
             }
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
@@ -104,8 +104,8 @@ __global__ void load_damped_kernel(const float* __restrict__ H, int64_t c, int64
         }
         if (i >= c && i >= j0 && i < j0 + 4) v[i - j0] = 1.0;        // identity on the padding
         double2* out = reinterpret_cast<double2*>(A + i * cp + j0);  // cp is a multiple of 128
-        out[0] = make_double2(v[0], v[1]);
-        out[1] = make_double2(v[2], v[3]);
+        LQ_AT(out) = make_double2(v[0], v[1]);
+        LQ_AT(out + 1) = make_double2(v[2], v[3]);
     }
 }
 
@@ -116,6 +116,7 @@ __device__ __forceinline__ void dmma(double& c0, double& c1, double a, double b)
 }
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc) {
     const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+    if (!LQ_DBG_OK(gsrc, 16) || !LQ_DBG_OK(smem_dst, 16)) return;       // debug build: a copy outside the registered buffers is skipped
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
@@ -225,15 +226,15 @@ __device__ __forceinline__ void gemm_tile(const double* __restrict__ A, int64_t 
             v.y = alpha * acc[i][j][1];
             double* cp = o.C + (int64_t)row * o.ldc + col;
             if (beta != 0.0) {
-                const double2 old = *reinterpret_cast<const double2*>(cp);
+                const double2 old = LQ_AT(reinterpret_cast<const double2*>(cp));
                 v.x += beta * old.x;
                 v.y += beta * old.y;
             }
-            *reinterpret_cast<double2*>(cp) = v;
-            if (o.C2) *reinterpret_cast<double2*>(o.C2 + (int64_t)row * o.ldc2 + col) = v;
+            LQ_AT(reinterpret_cast<double2*>(cp)) = v;
+            if (o.C2) LQ_AT(reinterpret_cast<double2*>(o.C2 + (int64_t)row * o.ldc2 + col)) = v;
             if (o.Ct) {
-                o.Ct[(int64_t)col * o.ldct + row] = v.x;
-                o.Ct[(int64_t)(col + 1) * o.ldct + row] = v.y;
+                LQ_AT(o.Ct + (int64_t)col * o.ldct + row) = v.x;
+                LQ_AT(o.Ct + (int64_t)(col + 1) * o.ldct + row) = v.y;
             }
         }
     }
@@ -333,7 +334,7 @@ slice_rows_kernel(const double* __restrict__ P, int64_t ldp, int K, int* __restr
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
         const int kx = threadIdx.x + 256 * u;
-        v[u] = kx < K ? p[kx] : 0.0;
+        v[u] = kx < K ? LQ_AT(p + kx) : 0.0;
         mx = fmax(mx, fabs(v[u]));
     }
 #pragma unroll
@@ -344,7 +345,7 @@ slice_rows_kernel(const double* __restrict__ P, int64_t ldp, int K, int* __restr
 #pragma unroll
     for (int w = 1; w < 8; ++w) mx = fmax(mx, red[w]);
     const int e = isfinite(mx) ? exp_for(mx) : 0;
-    if (threadIdx.x == 0) ex[row] = e;
+    if (threadIdx.x == 0) LQ_AT(ex + row) = e;
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
         const int kx = threadIdx.x + 256 * u;
@@ -352,7 +353,7 @@ slice_rows_kernel(const double* __restrict__ P, int64_t ldp, int K, int* __restr
         __nv_bfloat16 d[NSL];
         digits_of(isfinite(v[u]) ? v[u] : 0.0, e, d);
 #pragma unroll
-        for (int s = 0; s < NSL; ++s) SL[(s * slice_rows + row) * LDP + kx] = d[s];
+        for (int s = 0; s < NSL; ++s) LQ_AT(SL + (s * slice_rows + row) * LDP + kx) = d[s];
     }
 }
 
@@ -362,8 +363,8 @@ col_exp_kernel(const double* __restrict__ A, int64_t cp, int64_t row0, int K, in
     const int64_t j = col0 + blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (j >= cp) return;
     double mx = 0.0;
-    for (int kx = 0; kx < K; ++kx) mx = fmax(mx, fabs(A[(row0 + kx) * cp + j]));
-    ex[j] = isfinite(mx) ? exp_for(mx) : 0;
+    for (int kx = 0; kx < K; ++kx) mx = fmax(mx, fabs(LQ_AT(A + (row0 + kx) * cp + j)));
+    LQ_AT(ex + j) = isfinite(mx) ? exp_for(mx) : 0;
 }
 
 // Slices of those columns, transposed: SL[s][j][kx] = digit s of A[row0 + kx][j].  64 x 64 tiles through shared memory.
@@ -376,7 +377,7 @@ slice_cols_kernel(const double* __restrict__ A, int64_t cp, int64_t row0, int K,
     for (int idx = threadIdx.x; idx < 64 * 64; idx += 256) {
         const int a = idx >> 6, b = idx & 63;            // row k0 + a, column j0 + b
         const int64_t j = j0 + b;
-        tile[a][b] = (k0 + a < K && j < cp) ? A[(row0 + k0 + a) * cp + j] : 0.0;
+        tile[a][b] = (k0 + a < K && j < cp) ? LQ_AT(A + (row0 + k0 + a) * cp + j) : 0.0;
     }
     __syncthreads();
     for (int idx = threadIdx.x; idx < 64 * 64; idx += 256) {
@@ -385,9 +386,9 @@ slice_cols_kernel(const double* __restrict__ A, int64_t cp, int64_t row0, int K,
         if (j >= cp || k0 + a >= K) continue;
         const double x = tile[a][b];
         __nv_bfloat16 d[NSL];
-        digits_of(isfinite(x) ? x : 0.0, ex[j], d);
+        digits_of(isfinite(x) ? x : 0.0, LQ_AT(ex + j), d);
 #pragma unroll
-        for (int s = 0; s < NSL; ++s) SL[(s * slice_rows + j) * LDP + k0 + a] = d[s];
+        for (int s = 0; s < NSL; ++s) LQ_AT(SL + (s * slice_rows + j) * LDP + k0 + a) = d[s];
     }
 }
 
@@ -398,17 +399,17 @@ apply_kernel(double* __restrict__ A, int64_t cp, const float* __restrict__ Ta, c
              const int* __restrict__ ex, int64_t row0, int64_t nrows, int64_t col0, int64_t ncols, int upper) {
     const int64_t i = blockIdx.y;
     const int64_t row = row0 + i;
-    const int er = ex[row];
+    const int er = LQ_AT(ex + row);
     for (int64_t j2 = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; 2 * j2 < ncols; j2 += (int64_t)gridDim.x * blockDim.x) {
         const int64_t col = col0 + 2 * j2;
         if (upper && col / NB < row / NB) continue;
-        const float2 a = *reinterpret_cast<const float2*>(Ta + i * ldt + col);
-        const float2 b = *reinterpret_cast<const float2*>(Tb + i * ldt + col);
+        const float2 a = LQ_AT(reinterpret_cast<const float2*>(Ta + i * ldt + col));
+        const float2 b = LQ_AT(reinterpret_cast<const float2*>(Tb + i * ldt + col));
         double2* ap = reinterpret_cast<double2*>(A + row * cp + col);
-        double2 v = *ap;
-        v.x -= scalbn(static_cast<double>(a.x) + static_cast<double>(b.x), er + ex[col]);
-        v.y -= scalbn(static_cast<double>(a.y) + static_cast<double>(b.y), er + ex[col + 1]);
-        *ap = v;
+        double2 v = LQ_AT(ap);
+        v.x -= scalbn(static_cast<double>(a.x) + static_cast<double>(b.x), er + LQ_AT(ex + col));
+        v.y -= scalbn(static_cast<double>(a.y) + static_cast<double>(b.y), er + LQ_AT(ex + col + 1));
+        LQ_AT(ap) = v;
     }
 }
 
@@ -604,7 +605,7 @@ diag_block_kernel(double* __restrict__ A, int64_t cp, int64_t blk, int64_t c_rea
         double2 v;
         v.x = (c2 >= row) ? S[row * DP + c2] : 0.0;
         v.y = (c2 + 1 >= row) ? S[row * DP + c2 + 1] : 0.0;
-        *reinterpret_cast<double2*>(base + (int64_t)row * cp + c2) = v;
+        LQ_AT(reinterpret_cast<double2*>(base + (int64_t)row * cp + c2)) = v;
     }
 }
 
@@ -625,10 +626,10 @@ finalize_kernel(const double* __restrict__ A, int64_t cp, int64_t c, float* __re
         for (int64_t i = i0 + ty; i < i1; i += 8) {
             double u = 0.0;
             if (i <= j) {
-                u = A[i * cp + j];
+                u = LQ_AT(A + i * cp + j);
                 s = fma(u, u, s);
             }
-            U[i * ldu + j] = static_cast<float>(u);
+            LQ_AT(U + i * ldu + j) = static_cast<float>(u);
         }
     }
     red[ty][tx] = s;
@@ -637,15 +638,15 @@ finalize_kernel(const double* __restrict__ A, int64_t cp, int64_t c, float* __re
         double t = 0.0;
 #pragma unroll
         for (int w = 0; w < 8; ++w) t += red[w][tx];
-        part[(int64_t)blockIdx.y * c + j] = t;
+        LQ_AT(part + (int64_t)blockIdx.y * c + j) = t;
     }
 }
 __global__ void dinv_kernel(const double* __restrict__ part, int64_t c, int n_chunks, float* __restrict__ dinv) {
     const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= c) return;
     double t = 0.0;
-    for (int q = 0; q * (int64_t)FIN_ROWS <= j && q < n_chunks; ++q) t += part[(int64_t)q * c + j];
-    dinv[j] = static_cast<float>(t);
+    for (int q = 0; q * (int64_t)FIN_ROWS <= j && q < n_chunks; ++q) t += LQ_AT(part + (int64_t)q * c + j);
+    LQ_AT(dinv + j) = static_cast<float>(t);
 }
 
 struct PrepLayout {
@@ -772,6 +773,15 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
     double* scal = reinterpret_cast<double*>(wsp + L.scal);
     double* A = reinterpret_cast<double*>(wsp + L.a);
 
+    {
+        LQ_DBG_SCOPE(h, st);
+        LQ_DBG_REG(H, (static_cast<size_t>(c - 1) * ldh + c) * sizeof(float));
+        LQ_DBG_REG(U, (static_cast<size_t>(c - 1) * ldu + c) * sizeof(float));
+        LQ_DBG_REG(dinv, static_cast<size_t>(c) * sizeof(float));
+        if (W) LQ_DBG_REG(W, (static_cast<size_t>(r - 1) * ldw + c) * (w_dtype == LQ_F32 ? 4 : 2));
+        LQ_DBG_REG(ws, L.total);
+        LQ_DBG_COMMIT();
+    }
     static lq_once_per_device attr_set;
     if (attr_set.first()) {
         LQ_CUDA_TRY(cudaFuncSetAttribute(diag_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DIAG_SMEM));
@@ -897,12 +907,18 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
 namespace {
 __global__ void chol_diag_kernel(const float* __restrict__ U, int64_t c, int64_t ldu, float* __restrict__ d) {
     const int64_t j = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (j < c) d[j] = U[j * ldu + j];
+    if (j < c) LQ_AT(d + j) = LQ_AT(U + j * ldu + j);
 }
 }  // namespace
 
 extern "C" int lq_chol_diag(lq_handle* h, void* stream, const float* U, int64_t c, int64_t ldu, float* d) {
     if (!h || !U || !d || c <= 0 || ldu < c) return LQ_ERR_INVALID_ARG;
+    {
+        LQ_DBG_SCOPE(h, static_cast<cudaStream_t>(stream));
+        LQ_DBG_REG(U, (static_cast<size_t>(c - 1) * ldu + c) * sizeof(float));
+        LQ_DBG_REG(d, static_cast<size_t>(c) * sizeof(float));
+        LQ_DBG_COMMIT();
+    }
     chol_diag_kernel<<<static_cast<unsigned>(lq_ceil_div(c, 256)), 256, 0, static_cast<cudaStream_t>(stream)>>>(U, c, ldu, d);
     LQ_LAUNCH_CHECK();
     return LQ_OK;

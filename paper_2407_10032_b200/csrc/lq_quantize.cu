@@ -27,10 +27,10 @@ __global__ void to_f32_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, f
             float v[8];
             if (sizeof(T) == 4) {
                 const float4* p = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(W) + row * ldw + 8 * j8);
-                const float4 x = p[0], y = p[1];
+                const float4 x = LQ_AT(p), y = LQ_AT(p + 1);
                 v[0] = x.x; v[1] = x.y; v[2] = x.z; v[3] = x.w; v[4] = y.x; v[5] = y.y; v[6] = y.z; v[7] = y.w;
             } else {
-                const uint4 x = *reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(W) + row * ldw + 8 * j8);
+                const uint4 x = LQ_AT(reinterpret_cast<const uint4*>(reinterpret_cast<const __nv_bfloat16*>(W) + row * ldw + 8 * j8));
                 const uint32_t u[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
@@ -39,27 +39,27 @@ __global__ void to_f32_kernel(const T* __restrict__ W, int64_t ldw, int64_t c, f
                 }
             }
             float4* q = reinterpret_cast<float4*>(Wc + row * ldc + 8 * j8);
-            q[0] = make_float4(v[0], v[1], v[2], v[3]);
-            q[1] = make_float4(v[4], v[5], v[6], v[7]);
+            LQ_AT(q) = make_float4(v[0], v[1], v[2], v[3]);
+            LQ_AT(q + 1) = make_float4(v[4], v[5], v[6], v[7]);
         }
         // the ragged end of the row, if any
         for (int64_t j = n8 * 8 + blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < ldc; j += (int64_t)gridDim.x * blockDim.x) {
             float v = 0.0f;
             if (j < c) {
-                if (sizeof(T) == 4) v = reinterpret_cast<const float*>(W)[row * ldw + j];
-                else v = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(W)[row * ldw + j]);
+                if (sizeof(T) == 4) v = LQ_AT(reinterpret_cast<const float*>(W) + row * ldw + j);
+                else v = __bfloat162float(LQ_AT(reinterpret_cast<const __nv_bfloat16*>(W) + row * ldw + j));
             }
-            Wc[row * ldc + j] = v;
+            LQ_AT(Wc + row * ldc + j) = v;
         }
         return;
     }
     for (int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < ldc; j += (int64_t)gridDim.x * blockDim.x) {
         float v = 0.0f;
         if (j < c) {
-            if (sizeof(T) == 4) v = reinterpret_cast<const float*>(W)[row * ldw + j];
-            else v = __bfloat162float(reinterpret_cast<const __nv_bfloat16*>(W)[row * ldw + j]);
+            if (sizeof(T) == 4) v = LQ_AT(reinterpret_cast<const float*>(W) + row * ldw + j);
+            else v = __bfloat162float(LQ_AT(reinterpret_cast<const __nv_bfloat16*>(W) + row * ldw + j));
         }
-        Wc[row * ldc + j] = v;
+        LQ_AT(Wc + row * ldc + j) = v;
     }
 }
 
@@ -76,12 +76,12 @@ split_transpose_kernel(const float* __restrict__ U, int64_t ldu, int64_t c, __nv
         const int64_t k = k0 + a, n = n0 + n4;
         float4 v = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
         if (k < c) {
-            if (vec_in && n + 3 < c) v = *reinterpret_cast<const float4*>(U + k * ldu + n);
+            if (vec_in && n + 3 < c) v = LQ_AT(reinterpret_cast<const float4*>(U + k * ldu + n));
             else {
-                if (n < c) v.x = U[k * ldu + n];
-                if (n + 1 < c) v.y = U[k * ldu + n + 1];
-                if (n + 2 < c) v.z = U[k * ldu + n + 2];
-                if (n + 3 < c) v.w = U[k * ldu + n + 3];
+                if (n < c) v.x = LQ_AT(U + k * ldu + n);
+                if (n + 1 < c) v.y = LQ_AT(U + k * ldu + n + 1);
+                if (n + 2 < c) v.z = LQ_AT(U + k * ldu + n + 2);
+                if (n + 3 < c) v.w = LQ_AT(U + k * ldu + n + 3);
             }
         }
         tile[a][n4] = v.x; tile[a][n4 + 1] = v.y; tile[a][n4 + 2] = v.z; tile[a][n4 + 3] = v.w;
@@ -102,9 +102,9 @@ split_transpose_kernel(const float* __restrict__ U, int64_t ldu, int64_t c, __nv
             pl[e] = static_cast<uint32_t>(__bfloat16_as_ushort(l0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(l1)) << 16);
         }
         // ldt is a multiple of 8 and k a multiple of 8: the eight entries are inside the row and 16-byte aligned
-        *reinterpret_cast<uint4*>(UT + n * ldt + k) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
-        *reinterpret_cast<uint4*>(UT + (c + n) * ldt + k) = make_uint4(pm[0], pm[1], pm[2], pm[3]);
-        *reinterpret_cast<uint4*>(UT + (2 * c + n) * ldt + k) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
+        LQ_AT(reinterpret_cast<uint4*>(UT + n * ldt + k)) = make_uint4(ph[0], ph[1], ph[2], ph[3]);
+        LQ_AT(reinterpret_cast<uint4*>(UT + (c + n) * ldt + k)) = make_uint4(pm[0], pm[1], pm[2], pm[3]);
+        LQ_AT(reinterpret_cast<uint4*>(UT + (2 * c + n) * ldt + k)) = make_uint4(pl[0], pl[1], pl[2], pl[3]);
     }
 }
 
@@ -155,15 +155,16 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
         const int jj = idx / (B / 4), k4 = (idx % (B / 4)) * 4;
         if (whole) {
             const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(Us + jj * B + k4));
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(U + (i0 + jj) * ldu + i0 + k4) : "memory");
+            if (LQ_DBG_OK(U + (i0 + jj) * ldu + i0 + k4, 16) && LQ_DBG_OK(Us + jj * B + k4, 16))
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(U + (i0 + jj) * ldu + i0 + k4) : "memory");
         } else {
             float t[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const int kk = k4 + u;
-                t[u] = (jj < bw && kk < bw) ? U[(i0 + jj) * ldu + i0 + kk] : (jj == kk ? 1.0f : 0.0f);
+                t[u] = (jj < bw && kk < bw) ? LQ_AT(U + (i0 + jj) * ldu + i0 + kk) : (jj == kk ? 1.0f : 0.0f);
             }
-            *reinterpret_cast<float4*>(Us + jj * B + k4) = make_float4(t[0], t[1], t[2], t[3]);
+            LQ_AT(reinterpret_cast<float4*>(Us + jj * B + k4)) = make_float4(t[0], t[1], t[2], t[3]);
         }
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
@@ -175,38 +176,38 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
     if (valid) {
         const float* wp = Wc + row * ldc + i0 + col0;
         if (col0 + 3 < bw) {
-            const float4 v = *reinterpret_cast<const float4*>(wp);
+            const float4 v = LQ_AT(reinterpret_cast<const float4*>(wp));
             w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
         } else {
 #pragma unroll
-            for (int u = 0; u < 4; ++u) w[u] = (col0 + u < bw) ? wp[u] : 0.0f;
+            for (int u = 0; u < 4; ++u) w[u] = (col0 + u < bw) ? LQ_AT(wp + u) : 0.0f;
         }
     }
     float gl = 0.0f, ml = INFINITY;        // this lane's grid point and the midpoint above it
     float S_mine = 1.0f, Z_mine = 0.0f;    // affine parameters of this lane's columns
     if (!AFFINE) {
-        if (valid && lane < K) gl = grid[row * K + lane];
+        if (valid && lane < K) gl = LQ_AT(grid + row * K + lane);
         const float gn = __shfl_down_sync(0xffffffffu, gl, 1);
         if (lane < K - 1) ml = 0.5f * (gl + gn);
     } else if (!REFIT && valid && col0 < bw) {
         const int64_t gi = (i0 + col0) / group;
         const int64_t gidx = row * n_groups + (gi < n_groups ? gi : n_groups - 1);
-        S_mine = scale[gidx];
-        Z_mine = static_cast<float>(zero[gidx]);
+        S_mine = LQ_AT(scale + gidx);
+        Z_mine = static_cast<float>(LQ_AT(zero + gidx));
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
-    if (tid < B) invd[tid] = 1.0f / Us[tid * B + tid];
+    if (tid < B) LQ_AT(invd + tid) = 1.0f / LQ_AT(Us + tid * B + tid);
     __syncthreads();
     // rows of the block scaled by the reciprocal of their diagonal entry: the column loop then feeds w - q straight
     // into the other columns, and only the lane that owns a column turns it into E = (w - q) / U_jj afterwards
     for (int idx = tid; idx < B * B / 4; idx += nthr) {
         const int jj = idx / (B / 4);
         float4* p4 = reinterpret_cast<float4*>(Us) + idx;
-        float4 v = *p4;
-        const float sc = invd[jj];
+        float4 v = LQ_AT(p4);
+        const float sc = LQ_AT(invd + jj);
         v.x *= sc; v.y *= sc; v.z *= sc; v.w *= sc;
-        *p4 = v;
+        LQ_AT(p4) = v;
     }
     __syncthreads();
     if (!valid) return;
@@ -225,17 +226,17 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
             const int gl = group / 4;                        // lanes per group
             if (lane >= jj && lane < jj + gl) {
 #pragma unroll
-                for (int u = 0; u < 4; ++u) wtmp[4 * (lane - jj) + u] = w[u];
+                for (int u = 0; u < 4; ++u) LQ_AT(wtmp + 4 * (lane - jj) + u) = w[u];
             }
             __syncwarp();
             double Sd, Zd;
-            lq_affine_warp_search([&](int j) { return wtmp[j]; }, refit.s64 + i0 + 4 * jj, group, ws, K, refit.T, refit.t_count, lane,
+            lq_affine_warp_search([&](int j) { return LQ_AT(wtmp + j); }, refit.s64 + i0 + 4 * jj, group, ws, K, refit.T, refit.t_count, lane,
                                   Sd, Zd);
             if (lane >= jj && lane < jj + gl) { S_mine = static_cast<float>(Sd); Z_mine = static_cast<float>(static_cast<int32_t>(Zd)); }
             if (lane == jj) {
                 const int64_t gidx = row * n_groups + (i0 + 4 * jj) / group;
-                refit.scale[gidx] = static_cast<float>(Sd);
-                refit.zero[gidx] = static_cast<int32_t>(Zd);
+                LQ_AT(refit.scale + gidx) = static_cast<float>(Sd);
+                LQ_AT(refit.zero + gidx) = static_cast<int32_t>(Zd);
             }
             __syncwarp();
         }
@@ -265,7 +266,7 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
                 dkeep[u] = d;
                 cpack |= static_cast<uint32_t>(code) << (8 * u);
             }
-            const float4 uv = *reinterpret_cast<const float4*>(Us + j * B + col0);
+            const float4 uv = LQ_AT(reinterpret_cast<const float4*>(Us + j * B + col0));
             w[0] = fmaf(-d, uv.x, w[0]);
             w[1] = fmaf(-d, uv.y, w[1]);
             w[2] = fmaf(-d, uv.z, w[2]);
@@ -281,7 +282,7 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
         const int code = static_cast<int>((cpack >> (8 * u)) & 0xffu);
         if (AFFINE) qkeep[u] = (static_cast<float>(code) - Z_mine) * S_mine;
         else qkeep[u] = __shfl_sync(0xffffffffu, gl, code);
-        ekeep[u] = (col0 + u < bw) ? dkeep[u] * invd[col0 + u] : 0.0f;
+        ekeep[u] = (col0 + u < bw) ? dkeep[u] * LQ_AT(invd + col0 + u) : 0.0f;
         loss = fmaf(ekeep[u], ekeep[u], loss);
     }
 #pragma unroll
@@ -290,18 +291,18 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
     if (col0 < bw) {
         const int64_t gcol = i0 + col0;
         if (col0 + 3 < bw && (c % 4 == 0)) {
-            *reinterpret_cast<uint32_t*>(out.codes + row * c + gcol) = cpack;
+            LQ_AT(reinterpret_cast<uint32_t*>(out.codes + row * c + gcol)) = cpack;
         } else {
 #pragma unroll
             for (int u = 0; u < 4; ++u)
-                if (col0 + u < bw) out.codes[row * c + gcol + u] = static_cast<uint8_t>((cpack >> (8 * u)) & 0xff);
+                if (col0 + u < bw) LQ_AT(out.codes + row * c + gcol + u) = static_cast<uint8_t>((cpack >> (8 * u)) & 0xff);
         }
         if (out.what) {
 #pragma unroll
             for (int u = 0; u < 4; ++u)
                 if (col0 + u < bw) {
-                    if (out.what_bf16) static_cast<__nv_bfloat16*>(out.what)[row * out.ldwh + gcol + u] = __float2bfloat16_rn(qkeep[u]);
-                    else static_cast<float*>(out.what)[row * out.ldwh + gcol + u] = qkeep[u];
+                    if (out.what_bf16) LQ_AT(static_cast<__nv_bfloat16*>(out.what) + row * out.ldwh + gcol + u) = __float2bfloat16_rn(qkeep[u]);
+                    else LQ_AT(static_cast<float*>(out.what) + row * out.ldwh + gcol + u) = qkeep[u];
                 }
         }
     }
@@ -319,11 +320,11 @@ inblock_kernel(const float* __restrict__ Wc, int64_t ldc, int64_t r, int64_t c, 
         __nv_bfloat16* e0 = out.esplit + row * out.e_ld + out.e_col + col0;
         __nv_bfloat16* e1 = e0 + r * out.e_ld;
         __nv_bfloat16* e2 = e1 + r * out.e_ld;
-        *reinterpret_cast<uint2*>(e0) = make_uint2(ph[0], ph[1]);
-        *reinterpret_cast<uint2*>(e1) = make_uint2(pm[0], pm[1]);
-        *reinterpret_cast<uint2*>(e2) = make_uint2(pl[0], pl[1]);
+        LQ_AT(reinterpret_cast<uint2*>(e0)) = make_uint2(ph[0], ph[1]);
+        LQ_AT(reinterpret_cast<uint2*>(e1)) = make_uint2(pm[0], pm[1]);
+        LQ_AT(reinterpret_cast<uint2*>(e2)) = make_uint2(pl[0], pl[1]);
     }
-    if (lane == 0) out.loss_rows[row] += static_cast<double>(loss);
+    if (lane == 0) LQ_AT(out.loss_rows + row) += static_cast<double>(loss);
 }
 
 // Packed output: the b-bit codes of a row as one little-endian bit stream (code j in bits
@@ -338,23 +339,23 @@ __global__ void pack_codes_kernel(const uint8_t* __restrict__ codes, int64_t r, 
         uint32_t acc = 0;
         for (int64_t j = j0; j <= j1 && j < c; ++j) {
             const int64_t sh = j * bits - bit0;                 // position of code j relative to this byte
-            const uint32_t v = codes[row * c + j] & ((1u << bits) - 1u);
+            const uint32_t v = LQ_AT(codes + row * c + j) & ((1u << bits) - 1u);
             acc |= sh >= 0 ? (v << sh) : (v >> (-sh));
         }
-        packed[row * ldp + b] = static_cast<uint8_t>(acc & 0xffu);
+        LQ_AT(packed + row * ldp + b) = static_cast<uint8_t>(acc & 0xffu);
     }
 }
 
 __global__ void zero_doubles_kernel(double* p, int64_t n) {
     const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (i < n) p[i] = 0.0;
+    if (i < n) LQ_AT(p + i) = 0.0;
 }
 
 // loss_out[0] = 1/2 * sum_rows loss_rows
 __global__ void loss_reduce_kernel(const double* __restrict__ loss_rows, int64_t r, double* __restrict__ loss_out) {
     __shared__ double red[1024];
     double s = 0.0;
-    for (int64_t i = threadIdx.x; i < r; i += blockDim.x) s += loss_rows[i];
+    for (int64_t i = threadIdx.x; i < r; i += blockDim.x) s += LQ_AT(loss_rows + i);
     red[threadIdx.x] = s;
     __syncthreads();
     for (int o = blockDim.x / 2; o > 0; o >>= 1) {
@@ -472,6 +473,20 @@ int quantize_impl(lq_handle* h, void* stream, const lq_config* cfg, const void* 
         s64 = reinterpret_cast<double*>(wsp + L.total + 256);
         e = lq_sample_weights(h, st, dinv, c, static_cast<double>(cfg->p), reinterpret_cast<double*>(wsp + L.total), s64);
         if (e) return e;
+    }
+    {
+        LQ_DBG_SCOPE(h, st);
+        const size_t wb = w_dtype == LQ_F32 ? 4 : 2;
+        LQ_DBG_REG(W, (static_cast<size_t>(r - 1) * ldw + c) * wb);
+        LQ_DBG_REG(U, (static_cast<size_t>(c - 1) * ldu + c) * sizeof(float));
+        LQ_DBG_REG(ws, L.total + lazy_bytes);
+        LQ_DBG_REG(codes, static_cast<size_t>(r) * c);
+        if (W_hat) LQ_DBG_REG(W_hat, (static_cast<size_t>(r - 1) * ldwh + c) * (what_dtype == LQ_F32 ? 4 : 2));
+        if (grid) LQ_DBG_REG(grid, static_cast<size_t>(r) * (size_t(1) << cfg->bits) * sizeof(float));
+        if (scale) LQ_DBG_REG(scale, static_cast<size_t>(r) * n_groups * sizeof(float));
+        if (zero) LQ_DBG_REG(zero, static_cast<size_t>(r) * n_groups * sizeof(int32_t));
+        if (loss_out) LQ_DBG_REG(loss_out, sizeof(double));
+        LQ_DBG_COMMIT();
     }
     float* Wc = reinterpret_cast<float*>(wsp + L.wc);
     __nv_bfloat16* UT = reinterpret_cast<__nv_bfloat16*>(wsp + L.ut);
@@ -623,6 +638,12 @@ extern "C" int lq_pack_codes(lq_handle* h, void* stream, const uint8_t* codes, i
         return LQ_OK;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    {
+        LQ_DBG_SCOPE(h, st);
+        LQ_DBG_REG(codes, static_cast<size_t>(r) * c);
+        LQ_DBG_REG(packed, static_cast<size_t>(r - 1) * ldp + nbytes);
+        LQ_DBG_COMMIT();
+    }
     dim3 g(static_cast<unsigned>(lq_ceil_div(nbytes, 256) < 64 ? lq_ceil_div(nbytes, 256) : 64), static_cast<unsigned>(r));
     pack_codes_kernel<<<g, 256, 0, st>>>(codes, r, c, bits, packed, ldp);
     LQ_LAUNCH_CHECK();

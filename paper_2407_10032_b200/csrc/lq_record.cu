@@ -59,17 +59,17 @@ __global__ void header_kernel(Header* dst, Header h) { *dst = h; }
 // fp16 copies of the per-row tables (non-uniform) or scales (affine); int16 copies of the zero points.
 __global__ void to_half_kernel(const float* __restrict__ src, int64_t n, __half* __restrict__ dst) {
     const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (i < n) dst[i] = __float2half_rn(src[i]);
+    if (i < n) LQ_AT(dst + i) = __float2half_rn(LQ_AT(src + i));
 }
 __global__ void to_int16_kernel(const int32_t* __restrict__ src, int64_t n, int16_t* __restrict__ dst, lq_dev_status* st) {
     const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (i >= n) return;
-    int32_t z = src[i];
+    int32_t z = LQ_AT(src + i);
     if (z > 32767 || z < -32768) {          // a zero point that 16 bits cannot hold: reported, stored saturated
         lq_report(st, LQ_ERR_UNSUPPORTED, i);
         z = z > 0 ? 32767 : -32768;
     }
-    dst[i] = static_cast<int16_t>(z);
+    LQ_AT(dst + i) = static_cast<int16_t>(z);
 }
 
 // One thread per weight: code from the bit stream, value from the row's table or the group's (S, Z).
@@ -89,17 +89,17 @@ __global__ void unpack_kernel(const uint8_t* __restrict__ rec, int64_t r, int64_
     const int K = 1 << bits;
     for (int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; j < c; j += (int64_t)gridDim.x * blockDim.x) {
         const int64_t bit0 = j * bits;
-        uint32_t w = codes[bit0 >> 3];
-        if (((bit0 & 7) + bits > 8) && (bit0 >> 3) + 1 < row_bytes) w |= static_cast<uint32_t>(codes[(bit0 >> 3) + 1]) << 8;
+        uint32_t w = LQ_AT(codes + (bit0 >> 3));
+        if (((bit0 & 7) + bits > 8) && (bit0 >> 3) + 1 < row_bytes) w |= static_cast<uint32_t>(LQ_AT(codes + (bit0 >> 3) + 1)) << 8;
         const int code = static_cast<int>((w >> (bit0 & 7)) & (K - 1));
         float v;
         if (affine) {
             const int64_t gi = row * n_groups + j / group;
-            v = (static_cast<float>(code) - static_cast<float>(zero[gi])) * __half2float(table[gi]);
+            v = (static_cast<float>(code) - static_cast<float>(LQ_AT(zero + gi))) * __half2float(LQ_AT(table + gi));
         } else {
-            v = __half2float(table[row * K + code]);
+            v = __half2float(LQ_AT(table + row * K + code));
         }
-        out[row * ldo + j] = T(v);
+        LQ_AT(out + row * ldo + j) = T(v);
     }
 }
 
@@ -139,6 +139,14 @@ extern "C" int lq_pack_layer(lq_handle* h, void* stream, const lq_config* cfg, c
     hd.table_offset = static_cast<long long>(L.table);
     hd.zero_offset = static_cast<long long>(L.zero);
     hd.total_bytes = static_cast<long long>(L.total);
+    {
+        LQ_DBG_SCOPE(h, st);
+        LQ_DBG_REG(record, L.total);
+        if (grid) LQ_DBG_REG(grid, static_cast<size_t>(r) * (size_t(1) << cfg->bits) * sizeof(float));
+        if (affine) LQ_DBG_REG(scale, static_cast<size_t>(r) * L.n_groups * sizeof(float));
+        if (affine) LQ_DBG_REG(zero, static_cast<size_t>(r) * L.n_groups * sizeof(int32_t));
+        LQ_DBG_COMMIT();
+    }
     header_kernel<<<1, 1, 0, st>>>(reinterpret_cast<Header*>(rec), hd);
     LQ_LAUNCH_CHECK();
     e = lq_pack_codes(h, stream, codes, r, c, cfg->bits, rec + L.codes, L.row_bytes);
@@ -169,6 +177,12 @@ extern "C" int lq_unpack_layer(lq_handle* h, void* stream, const lq_config* cfg,
     const int affine = cfg->grid_type == LQ_GRID_AFFINE ? 1 : 0;
     const int64_t g = cfg->group_size == 0 ? c : cfg->group_size;
     const uint8_t* rec = static_cast<const uint8_t*>(record);
+    {
+        LQ_DBG_SCOPE(h, st);
+        LQ_DBG_REG(record, L.total);
+        LQ_DBG_REG(W_hat, (static_cast<size_t>(r - 1) * ldwh + c) * (what_dtype == LQ_F32 ? 4 : 2));
+        LQ_DBG_COMMIT();
+    }
     for (int64_t r0 = 0; r0 < r; r0 += 65535) {          // rows in slabs: the second grid dimension holds 65535 at most
         const int64_t rr = r - r0 < 65535 ? r - r0 : 65535;
         dim3 grid(static_cast<unsigned>(lq_ceil_div(c, 256) < 64 ? lq_ceil_div(c, 256) : 64), static_cast<unsigned>(rr));
@@ -193,8 +207,8 @@ namespace {
 template <typename T>
 __global__ void zero_dead_kernel(const float* __restrict__ H, int64_t c, int64_t ldh, T* __restrict__ W, int64_t r, int64_t ldw) {
     const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (j >= c || H[j * ldh + j] != 0.0f) return;
-    for (int64_t i = blockIdx.y; i < r; i += gridDim.y) W[i * ldw + j] = T(0.0f);
+    if (j >= c || LQ_AT(H + j * ldh + j) != 0.0f) return;
+    for (int64_t i = blockIdx.y; i < r; i += gridDim.y) LQ_AT(W + i * ldw + j) = T(0.0f);
 }
 }  // namespace
 
@@ -202,6 +216,12 @@ extern "C" int lq_zero_dead_columns(lq_handle* h, void* stream, const float* H, 
                                     int64_t r, int64_t ldw) {
     if (!h || !H || !W || c <= 0 || r <= 0 || ldh < c || ldw < c || (w_dtype != LQ_F32 && w_dtype != LQ_BF16)) return LQ_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    {
+        LQ_DBG_SCOPE(h, st);
+        LQ_DBG_REG(H, (static_cast<size_t>(c - 1) * ldh + c) * sizeof(float));
+        LQ_DBG_REG(W, (static_cast<size_t>(r - 1) * ldw + c) * (w_dtype == LQ_F32 ? 4 : 2));
+        LQ_DBG_COMMIT();
+    }
     dim3 g(static_cast<unsigned>(lq_ceil_div(c, 256)), static_cast<unsigned>(r < 64 ? r : 64));
     if (w_dtype == LQ_F32) zero_dead_kernel<float><<<g, 256, 0, st>>>(H, c, ldh, static_cast<float*>(W), r, ldw);
     else zero_dead_kernel<__nv_bfloat16><<<g, 256, 0, st>>>(H, c, ldh, static_cast<__nv_bfloat16*>(W), r, ldw);

@@ -12,7 +12,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 @pytest.fixture(scope="module")
 def lib():
     from paper_2407_10032_b200 import build
-    build.build()
+    build.build(debug_bounds=os.environ.get("LQ_LIBRARY_VARIANT") == "debug")
     import paper_2407_10032_b200 as lq
     return lq
 

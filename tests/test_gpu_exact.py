@@ -4,6 +4,8 @@ Isolated: the oracle runs on the inverse U^T U of the factor the GPU produced (w
 the GPU's grid, so that only the greedy loop itself is compared: its order, codes and loss must agree to
 rounding.  Chained: everything from X on, against the oracle's own float64 pass, within the tolerances of the
 other parity tests (0.1 % of codes, 1e-3 on the loss)."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -21,7 +23,7 @@ LOSS_TOL = 1e-3
 def lq():
     import paper_2407_10032_b200 as m
     from paper_2407_10032_b200 import build
-    build.build()
+    build.build(debug_bounds=os.environ.get("LQ_LIBRARY_VARIANT") == "debug")
     return m
 
 

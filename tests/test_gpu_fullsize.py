@@ -13,6 +13,8 @@ benchmark times.  The float64 oracle cannot redo these layers in full within min
            tr((W - W_hat) H_d (W - W_hat)^T) equals twice the summed loss error the library
            returns (an identity of the column loop, Eq. 3 with the Cholesky rows);
   Eq. 7 at T = 2048 on the 8B-shaped down_proj and Algorithm 2 on a 768 x 768 layer: sampled groups / rows."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -31,7 +33,7 @@ CENT_TOL = 1e-4
 def lq():
     import paper_2407_10032_b200 as m
     from paper_2407_10032_b200 import build
-    build.build()
+    build.build(debug_bounds=os.environ.get("LQ_LIBRARY_VARIANT") == "debug")
     return m
 
 

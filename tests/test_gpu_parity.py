@@ -1,6 +1,8 @@
 """Parity of the CUDA path (through the C ABI) with the float64 oracle, stage by stage and
 chained, on seeded synthetic layers.  Tolerances: centroids within
 1e-4 relative, at most 0.1 % of integer codes differing, layer loss within 1e-3 relative."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -19,7 +21,7 @@ CENT_TOL = 1e-4
 def lq():
     import paper_2407_10032_b200 as m
     from paper_2407_10032_b200 import build
-    build.build()
+    build.build(debug_bounds=os.environ.get("LQ_LIBRARY_VARIANT") == "debug")
     return m
 
 

@@ -1,4 +1,6 @@
 """The packed layer record (codes + fp16 tables / (S, Z)) and the stack driver, through the C ABI, against the oracle."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -15,7 +17,7 @@ CODE_TOL, LOSS_TOL, CENT_TOL = 1e-3, 1e-3, 1e-4
 def lq():
     import paper_2407_10032_b200 as m
     from paper_2407_10032_b200 import build
-    build.build()
+    build.build(debug_bounds=os.environ.get("LQ_LIBRARY_VARIANT") == "debug")
     return m
 
 

@@ -7,6 +7,8 @@ what lq_fit_grid gives.  Checked here through the C ABI on two calls in a row wi
 shapes, so that the second call runs on whatever the first left in the shared array.
 This file is named to be collected last: a run that stops at the first failure has then
 already run every other test."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -23,7 +25,7 @@ CENT_TOL = 1e-4      # the centroid tolerance of the parity tests
 def lq():
     import paper_2407_10032_b200 as m
     from paper_2407_10032_b200 import build
-    build.build()
+    build.build(debug_bounds=os.environ.get("LQ_LIBRARY_VARIANT") == "debug")
     return m
 
 
