@@ -288,6 +288,14 @@ def stage_rooflines(st, r, c, n, stage_ms, pk, pipes, w_bytes, exact=False):
                            "executed_frac": STAGE4_PRODUCTS * s4 / pk["tf_burst"],
                            "executed_frac_of_sustained": STAGE4_PRODUCTS * s4 / pk["tf_sust"]},
     }
+    dfrac = stage2_deferred_fraction(c)
+    if dfrac > 0.0:
+        # wide layers: most update products run on the bf16 tensor cores as 15 digit-slice products each, so the
+        # algorithmic rate can exceed the FP64 pipe's peak; what the tensor pipe executes is reported beside it
+        ex = STAGE2_PRODUCTS * dfrac * s2
+        out["prepare_hinv"].update({"bound": "tensor (bf16 digit slices) for the deferred updates, fp64 tensor for the rest",
+                                    "deferred_fraction": dfrac, "executed_bf16": ex,
+                                    "executed_frac_of_sustained": ex / pk["tf_sust"]})
     if exact:
         # Algorithm 2: r rows x c steps x a c x c downdate = r c^3 fp64 FMAs, half of which touch weights already
         # quantised and need not be done
@@ -298,6 +306,30 @@ def stage_rooflines(st, r, c, n, stage_ms, pk, pipes, w_bytes, exact=False):
 
 
 STAGE4_PRODUCTS = 6     # bf16 products the library issues per fp32 product of the lazy update
+STAGE2_PRODUCTS = 15    # bf16 digit-slice products per fp64 product of stage 2's deferred updates
+STAGE2_DEFER_MIN_BLOCKS, STAGE2_OUTER = 48, 8
+
+
+def stage2_deferred_fraction(c):
+    """Share of stage 2's update products (128 x 128 x 128 tile products) that the library defers to the bf16 tensor
+    cores: it counts, step by step as the library's sweep goes, the tiles updated at once on the FP64 MMA (the rows
+    and columns of the current outer block of 8 block columns) and the tiles that wait for the outer block's end."""
+    nblk = -(-c // 128)
+    if nblk < STAGE2_DEFER_MIN_BLOCKS:
+        return 0.0
+    eager = deferred = 0
+    for o_lo in range(0, nblk, STAGE2_OUTER):
+        o_hi = min(o_lo + STAGE2_OUTER, nblk) - 1
+        for k in range(o_lo, o_hi + 1):
+            for i in range(k):                       # block row i < k gets tiles j >= i
+                n_all = nblk - i
+                if i >= o_lo:
+                    eager += n_all
+                else:
+                    n_in = o_hi - o_lo + 1           # columns of the outer block
+                    eager += n_in
+                    deferred += n_all - n_in
+    return deferred / float(eager + deferred)
 
 
 class LayerRun:
@@ -428,6 +460,8 @@ def extra_workloads(lq, h, dev, rank, pk, pipes, args):
                                   "fit_grid": float(stage_ms[2]), "quantize_layer": float(stage_ms[3])},
                      "stage_roofline_frac": {k: v["frac"] for k, v in roofs.items()},
                      "quantize_layer_executed_frac_of_sustained": roofs["quantize_layer"].get("executed_frac_of_sustained"),
+                     "prepare_hinv_deferred_fraction": roofs["prepare_hinv"].get("deferred_fraction"),
+                     "prepare_hinv_executed_bf16_frac_of_sustained": roofs["prepare_hinv"].get("executed_frac_of_sustained"),
                      "gpu_launches_per_step": launches // steps}
             if share is not None:
                 entry["note"] = f"stages 1-2 shared with {share_name} (same layer, same Hessian); their times are that run's"
