@@ -34,6 +34,11 @@ int lq_testing_inject_stall(lq_handle* h, int32_t on);
  * default), so that tests can run the deferred path on matrices small enough for a float64 check in full. */
 int lq_testing_set_prepare_defer_min_blocks(lq_handle* h, int32_t n_blocks);
 
+/* The deferred updates of lq_prepare_hinv multiply digit slices of their fp64 operands: as 8-bit integers on the integer
+ * tensor-core path (the default) or, with on = 0, as bf16 values on the bf16 path.  Both are exact products; tests run
+ * both and compare. */
+int lq_testing_set_prepare_slices_int8(lq_handle* h, int32_t on);
+
 #ifdef __cplusplus
 }
 #endif

@@ -82,6 +82,7 @@ def LQ():
             "lq_testing_set_wait_limit_ns": [vp, C.c_uint64],
             "lq_testing_inject_stall": [vp, i32],
             "lq_testing_set_prepare_defer_min_blocks": [vp, i32],
+            "lq_testing_set_prepare_slices_int8": [vp, i32],
             "lq_quantize_layer_lazy_workspace": [P(Config), i64, i64, P(sz)],
             "lq_quantize_layer_lazy": [vp, vp, P(Config), vp, i32, i64, i64, i64, vp, i64, vp, vp, vp, vp, vp, i32, i64,
                                        vp, vp, sz],
@@ -288,6 +289,11 @@ def lq_testing_inject_stall(h, on):
 def lq_testing_set_prepare_defer_min_blocks(h, n_blocks):
     """Test hook (include/lq_testing.h): matrix size from which stage 2 defers far updates to the bf16 tensor cores."""
     _check(LQ().lq_testing_set_prepare_defer_min_blocks(h, n_blocks), "lq_testing_set_prepare_defer_min_blocks")
+
+
+def lq_testing_set_prepare_slices_int8(h, on):
+    """Test hook (include/lq_testing.h): digit slices of stage 2's deferred updates as 8-bit integers (default) or bf16."""
+    _check(LQ().lq_testing_set_prepare_slices_int8(h, 1 if on else 0), "lq_testing_set_prepare_slices_int8")
 
 
 def lq_pack_codes(h, codes, bits, packed=None, stream=None):

@@ -25,6 +25,12 @@ extern "C" int lq_testing_set_prepare_defer_min_blocks(lq_handle* h, int32_t n_b
     return LQ_OK;
 }
 
+extern "C" int lq_testing_set_prepare_slices_int8(lq_handle* h, int32_t on) {
+    if (!h) return LQ_ERR_INVALID_ARG;
+    h->prep_slices_int8 = on ? 1 : 0;
+    return LQ_OK;
+}
+
 extern "C" const char* lq_version(void) { return "lq 0.1 (sm_100a)"; }
 
 extern "C" int lq_create(lq_handle** out, int device) {
@@ -45,6 +51,7 @@ extern "C" int lq_create(lq_handle** out, int device) {
     h->wait_limit_ns = LQ_DEFAULT_WAIT_LIMIT_NS;
     h->inject_stall = 0;
     h->prep_defer_min_blocks = LQ_DEFAULT_PREP_DEFER_MIN_BLOCKS;
+    h->prep_slices_int8 = 1;
     if (cudaStreamCreateWithFlags(&h->aux, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_next, cudaEventDisableTiming) != cudaSuccess ||

@@ -33,6 +33,8 @@ struct lq_handle {
     // Stage 2 defers the updates of far tiles to the bf16 tensor cores when the matrix has at least this many
     // 128-column blocks; below that the whole sweep stays on the FP64 MMA (a test hook can change the threshold).
     int prep_defer_min_blocks;
+    // Digit slices of the deferred updates as 8-bit integers (tcgen05 kind::i8, the default) or as bf16 values.
+    int prep_slices_int8;
 };
 constexpr int LQ_DEFAULT_PREP_DEFER_MIN_BLOCKS = 48;
 constexpr unsigned long long LQ_DEFAULT_WAIT_LIMIT_NS = 5ull * 1000ull * 1000ull * 1000ull;
@@ -152,8 +154,8 @@ static inline int64_t lq_ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b
 constexpr int LQ_TC_MAX_PASS = 16;
 constexpr int LQ_TC_MAX_LVL = 5;
 struct lq_tc_gemm_args {
-    const __nv_bfloat16* A_all; int64_t a_rows; int64_t lda;   // a_rows = total rows of A_all
-    const __nv_bfloat16* B_all; int64_t b_rows; int64_t ldb;
+    const void* A_all; int64_t a_rows; int64_t lda;   // a_rows = total rows of A_all; bf16, or 8-bit integers with int8_ops
+    const void* B_all; int64_t b_rows; int64_t ldb;
     float* D; int64_t ldd;
     int64_t M, N, K;
     int n_pass;
@@ -172,6 +174,13 @@ struct lq_tc_gemm_args {
     int n_lvl;
     int lvl_npass[LQ_TC_MAX_LVL];
     int chunk_kb;
+    // 8-bit integer operands (int8_ops != 0): A_all / B_all hold bytes, pass p reads them as signed (a_signed[p] != 0)
+    // or unsigned integers, the products are summed in int32 (exactly), and every partial sum is converted to fp32 and
+    // multiplied by lvl_scale[level] (lvl_scale[0] without levels) as it is added to the running sum.  A k-step and
+    // chunk_kb count 128 integers instead of 64 bf16.
+    int int8_ops;
+    int a_signed[LQ_TC_MAX_PASS], b_signed[LQ_TC_MAX_PASS];
+    float lvl_scale[LQ_TC_MAX_LVL];
 };
 int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a);
 

@@ -1000,6 +1000,7 @@ extern "C" int lq_fit_grid_noalloc(lq_handle* h, void* stream, const lq_config* 
     local.wait_limit_ns = LQ_DEFAULT_WAIT_LIMIT_NS;
     local.inject_stall = 0;
     local.prep_defer_min_blocks = LQ_DEFAULT_PREP_DEFER_MIN_BLOCKS;
+    local.prep_slices_int8 = 1;
     return lq_fit_grid(h ? h : &local, stream, cfg, W, w_dtype, r, c, ldw, dinv, grid, scale, zero, d.scratch,
                        kNoAllocScratchBytes);
 }

@@ -1,4 +1,4 @@
-// bf16 x bf16 -> fp32 "NT" GEMM on the sm_100a tensor cores.
+// bf16 x bf16 -> fp32 (or 8-bit integer x 8-bit integer -> int32) "NT" GEMM on the sm_100a tensor cores.
 //
 //   D[M x N] (+)= alpha * sum_p A_p[M x K] * B_p[N x K]^T        (all row-major, K contiguous)
 //
@@ -23,6 +23,9 @@
 //                 add it (round-to-nearest) to running sums held in registers.  After the
 //                 piece's last segment: scale -> swizzled smem slab -> TMA store, or a TMA
 //                 reduce-add when accumulating into D (no read of D by the SM).
+// With 8-bit integer operands (the digit slices of stage 2's deferred updates) the same pipeline runs tcgen05.mma
+// kind::i8: a k-step is still 128 bytes (128 digits instead of 64 bf16), the accumulator holds int32 sums, which
+// are exact, and the epilogue converts each partial sum to fp32 and scales it by its level's power of two.
 // Every wait on an mbarrier is bounded: when the time limit passes the CTA records
 // LQ_ERR_TIMEOUT in the handle's status word, stops issuing work and leaves.
 #include <cuda.h>
@@ -52,6 +55,11 @@ template <int CTAS> struct Cfg {
     static constexpr int TILE_M = BM * CTAS;
     // Instruction descriptor: D fp32, A and B bf16, both K-major, M = TILE_M, N = 256.
     static constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(BN >> 3) << 17) | (uint32_t(TILE_M >> 4) << 24);
+    // The same for kind::i8: D int32 (2 in bits 4-5), A and B unsigned (0) or signed (1) 8-bit integers in bits 7-9 / 10-12.
+    static constexpr uint32_t idesc_i8(bool a_signed, bool b_signed) {
+        return (2u << 4) | ((a_signed ? 1u : 0u) << 7) | ((b_signed ? 1u : 0u) << 10) | (uint32_t(BN >> 3) << 17) |
+               (uint32_t(TILE_M >> 4) << 24);
+    }
 };
 
 struct KParams {
@@ -80,6 +88,12 @@ struct KParams {
     lq_dev_status* status;
     unsigned long long timeout_ns;
     int stall_bytes;          // test hook: bytes a load barrier expects on top of what its loads deliver (0 in normal use)
+    // 8-bit integer operands: elements per 128-byte k-step, one instruction descriptor per pass (its operands may be
+    // signed or unsigned), and the factor each level's int32 partial sums are scaled by on their way into the fp32 sum
+    int int8_ops;
+    int bk_elems;
+    uint32_t idesc_pass[LQ_TC_MAX_PASS];
+    float lvl_scale[LQ_TC_MAX_LVL];
 };
 
 // ---------------------------------------------------------------- PTX wrappers ----
@@ -200,6 +214,19 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint
         asm volatile(
             "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
             "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(acc) : "memory");
+}
+template <int CTAS>
+__device__ __forceinline__ void umma_i8(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t acc) {
+    if (CTAS == 1)
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+            ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(acc) : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+            "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
             ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(acc) : "memory");
 }
 // The barrier is signalled when all MMAs issued so far by this thread have completed; with two
@@ -381,7 +408,7 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&tmem_base_slot);
     volatile int* abortp = &abort_flag;
 
-    const int k_blocks = (p.K + BK - 1) / BK;
+    const int k_blocks = (p.K + p.bk_elems - 1) / p.bk_elems;
     const int k_iters = k_blocks * p.n_pass;
     const long long u_begin = blockIdx.x / CTAS;
     const long long u_stride = gridDim.x / CTAS;
@@ -404,7 +431,7 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 if (lane == 0) {
                     int pass, kb;
                     seg_item(g, q, pass, kb);
-                    const int k0 = kb * BK;
+                    const int k0 = kb * p.bk_elems;
                     const uint32_t sa = smem_base + stage * C::STAGE_BYTES;
                     const uint32_t sb = sa + A_STAGE_BYTES;
                     if (!PAIR) {
@@ -433,7 +460,8 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         Piece pc;
         while (alive && next_piece(p, u, u_stride, pc)) {
             for (int sg = pc.s0; sg < pc.s1 && alive; ++sg, ++it) {
-                const int seg_len = seg_of(p, k_blocks, k_iters, sg).len;
+                const Seg seg = seg_of(p, k_blocks, k_iters, sg);
+                const int seg_len = seg.len;
                 const uint32_t acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
                 if (!mbar_wait(bar_tempty + 8 * acc, acc_phase ^ 1u, abortp, p, 2)) { alive = false; break; }
@@ -447,9 +475,19 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                         const uint64_t da = make_desc_sw128(sa);
                         const uint64_t db = make_desc_sw128(sa + A_STAGE_BYTES);
 #pragma unroll
-                        for (int kk = 0; kk < BK / UMMA_K; ++kk) {
-                            // advancing 16 bf16 = 32 bytes inside the swizzle row: +2 in the address field
-                            umma_bf16<CTAS>(tmem_d, da + 2 * kk, db + 2 * kk, C::IDESC, (q > 0 || kk > 0) ? 1u : 0u);
+                        if (p.int8_ops) {
+                            int pass, kb;
+                            seg_item(seg, q, pass, kb);
+                            const uint32_t idesc = p.idesc_pass[pass];
+#pragma unroll
+                            for (int kk = 0; kk < BK / UMMA_K; ++kk)      // 32 digits = 32 bytes per instruction: the same +2
+                                umma_i8<CTAS>(tmem_d, da + 2 * kk, db + 2 * kk, idesc, (q > 0 || kk > 0) ? 1u : 0u);
+                        } else {
+#pragma unroll
+                            for (int kk = 0; kk < BK / UMMA_K; ++kk) {
+                                // advancing 16 bf16 = 32 bytes inside the swizzle row: +2 in the address field
+                                umma_bf16<CTAS>(tmem_d, da + 2 * kk, db + 2 * kk, C::IDESC, (q > 0 || kk > 0) ? 1u : 0u);
+                            }
                         }
                         umma_commit<CTAS>(bar_empty + 8 * stage);
                     }
@@ -494,7 +532,17 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     uint32_t v[32];
                     tmem_ld32(tmem_base + ((q * 32u) << 16) + acc * BN + hf * (BN / 2) + ch * EPI_COLS, v);
                     tmem_wait_ld();
-                    if (sg == pc.s0) {
+                    if (p.int8_ops) {
+                        // int32 partial sums (exact) -> fp32, scaled by the level's power of two
+                        const float sc = p.lvl_scale[p.n_lvl > 0 ? sg / p.n_chunks : 0];
+                        if (sg == pc.s0) {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) accr[ch * 32 + i] = static_cast<float>(static_cast<int>(v[i])) * sc;
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) accr[ch * 32 + i] = fmaf(static_cast<float>(static_cast<int>(v[i])), sc, accr[ch * 32 + i]);
+                        }
+                    } else if (sg == pc.s0) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) accr[ch * 32 + i] = __uint_as_float(v[i]);
                     } else {
@@ -627,7 +675,7 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
     if (a.n_pass < 1 || a.n_pass > LQ_TC_MAX_PASS) return LQ_ERR_INVALID_ARG;
     if (a.n_lvl < 0 || a.n_lvl > LQ_TC_MAX_LVL || (a.n_lvl > 0 && a.chunk_kb < 1)) return LQ_ERR_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(a.A_all) & 15) || (reinterpret_cast<uintptr_t>(a.B_all) & 15) ||
-        (reinterpret_cast<uintptr_t>(a.D) & 15) || (a.lda % 8) || (a.ldb % 8) || (a.ldd % 4))
+        (reinterpret_cast<uintptr_t>(a.D) & 15) || (a.lda % (a.int8_ops ? 16 : 8)) || (a.ldb % (a.int8_ops ? 16 : 8)) || (a.ldd % 4))
         return LQ_ERR_INVALID_ARG;
     if (a.a_rows > 0x7fffffffLL || a.b_rows > 0x7fffffffLL || a.K > 0x7fffffffLL || a.M > 0x7fffffffLL ||
         a.N > 0x7fffffffLL)
@@ -643,8 +691,12 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
     const int b_rows_box = BN / ctas_per_tile;
 
     CUtensorMap map_a, map_b, map_d;
-    if (!make_map_2d(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.A_all, a.K, a.a_rows, a.lda, BK, BM) ||
-        !make_map_2d(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.B_all, a.K, a.b_rows, a.ldb, BK, b_rows_box) ||
+    const bool i8 = a.int8_ops != 0;
+    const int bk_elems = i8 ? 2 * BK : BK;                 // a k-step is one 128-byte swizzle row of either type
+    const CUtensorMapDataType op_dt = i8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    const int op_bytes = i8 ? 1 : 2;
+    if (!make_map_2d(&map_a, op_dt, op_bytes, a.A_all, a.K, a.a_rows, a.lda, bk_elems, BM) ||
+        !make_map_2d(&map_b, op_dt, op_bytes, a.B_all, a.K, a.b_rows, a.ldb, bk_elems, b_rows_box) ||
         !make_map_2d(&map_d, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.D, a.N, a.M, a.ldd, EPI_COLS, BM))
         return LQ_ERR_CUDA;
 
@@ -677,9 +729,15 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
     p.status = h->dstatus;
     p.timeout_ns = h->wait_limit_ns;
     p.stall_bytes = h->inject_stall ? 16 : 0;
+    p.int8_ops = i8 ? 1 : 0;
+    p.bk_elems = bk_elems;
+    for (int i = 0; i < LQ_TC_MAX_PASS; ++i)
+        p.idesc_pass[i] = ctas_per_tile == 2 ? Cfg<2>::idesc_i8(a.a_signed[i] != 0, a.b_signed[i] != 0)
+                                             : Cfg<1>::idesc_i8(a.a_signed[i] != 0, a.b_signed[i] != 0);
+    for (int i = 0; i < LQ_TC_MAX_LVL; ++i) p.lvl_scale[i] = a.lvl_scale[i];
     if (p.num_tiles == 0) return LQ_OK;
     {
-        const int k_blocks = static_cast<int>(lq_ceil_div(a.K, BK));
+        const int k_blocks = static_cast<int>(lq_ceil_div(a.K, bk_elems));
         const int k_iters = k_blocks * a.n_pass;
         p.seg_iters = (a.seg_iters > 0 && a.seg_iters < k_iters) ? a.seg_iters : k_iters;
         p.segs_per_tile = static_cast<int>(lq_ceil_div(k_iters, p.seg_iters));

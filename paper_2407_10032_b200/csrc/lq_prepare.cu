@@ -321,10 +321,33 @@ __device__ __forceinline__ void digits_of(double x, int e, __nv_bfloat16 (&d)[NS
         w *= 0.00390625;
     }
 }
+// The same number as signed 8-bit integers for the integer tensor-core path: balanced digits in [-128, 127].  With
+// that range the digits after position s can make up anything in [-128/255, 127/255] of position s, so a digit is
+// chosen to leave its remainder in that interval: q = floor(rest + 128/255).  (Unsigned lower digits would be simpler,
+// but their mean of 127 puts a large common component into every lower level, and the fp32 rounding of that level's
+// sum then costs five bits of the result: measured, 1e-7 instead of 4e-8 on U.)
+__device__ __forceinline__ void digits_of(double x, int e, uint8_t (&d)[NSL]) {
+    double rest = scalbn(x, 8 - e);                     // |rest| <= 127 (exp_for8)
+#pragma unroll
+    for (int s = 0; s < NSL; ++s) {
+        double q = s + 1 < NSL ? floor(rest + 128.0 / 255.0) : rint(rest);
+        q = fmin(fmax(q, -128.0), 127.0);
+        d[s] = static_cast<uint8_t>(static_cast<int8_t>(static_cast<int>(q)));
+        rest = (rest - q) * 256.0;
+    }
+}
+// Exponent for the integer digits: the leading digit must not reach 128.
+__device__ __forceinline__ int exp_for8(double mx) {
+    if (!(mx > 0.0)) return 0;
+    int e = ilogb(mx) + 2;                              // mx 2^(8 - e) < 128
+    if (scalbn(mx, 8 - e) > 127.0) ++e;
+    return e;
+}
 
 // Rows [0, rows) of the panel buffer (K columns each): exponent and slices.  One CTA per row.
+template <typename D>
 __global__ void __launch_bounds__(256)
-slice_rows_kernel(const double* __restrict__ P, int64_t ldp, int K, int* __restrict__ ex, __nv_bfloat16* __restrict__ SL,
+slice_rows_kernel(const double* __restrict__ P, int64_t ldp, int K, int* __restrict__ ex, D* __restrict__ SL,
                   int64_t slice_rows) {
     __shared__ double red[8];
     const int64_t row = blockIdx.x;
@@ -344,13 +367,13 @@ slice_rows_kernel(const double* __restrict__ P, int64_t ldp, int K, int* __restr
     mx = red[0];
 #pragma unroll
     for (int w = 1; w < 8; ++w) mx = fmax(mx, red[w]);
-    const int e = isfinite(mx) ? exp_for(mx) : 0;
+    const int e = isfinite(mx) ? (sizeof(D) == 1 ? exp_for8(mx) : exp_for(mx)) : 0;
     if (threadIdx.x == 0) LQ_AT(ex + row) = e;
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
         const int kx = threadIdx.x + 256 * u;
         if (kx >= K) continue;
-        __nv_bfloat16 d[NSL];
+        D d[NSL];
         digits_of(isfinite(v[u]) ? v[u] : 0.0, e, d);
 #pragma unroll
         for (int s = 0; s < NSL; ++s) LQ_AT(SL + (s * slice_rows + row) * LDP + kx) = d[s];
@@ -359,18 +382,19 @@ slice_rows_kernel(const double* __restrict__ P, int64_t ldp, int K, int* __restr
 
 // Exponents of the columns j >= col0 of the K rows of A that start at row0 (the final rows of U of an outer block).
 __global__ void __launch_bounds__(256)
-col_exp_kernel(const double* __restrict__ A, int64_t cp, int64_t row0, int K, int64_t col0, int* __restrict__ ex) {
+col_exp_kernel(const double* __restrict__ A, int64_t cp, int64_t row0, int K, int64_t col0, int* __restrict__ ex, int int8) {
     const int64_t j = col0 + blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     if (j >= cp) return;
     double mx = 0.0;
     for (int kx = 0; kx < K; ++kx) mx = fmax(mx, fabs(LQ_AT(A + (row0 + kx) * cp + j)));
-    LQ_AT(ex + j) = isfinite(mx) ? exp_for(mx) : 0;
+    LQ_AT(ex + j) = isfinite(mx) ? (int8 ? exp_for8(mx) : exp_for(mx)) : 0;
 }
 
 // Slices of those columns, transposed: SL[s][j][kx] = digit s of A[row0 + kx][j].  64 x 64 tiles through shared memory.
+template <typename D>
 __global__ void __launch_bounds__(256)
 slice_cols_kernel(const double* __restrict__ A, int64_t cp, int64_t row0, int K, int64_t col0, const int* __restrict__ ex,
-                  __nv_bfloat16* __restrict__ SL, int64_t slice_rows) {
+                  D* __restrict__ SL, int64_t slice_rows) {
     __shared__ double tile[64][65];
     const int64_t j0 = col0 + (int64_t)blockIdx.x * 64;
     const int k0 = blockIdx.y * 64;
@@ -385,7 +409,7 @@ slice_cols_kernel(const double* __restrict__ A, int64_t cp, int64_t row0, int K,
         const int64_t j = j0 + b;
         if (j >= cp || k0 + a >= K) continue;
         const double x = tile[a][b];
-        __nv_bfloat16 d[NSL];
+        D d[NSL];
         digits_of(isfinite(x) ? x : 0.0, LQ_AT(ex + j), d);
 #pragma unroll
         for (int s = 0; s < NSL; ++s) LQ_AT(SL + (s * slice_rows + j) * LDP + k0 + a) = d[s];
@@ -677,18 +701,22 @@ PrepLayout prep_layout(int64_t c) {
 // with Q_j^(k) = P_j^(k)^T left of the outer block (the Cholesky part) and the final row k of U right of it (the
 // Gauss-Jordan part).  Both operands go through the digit slices; row bands of at most `band` rows at a time.
 int deferred_update(lq_handle* h, cudaStream_t st, double* A, int64_t cp, int64_t o_lo, int64_t o_hi, const double* Pob, int* ex,
-                    __nv_bfloat16* SL, float* Ta, float* Tb, int64_t band) {
+                    void* SL, float* Ta, float* Tb, int64_t band) {
     const int K = static_cast<int>((o_hi - o_lo + 1) * NB);
     const int64_t top = o_lo * NB;                     // rows [0, top) are updated
     const int64_t right0 = (o_hi + 1) * NB;            // columns [right0, cp) on the right of the outer block
     const int64_t n_right = cp - right0;
-    slice_rows_kernel<<<static_cast<unsigned>(top), 256, 0, st>>>(Pob, LDP, K, ex, SL, cp);
+    // digits as 8-bit integers for tcgen05 kind::i8 (twice the rate of the bf16 form), or as bf16 values
+    const bool i8 = h->prep_slices_int8 != 0;
+    if (i8) slice_rows_kernel<uint8_t><<<static_cast<unsigned>(top), 256, 0, st>>>(Pob, LDP, K, ex, static_cast<uint8_t*>(SL), cp);
+    else slice_rows_kernel<__nv_bfloat16><<<static_cast<unsigned>(top), 256, 0, st>>>(Pob, LDP, K, ex, static_cast<__nv_bfloat16*>(SL), cp);
     LQ_LAUNCH_CHECK();
     if (n_right > 0) {
-        col_exp_kernel<<<static_cast<unsigned>(lq_ceil_div(n_right, 256)), 256, 0, st>>>(A, cp, top, K, right0, ex);
+        col_exp_kernel<<<static_cast<unsigned>(lq_ceil_div(n_right, 256)), 256, 0, st>>>(A, cp, top, K, right0, ex, i8 ? 1 : 0);
         LQ_LAUNCH_CHECK();
         dim3 g(static_cast<unsigned>(lq_ceil_div(n_right, 64)), static_cast<unsigned>(lq_ceil_div(K, 64)));
-        slice_cols_kernel<<<g, 256, 0, st>>>(A, cp, top, K, right0, ex, SL, cp);
+        if (i8) slice_cols_kernel<uint8_t><<<g, 256, 0, st>>>(A, cp, top, K, right0, ex, static_cast<uint8_t*>(SL), cp);
+        else slice_cols_kernel<__nv_bfloat16><<<g, 256, 0, st>>>(A, cp, top, K, right0, ex, static_cast<__nv_bfloat16*>(SL), cp);
         LQ_LAUNCH_CHECK();
     }
     // passes: the leading pair alone (exact), then the pairs of levels s + t = NSL + 1 down to 3, least significant first
@@ -700,12 +728,16 @@ int deferred_update(lq_handle* h, cudaStream_t st, double* A, int64_t cp, int64_
     lead.K = K;
     lead.alpha = 1.0f;
     lead.n_pass = 1;
-    lead.seg_iters = 4;                                // 256 digit products per partial sum: far below 2^24
+    lead.seg_iters = i8 ? 2 : 4;                       // 256 digit products per partial sum: far below 2^24
+    lead.int8_ops = i8 ? 1 : 0;
+    lead.a_signed[0] = lead.b_signed[0] = 1;           // all digits are signed
+    lead.lvl_scale[0] = 1.0f / 65536.0f;               // 2^-8 2^-8 (the bf16 digits carry their power of two themselves)
     lq_tc_gemm_args tail = lead;
     tail.seg_iters = 0;
     tail.n_pass = 0;
     tail.n_lvl = 0;
-    tail.chunk_kb = 2;                                 // 128 of the inner dimension per segment: at most 5 x 128 x 2^14 < 2^24 per sum
+    tail.chunk_kb = i8 ? 1 : 2;                        // 128 of the inner dimension per segment: at most 5 x 128 x 2^14 < 2^24 per sum
+                                                       // (the same bound for the integer digits)
     int pair_s[LQ_TC_MAX_PASS], pair_t[LQ_TC_MAX_PASS];
     for (int lvl = NSL + 1; lvl >= 3; --lvl) {
         int cnt = 0;
@@ -714,9 +746,11 @@ int deferred_update(lq_handle* h, cudaStream_t st, double* A, int64_t cp, int64_
             if (tdig < 1 || tdig > NSL) continue;
             pair_s[tail.n_pass] = sdig - 1;
             pair_t[tail.n_pass] = tdig - 1;
+            tail.a_signed[tail.n_pass] = tail.b_signed[tail.n_pass] = 1;
             ++tail.n_pass;
             ++cnt;
         }
+        tail.lvl_scale[tail.n_lvl] = static_cast<float>(ldexp(1.0, -8 * lvl));
         tail.lvl_npass[tail.n_lvl++] = cnt;
     }
     for (int64_t b0 = 0; b0 < top; b0 += band) {
@@ -884,7 +918,7 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
             if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_rest, 0));
             rest_pending = false;
             int rc = deferred_update(h, st, A, cp, o_lo, o_hi, Pob, reinterpret_cast<int*>(wsp + L.ex),
-                                     reinterpret_cast<__nv_bfloat16*>(wsp + L.sl), reinterpret_cast<float*>(wsp + L.ta),
+                                     wsp + L.sl, reinterpret_cast<float*>(wsp + L.ta),
                                      reinterpret_cast<float*>(wsp + L.tb), L.band);
             if (rc) return rc;
         }

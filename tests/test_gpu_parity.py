@@ -198,17 +198,20 @@ def test_stage2_prepare(lq, h, c):                                              
     ws = ws_for(lq, lq.lq_prepare_hinv_workspace(c))
     # both forms of the sweep: everything on the FP64 MMA (what matrices of this size get by default), and with the
     # far tiles' updates deferred to the bf16 tensor cores (what wide layers get; forced here through the test hook)
-    for defer_from in ((-1, 0) if c > 1024 else (-1,)):
+    # (the deferred products with their digit slices as 8-bit integers, the default, and as bf16 values)
+    for defer_from, int8 in (((-1, True), (0, True), (0, False)) if c > 1024 else ((-1, True),)):
         lq.lq_testing_set_prepare_defer_min_blocks(h, defer_from)
+        lq.lq_testing_set_prepare_slices_int8(h, int8)
         try:
             U.fill_(float("nan"))
             lq.lq_prepare_hinv(h, H32.cuda(), U, dinv, ws, 0.01)
             lq.lq_sync_status(h)
         finally:
             lq.lq_testing_set_prepare_defer_min_blocks(h, -1)
+            lq.lq_testing_set_prepare_slices_int8(h, True)
         Ug, dg = f64(U), f64(dinv)
         assert np.array_equal(Ug, np.triu(Ug)) and (np.diag(Ug) > 0).all()
-        print(f"stage 2 c={c} ({'deferred' if defer_from == 0 else 'default'}): max |dU| / max |U| = "
+        print(f"stage 2 c={c} ({('deferred, int8 slices' if int8 else 'deferred, bf16 slices') if defer_from == 0 else 'default'}): max |dU| / max |U| = "
               f"{np.abs(Ug - Uo).max() / np.abs(Uo).max():.2e}, dinv rel err {np.abs(dg / dinvo - 1).max():.2e}")
         assert np.abs(Ug - Uo).max() <= 2e-7 * np.abs(Uo).max() + 1e-7 * np.abs(Uo).max()
         np.testing.assert_allclose(dg, dinvo, rtol=3e-7)
