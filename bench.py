@@ -290,12 +290,14 @@ def stage_rooflines(st, r, c, n, stage_ms, pk, pipes, w_bytes, exact=False):
     }
     dfrac = stage2_deferred_fraction(c)
     if dfrac > 0.0:
-        # wide layers: most update products run on the bf16 tensor cores as 15 digit-slice products each, so the
-        # algorithmic rate can exceed the FP64 pipe's peak; what the tensor pipe executes is reported beside it
+        # wide layers: most update products run on the integer tensor cores as 15 digit-slice products each, so the
+        # algorithmic rate can exceed the FP64 pipe's peak; what the tensor pipe executes is reported beside it, against
+        # the measured sustained bf16 rate times the nominal int8 / bf16 ratio (there is no measured int8 figure)
         ex = STAGE2_PRODUCTS * dfrac * s2
-        out["prepare_hinv"].update({"bound": "tensor (bf16 digit slices) for the deferred updates, fp64 tensor for the rest",
-                                    "deferred_fraction": dfrac, "executed_bf16": ex,
-                                    "executed_frac_of_sustained": ex / pk["tf_sust"]})
+        out["prepare_hinv"].update({"bound": "tensor (int8 digit slices) for the deferred updates, fp64 tensor for the rest",
+                                    "deferred_fraction": dfrac, "executed_int8_tops": ex,
+                                    "int8_peak": INT8_OVER_BF16 * pk["tf_sust"],
+                                    "executed_frac_of_sustained": ex / (INT8_OVER_BF16 * pk["tf_sust"])})
     if exact:
         # Algorithm 2: r rows x c steps x a c x c downdate = r c^3 fp64 FMAs, half of which touch weights already
         # quantised and need not be done
@@ -306,7 +308,8 @@ def stage_rooflines(st, r, c, n, stage_ms, pk, pipes, w_bytes, exact=False):
 
 
 STAGE4_PRODUCTS = 6     # bf16 products the library issues per fp32 product of the lazy update
-STAGE2_PRODUCTS = 15    # bf16 digit-slice products per fp64 product of stage 2's deferred updates
+STAGE2_PRODUCTS = 15    # 8-bit integer digit-slice products per fp64 product of stage 2's deferred updates
+INT8_OVER_BF16 = 2.0    # nominal ratio of the dense int8 and bf16 tensor rates (4.5 vs 2.25 P op/s)
 STAGE2_DEFER_MIN_BLOCKS, STAGE2_OUTER = 48, 8
 
 
@@ -461,7 +464,7 @@ def extra_workloads(lq, h, dev, rank, pk, pipes, args):
                      "stage_roofline_frac": {k: v["frac"] for k, v in roofs.items()},
                      "quantize_layer_executed_frac_of_sustained": roofs["quantize_layer"].get("executed_frac_of_sustained"),
                      "prepare_hinv_deferred_fraction": roofs["prepare_hinv"].get("deferred_fraction"),
-                     "prepare_hinv_executed_bf16_frac_of_sustained": roofs["prepare_hinv"].get("executed_frac_of_sustained"),
+                     "prepare_hinv_executed_int8_frac_of_sustained": roofs["prepare_hinv"].get("executed_frac_of_sustained"),
                      "gpu_launches_per_step": launches // steps}
             if share is not None:
                 entry["note"] = f"stages 1-2 shared with {share_name} (same layer, same Hessian); their times are that run's"

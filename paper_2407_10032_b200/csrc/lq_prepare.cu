@@ -27,16 +27,17 @@
 //              outer block's own diagonal and panel kernels read;
 //   deferred : all other tiles (rows above the outer block, columns outside it) get the updates of the outer
 //              block's steps in one product of inner dimension 1024 when the outer block is complete, on the
-//              bf16 tensor cores (tcgen05, lq_tc_gemm).  The fp64 operands are cut into S = 5 slices of 8-bit
-//              integer digits below a per-row power of two; a product of two slices is a sum of integers that
-//              the fp32 accumulator holds exactly, the leading slice pair (s = t = 1) is kept as a result of its
-//              own and the other pairs with s + t <= S + 1 are combined, least significant level first, in fp32;
-//              the two results are added in fp64 and scaled back (15 bf16 products in all).  Worth ~39 bits relative
-//              to the largest entry of a row; entries of one row of a panel differ by the ratio of the channel scales,
-//              several bits, which is why four slices are not enough (U then comes out 1e-7 to 5e-7 of its largest
-//              entry off, measured here and in the CPU emulation alike; five hold it to 1e-8).  An fp32 accumulation
-//              of split floating-point operands keeps ~20 bits whatever the number of terms and moves 0.1 - 0.2 % of
-//              the codes.
+//              integer tensor cores (tcgen05 kind::i8, lq_tc_gemm).  The fp64 operands are cut into S = 5 slices of
+//              balanced 8-bit integer digits below a per-row power of two; a product of two slices is a sum of
+//              integers that the int32 accumulator holds exactly, the leading slice pair (s = t = 1) is kept as a
+//              result of its own and the other pairs with s + t <= S + 1 are combined, least significant level first,
+//              in fp32; the two results are added in fp64 and scaled back (15 integer products in all).  Worth ~39 bits
+//              relative to the largest entry of a row; entries of one row of a panel differ by several bits, which is
+//              why four slices are not enough (U then comes out 1e-7 to 5e-7 of its largest entry off, measured here and
+//              in the CPU emulation alike; five hold it to 1e-8).  An fp32 accumulation of split floating-point
+//              operands keeps ~20 bits whatever the number of terms and moves 0.1 - 0.2 % of the codes.  The same
+//              slices as bf16 values on the bf16 path (exact in its fp32 accumulator per 128 of the inner dimension)
+//              remain selectable for tests; the integer path runs the stage 1.2 - 1.5 x faster.
 #include "lq_common.cuh"
 
 namespace {
@@ -728,7 +729,8 @@ int deferred_update(lq_handle* h, cudaStream_t st, double* A, int64_t cp, int64_
     lead.K = K;
     lead.alpha = 1.0f;
     lead.n_pass = 1;
-    lead.seg_iters = i8 ? 2 : 4;                       // 256 digit products per partial sum: far below 2^24
+    lead.seg_iters = i8 ? 0 : 4;                       // bf16: 256 digit products per partial sum, far below 2^24; integers: the
+                                                       // whole inner dimension in int32, at most 1024 x 2^14 = 2^24, exact in fp32 too
     lead.int8_ops = i8 ? 1 : 0;
     lead.a_signed[0] = lead.b_signed[0] = 1;           // all digits are signed
     lead.lvl_scale[0] = 1.0f / 65536.0f;               // 2^-8 2^-8 (the bf16 digits carry their power of two themselves)
@@ -736,8 +738,11 @@ int deferred_update(lq_handle* h, cudaStream_t st, double* A, int64_t cp, int64_
     tail.seg_iters = 0;
     tail.n_pass = 0;
     tail.n_lvl = 0;
-    tail.chunk_kb = i8 ? 1 : 2;                        // 128 of the inner dimension per segment: at most 5 x 128 x 2^14 < 2^24 per sum
-                                                       // (the same bound for the integer digits)
+    // bf16 digits: 128 of the inner dimension per segment, at most 5 x 128 x 2^14 < 2^24 per partial sum, which the fp32
+    // accumulator holds exactly.  Integer digits: the int32 accumulator holds a level's sum over the whole inner
+    // dimension exactly (5 x 1024 x 2^14 < 2^27), so a level is one segment; its conversion to fp32 rounds at 2^-24 of
+    // a level that lies 2^-8 or more below the leading one.
+    tail.chunk_kb = i8 ? 8 : 2;
     int pair_s[LQ_TC_MAX_PASS], pair_t[LQ_TC_MAX_PASS];
     for (int lvl = NSL + 1; lvl >= 3; --lvl) {
         int cnt = 0;
