@@ -711,8 +711,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama3-8b-q_proj-nu4", choices=sorted(WORKLOADS) + sorted(BLOCKS))
-    ap.add_argument("--ref-tokens", type=int, default=32768)
-    ap.add_argument("--ref-rows", type=int, default=512)
+    ap.add_argument("--ref-tokens", type=int, default=65536)
+    ap.add_argument("--ref-rows", type=int, default=1024)
     ap.add_argument("--chunk", type=int, default=0, help="tokens per Hessian call (0 = all at once)")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer end-to-end leg (e2e is then null)")
     ap.add_argument("--no-cpu-baseline", action="store_true",
