@@ -47,18 +47,29 @@ extern "C" int lq_create(lq_handle** out, int device) {
     h->sm_count = prop.multiProcessorCount;
     h->dstatus = nullptr;
     h->aux = nullptr;
-    h->ev_fork = h->ev_next = h->ev_rest = nullptr;
+    h->chain = h->mid = nullptr;
+    h->ev_fork = h->ev_next = h->ev_rest = h->ev_join = h->ev_next2 = nullptr;
     h->wait_limit_ns = LQ_DEFAULT_WAIT_LIMIT_NS;
     h->inject_stall = 0;
     h->prep_defer_min_blocks = LQ_DEFAULT_PREP_DEFER_MIN_BLOCKS;
     h->prep_slices_int8 = 1;
-    if (cudaStreamCreateWithFlags(&h->aux, cudaStreamNonBlocking) != cudaSuccess ||
+    int prio_least = 0, prio_greatest = 0;
+    if (cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest) != cudaSuccess) prio_least = prio_greatest = 0;
+    if (cudaStreamCreateWithPriority(&h->aux, cudaStreamNonBlocking, prio_least) != cudaSuccess ||
+        cudaStreamCreateWithPriority(&h->chain, cudaStreamNonBlocking, prio_greatest) != cudaSuccess ||
+        cudaStreamCreateWithPriority(&h->mid, cudaStreamNonBlocking, prio_greatest < prio_least ? prio_greatest + 1 : prio_least) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_next2, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_next, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_rest, cudaEventDisableTiming) != cudaSuccess) {
         if (h->ev_rest) cudaEventDestroy(h->ev_rest);
         if (h->ev_next) cudaEventDestroy(h->ev_next);
         if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+        if (h->ev_join) cudaEventDestroy(h->ev_join);
+        if (h->ev_next2) cudaEventDestroy(h->ev_next2);
+        if (h->mid) cudaStreamDestroy(h->mid);
+        if (h->chain) cudaStreamDestroy(h->chain);
         if (h->aux) cudaStreamDestroy(h->aux);
         delete h;
         return LQ_ERR_CUDA;
@@ -69,6 +80,10 @@ extern "C" int lq_create(lq_handle** out, int device) {
         cudaEventDestroy(h->ev_rest);
         cudaEventDestroy(h->ev_next);
         cudaEventDestroy(h->ev_fork);
+        cudaEventDestroy(h->ev_join);
+        cudaEventDestroy(h->ev_next2);
+        cudaStreamDestroy(h->mid);
+        cudaStreamDestroy(h->chain);
         cudaStreamDestroy(h->aux);
         delete h;
         return LQ_ERR_CUDA;
@@ -82,6 +97,12 @@ extern "C" int lq_destroy(lq_handle* h) {
     cudaFree(h->dstatus);
     if (h->aux) {
         cudaStreamSynchronize(h->aux);
+        cudaStreamSynchronize(h->chain);
+        cudaStreamSynchronize(h->mid);
+        cudaEventDestroy(h->ev_join);
+        cudaEventDestroy(h->ev_next2);
+        cudaStreamDestroy(h->mid);
+        cudaStreamDestroy(h->chain);
         cudaEventDestroy(h->ev_rest);
         cudaEventDestroy(h->ev_next);
         cudaEventDestroy(h->ev_fork);

@@ -24,7 +24,11 @@ struct lq_handle {
     // stream already works on the next block column.  Null in a handle that owns no stream
     // (everything then runs on the caller's stream).
     cudaStream_t aux;
-    cudaEvent_t ev_fork, ev_next, ev_rest;
+    // Stage 2's serial chain (diagonal block, panel, "next" update) runs on a stream of the highest priority, so that
+    // its CTAs are placed ahead of the queued CTAs of the bulk update; `mid` (one priority level below) takes the
+    // updates that the chain needs two steps later.
+    cudaStream_t chain, mid;
+    cudaEvent_t ev_fork, ev_next, ev_rest, ev_join, ev_next2;
     // Time limit of every bounded wait inside a kernel launched through this handle (nanoseconds).
     unsigned long long wait_limit_ns;
     // Test hook: nonzero makes the load barriers of the tensor-core contraction expect bytes that never arrive, so that

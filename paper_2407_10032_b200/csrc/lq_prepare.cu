@@ -125,6 +125,14 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
+// Programmatic dependent launch along the serial chain: a kernel launched with launch_chained() may be placed on the
+// SMs while its predecessor in the stream still runs; it calls chain_wait() before it touches anything the predecessor
+// wrote (the wait returns when the predecessor has completed and its writes are visible).  chain_release() in the
+// predecessor says that the successor's CTAs may be placed from now on; without it they are placed when the
+// predecessor ends.  In a kernel launched the plain way both are no-ops.
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ------------------------------------------------------------ tile product, K = 128 --
 // C[TM x TN] = beta * C + alpha * A[TM x 128] * op(B), all fp64 row-major, by 256 threads = 8 warps
 // arranged WMW x (8 / WMW); each warp owns an (8 MI) x 32 patch as MI x 4 MMA tiles, so
@@ -250,6 +258,7 @@ __global__ void __launch_bounds__(GEMM_THREADS, 2)
 panel_kernel(double* __restrict__ A, int64_t cp, int k, double* __restrict__ Pbuf, int64_t ldp, double* __restrict__ Q) {
     extern __shared__ double smem[];
     const int t = blockIdx.x >> 2, q = blockIdx.x & 3;
+    chain_wait();                                       // launched behind the diagonal kernel of this step
     const double* Vk = A + (int64_t)k * NB * cp + (int64_t)k * NB;
     TileOut o = {};
     if (t < k) {
@@ -270,34 +279,42 @@ panel_kernel(double* __restrict__ A, int64_t cp, int k, double* __restrict__ Pbu
 // Step k, eager update of tiles (i, j), i < k: A[i][j] -= P_i Q[:, j] (A[i][k] = -P_i V_k).  A launch covers the
 // block rows i_base + blockIdx.y and the block columns j_base + (blockIdx.x >> 1) (128 x 64 tiles).  The tiles of
 // block column k-1 and of block row k-1 are all that step k-1's diagonal and panel kernels read, so they can be
-// updated first ("next") and the remainder ("rest") left to run beside step k-1:
+// updated first ("next") and the remainder ("rest") left to run beside step k-1.  With a look-ahead of two steps the
+// tiles of block row and column k-2 ("next2") leave the rest as well, so that step k-1's "next" update waits for a
+// short launch only and the rest of step k has two chain steps to finish:
 //   part 0: every tile of the launch;  part 2: all but block row and block column k-1;
-//   part 1: next only, grid 4 nblk x 1, 64 x 64 tiles -- block tile t < k is (t, k-1), t >= k is (k-1, t).
+//   part 4: all but block rows and block columns k-1 and k-2;
+//   part 1: next only, grid 4 nblk x 1, 64 x 64 tiles -- block tile t < k is (t, k-1), t >= k is (k-1, t);
+//   part 3: next2 only, same grid -- block tile t < k-1 is (t, k-2), t >= k is (k-2, t) (tile (k-2, k-1) belongs to next).
 __global__ void __launch_bounds__(GEMM_THREADS, 2)
 update_kernel(double* __restrict__ A, int64_t cp, int k, int part, int i_base, int j_base, const double* __restrict__ Pbuf,
               int64_t ldp, const double* __restrict__ Q) {
     extern __shared__ double smem[];
     int i, j, r0, c0;
-    if (part == 1) {
+    if (part == 1 || part == 3) {
         const int t = blockIdx.x >> 2;
-        if (t < k) { i = t; j = k - 1; } else { i = k - 1; j = t; }
+        const int nx = part == 1 ? k - 1 : k - 2;         // the block row and column this launch brings up to date
+        if (part == 3 && t == k - 1) return;
+        if (t <= nx) { i = t; j = nx; } else { i = nx; j = t; }
         r0 = ((blockIdx.x >> 1) & 1) * 64;
         c0 = (blockIdx.x & 1) * 64;
     } else {
         j = j_base + (blockIdx.x >> 1);
         i = i_base + blockIdx.y;
-        if (part == 2 && (j == k - 1 || i == k - 1)) return;
+        if (part >= 2 && (j == k - 1 || i == k - 1)) return;
+        if (part == 4 && (j == k - 2 || i == k - 2)) return;
         r0 = 0;
         c0 = (blockIdx.x & 1) * 64;
     }
     if (j < i) return;                                  // strictly lower tiles of the symmetric part
+    if (part == 1) chain_release();                     // the next step's diagonal kernel may take its SM now; it waits for this launch to end
     const double* Pi = Pbuf + ((int64_t)i * NB + r0) * ldp;
     TileOut o = {};
     o.C = A + ((int64_t)i * NB + r0) * cp + (int64_t)j * NB + c0; o.ldc = cp;
     // A[i][k] = -P_i V_k;  A[i][j] -= P_i Q[:, j] otherwise
     const double* Bsrc = (j == k) ? A + (int64_t)k * NB * cp + (int64_t)k * NB + c0 : Q + (int64_t)j * NB + c0;
     const double beta = (j == k) ? 0.0 : 1.0;
-    if (part == 1) gemm_tile<2, 4, false>(Pi, ldp, Bsrc, cp, -1.0, beta, o, smem);
+    if (part == 1 || part == 3) gemm_tile<2, 4, false>(Pi, ldp, Bsrc, cp, -1.0, beta, o, smem);
     else gemm_tile<4, 4, false>(Pi, ldp, Bsrc, cp, -1.0, beta, o, smem);
 }
 
@@ -538,6 +555,7 @@ diag_block_kernel(double* __restrict__ A, int64_t cp, int64_t blk, int64_t c_rea
     const int fr = lane >> 2, fk = lane & 3;
     constexpr int NW = DIAG_THREADS / 32;
 
+    chain_wait();                                       // launched behind the previous step's "next" update
     for (int idx = tid; idx < NB * (NB / 2); idx += DIAG_THREADS) {
         const int row = idx >> 6, c2 = (idx & 63) * 2;
         cp_async16(S + row * DP + c2, base + (int64_t)row * cp + c2);
@@ -625,6 +643,7 @@ diag_block_kernel(double* __restrict__ A, int64_t cp, int64_t blk, int64_t c_rea
         __syncthreads();
     }
 
+    chain_release();                                    // the panel kernel's CTAs may be placed while the block is written back
     for (int idx = tid; idx < NB * (NB / 2); idx += DIAG_THREADS) {
         const int row = idx >> 6, c2 = (idx & 63) * 2;
         double2 v;
@@ -674,6 +693,19 @@ __global__ void dinv_kernel(const double* __restrict__ part, int64_t c, int n_ch
     LQ_AT(dinv + j) = static_cast<float>(t);
 }
 
+// Launches a kernel of the chain so that it may be placed before its predecessor in the stream has ended (the kernel
+// itself waits with chain_wait()).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 struct PrepLayout {
     int64_t nblk, cp, band;
     size_t scal, a, pbuf, q, ex, sl, ta, tb, total, panel_bytes;
@@ -688,7 +720,7 @@ PrepLayout prep_layout(int64_t c) {
     L.a = off;    off += lq_align_up(static_cast<size_t>(L.cp) * L.cp * sizeof(double), 256);
     L.panel_bytes = lq_align_up(static_cast<size_t>(L.cp) * NB * sizeof(double), 256);
     L.pbuf = off; off += lq_align_up(static_cast<size_t>(L.cp) * LDP * sizeof(double), 256);   // the panels of one outer block
-    L.q = off;    off += 2 * L.panel_bytes;            // Q is double-buffered: one step's update may still read it while the next is written
+    L.q = off;    off += 4 * L.panel_bytes;            // Q of the last four steps: with a look-ahead of two steps the rest of step k+2's update may still read its Q while step k's is written
     L.ex = off;   off += lq_align_up(static_cast<size_t>(L.cp) * sizeof(int), 256);
     L.sl = off;   off += lq_align_up(static_cast<size_t>(NSL) * L.cp * LDP * sizeof(__nv_bfloat16), 256);
     L.ta = off;   off += lq_align_up(static_cast<size_t>(L.band) * L.cp * sizeof(float), 256);
@@ -851,59 +883,91 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
     // all other tiles get its steps' updates in one product on the bf16 tensor cores (deferred_update).
     cudaStream_t aux = h->aux;
     const bool fork = aux != nullptr && nblk > 2;
+    // With the fork the sweep leaves the caller's stream: the chain goes to the handle's high-priority stream `cs`, the
+    // bulk of the eager updates to the low-priority `aux`; the caller's stream joins again after the last step.
+    cudaStream_t cs = fork ? h->chain : st;
     if (fork) {
         LQ_CUDA_TRY(cudaEventRecord(h->ev_fork, st));
         LQ_CUDA_TRY(cudaStreamWaitEvent(aux, h->ev_fork, 0));
+        LQ_CUDA_TRY(cudaStreamWaitEvent(cs, h->ev_fork, 0));
     }
     double* Pob = reinterpret_cast<double*>(wsp + L.pbuf);
     // Small matrices are bound by the serial chain of diagonal blocks, not by the updates: they stay on the FP64 MMA
     // throughout (one outer block as wide as the matrix).
     const bool defer = nblk > OBB && nblk >= h->prep_defer_min_blocks;
     const int64_t obb = defer ? OBB : nblk;
-    if (defer) LQ_CUDA_TRY(cudaMemsetAsync(wsp + L.sl, 0, static_cast<size_t>(NSL) * cp * LDP * sizeof(__nv_bfloat16), st));
-    bool rest_pending = false;
+    if (defer) LQ_CUDA_TRY(cudaMemsetAsync(wsp + L.sl, 0, static_cast<size_t>(NSL) * cp * LDP * sizeof(__nv_bfloat16), cs));
+    bool rest_pending = false, next2_pending = false;
+    const bool deep = fork && !defer && h->mid != nullptr;
     const int64_t n_ob = lq_ceil_div(nblk, obb);
     for (int64_t m = n_ob - 1; m >= 0; --m) {
         const int64_t o_lo = m * obb;
         const int64_t o_hi = (o_lo + obb < nblk ? o_lo + obb : nblk) - 1;
         const int obw = static_cast<int>(o_hi - o_lo + 1);
         for (int64_t k = o_hi; k >= o_lo; --k) {
-            // this step's 128 columns of the panel buffer: its place in the outer block, or one of two alternating
-            // slots when nothing is deferred (the previous step's update may still be reading the other one)
-            double* Pk = Pob + (defer ? k - o_lo : (k & 1)) * NB;
-            double* Qk = reinterpret_cast<double*>(wsp + L.q + (k & 1) * L.panel_bytes);
+            // this step's 128 columns of the panel buffer: its place in the outer block, or one of four alternating
+            // slots when nothing is deferred (the updates of the two steps before may still be reading theirs)
+            double* Pk = Pob + (defer ? k - o_lo : (k & 3)) * NB;
+            double* Qk = reinterpret_cast<double*>(wsp + L.q + (k & 3) * L.panel_bytes);
             const int ki = static_cast<int>(k);
-            diag_block_kernel<<<1, DIAG_THREADS, DIAG_SMEM, st>>>(A, cp, k, c, h->dstatus);
-            LQ_LAUNCH_CHECK();
+            LQ_CUDA_TRY(launch_chained(diag_block_kernel, dim3(1), dim3(DIAG_THREADS), DIAG_SMEM, cs, A, cp, k, c, h->dstatus));
             if (nblk > 1) {
-                panel_kernel<<<static_cast<unsigned>(4 * (nblk - 1)), GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, ki, Pk, LDP, Qk);
-                LQ_LAUNCH_CHECK();
+                LQ_CUDA_TRY(launch_chained(panel_kernel, dim3(static_cast<unsigned>(4 * (nblk - 1))), dim3(GEMM_THREADS), GEMM_SMEM, cs,
+                                           A, cp, ki, Pk, LDP, Qk));
             }
             if (k == 0) break;
             // eager tiles of step k: block rows [o_lo, k) over the whole width, block rows [0, o_lo) over the
             // outer block's columns
             const int rows_in = static_cast<int>(k - o_lo);
             if (!fork || k == o_lo) {
-                if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_rest, 0));
+                if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(cs, h->ev_rest, 0));
                 rest_pending = false;
                 if (rows_in > 0) {
                     dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(rows_in));
-                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, ki, 0, static_cast<int>(o_lo), 0, Pk, LDP, Qk);
+                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, cs>>>(A, cp, ki, 0, static_cast<int>(o_lo), 0, Pk, LDP, Qk);
                     LQ_LAUNCH_CHECK();
                 }
                 if (o_lo > 0) {
                     dim3 g(static_cast<unsigned>(2 * obw), static_cast<unsigned>(o_lo));
-                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, ki, 0, 0, static_cast<int>(o_lo), Pk, LDP, Qk);
+                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, cs>>>(A, cp, ki, 0, 0, static_cast<int>(o_lo), Pk, LDP, Qk);
                     LQ_LAUNCH_CHECK();
                 }
                 continue;
             }
-            if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_rest, 0));     // step k+1's rest touched the same tiles
-            update_kernel<<<static_cast<unsigned>(4 * nblk), GEMM_THREADS, GEMM_SMEM, st>>>(A, cp, ki, 1, 0, 0, Pk, LDP, Qk);
+            if (deep) {
+                // Look-ahead of two steps (nothing deferred, o_lo = 0).  "next" (block row and column k-1) stays on the
+                // chain and waits only for step k+1's "next2", which touched the same tiles; "next2" (block row and
+                // column k-2) runs on the middle stream once step k+1's rest has left those tiles; the rest of step k
+                // follows step k+1's on the low-priority stream.
+                if (k >= 2) LQ_CUDA_TRY(cudaEventRecord(h->ev_next, cs));      // the panel of step k is complete (next2 and the rest need no more)
+                if (next2_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(cs, h->ev_next2, 0));
+                next2_pending = false;
+                update_kernel<<<static_cast<unsigned>(4 * nblk), GEMM_THREADS, GEMM_SMEM, cs>>>(A, cp, ki, 1, 0, 0, Pk, LDP, Qk);
+                LQ_LAUNCH_CHECK();
+                if (k >= 2) {
+                    LQ_CUDA_TRY(cudaStreamWaitEvent(h->mid, h->ev_next, 0));
+                    if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(h->mid, h->ev_rest, 0));
+                    update_kernel<<<static_cast<unsigned>(4 * nblk), GEMM_THREADS, GEMM_SMEM, h->mid>>>(A, cp, ki, 3, 0, 0, Pk, LDP, Qk);
+                    LQ_LAUNCH_CHECK();
+                    LQ_CUDA_TRY(cudaEventRecord(h->ev_next2, h->mid));
+                    next2_pending = true;
+                }
+                if (k >= 3) {
+                    LQ_CUDA_TRY(cudaStreamWaitEvent(aux, h->ev_next, 0));
+                    dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(k - 2));
+                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, aux>>>(A, cp, ki, 4, 0, 0, Pk, LDP, Qk);
+                    LQ_LAUNCH_CHECK();
+                    LQ_CUDA_TRY(cudaEventRecord(h->ev_rest, aux));
+                    rest_pending = true;
+                }
+                continue;
+            }
+            if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(cs, h->ev_rest, 0));     // step k+1's rest touched the same tiles
+            update_kernel<<<static_cast<unsigned>(4 * nblk), GEMM_THREADS, GEMM_SMEM, cs>>>(A, cp, ki, 1, 0, 0, Pk, LDP, Qk);
             LQ_LAUNCH_CHECK();
             rest_pending = false;
             if (rows_in > 1 || o_lo > 0) {
-                LQ_CUDA_TRY(cudaEventRecord(h->ev_next, st));
+                LQ_CUDA_TRY(cudaEventRecord(h->ev_next, cs));
                 LQ_CUDA_TRY(cudaStreamWaitEvent(aux, h->ev_next, 0));
                 if (rows_in > 1) {             // block row k-1 is part of "next"
                     dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(rows_in - 1));
@@ -920,15 +984,20 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
             }
         }
         if (o_lo > 0) {
-            if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_rest, 0));
+            if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(cs, h->ev_rest, 0));
             rest_pending = false;
-            int rc = deferred_update(h, st, A, cp, o_lo, o_hi, Pob, reinterpret_cast<int*>(wsp + L.ex),
+            int rc = deferred_update(h, cs, A, cp, o_lo, o_hi, Pob, reinterpret_cast<int*>(wsp + L.ex),
                                      wsp + L.sl, reinterpret_cast<float*>(wsp + L.ta),
                                      reinterpret_cast<float*>(wsp + L.tb), L.band);
             if (rc) return rc;
         }
     }
-    if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_rest, 0));
+    if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(cs, h->ev_rest, 0));
+    if (next2_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(cs, h->ev_next2, 0));
+    if (fork) {
+        LQ_CUDA_TRY(cudaEventRecord(h->ev_join, cs));
+        LQ_CUDA_TRY(cudaStreamWaitEvent(st, h->ev_join, 0));
+    }
     {
         // the panel buffers are free now: they hold the per-chunk column sums (c / 256 x c doubles <= 2 panels for c <= 65536)
         double* part = reinterpret_cast<double*>(wsp + L.pbuf);
