@@ -288,6 +288,339 @@ kmeans_sorted_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
     }
 }
 
+// ------------------------------------------------- rows that fit shared memory, Eq. 6 start: grouped by value ---
+// A total order is more than the iterations need.  The row is grouped once into 2^14 buckets of equal width between
+// its smallest and its largest weight with a counting pass: histogram, exclusive scan, scatter.  Positions inside a
+// bucket keep no order.  The prefix sums of s and s*w over the positions are taken as in the sorted kernel; the prefix
+// at a bucket's first position does not depend on the order inside the buckets.  The bucket index
+// floor((w - lo) * scale), clamped, is monotone in w, and a boundary m takes its bucket through the same expression:
+// every member of a lower bucket is < m, every member of a higher bucket is > m, and the members of that one bucket
+// are compared with m one by one.  So ub(m) = first position of the bucket + its members <= m, and F(ub(m)) = the
+// prefix at the bucket's first position + the terms of those members: the same assignments as the sorted kernel,
+// without the sort.  The buckets are much narrower than the spacing of bf16 values around the bulk of a row, so a
+// boundary's bucket is empty more often than not.
+//   offs : 2^14 16-bit counters, two to a 32-bit word (a row has at most 16384 weights, so a half never carries);
+//          after the scatter half b holds the position behind bucket b's last member.
+constexpr int KB_BITS = 14;
+constexpr int KB_BUCKETS = 1 << KB_BITS;
+constexpr int KB_MIN_N = 4096;           // shorter rows are sorted: the counters' fixed cost (clearing, scan) would dominate
+constexpr int KB_SERIAL_MAX = 24;        // boundary scans longer than this are shared out over the warp
+__device__ __forceinline__ int value_bucket(double w, double lo, double scale) {
+    const double x = __dmul_rn(__dsub_rn(w, lo), scale);
+    int b = x < static_cast<double>(KB_BUCKETS - 1) ? static_cast<int>(x) : KB_BUCKETS - 1;      // x >= 0 for a member; NaN goes to the top bucket
+    return b < 0 ? 0 : b;
+}
+__device__ __forceinline__ int offs_half(const uint32_t* offs, int b) { return static_cast<int>((offs[b >> 1] >> ((b & 1) * 16)) & 0xffffu); }
+
+template <int K, typename T>
+__global__ void __launch_bounds__(KS_THREADS, 3)
+kmeans_bucket_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int n, const double* __restrict__ s64,
+                     float* __restrict__ grid, int n_iter) {
+    typedef typename KeyOf<T>::type KeyT;
+    extern __shared__ __align__(16) unsigned char ks_smem[];
+    dd2* coarse = reinterpret_cast<dd2*>(ks_smem);            // n / 8 + 1 coarse prefixes, then the n keys, then the counters
+    KeyT* keys = reinterpret_cast<KeyT*>(coarse + (n / KS_CHUNK + 1));
+    uint32_t* offs = reinterpret_cast<uint32_t*>(ks_smem + (((n / KS_CHUNK + 1) * sizeof(dd2) + (n + n / 32) * sizeof(KeyT) + 15) & ~size_t(15)));
+    __shared__ dd2 tot[KS_THREADS];                            // per-thread totals, then their exclusive scan
+    __shared__ double g[K];
+    __shared__ dd2 F[K + 1];
+    __shared__ KeyT ext[2][KS_THREADS / 32];                   // per-warp smallest and largest key
+    __shared__ int wsum[KS_THREADS / 32];
+    __shared__ double rng[2];                                  // smallest weight of the row, buckets per unit of weight
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nch = n / KS_CHUNK;
+    const int cpt = nch > KS_THREADS ? nch / KS_THREADS : 1;   // chunks per thread
+    constexpr int WPT = KB_BUCKETS / 2 / KS_THREADS;           // counter words per thread in the scan
+
+    for (int64_t row = blockIdx.x; row < r; row += gridDim.x) {
+        const T* wp = W + row * ldw;
+        for (int i = tid; i < KB_BUCKETS / 8; i += KS_THREADS) reinterpret_cast<uint4*>(offs)[i] = make_uint4(0u, 0u, 0u, 0u);
+        // smallest and largest weight of the row
+        KeyT kmin = KeyOf<T>::pad(), kmax = 0;
+        for (int i = tid; i < c; i += KS_THREADS) {
+            const KeyT key = KeyOf<T>::make(LQ_AT(wp + i), i);
+            kmin = key < kmin ? key : kmin;
+            kmax = key > kmax ? key : kmax;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const KeyT a = __shfl_xor_sync(0xffffffffu, kmin, o), b = __shfl_xor_sync(0xffffffffu, kmax, o);
+            kmin = a < kmin ? a : kmin;
+            kmax = b > kmax ? b : kmax;
+        }
+        if (lane == 0) { ext[0][warp] = kmin; ext[1][warp] = kmax; }
+        __syncthreads();
+        if (tid == 0) {
+            KeyT k0 = ext[0][0], k1 = ext[1][0];
+#pragma unroll
+            for (int w = 1; w < KS_THREADS / 32; ++w) {
+                k0 = ext[0][w] < k0 ? ext[0][w] : k0;
+                k1 = ext[1][w] > k1 ? ext[1][w] : k1;
+            }
+            const double lo = static_cast<double>(key_weight(k0)), hi = static_cast<double>(key_weight(k1));
+            rng[0] = lo;
+            rng[1] = hi > lo ? static_cast<double>(KB_BUCKETS) / (hi - lo) : 0.0;
+            ext[0][0] = k0;
+            ext[1][0] = k1;
+        }
+        __syncthreads();
+        const double lo = rng[0], scale = rng[1];
+        // histogram of the buckets
+        for (int i = tid; i < c; i += KS_THREADS) {
+            const int b = value_bucket(static_cast<double>(key_weight(KeyOf<T>::make(LQ_AT(wp + i), i))), lo, scale);
+            atomicAdd(offs + (b >> 1), (b & 1) ? 0x10000u : 1u);
+        }
+        __syncthreads();
+        // exclusive scan of the counters: 64 buckets per thread, then across the CTA
+        {
+            uint32_t wv[WPT];
+            int sum = 0;
+#pragma unroll
+            for (int e = 0; e < WPT / 4; ++e) {
+                const uint4 v = reinterpret_cast<const uint4*>(offs)[tid * (WPT / 4) + e];
+                wv[4 * e] = v.x; wv[4 * e + 1] = v.y; wv[4 * e + 2] = v.z; wv[4 * e + 3] = v.w;
+            }
+#pragma unroll
+            for (int e = 0; e < WPT; ++e) sum += static_cast<int>((wv[e] & 0xffffu) + (wv[e] >> 16));
+            int inc = sum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int up = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += up;
+            }
+            if (lane == 31) wsum[warp] = inc;
+            __syncthreads();
+            int run = inc - sum;
+            for (int w = 0; w < warp; ++w) run += wsum[w];
+#pragma unroll
+            for (int e = 0; e < WPT; ++e) {
+                const uint32_t lo = wv[e] & 0xffffu, hi = wv[e] >> 16;
+                wv[e] = static_cast<uint32_t>(run) | (static_cast<uint32_t>(run + lo) << 16);
+                run += static_cast<int>(lo + hi);
+            }
+#pragma unroll
+            for (int e = 0; e < WPT / 4; ++e)
+                reinterpret_cast<uint4*>(offs)[tid * (WPT / 4) + e] = make_uint4(wv[4 * e], wv[4 * e + 1], wv[4 * e + 2], wv[4 * e + 3]);
+        }
+        __syncthreads();
+        // scatter: a bucket's counter hands out its positions
+        for (int i = tid; i < c; i += KS_THREADS) {
+            const KeyT key = KeyOf<T>::make(LQ_AT(wp + i), i);
+            const int b = value_bucket(static_cast<double>(key_weight(key)), lo, scale);
+            const uint32_t old = atomicAdd(offs + (b >> 1), (b & 1) ? 0x10000u : 1u);
+            const int pos = static_cast<int>((b & 1) ? old >> 16 : old & 0xffffu);
+            LQ_AT(keys + ks_slot(pos)) = key;
+        }
+        __syncthreads();
+        // chunk totals, thread-local exclusive prefixes (positions in bucket order).  A chunk's eight terms are loaded
+        // first and summed as two chains of four (the double-double sums are exact far below the tolerance, so
+        // their grouping is free).
+        dd2 run;
+        run.s.hi = run.s.lo = run.sw.hi = run.sw.lo = 0.0;
+        for (int q = tid * cpt; q < (tid + 1) * cpt && q < nch; ++q) {
+            LQ_AT(coarse + q) = run;
+            double sv[KS_CHUNK], swv[KS_CHUNK];
+#pragma unroll
+            for (int e = 0; e < KS_CHUNK; ++e) {
+                const int i = q * KS_CHUNK + e;
+                sv[e] = swv[e] = 0.0;
+                if (i < c) {
+                    const KeyT key = LQ_AT(keys + ks_slot(i));
+                    sv[e] = LQ_AT(s64 + key_index(key));
+                    swv[e] = __dmul_rn(sv[e], static_cast<double>(key_weight(key)));
+                }
+            }
+            dd2 half;
+            half.s.hi = sv[KS_CHUNK / 2]; half.s.lo = 0.0; half.sw.hi = swv[KS_CHUNK / 2]; half.sw.lo = 0.0;
+#pragma unroll
+            for (int e = 0; e < KS_CHUNK / 2; ++e) {
+                run.s = dd_add_d(run.s, sv[e]);
+                run.sw = dd_add_d(run.sw, swv[e]);
+                if (e > 0) {
+                    half.s = dd_add_d(half.s, sv[KS_CHUNK / 2 + e]);
+                    half.sw = dd_add_d(half.sw, swv[KS_CHUNK / 2 + e]);
+                }
+            }
+            run.s = dd_add(run.s, half.s);
+            run.sw = dd_add(run.sw, half.sw);
+        }
+        tot[tid] = run;
+        __syncthreads();
+        if (warp == 0) {       // exclusive scan of the 256 thread totals: 8 per lane, then across the warp
+            dd2 loc[KS_THREADS / 32];
+            dd2 acc;
+            acc.s.hi = acc.s.lo = acc.sw.hi = acc.sw.lo = 0.0;
+#pragma unroll
+            for (int e = 0; e < KS_THREADS / 32; ++e) {
+                loc[e] = acc;
+                const dd2 v = tot[lane * (KS_THREADS / 32) + e];
+                acc.s = dd_add(acc.s, v.s);
+                acc.sw = dd_add(acc.sw, v.sw);
+            }
+            dd2 inc = acc;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                dd2 up;
+                up.s.hi = __shfl_up_sync(0xffffffffu, inc.s.hi, o);
+                up.s.lo = __shfl_up_sync(0xffffffffu, inc.s.lo, o);
+                up.sw.hi = __shfl_up_sync(0xffffffffu, inc.sw.hi, o);
+                up.sw.lo = __shfl_up_sync(0xffffffffu, inc.sw.lo, o);
+                if (lane >= o) { inc.s = dd_add(up.s, inc.s); inc.sw = dd_add(up.sw, inc.sw); }
+            }
+            dd2 excl;                                           // sum of the lanes before this one
+            excl.s.hi = __shfl_up_sync(0xffffffffu, inc.s.hi, 1);
+            excl.s.lo = __shfl_up_sync(0xffffffffu, inc.s.lo, 1);
+            excl.sw.hi = __shfl_up_sync(0xffffffffu, inc.sw.hi, 1);
+            excl.sw.lo = __shfl_up_sync(0xffffffffu, inc.sw.lo, 1);
+            if (lane == 0) excl.s.hi = excl.s.lo = excl.sw.hi = excl.sw.lo = 0.0;
+#pragma unroll
+            for (int e = 0; e < KS_THREADS / 32; ++e) {
+                dd2 v;
+                v.s = dd_add(excl.s, loc[e].s);
+                v.sw = dd_add(excl.sw, loc[e].sw);
+                tot[lane * (KS_THREADS / 32) + e] = v;
+            }
+            if (lane == 31) LQ_AT(coarse + nch) = inc;          // grand total
+        }
+        __syncthreads();
+        {
+            const dd2 off = tot[tid];
+            for (int q = tid * cpt; q < (tid + 1) * cpt && q < nch; ++q) {
+                dd2 v = LQ_AT(coarse + q);
+                v.s = dd_add(off.s, v.s);
+                v.sw = dd_add(off.sw, v.sw);
+                LQ_AT(coarse + q) = v;
+            }
+        }
+        __syncthreads();
+
+        if (warp == 0) {
+            const double hi = static_cast<double>(key_weight(ext[1][0]));
+            if (lane < K) g[lane] = lo + (hi - lo) * static_cast<double>(lane) / static_cast<double>(K - 1);   // Eq. 6
+            if (lane == 0) {
+                F[0].s.hi = F[0].s.lo = F[0].sw.hi = F[0].sw.lo = 0.0;
+                F[K] = coarse[nch];
+            }
+            __syncwarp();
+            int b_prev = -1;
+            for (int it = 0; it < n_iter; ++it) {
+                // boundary of lane: its bucket's members [start, end), of which cnt do not exceed m
+                int start = 0, end = 0, cnt = 0;
+                double m = 0.0;
+                if (lane < K - 1) {
+                    m = 0.5 * (g[lane] + g[lane + 1]);
+                    const int B = value_bucket(m, lo, scale);
+                    start = B > 0 ? offs_half(offs, B - 1) : 0;
+                    end = offs_half(offs, B);
+                }
+                const bool wide = end - start > KB_SERIAL_MAX;
+                const unsigned big = __ballot_sync(0xffffffffu, wide);
+                if (!wide)
+                    for (int p = start; p < end; ++p) cnt += !(static_cast<double>(key_weight(LQ_AT(keys + ks_slot(p)))) > m);
+                for (unsigned todo = big; todo;) {              // a long bucket (many equal or nearly equal weights): all lanes count
+                    const int src = __ffs(todo) - 1;
+                    todo &= todo - 1;
+                    const int ss = __shfl_sync(0xffffffffu, start, src), es = __shfl_sync(0xffffffffu, end, src);
+                    const double ms = __shfl_sync(0xffffffffu, m, src);
+                    int ac = 0;
+                    for (int p = ss + lane; p < es; p += 32) ac += !(static_cast<double>(key_weight(LQ_AT(keys + ks_slot(p)))) > ms);
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) ac += __shfl_xor_sync(0xffffffffu, ac, o);
+                    if (lane == src) cnt = ac;
+                }
+                const int b0 = start + cnt;                     // ub(m)
+                // Unchanged boundaries give back the same centroids, and so would every later
+                // iteration: the fixed point has been reached and the remaining iterations are skipped.
+                if (__all_sync(0xffffffffu, b0 == b_prev)) break;
+                b_prev = b0;
+                // F(ub(m)).  Nearly always the bucket's members lie on one side of m (a bucket is narrower than the
+                // spacing of the values around it): every position below b0 counts, and the prefix there is the nearer
+                // coarse prefix plus or minus at most four terms.  A bucket with members on both sides adds its
+                // members <= m to the prefix at its first position.
+                const bool mixed = cnt != 0 && cnt != end - start;
+                const int at = mixed ? start : b0;
+                dd2 f;
+                f.s.hi = f.s.lo = f.sw.hi = f.sw.lo = 0.0;
+                if (lane < K - 1) {
+                    const int q = at >> 3, rem = at & (KS_CHUNK - 1);
+                    if (rem <= KS_CHUNK / 2) {
+                        f = LQ_AT(coarse + q);
+                        for (int e = 0; e < rem; ++e) {
+                            const KeyT key = LQ_AT(keys + ks_slot(q * KS_CHUNK + e));
+                            const double sv = LQ_AT(s64 + key_index(key));
+                            f.s = dd_add_d(f.s, sv);
+                            f.sw = dd_add_d(f.sw, __dmul_rn(sv, static_cast<double>(key_weight(key))));
+                        }
+                    } else {
+                        f = LQ_AT(coarse + q + 1);
+                        for (int e = rem; e < KS_CHUNK; ++e) {
+                            const int i = q * KS_CHUNK + e;
+                            if (i < c) {
+                                const KeyT key = LQ_AT(keys + ks_slot(i));
+                                const double sv = LQ_AT(s64 + key_index(key));
+                                f.s = dd_add_d(f.s, -sv);
+                                f.sw = dd_add_d(f.sw, -__dmul_rn(sv, static_cast<double>(key_weight(key))));
+                            }
+                        }
+                    }
+                    if (mixed && !wide) {
+                        for (int p = start; p < end; ++p) {
+                            const KeyT key = LQ_AT(keys + ks_slot(p));
+                            const double wv = static_cast<double>(key_weight(key));
+                            if (!(wv > m)) {
+                                const double sv = LQ_AT(s64 + key_index(key));
+                                f.s = dd_add_d(f.s, sv);
+                                f.sw = dd_add_d(f.sw, __dmul_rn(sv, wv));
+                            }
+                        }
+                    }
+                }
+                for (unsigned todo = __ballot_sync(0xffffffffu, mixed && wide); todo;) {      // long and mixed: all lanes sum
+                    const int src = __ffs(todo) - 1;
+                    todo &= todo - 1;
+                    const int ss = __shfl_sync(0xffffffffu, start, src), es = __shfl_sync(0xffffffffu, end, src);
+                    const double ms = __shfl_sync(0xffffffffu, m, src);
+                    dd2 a;
+                    a.s.hi = a.s.lo = a.sw.hi = a.sw.lo = 0.0;
+                    for (int p = ss + lane; p < es; p += 32) {
+                        const KeyT key = LQ_AT(keys + ks_slot(p));
+                        const double wv = static_cast<double>(key_weight(key));
+                        if (!(wv > ms)) {
+                            const double sv = LQ_AT(s64 + key_index(key));
+                            a.s = dd_add_d(a.s, sv);
+                            a.sw = dd_add_d(a.sw, __dmul_rn(sv, wv));
+                        }
+                    }
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+                        dd2 u;
+                        u.s.hi = __shfl_xor_sync(0xffffffffu, a.s.hi, o);
+                        u.s.lo = __shfl_xor_sync(0xffffffffu, a.s.lo, o);
+                        u.sw.hi = __shfl_xor_sync(0xffffffffu, a.sw.hi, o);
+                        u.sw.lo = __shfl_xor_sync(0xffffffffu, a.sw.lo, o);
+                        a.s = dd_add(a.s, u.s);
+                        a.sw = dd_add(a.sw, u.sw);
+                    }
+                    if (lane == src) {
+                        f.s = dd_add(f.s, a.s);
+                        f.sw = dd_add(f.sw, a.sw);
+                    }
+                }
+                if (lane < K - 1) F[lane + 1] = f;
+                __syncwarp();
+                if (lane < K) {
+                    const double den = dd_diff(F[lane + 1].s, F[lane].s);
+                    const double num = dd_diff(F[lane + 1].sw, F[lane].sw);
+                    if (den > 0.0) g[lane] = num / den;         // an empty cluster keeps its centroid
+                }
+                __syncwarp();
+            }
+            if (lane < K) LQ_AT(grid + row * K + lane) = static_cast<float>(g[lane]);
+        }
+        __syncthreads();
+    }
+}
+
 // ------------------------------------------------- long rows: direct k-means --------
 // Rows too long to sort in shared memory: the row is staged once in shared memory in its own
 // type and every iteration visits every weight (compares and cluster sums in fp64).
@@ -381,6 +714,22 @@ int launch_kmeans(cudaStream_t st, int sms, const T* W, int64_t ldw, int64_t r, 
         while (n < c) n <<= 1;
         const size_t smem = (static_cast<size_t>(n) / KS_CHUNK + 1) * sizeof(dd2) +
                             static_cast<size_t>(n + n / 32) * sizeof(typename KeyOf<T>::type);
+        const size_t bsmem = ((smem + 15) & ~size_t(15)) + KB_BUCKETS * 2;
+        // the start of Eq. 6 needs no order inside a bucket: the counting pass replaces the sort (where its counters fit
+        // and pays: below 4096 weights the fixed cost of the 2^14 counters exceeds the sort's)
+        if (init == LQ_INIT_UNIFORM && n >= KB_MIN_N && bsmem <= 216 * 1024) {
+            static lq_once_per_device battr_set;
+            if (battr_set.first()) {
+                LQ_CUDA_TRY(cudaFuncSetAttribute(kmeans_bucket_kernel<K, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 216 * 1024));
+            }
+            int per_sm = static_cast<int>((228 * 1024) / (bsmem + 10 * 1024));
+            per_sm = per_sm < 1 ? 1 : (per_sm > 3 ? 3 : per_sm);
+            const int64_t cap = static_cast<int64_t>(sms) * per_sm;
+            kmeans_bucket_kernel<K, T><<<static_cast<unsigned>(r < cap ? r : cap), KS_THREADS, bsmem, st>>>(
+                W, ldw, r, static_cast<int>(c), n, s64, grid, n_iter);
+            LQ_LAUNCH_CHECK();
+            return LQ_OK;
+        }
         static lq_once_per_device attr_set;
         if (attr_set.first()) {
             LQ_CUDA_TRY(cudaFuncSetAttribute(kmeans_sorted_kernel<K, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));

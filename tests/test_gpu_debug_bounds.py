@@ -13,7 +13,7 @@ pytestmark = pytest.mark.gpu
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 CASES = ("tiny_and_ragged or stage1_hessian or stage1_token_major or stage1_empty or stage2_prepare or stage2_dead or "
-         "stage3_nonuniform or stage3_weighted or stage3_degenerate or stage3_affine or stage4 or lazy_refit or pack_codes or "
+         "stage3_nonuniform or stage3_grouped or stage3_weighted or stage3_degenerate or stage3_affine or stage4 or lazy_refit or pack_codes or "
          "activation_order or act_order or record or stack_of_layers or chained_affine or noalloc")
 
 

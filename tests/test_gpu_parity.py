@@ -307,6 +307,35 @@ def test_stage3_degenerate_rows(lq, h):
     assert np.all(f64(grid)[1] == 0.125)
 
 
+@pytest.mark.parametrize("c,dtype", [(4096, torch.bfloat16), (5000, torch.bfloat16), (9000, torch.float32), (16384, torch.bfloat16)])
+def test_stage3_grouped_rows(lq, h, c, dtype):
+    """Rows of 4096 weights and more are grouped by value instead of sorted: ordinary rows, and the rows that stress the
+    grouping -- one value only, one far outlier (every other weight in a few buckets, boundaries inside long buckets),
+    a handful of distinct values, and sample weights that span many decades next to each other."""
+    r = 12
+    g = torch.Generator().manual_seed(c)
+    W = torch.randn(r, c, generator=g) * 0.02
+    W[1] = -0.375                                   # one value
+    W[2, 17] = 40.0                                 # a far outlier: the bulk of the row shares a few buckets
+    W[3] = torch.tensor([-0.5, -0.25, 0.0, 0.125, 0.75])[torch.randint(0, 5, (c,), generator=g)]      # five values
+    W[4] = 0.0
+    W[4, c - 1] = -1.0
+    W[5] = (W[5] * 64).round() / 64                 # many ties
+    W = W.to(dtype)
+    dinv = torch.exp(torch.randn(c, generator=g) * 1.5).float()       # s = dinv^-4 spans ~10 decades
+    for bits in (2, 4):
+        cfg = lq.Config.make(grid="nonuniform", bits=bits, p=4.0, n_iter=20)
+        Gref = O.fit_grid_nonuniform(f64(W), f64(dinv), bits, 4.0, 20)
+        grid = torch.empty(r, 1 << bits, device="cuda")
+        ws = ws_for(lq, lq.lq_fit_grid_workspace(cfg, r, c))
+        lq.lq_fit_grid(h, cfg, W.cuda(), dinv.cuda(), ws, grid=grid)
+        lq.lq_sync_status(h)
+        G = f64(grid)
+        assert (np.diff(G, axis=1) >= 0).all()
+        assert centroid_ok(G, Gref, f64(W))
+        assert np.all(G[1] == -0.375)
+
+
 @pytest.mark.parametrize("r,c,bits,group,T,t", [(64, 512, 4, 128, 45, 9), (32, 256, 3, 64, 40, 12),
                                                (16, 384, 4, 0, 45, 9), (8, 256, 2, 128, 2048, 40)])
 def test_stage3_affine(lq, h, r, c, bits, group, T, t):
