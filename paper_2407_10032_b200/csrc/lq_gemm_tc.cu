@@ -358,7 +358,8 @@ __device__ __forceinline__ void seg_item(const Seg& g, int q, int& pass, int& kb
     kb = g.kb0 + kit - ps * g.kbn;
 }
 
-template <int CTAS>
+// I8: the instantiation for 8-bit integer operands; the bf16 instantiation carries none of that code.
+template <int CTAS, bool I8>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const __grid_constant__ CUtensorMap map_d, const __grid_constant__ KParams p) {
@@ -475,7 +476,7 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                         const uint64_t da = make_desc_sw128(sa);
                         const uint64_t db = make_desc_sw128(sa + A_STAGE_BYTES);
 #pragma unroll
-                        if (p.int8_ops) {
+                        if (I8) {
                             int pass, kb;
                             seg_item(seg, q, pass, kb);
                             const uint32_t idesc = p.idesc_pass[pass];
@@ -532,7 +533,7 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     uint32_t v[32];
                     tmem_ld32(tmem_base + ((q * 32u) << 16) + acc * BN + hf * (BN / 2) + ch * EPI_COLS, v);
                     tmem_wait_ld();
-                    if (p.int8_ops) {
+                    if (I8) {
                         // int32 partial sums (exact) -> fp32, scaled by the level's power of two
                         const float sc = p.lvl_scale[p.n_lvl > 0 ? sg / p.n_chunks : 0];
                         if (sg == pc.s0) {
@@ -645,7 +646,8 @@ int max_pairs(int sm_count) {
     int& cached = cached_per_device[dev];
     if (!once.first()) return cached;
     cached = 0;
-    if (cudaFuncSetAttribute(lq_tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::SMEM_BYTES) != cudaSuccess) {
+    if (cudaFuncSetAttribute(lq_tc_gemm_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::SMEM_BYTES) != cudaSuccess ||
+        cudaFuncSetAttribute(lq_tc_gemm_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<2>::SMEM_BYTES) != cudaSuccess) {
         cudaGetLastError();
         return cached;
     }
@@ -659,7 +661,7 @@ int max_pairs(int sm_count) {
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     int n = 0;
-    if (cudaOccupancyMaxActiveClusters(&n, lq_tc_gemm_kernel<2>, &cfg) != cudaSuccess) {
+    if (cudaOccupancyMaxActiveClusters(&n, lq_tc_gemm_kernel<2, false>, &cfg) != cudaSuccess) {
         cudaGetLastError();
         return cached;
     }
@@ -683,7 +685,8 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
 
     static lq_once_per_device attr_set;
     if (attr_set.first()) {
-        LQ_CUDA_TRY(cudaFuncSetAttribute(lq_tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<1>::SMEM_BYTES));
+        LQ_CUDA_TRY(cudaFuncSetAttribute(lq_tc_gemm_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<1>::SMEM_BYTES));
+        LQ_CUDA_TRY(cudaFuncSetAttribute(lq_tc_gemm_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg<1>::SMEM_BYTES));
     }
     // The pair form pays off once there are at least a few 256-row tiles; below that one CTA per tile.
     const int pairs = (a.M > BM) ? max_pairs(h->sm_count) : 0;
@@ -781,13 +784,16 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
         attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, lq_tc_gemm_kernel<2>, map_a, map_b, map_d, p) != cudaSuccess) {
+        const cudaError_t le = i8 ? cudaLaunchKernelEx(&cfg, lq_tc_gemm_kernel<2, true>, map_a, map_b, map_d, p)
+                                  : cudaLaunchKernelEx(&cfg, lq_tc_gemm_kernel<2, false>, map_a, map_b, map_d, p);
+        if (le != cudaSuccess) {
             cudaGetLastError();
             return LQ_ERR_CUDA;
         }
         lq_launches_total.fetch_add(1, std::memory_order_relaxed);
     } else {
-        lq_tc_gemm_kernel<1><<<active, NUM_THREADS, Cfg<1>::SMEM_BYTES, stream>>>(map_a, map_b, map_d, p);
+        if (i8) lq_tc_gemm_kernel<1, true><<<active, NUM_THREADS, Cfg<1>::SMEM_BYTES, stream>>>(map_a, map_b, map_d, p);
+        else lq_tc_gemm_kernel<1, false><<<active, NUM_THREADS, Cfg<1>::SMEM_BYTES, stream>>>(map_a, map_b, map_d, p);
         LQ_LAUNCH_CHECK();
     }
     return LQ_OK;
