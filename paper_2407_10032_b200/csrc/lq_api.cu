@@ -48,7 +48,7 @@ extern "C" int lq_create(lq_handle** out, int device) {
     h->dstatus = nullptr;
     h->aux = nullptr;
     h->chain = h->mid = nullptr;
-    h->ev_fork = h->ev_next = h->ev_rest = h->ev_join = h->ev_next2 = nullptr;
+    h->ev_fork = h->ev_next = h->ev_rest = h->ev_join = h->ev_next2 = h->ev_diag = h->ev_crit = nullptr;
     h->wait_limit_ns = LQ_DEFAULT_WAIT_LIMIT_NS;
     h->inject_stall = 0;
     h->prep_defer_min_blocks = LQ_DEFAULT_PREP_DEFER_MIN_BLOCKS;
@@ -59,6 +59,8 @@ extern "C" int lq_create(lq_handle** out, int device) {
         cudaStreamCreateWithPriority(&h->chain, cudaStreamNonBlocking, prio_greatest) != cudaSuccess ||
         cudaStreamCreateWithPriority(&h->mid, cudaStreamNonBlocking, prio_greatest < prio_least ? prio_greatest + 1 : prio_least) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_next2, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_diag, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&h->ev_crit, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_join, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&h->ev_next, cudaEventDisableTiming) != cudaSuccess ||
@@ -68,6 +70,8 @@ extern "C" int lq_create(lq_handle** out, int device) {
         if (h->ev_fork) cudaEventDestroy(h->ev_fork);
         if (h->ev_join) cudaEventDestroy(h->ev_join);
         if (h->ev_next2) cudaEventDestroy(h->ev_next2);
+        if (h->ev_diag) cudaEventDestroy(h->ev_diag);
+        if (h->ev_crit) cudaEventDestroy(h->ev_crit);
         if (h->mid) cudaStreamDestroy(h->mid);
         if (h->chain) cudaStreamDestroy(h->chain);
         if (h->aux) cudaStreamDestroy(h->aux);
@@ -82,6 +86,8 @@ extern "C" int lq_create(lq_handle** out, int device) {
         cudaEventDestroy(h->ev_fork);
         cudaEventDestroy(h->ev_join);
         cudaEventDestroy(h->ev_next2);
+        cudaEventDestroy(h->ev_diag);
+        cudaEventDestroy(h->ev_crit);
         cudaStreamDestroy(h->mid);
         cudaStreamDestroy(h->chain);
         cudaStreamDestroy(h->aux);
@@ -101,6 +107,8 @@ extern "C" int lq_destroy(lq_handle* h) {
         cudaStreamSynchronize(h->mid);
         cudaEventDestroy(h->ev_join);
         cudaEventDestroy(h->ev_next2);
+        cudaEventDestroy(h->ev_diag);
+        cudaEventDestroy(h->ev_crit);
         cudaStreamDestroy(h->mid);
         cudaStreamDestroy(h->chain);
         cudaEventDestroy(h->ev_rest);

@@ -28,7 +28,7 @@ struct lq_handle {
     // its CTAs are placed ahead of the queued CTAs of the bulk update; `mid` (one priority level below) takes the
     // updates that the chain needs two steps later.
     cudaStream_t chain, mid;
-    cudaEvent_t ev_fork, ev_next, ev_rest, ev_join, ev_next2;
+    cudaEvent_t ev_fork, ev_next, ev_rest, ev_join, ev_next2, ev_diag, ev_crit;
     // Time limit of every bounded wait inside a kernel launched through this handle (nanoseconds).
     unsigned long long wait_limit_ns;
     // Test hook: nonzero makes the load barriers of the tensor-core contraction expect bytes that never arrive, so that

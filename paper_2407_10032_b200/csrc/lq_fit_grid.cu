@@ -1346,7 +1346,7 @@ extern "C" int lq_fit_grid_noalloc(lq_handle* h, void* stream, const lq_config* 
     local.dstatus = d.status;
     local.aux = nullptr;
     local.chain = local.mid = nullptr;
-    local.ev_fork = local.ev_next = local.ev_rest = local.ev_join = local.ev_next2 = nullptr;
+    local.ev_fork = local.ev_next = local.ev_rest = local.ev_join = local.ev_next2 = local.ev_diag = local.ev_crit = nullptr;
     local.wait_limit_ns = LQ_DEFAULT_WAIT_LIMIT_NS;
     local.inject_stall = 0;
     local.prep_defer_min_blocks = LQ_DEFAULT_PREP_DEFER_MIN_BLOCKS;

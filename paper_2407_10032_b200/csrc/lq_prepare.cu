@@ -285,16 +285,18 @@ panel_kernel(double* __restrict__ A, int64_t cp, int k, double* __restrict__ Pbu
 //   part 0: every tile of the launch;  part 2: all but block row and block column k-1;
 //   part 4: all but block rows and block columns k-1 and k-2;
 //   part 1: next only, grid 4 nblk x 1, 64 x 64 tiles -- block tile t < k is (t, k-1), t >= k is (k-1, t);
-//   part 3: next2 only, same grid -- block tile t < k-1 is (t, k-2), t >= k is (k-2, t) (tile (k-2, k-1) belongs to next).
+//   part 3: next2 only, same grid -- block tile t < k-1 is (t, k-2), t >= k is (k-2, t) (tile (k-2, k-1) belongs to next);
+//   part 5: next without the diagonal tile (k-1, k-1), which crit_kernel has updated already.
 __global__ void __launch_bounds__(GEMM_THREADS, 2)
 update_kernel(double* __restrict__ A, int64_t cp, int k, int part, int i_base, int j_base, const double* __restrict__ Pbuf,
               int64_t ldp, const double* __restrict__ Q) {
     extern __shared__ double smem[];
     int i, j, r0, c0;
-    if (part == 1 || part == 3) {
+    if (part == 1 || part == 3 || part == 5) {
         const int t = blockIdx.x >> 2;
-        const int nx = part == 1 ? k - 1 : k - 2;         // the block row and column this launch brings up to date
+        const int nx = part == 3 ? k - 2 : k - 1;         // the block row and column this launch brings up to date
         if (part == 3 && t == k - 1) return;
+        if (part == 5 && t == k - 1) return;              // the diagonal tile was updated by crit_kernel
         if (t <= nx) { i = t; j = nx; } else { i = nx; j = t; }
         r0 = ((blockIdx.x >> 1) & 1) * 64;
         c0 = (blockIdx.x & 1) * 64;
@@ -314,8 +316,28 @@ update_kernel(double* __restrict__ A, int64_t cp, int k, int part, int i_base, i
     // A[i][k] = -P_i V_k;  A[i][j] -= P_i Q[:, j] otherwise
     const double* Bsrc = (j == k) ? A + (int64_t)k * NB * cp + (int64_t)k * NB + c0 : Q + (int64_t)j * NB + c0;
     const double beta = (j == k) ? 0.0 : 1.0;
-    if (part == 1 || part == 3) gemm_tile<2, 4, false>(Pi, ldp, Bsrc, cp, -1.0, beta, o, smem);
+    if (part == 1 || part == 3 || part == 5) gemm_tile<2, 4, false>(Pi, ldp, Bsrc, cp, -1.0, beta, o, smem);
     else gemm_tile<4, 4, false>(Pi, ldp, Bsrc, cp, -1.0, beta, o, smem);
+}
+
+// Step k, the one tile the next diagonal block waits for.  phase 0: P' = A[k-1][k] V_k^T (the panel tile of block row
+// k-1, into the scratch Pc, 128 x 128); phase 1: A[k-1][k-1] -= P' P'^T.  Four CTAs of 64 x 64 each: they find free
+// places on the SMs at once, where the panel and "next" launches (over a hundred CTAs) queue behind the bulk update.
+// The panel launch computes the same P' again for everybody else.
+__global__ void __launch_bounds__(GEMM_THREADS, 2)
+crit_kernel(double* __restrict__ A, int64_t cp, int k, int phase, double* __restrict__ Pc) {
+    extern __shared__ double smem[];
+    chain_wait();
+    const int mh = blockIdx.x >> 1, hh = blockIdx.x & 1;
+    TileOut o = {};
+    if (phase == 0) {
+        const double* Vk = A + (int64_t)k * NB * cp + (int64_t)k * NB;
+        o.C = Pc + (int64_t)(mh * 64) * NB + hh * 64; o.ldc = NB;
+        gemm_tile<2, 4, true>(A + ((int64_t)(k - 1) * NB + mh * 64) * cp + (int64_t)k * NB, cp, Vk + (int64_t)(hh * 64) * cp, cp, 1.0, 0.0, o, smem);
+    } else {
+        o.C = A + ((int64_t)(k - 1) * NB + mh * 64) * cp + (int64_t)(k - 1) * NB + hh * 64; o.ldc = cp;
+        gemm_tile<2, 4, true>(Pc + (int64_t)(mh * 64) * NB, NB, Pc + (int64_t)(hh * 64) * NB, NB, -1.0, 1.0, o, smem);
+    }
 }
 
 // ------------------------------------------------ deferred update: operands as digit slices ----
@@ -858,6 +880,7 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
         LQ_CUDA_TRY(cudaFuncSetAttribute(diag_block_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, DIAG_SMEM));
         LQ_CUDA_TRY(cudaFuncSetAttribute(panel_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
         LQ_CUDA_TRY(cudaFuncSetAttribute(update_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
+        LQ_CUDA_TRY(cudaFuncSetAttribute(crit_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM));
     }
 
     diag_mean_kernel<<<1, 1024, 0, st>>>(H, c, ldh, static_cast<double>(damp_frac), scal);
@@ -900,6 +923,62 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
     bool rest_pending = false, next2_pending = false;
     const bool deep = fork && !defer && h->mid != nullptr;
     const int64_t n_ob = lq_ceil_div(nblk, obb);
+    if (deep) {
+        // Nothing deferred (o_lo = 0): look-ahead of two steps, and only what the next diagonal block waits for on the chain.
+        //   chain (highest priority): diagonal kernel of step k, then crit_kernel: the panel tile of block row k-1 and the
+        //                             update of tile (k-1, k-1) -- the next diagonal block;
+        //   middle stream           : panel of step k (after the diagonal kernel), "next" (block row and column k-1 but for
+        //                             its diagonal tile; after crit_kernel, which read the tile (k-1, k) that "next"
+        //                             overwrites), "next2" (block row and column k-2; after the rest of step k+1);
+        //   low-priority stream     : the rest of step k (after the panel of step k and, in stream order, the rest of step k+1).
+        // crit_kernel of step k waits for "next2" of step k+1 (and with it for "next" of step k+1 and the rest of step
+        // k+2), which wrote the tiles it reads and updates.
+        cudaStream_t mid = h->mid;
+        LQ_CUDA_TRY(cudaStreamWaitEvent(mid, h->ev_fork, 0));
+        double* Pc = reinterpret_cast<double*>(wsp + L.sl);          // 128 x 128 scratch of crit_kernel (the slices' space is free here)
+        for (int64_t k = nblk - 1; k >= 0; --k) {
+            double* Pk = Pob + (k & 3) * NB;
+            double* Qk = reinterpret_cast<double*>(wsp + L.q + (k & 3) * L.panel_bytes);
+            const int ki = static_cast<int>(k);
+            LQ_CUDA_TRY(launch_chained(diag_block_kernel, dim3(1), dim3(DIAG_THREADS), DIAG_SMEM, cs, A, cp, k, c, h->dstatus));
+            LQ_CUDA_TRY(cudaEventRecord(h->ev_diag, cs));
+            if (k > 0) {
+                if (next2_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(cs, h->ev_next2, 0));
+                next2_pending = false;
+                crit_kernel<<<4, GEMM_THREADS, GEMM_SMEM, cs>>>(A, cp, ki, 0, Pc);
+                LQ_LAUNCH_CHECK();
+                LQ_CUDA_TRY(launch_chained(crit_kernel, dim3(4), dim3(GEMM_THREADS), GEMM_SMEM, cs, A, cp, ki, 1, Pc));
+                LQ_CUDA_TRY(cudaEventRecord(h->ev_crit, cs));
+            }
+            LQ_CUDA_TRY(cudaStreamWaitEvent(mid, h->ev_diag, 0));
+            panel_kernel<<<static_cast<unsigned>(4 * (nblk - 1)), GEMM_THREADS, GEMM_SMEM, mid>>>(A, cp, ki, Pk, LDP, Qk);
+            LQ_LAUNCH_CHECK();
+            if (k == 0) {
+                LQ_CUDA_TRY(cudaEventRecord(h->ev_next2, mid));
+                next2_pending = true;
+                break;
+            }
+            if (k >= 3) LQ_CUDA_TRY(cudaEventRecord(h->ev_next, mid));       // the panel of step k is complete
+            LQ_CUDA_TRY(cudaStreamWaitEvent(mid, h->ev_crit, 0));
+            update_kernel<<<static_cast<unsigned>(4 * nblk), GEMM_THREADS, GEMM_SMEM, mid>>>(A, cp, ki, 5, 0, 0, Pk, LDP, Qk);
+            LQ_LAUNCH_CHECK();
+            if (k >= 2) {
+                if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(mid, h->ev_rest, 0));
+                update_kernel<<<static_cast<unsigned>(4 * nblk), GEMM_THREADS, GEMM_SMEM, mid>>>(A, cp, ki, 3, 0, 0, Pk, LDP, Qk);
+                LQ_LAUNCH_CHECK();
+            }
+            LQ_CUDA_TRY(cudaEventRecord(h->ev_next2, mid));
+            next2_pending = true;
+            if (k >= 3) {
+                LQ_CUDA_TRY(cudaStreamWaitEvent(aux, h->ev_next, 0));
+                dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(k - 2));
+                update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, aux>>>(A, cp, ki, 4, 0, 0, Pk, LDP, Qk);
+                LQ_LAUNCH_CHECK();
+                LQ_CUDA_TRY(cudaEventRecord(h->ev_rest, aux));
+                rest_pending = true;
+            }
+        }
+    } else
     for (int64_t m = n_ob - 1; m >= 0; --m) {
         const int64_t o_lo = m * obb;
         const int64_t o_hi = (o_lo + obb < nblk ? o_lo + obb : nblk) - 1;
@@ -931,34 +1010,6 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
                     dim3 g(static_cast<unsigned>(2 * obw), static_cast<unsigned>(o_lo));
                     update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, cs>>>(A, cp, ki, 0, 0, static_cast<int>(o_lo), Pk, LDP, Qk);
                     LQ_LAUNCH_CHECK();
-                }
-                continue;
-            }
-            if (deep) {
-                // Look-ahead of two steps (nothing deferred, o_lo = 0).  "next" (block row and column k-1) stays on the
-                // chain and waits only for step k+1's "next2", which touched the same tiles; "next2" (block row and
-                // column k-2) runs on the middle stream once step k+1's rest has left those tiles; the rest of step k
-                // follows step k+1's on the low-priority stream.
-                if (k >= 2) LQ_CUDA_TRY(cudaEventRecord(h->ev_next, cs));      // the panel of step k is complete (next2 and the rest need no more)
-                if (next2_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(cs, h->ev_next2, 0));
-                next2_pending = false;
-                update_kernel<<<static_cast<unsigned>(4 * nblk), GEMM_THREADS, GEMM_SMEM, cs>>>(A, cp, ki, 1, 0, 0, Pk, LDP, Qk);
-                LQ_LAUNCH_CHECK();
-                if (k >= 2) {
-                    LQ_CUDA_TRY(cudaStreamWaitEvent(h->mid, h->ev_next, 0));
-                    if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(h->mid, h->ev_rest, 0));
-                    update_kernel<<<static_cast<unsigned>(4 * nblk), GEMM_THREADS, GEMM_SMEM, h->mid>>>(A, cp, ki, 3, 0, 0, Pk, LDP, Qk);
-                    LQ_LAUNCH_CHECK();
-                    LQ_CUDA_TRY(cudaEventRecord(h->ev_next2, h->mid));
-                    next2_pending = true;
-                }
-                if (k >= 3) {
-                    LQ_CUDA_TRY(cudaStreamWaitEvent(aux, h->ev_next, 0));
-                    dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(k - 2));
-                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, aux>>>(A, cp, ki, 4, 0, 0, Pk, LDP, Qk);
-                    LQ_LAUNCH_CHECK();
-                    LQ_CUDA_TRY(cudaEventRecord(h->ev_rest, aux));
-                    rest_pending = true;
                 }
                 continue;
             }
