@@ -391,7 +391,9 @@ def _check_affine_picks(W, dinv, bits, group, T, t, scale, zero, So, Zo, p=4.0):
                                                       (6, 512, 4, 0, 256, 51, "c3"), (4, 256, 2, 128, 256, 102, "c2"),
                                                       (5, 384, 4, 128, 100, 30, "c1"), (6, 384, 4, 128, 45, 9, "c1"),
                                                       (8, 512, 3, 128, 45, 13, "c2"),
-                                                      (3, 256, 4, 128, 2048, 409, "c3")])
+                                                      (3, 256, 4, 128, 2048, 409, "c3"),
+                                                      # the paper's t for 3 and 2 bits (377 000 and 672 000 candidates per group)
+                                                      (1, 256, 3, 128, 2048, 614, "c3"), (1, 128, 2, 128, 2048, 819, "c2")])
 def test_stage3_affine_fine_partition(lq, h, r, c, bits, group, T, t, recipe):
     L = synth.make_layer(recipe, r, c, 2 * c, seed=T + bits)
     _, dinv, _, _ = O.prepare_hinv(O.hessian(f64(L.X)), 0.01)
