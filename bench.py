@@ -282,6 +282,9 @@ def stage_rooflines(st, r, c, n, stage_ms, pk, pipes, w_bytes, exact=False):
                          "peak_source": "measured: dependent-free mma.sync m8n8k4 f64 loop"},
         "fit_grid": {"bound": "alu", "achieved": s3_ops, "peak": lane_peak, "unit": "T lane-op/s", "frac": s3_ops / lane_peak,
                      "peak_source": "measured: dependent-free fp32 FMA loop",
+                     "kind": "notional: the point-iterations of Eq. 5 (the candidate evaluations of Eq. 7) at their lane-operations each; "
+                             "the k-means kernels sort or group a row once and then move K-1 boundaries on prefix sums, "
+                             "so what binds them is latency (one warp per row runs the fp64 iterations), not this work",
                      "hbm_gbs": s3_gbs, "hbm_frac": s3_gbs / pk["hbm"],
                      "executed": s3_exec, "executed_frac": None if s3_exec is None else s3_exec / lane_peak},
         "quantize_layer": {"bound": "tensor", "achieved": s4, "peak": pk["tf_burst"], "unit": "TFLOP/s", "frac": s4 / pk["tf_burst"],
