@@ -475,6 +475,34 @@ def test_stage4_affine_isolated(lq, h, r, c, bits, group):
     assert abs(loss / loss_o - 1) <= LOSS_TOL
 
 
+@pytest.mark.parametrize("grid_type", ["nonuniform", "affine"])
+def test_stage4_many_rows_odd_count(lq, h, grid_type):
+    """From 24 rows per SM on a warp of the in-block kernel carries two rows: an odd row count (the last warp has one
+    row), a ragged last block, both grid types."""
+    r, c, bits = 3601, 200, 3
+    L = synth.make_layer("c2", r, c, 2 * c, seed=77)
+    W = f64(L.W)
+    U, dinv, _, _ = O.prepare_hinv(O.hessian(f64(L.X)), 0.01)
+    U32 = torch.from_numpy(U).float()
+    if grid_type == "nonuniform":
+        G32 = torch.from_numpy(O.fit_grid_nonuniform(W, dinv, bits, 4.0, 20)).float()
+        codes_o, What_o, loss_o, Wpre = O.quantize_layer(W, f64(U32), grid=f64(G32), bits=bits, block=128, return_pre=True)
+        cfg = lq.Config.make(grid="nonuniform", bits=bits)
+        codes, What, loss = run_stage4(lq, h, L.W, U32, cfg, grid=G32)
+        frac, n_rows = codes_agree(codes, codes_o, Wpre, nu_points(G32))
+        assert np.array_equal(What, np.take_along_axis(f64(G32), codes, 1))
+    else:
+        So, Zo = O.fit_grid_affine(W, dinv, bits, 4.0, 100, 40, 8)
+        S32, Z32 = torch.from_numpy(So).float(), torch.from_numpy(Zo).int()
+        codes_o, What_o, loss_o, Wpre = O.quantize_layer(W, f64(U32), scale=f64(S32), zero=f64(Z32), bits=bits,
+                                                         group=100, block=128, return_pre=True)
+        cfg = lq.Config.make(grid="affine", bits=bits, group=100, T=40, t=8)
+        codes, What, loss = run_stage4(lq, h, L.W, U32, cfg, scale=S32, zero=Z32)
+        frac, n_rows = codes_agree(codes, codes_o, Wpre, aff_points(f64(S32), f64(Z32), 1 << bits, 100, c))
+    print(f"stage 4, {r} rows, {grid_type}: {100 * frac:.4f} % of codes differ ({n_rows} rows)")
+    assert abs(loss / loss_o - 1) <= LOSS_TOL
+
+
 def test_stage4_identity_hessian_is_round_to_nearest(lq, h):
     g = torch.Generator().manual_seed(2)
     r, c = 48, 256
