@@ -300,6 +300,26 @@ update_kernel(double* __restrict__ A, int64_t cp, int k, int part, int i_base, i
         if (t <= nx) { i = t; j = nx; } else { i = nx; j = t; }
         r0 = ((blockIdx.x >> 1) & 1) * 64;
         c0 = (blockIdx.x & 1) * 64;
+    } else if (part >= 10) {
+        // parts 0 and 2 of the deferred sweep in one launch (part - 10): first the block rows [i_base, k) (part 2:
+        // [i_base, k-1)) over the whole width, one grid row each; then the block rows [0, i_base) over the j_base block
+        // columns of the outer block, packed into grid rows of the same width
+        const int o_lo = i_base, obw = j_base;
+        const int nA = k - o_lo - (part == 12 ? 1 : 0);
+        if (static_cast<int>(blockIdx.y) < nA) {
+            i = o_lo + blockIdx.y;
+            j = blockIdx.x >> 1;
+            c0 = (blockIdx.x & 1) * 64;
+        } else {
+            const int64_t lin = static_cast<int64_t>(blockIdx.y - nA) * gridDim.x + blockIdx.x;
+            i = static_cast<int>(lin / (2 * obw));
+            if (i >= o_lo) return;
+            const int xx = static_cast<int>(lin - static_cast<int64_t>(i) * (2 * obw));
+            j = o_lo + (xx >> 1);
+            c0 = (xx & 1) * 64;
+        }
+        if (part == 12 && (j == k - 1 || i == k - 1)) return;
+        r0 = 0;
     } else {
         j = j_base + (blockIdx.x >> 1);
         i = i_base + blockIdx.y;
@@ -423,11 +443,21 @@ slice_rows_kernel(const double* __restrict__ P, int64_t ldp, int K, int* __restr
 // Exponents of the columns j >= col0 of the K rows of A that start at row0 (the final rows of U of an outer block).
 __global__ void __launch_bounds__(256)
 col_exp_kernel(const double* __restrict__ A, int64_t cp, int64_t row0, int K, int64_t col0, int* __restrict__ ex, int int8) {
-    const int64_t j = col0 + blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (j >= cp) return;
+    // 32 columns per CTA, eight threads per column (each takes every eighth row), so that a column's K loads do not queue
+    // behind one another in one thread
+    __shared__ double part[8][32];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int64_t j = col0 + blockIdx.x * 32LL + tx;
     double mx = 0.0;
-    for (int kx = 0; kx < K; ++kx) mx = fmax(mx, fabs(LQ_AT(A + (row0 + kx) * cp + j)));
-    LQ_AT(ex + j) = isfinite(mx) ? (int8 ? exp_for8(mx) : exp_for(mx)) : 0;
+    if (j < cp)
+        for (int kx = ty; kx < K; kx += 8) mx = fmax(mx, fabs(LQ_AT(A + (row0 + kx) * cp + j)));
+    part[ty][tx] = mx;
+    __syncthreads();
+    if (ty == 0 && j < cp) {
+#pragma unroll
+        for (int q = 1; q < 8; ++q) mx = fmax(mx, part[q][tx]);
+        LQ_AT(ex + j) = isfinite(mx) ? (int8 ? exp_for8(mx) : exp_for(mx)) : 0;
+    }
 }
 
 // Slices of those columns, transposed: SL[s][j][kx] = digit s of A[row0 + kx][j].  64 x 64 tiles through shared memory.
@@ -767,7 +797,7 @@ int deferred_update(lq_handle* h, cudaStream_t st, double* A, int64_t cp, int64_
     else slice_rows_kernel<__nv_bfloat16><<<static_cast<unsigned>(top), 256, 0, st>>>(Pob, LDP, K, ex, static_cast<__nv_bfloat16*>(SL), cp);
     LQ_LAUNCH_CHECK();
     if (n_right > 0) {
-        col_exp_kernel<<<static_cast<unsigned>(lq_ceil_div(n_right, 256)), 256, 0, st>>>(A, cp, top, K, right0, ex, i8 ? 1 : 0);
+        col_exp_kernel<<<static_cast<unsigned>(lq_ceil_div(n_right, 32)), 256, 0, st>>>(A, cp, top, K, right0, ex, i8 ? 1 : 0);
         LQ_LAUNCH_CHECK();
         dim3 g(static_cast<unsigned>(lq_ceil_div(n_right, 64)), static_cast<unsigned>(lq_ceil_div(K, 64)));
         if (i8) slice_cols_kernel<uint8_t><<<g, 256, 0, st>>>(A, cp, top, K, right0, ex, static_cast<uint8_t*>(SL), cp);
@@ -1001,14 +1031,10 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
             if (!fork || k == o_lo) {
                 if (rest_pending) LQ_CUDA_TRY(cudaStreamWaitEvent(cs, h->ev_rest, 0));
                 rest_pending = false;
-                if (rows_in > 0) {
-                    dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(rows_in));
-                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, cs>>>(A, cp, ki, 0, static_cast<int>(o_lo), 0, Pk, LDP, Qk);
-                    LQ_LAUNCH_CHECK();
-                }
-                if (o_lo > 0) {
-                    dim3 g(static_cast<unsigned>(2 * obw), static_cast<unsigned>(o_lo));
-                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, cs>>>(A, cp, ki, 0, 0, static_cast<int>(o_lo), Pk, LDP, Qk);
+                if (rows_in > 0 || o_lo > 0) {      // both regions in one launch: one partial round of CTAs instead of two
+                    const int64_t rows_b = lq_ceil_div(o_lo * 2 * obw, 2 * nblk);
+                    dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(rows_in + rows_b));
+                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, cs>>>(A, cp, ki, 10, static_cast<int>(o_lo), obw, Pk, LDP, Qk);
                     LQ_LAUNCH_CHECK();
                 }
                 continue;
@@ -1020,14 +1046,10 @@ extern "C" int lq_prepare_hinv(lq_handle* h, void* stream, const float* H, int64
             if (rows_in > 1 || o_lo > 0) {
                 LQ_CUDA_TRY(cudaEventRecord(h->ev_next, cs));
                 LQ_CUDA_TRY(cudaStreamWaitEvent(aux, h->ev_next, 0));
-                if (rows_in > 1) {             // block row k-1 is part of "next"
-                    dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(rows_in - 1));
-                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, aux>>>(A, cp, ki, 2, static_cast<int>(o_lo), 0, Pk, LDP, Qk);
-                    LQ_LAUNCH_CHECK();
-                }
-                if (o_lo > 0) {
-                    dim3 g(static_cast<unsigned>(2 * obw), static_cast<unsigned>(o_lo));
-                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, aux>>>(A, cp, ki, 2, 0, static_cast<int>(o_lo), Pk, LDP, Qk);
+                {                              // block row k-1 is part of "next"; both regions in one launch
+                    const int64_t rows_b = lq_ceil_div(o_lo * 2 * obw, 2 * nblk);
+                    dim3 g(static_cast<unsigned>(2 * nblk), static_cast<unsigned>(rows_in - 1 + rows_b));
+                    update_kernel<<<g, GEMM_THREADS, GEMM_SMEM, aux>>>(A, cp, ki, 12, static_cast<int>(o_lo), obw, Pk, LDP, Qk);
                     LQ_LAUNCH_CHECK();
                 }
                 LQ_CUDA_TRY(cudaEventRecord(h->ev_rest, aux));
