@@ -185,6 +185,10 @@ struct lq_tc_gemm_args {
     int int8_ops;
     int a_signed[LQ_TC_MAX_PASS], b_signed[LQ_TC_MAX_PASS];
     float lvl_scale[LQ_TC_MAX_LVL];
+    // D_first != nullptr (integer operands, n_lvl >= 2, one chunk per level, accumulate == 0): the first level's scaled
+    // sum is stored to D_first (same shape and leading dimension as D) and does not enter the running sum that goes to
+    // D.  An exact leading level and the rounded sum of the other levels then come out of one launch.
+    float* D_first;
 };
 int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a);
 

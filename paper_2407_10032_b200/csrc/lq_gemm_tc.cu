@@ -94,6 +94,7 @@ struct KParams {
     int bk_elems;
     uint32_t idesc_pass[LQ_TC_MAX_PASS];
     float lvl_scale[LQ_TC_MAX_LVL];
+    int first_out;            // the first level's sum is stored through the second output map and leaves the running sum
 };
 
 // ---------------------------------------------------------------- PTX wrappers ----
@@ -362,7 +363,8 @@ __device__ __forceinline__ void seg_item(const Seg& g, int q, int& pass, int& kb
 template <int CTAS, bool I8>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                  const __grid_constant__ CUtensorMap map_d, const __grid_constant__ KParams p) {
+                  const __grid_constant__ CUtensorMap map_d, const __grid_constant__ CUtensorMap map_d1,
+                  const __grid_constant__ KParams p) {
     typedef Cfg<CTAS> C;
     constexpr int STAGES = C::STAGES;
     constexpr bool PAIR = CTAS == 2;
@@ -523,11 +525,42 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             int tm, tn;
             tile_coords(p, pc.tile, tm, tn);
             const int m0 = tm * C::TILE_M + static_cast<int>(rank) * BM, n0 = tn * BN;
+            // the running sums of this thread's row go to D: scale -> swizzled slab -> TMA store or reduce-add
+            auto store_tile = [&](const CUtensorMap* md, bool reduce) {
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) {
+                    const int col0 = n0 + hf * (BN / 2) + ch * EPI_COLS;
+                    if (col0 < p.N && m0 < p.M) {
+                        if (leader) bulk_wait_read<0>();          // the slab buffer has been read out
+                        group_bar_sync(1 + hf);
+                        uint8_t* rowp = my_buf + row * 128u;
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            float4 o;
+                            o.x = p.alpha * accr[ch * 32 + 4 * j + 0];
+                            o.y = p.alpha * accr[ch * 32 + 4 * j + 1];
+                            o.z = p.alpha * accr[ch * 32 + 4 * j + 2];
+                            o.w = p.alpha * accr[ch * 32 + 4 * j + 3];
+                            *reinterpret_cast<float4*>(rowp + ((j ^ (row & 7u)) << 4)) = o;
+                        }
+                        fence_async_smem();
+                        group_bar_sync(1 + hf);
+                        if (leader) {
+                            if (reduce) tma_reduce_add_2d(md, my_buf_s, col0, m0);
+                            else tma_store_2d(md, my_buf_s, col0, m0);
+                            bulk_commit();
+                        }
+                    }
+                }
+            };
+            const bool first_out = I8 && p.first_out != 0;
+            bool voted_out = false;
             for (int sg = pc.s0; sg < pc.s1; ++sg, ++it) {
                 const uint32_t acc = it & 1;
                 const uint32_t acc_phase = (it >> 1) & 1;
                 if (!mbar_wait(bar_tfull + 8 * acc, acc_phase, abortp, p, 4)) { alive = false; break; }
                 tc_fence_after();
+                const bool fresh = sg == pc.s0 || (first_out && sg == pc.s0 + 1);       // this segment starts the running sum
 #pragma unroll
                 for (int ch = 0; ch < 4; ++ch) {
                     uint32_t v[32];
@@ -536,14 +569,14 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     if (I8) {
                         // int32 partial sums (exact) -> fp32, scaled by the level's power of two
                         const float sc = p.lvl_scale[p.n_lvl > 0 ? sg / p.n_chunks : 0];
-                        if (sg == pc.s0) {
+                        if (fresh) {
 #pragma unroll
                             for (int i = 0; i < 32; ++i) accr[ch * 32 + i] = static_cast<float>(static_cast<int>(v[i])) * sc;
                         } else {
 #pragma unroll
                             for (int i = 0; i < 32; ++i) accr[ch * 32 + i] = fmaf(static_cast<float>(static_cast<int>(v[i])), sc, accr[ch * 32 + i]);
                         }
-                    } else if (sg == pc.s0) {
+                    } else if (fresh) {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) accr[ch * 32 + i] = __uint_as_float(v[i]);
                     } else {
@@ -557,35 +590,18 @@ lq_tc_gemm_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     if (mma_cta) mbar_arrive(bar_tempty + 8 * acc);
                     else mbar_arrive_remote(bar_tempty + 8 * acc, 0);
                 }
+                if (first_out && sg == pc.s0) {
+                    // The first level on its own goes out now, while the tensor core works on the next level.  The vote is
+                    // the same barrier as the one behind the loop: a warp whose wait ran out above meets this one there.
+                    if (group_bar_or(1 + hf, false)) { voted_out = true; break; }
+                    store_tile(&map_d1, false);
+                }
             }
+            if (voted_out) { alive = false; break; }
             // A wait may have run out in some warps of the group and not in others: the group leaves together, or
             // the warps that went on would wait at the slab barriers below for warps that never come.
             if (group_bar_or(1 + hf, !alive)) { alive = false; break; }
-#pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-                const int col0 = n0 + hf * (BN / 2) + ch * EPI_COLS;
-                if (col0 < p.N && m0 < p.M) {
-                    if (leader) bulk_wait_read<0>();          // the slab buffer has been read out
-                    group_bar_sync(1 + hf);
-                    uint8_t* rowp = my_buf + row * 128u;
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        float4 o;
-                        o.x = p.alpha * accr[ch * 32 + 4 * j + 0];
-                        o.y = p.alpha * accr[ch * 32 + 4 * j + 1];
-                        o.z = p.alpha * accr[ch * 32 + 4 * j + 2];
-                        o.w = p.alpha * accr[ch * 32 + 4 * j + 3];
-                        *reinterpret_cast<float4*>(rowp + ((j ^ (row & 7u)) << 4)) = o;
-                    }
-                    fence_async_smem();
-                    group_bar_sync(1 + hf);
-                    if (leader) {
-                        if (p.accumulate) tma_reduce_add_2d(&map_d, my_buf_s, col0, m0);
-                        else tma_store_2d(&map_d, my_buf_s, col0, m0);
-                        bulk_commit();
-                    }
-                }
-            }
+            store_tile(&map_d, p.accumulate != 0);
         }
         if (leader) bulk_wait<0>();
     }
@@ -693,7 +709,7 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
     const int ctas_per_tile = pairs > 0 ? 2 : 1;
     const int b_rows_box = BN / ctas_per_tile;
 
-    CUtensorMap map_a, map_b, map_d;
+    CUtensorMap map_a, map_b, map_d, map_d1;
     const bool i8 = a.int8_ops != 0;
     const int bk_elems = i8 ? 2 * BK : BK;                 // a k-step is one 128-byte swizzle row of either type
     const CUtensorMapDataType op_dt = i8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
@@ -702,6 +718,14 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
         !make_map_2d(&map_b, op_dt, op_bytes, a.B_all, a.K, a.b_rows, a.ldb, bk_elems, b_rows_box) ||
         !make_map_2d(&map_d, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.D, a.N, a.M, a.ldd, EPI_COLS, BM))
         return LQ_ERR_CUDA;
+    map_d1 = map_d;
+    if (a.D_first) {
+        // the first level's sum on its own: integer operands, at least two levels, one segment per level, nothing added to D
+        if (!i8 || a.n_lvl < 2 || a.accumulate || (reinterpret_cast<uintptr_t>(a.D_first) & 15) ||
+            a.chunk_kb < lq_ceil_div(a.K, bk_elems))
+            return LQ_ERR_INVALID_ARG;
+        if (!make_map_2d(&map_d1, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, a.D_first, a.N, a.M, a.ldd, EPI_COLS, BM)) return LQ_ERR_CUDA;
+    }
 
     KParams p;
     p.M = static_cast<int>(a.M);
@@ -738,6 +762,7 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
         p.idesc_pass[i] = ctas_per_tile == 2 ? Cfg<2>::idesc_i8(a.a_signed[i] != 0, a.b_signed[i] != 0)
                                              : Cfg<1>::idesc_i8(a.a_signed[i] != 0, a.b_signed[i] != 0);
     for (int i = 0; i < LQ_TC_MAX_LVL; ++i) p.lvl_scale[i] = a.lvl_scale[i];
+    p.first_out = a.D_first ? 1 : 0;
     if (p.num_tiles == 0) return LQ_OK;
     {
         const int k_blocks = static_cast<int>(lq_ceil_div(a.K, bk_elems));
@@ -784,16 +809,16 @@ int lq_tc_gemm(lq_handle* h, cudaStream_t stream, const lq_tc_gemm_args& a) {
         attr.val.clusterDim.x = 2; attr.val.clusterDim.y = 1; attr.val.clusterDim.z = 1;
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
-        const cudaError_t le = i8 ? cudaLaunchKernelEx(&cfg, lq_tc_gemm_kernel<2, true>, map_a, map_b, map_d, p)
-                                  : cudaLaunchKernelEx(&cfg, lq_tc_gemm_kernel<2, false>, map_a, map_b, map_d, p);
+        const cudaError_t le = i8 ? cudaLaunchKernelEx(&cfg, lq_tc_gemm_kernel<2, true>, map_a, map_b, map_d, map_d1, p)
+                                  : cudaLaunchKernelEx(&cfg, lq_tc_gemm_kernel<2, false>, map_a, map_b, map_d, map_d1, p);
         if (le != cudaSuccess) {
             cudaGetLastError();
             return LQ_ERR_CUDA;
         }
         lq_launches_total.fetch_add(1, std::memory_order_relaxed);
     } else {
-        if (i8) lq_tc_gemm_kernel<1, true><<<active, NUM_THREADS, Cfg<1>::SMEM_BYTES, stream>>>(map_a, map_b, map_d, p);
-        else lq_tc_gemm_kernel<1, false><<<active, NUM_THREADS, Cfg<1>::SMEM_BYTES, stream>>>(map_a, map_b, map_d, p);
+        if (i8) lq_tc_gemm_kernel<1, true><<<active, NUM_THREADS, Cfg<1>::SMEM_BYTES, stream>>>(map_a, map_b, map_d, map_d1, p);
+        else lq_tc_gemm_kernel<1, false><<<active, NUM_THREADS, Cfg<1>::SMEM_BYTES, stream>>>(map_a, map_b, map_d, map_d1, p);
         LQ_LAUNCH_CHECK();
     }
     return LQ_OK;

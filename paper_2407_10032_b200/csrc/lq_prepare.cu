@@ -849,6 +849,30 @@ int deferred_update(lq_handle* h, cudaStream_t st, double* A, int64_t cp, int64_
             const int64_t col0 = side == 0 ? b0 : right0;
             const int64_t ncols = side == 0 ? top - b0 : n_right;
             if (ncols <= 0) continue;
+            if (i8) {
+                // integer digits: one launch, the leading pair as its first level with an output of its own
+                lq_tc_gemm_args g = tail;
+                for (int ps = tail.n_pass; ps > 0; --ps) {
+                    g.a_signed[ps] = tail.a_signed[ps - 1]; g.b_signed[ps] = tail.b_signed[ps - 1];
+                    g.a_row_off[ps] = pair_s[ps - 1] * cp + b0;
+                    g.b_row_off[ps] = pair_t[ps - 1] * cp + col0;
+                }
+                g.a_signed[0] = g.b_signed[0] = 1;
+                g.a_row_off[0] = b0;
+                g.b_row_off[0] = col0;
+                g.n_pass = tail.n_pass + 1;
+                for (int l = tail.n_lvl; l > 0; --l) { g.lvl_npass[l] = tail.lvl_npass[l - 1]; g.lvl_scale[l] = tail.lvl_scale[l - 1]; }
+                g.lvl_npass[0] = 1;
+                g.lvl_scale[0] = lead.lvl_scale[0];
+                g.n_lvl = tail.n_lvl + 1;
+                g.D_first = Ta + col0;
+                g.D = Tb + col0;
+                g.M = b1 - b0;
+                g.N = ncols;
+                g.upper_only = side == 0 ? 1 : 0;
+                int rc = lq_tc_gemm(h, st, g);
+                if (rc) return rc;
+            } else
             for (int which = 0; which < 2; ++which) {
                 lq_tc_gemm_args g = which == 0 ? lead : tail;
                 g.D = (which == 0 ? Ta : Tb) + col0;
