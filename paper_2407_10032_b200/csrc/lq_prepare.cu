@@ -366,7 +366,7 @@ crit_kernel(double* __restrict__ A, int64_t cp, int k, int phase, double* __rest
 constexpr int OBB = 8;                   // block columns per outer block
 constexpr int LDP = OBB * NB;            // row stride of the panel buffer and of the slices
 constexpr int NSL = 5;                   // slices
-constexpr int64_t BAND = 4096;           // rows of the deferred region handled per product
+constexpr int64_t BAND = 8192;           // rows of the deferred region handled per product
 
 __device__ __forceinline__ int exp_for(double mx) { return mx > 0.0 ? ilogb(mx) + 2 : 0; }
 
