@@ -567,7 +567,7 @@ def run_ours(args):
         flops = float(c) * c * n
         ach = flops / (stage_ms[0] * 1e-3) / 1e12
         peak = pk["tf_burst"]
-        traffic = 6680238080 if args.workload == "llama3-8b-q_proj-nu4" else None      # dram read + write of this launch, one ncu capture (it varies with how far the CTA pairs drift apart: 4.8 - 7.7 GB seen)
+        traffic = 4777421056 if args.workload == "llama3-8b-q_proj-nu4" else None      # dram read + write of this launch, one ncu capture (it varies with how far the CTA pairs drift apart: 4.8 - 7.7 GB seen)
         roof = {"bound": "tensor", "kernel": "lq_tc_gemm_kernel (stage 1, H += 2XX^T)", "achieved": ach, "peak": peak,
                 "unit": "TFLOP/s", "frac": ach / peak, "traffic": traffic, "peak_source": pk["src"] + " burst bf16",
                 "frac_of_sustained": ach / pk["tf_sust"], "flops_per_launch": flops,
