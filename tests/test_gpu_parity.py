@@ -742,6 +742,34 @@ def test_bounded_wait_runs_out_and_the_handle_recovers(lq):
         lq.lq_destroy(hh)
 
 
+def test_bounded_wait_runs_out_in_the_integer_product_of_stage2(lq):
+    """The same host-made failure in the product that stage 2 runs on the integer tensor-core path (levels, the leading
+    pair stored on its own from inside the segment loop): every wait runs into its limit, the call returns, the first
+    recorded status is LQ_ERR_TIMEOUT, and the handle then factorises the same matrix correctly."""
+    hh = lq.lq_create(0)
+    try:
+        c = 1536
+        L = synth.make_layer("c2", 8, c, 2 * c, seed=21)
+        H32 = torch.from_numpy(O.hessian(f64(L.X))).float().cuda()
+        U = torch.empty(c, c, device="cuda")
+        dinv = torch.empty(c, device="cuda")
+        ws = ws_for(lq, lq.lq_prepare_hinv_workspace(c))
+        lq.lq_testing_set_prepare_defer_min_blocks(hh, 0)      # 12 blocks: the updates of the tiles outside an outer block are deferred
+        lq.lq_testing_set_wait_limit_ns(hh, 2_000_000)
+        lq.lq_testing_inject_stall(hh, True)
+        lq.lq_prepare_hinv(hh, H32, U, dinv, ws, 0.01)
+        st, info = lq.lq_sync_status(hh, raise_on_error=False)
+        assert st == 7, (st, info)
+        lq.lq_testing_inject_stall(hh, False)
+        lq.lq_testing_set_wait_limit_ns(hh, 0)
+        lq.lq_prepare_hinv(hh, H32, U, dinv, ws, 0.01)
+        assert lq.lq_sync_status(hh, raise_on_error=False)[0] == 0
+        Uo, dinvo, _, _ = O.prepare_hinv(f64(H32), 0.01)
+        assert np.abs(f64(U) - Uo).max() <= 3e-7 * np.abs(Uo).max()
+    finally:
+        lq.lq_destroy(hh)
+
+
 def test_more_rows_than_one_grid_dimension_holds(lq, h):
     """r > 65535: the launches that put rows on the second grid dimension go in slabs."""
     r, c = 65600, 128
