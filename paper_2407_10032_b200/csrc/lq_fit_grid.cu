@@ -21,8 +21,8 @@
 
 namespace {
 
-constexpr int KM_THREADS = 256;
-constexpr int KM_WARPS = KM_THREADS / 32;
+// threads of the long-row kernel (1024 were no faster for K = 4 and do not fit the 2 K doubles of cluster sums per thread for K = 16)
+__host__ __device__ constexpr int km_threads(int) { return 512; }
 
 // scal[1] = mean_j ln(dinv_j)
 __global__ void log_mean_kernel(const float* __restrict__ dinv, int64_t c, double* __restrict__ scal, lq_dev_status* st) {
@@ -625,9 +625,10 @@ kmeans_bucket_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
 // Rows too long to sort in shared memory: the row is staged once in shared memory in its own
 // type and every iteration visits every weight (compares and cluster sums in fp64).
 template <int K, typename T>
-__global__ void __launch_bounds__(KM_THREADS)
+__global__ void __launch_bounds__(km_threads(K))
 kmeans_rows_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int64_t c, const double* __restrict__ s64,
                    float* __restrict__ grid, int n_iter) {
+    constexpr int KM_THREADS = km_threads(K), KM_WARPS = KM_THREADS / 32;
     extern __shared__ unsigned char wrow_raw[];
     T* wrow = reinterpret_cast<T*>(wrow_raw);
     __shared__ double g[K];
@@ -747,7 +748,9 @@ int launch_kmeans(cudaStream_t st, int sms, const T* W, int64_t ldw, int64_t r, 
         if (attr_set.first()) {
             LQ_CUDA_TRY(cudaFuncSetAttribute(kmeans_rows_kernel<K, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
         }
-        kmeans_rows_kernel<K, T><<<static_cast<unsigned>(r < sms ? r : sms), KM_THREADS, smem, st>>>(W, ldw, r, c, s64, grid, n_iter);
+        // two CTAs per SM where two rows fit the shared memory: the loop is bound by the latency of its fp64 sums
+        const int64_t cap = static_cast<int64_t>(sms) * (2 * (smem + 8 * 1024) <= 227 * 1024 ? 2 : 1);
+        kmeans_rows_kernel<K, T><<<static_cast<unsigned>(r < cap ? r : cap), km_threads(K), smem, st>>>(W, ldw, r, c, s64, grid, n_iter);
     }
     LQ_LAUNCH_CHECK();
     return LQ_OK;
