@@ -312,8 +312,10 @@ __device__ __forceinline__ int value_bucket(double w, double lo, double scale) {
 }
 __device__ __forceinline__ int offs_half(const uint32_t* offs, int b) { return static_cast<int>((offs[b >> 1] >> ((b & 1) * 16)) & 0xffffu); }
 
-template <int K, typename T>
-__global__ void __launch_bounds__(KS_THREADS, 3)
+// NT threads: 256 for rows of 4096 weights (three CTAs per SM), 512 for longer ones (one or two CTAs per SM: more
+// threads for the phases that all of them share).
+template <int K, typename T, int NT>
+__global__ void __launch_bounds__(NT, NT == 256 ? 3 : 1)
 kmeans_bucket_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int n, const double* __restrict__ s64,
                      float* __restrict__ grid, int n_iter) {
     typedef typename KeyOf<T>::type KeyT;
@@ -321,23 +323,23 @@ kmeans_bucket_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
     dd2* coarse = reinterpret_cast<dd2*>(ks_smem);            // n / 8 + 1 coarse prefixes, then the n keys, then the counters
     KeyT* keys = reinterpret_cast<KeyT*>(coarse + (n / KS_CHUNK + 1));
     uint32_t* offs = reinterpret_cast<uint32_t*>(ks_smem + (((n / KS_CHUNK + 1) * sizeof(dd2) + (n + n / 32) * sizeof(KeyT) + 15) & ~size_t(15)));
-    __shared__ dd2 tot[KS_THREADS];                            // per-thread totals, then their exclusive scan
+    __shared__ dd2 tot[NT];                            // per-thread totals, then their exclusive scan
     __shared__ double g[K];
     __shared__ dd2 F[K + 1];
-    __shared__ KeyT ext[2][KS_THREADS / 32];                   // per-warp smallest and largest key
-    __shared__ int wsum[KS_THREADS / 32];
+    __shared__ KeyT ext[2][NT / 32];                   // per-warp smallest and largest key
+    __shared__ int wsum[NT / 32];
     __shared__ double rng[2];                                  // smallest weight of the row, buckets per unit of weight
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nch = n / KS_CHUNK;
-    const int cpt = nch > KS_THREADS ? nch / KS_THREADS : 1;   // chunks per thread
-    constexpr int WPT = KB_BUCKETS / 2 / KS_THREADS;           // counter words per thread in the scan
+    const int cpt = nch > NT ? nch / NT : 1;   // chunks per thread
+    constexpr int WPT = KB_BUCKETS / 2 / NT;           // counter words per thread in the scan
 
     for (int64_t row = blockIdx.x; row < r; row += gridDim.x) {
         const T* wp = W + row * ldw;
-        for (int i = tid; i < KB_BUCKETS / 8; i += KS_THREADS) reinterpret_cast<uint4*>(offs)[i] = make_uint4(0u, 0u, 0u, 0u);
+        for (int i = tid; i < KB_BUCKETS / 8; i += NT) reinterpret_cast<uint4*>(offs)[i] = make_uint4(0u, 0u, 0u, 0u);
         // smallest and largest weight of the row
         KeyT kmin = KeyOf<T>::pad(), kmax = 0;
-        for (int i = tid; i < c; i += KS_THREADS) {
+        for (int i = tid; i < c; i += NT) {
             const KeyT key = KeyOf<T>::make(LQ_AT(wp + i), i);
             kmin = key < kmin ? key : kmin;
             kmax = key > kmax ? key : kmax;
@@ -353,7 +355,7 @@ kmeans_bucket_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
         if (tid == 0) {
             KeyT k0 = ext[0][0], k1 = ext[1][0];
 #pragma unroll
-            for (int w = 1; w < KS_THREADS / 32; ++w) {
+            for (int w = 1; w < NT / 32; ++w) {
                 k0 = ext[0][w] < k0 ? ext[0][w] : k0;
                 k1 = ext[1][w] > k1 ? ext[1][w] : k1;
             }
@@ -366,7 +368,7 @@ kmeans_bucket_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
         __syncthreads();
         const double lo = rng[0], scale = rng[1];
         // histogram of the buckets
-        for (int i = tid; i < c; i += KS_THREADS) {
+        for (int i = tid; i < c; i += NT) {
             const int b = value_bucket(static_cast<double>(key_weight(KeyOf<T>::make(LQ_AT(wp + i), i))), lo, scale);
             atomicAdd(offs + (b >> 1), (b & 1) ? 0x10000u : 1u);
         }
@@ -404,7 +406,7 @@ kmeans_bucket_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
         }
         __syncthreads();
         // scatter: a bucket's counter hands out its positions
-        for (int i = tid; i < c; i += KS_THREADS) {
+        for (int i = tid; i < c; i += NT) {
             const KeyT key = KeyOf<T>::make(LQ_AT(wp + i), i);
             const int b = value_bucket(static_cast<double>(key_weight(key)), lo, scale);
             const uint32_t old = atomicAdd(offs + (b >> 1), (b & 1) ? 0x10000u : 1u);
@@ -447,13 +449,13 @@ kmeans_bucket_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
         tot[tid] = run;
         __syncthreads();
         if (warp == 0) {       // exclusive scan of the 256 thread totals: 8 per lane, then across the warp
-            dd2 loc[KS_THREADS / 32];
+            dd2 loc[NT / 32];
             dd2 acc;
             acc.s.hi = acc.s.lo = acc.sw.hi = acc.sw.lo = 0.0;
 #pragma unroll
-            for (int e = 0; e < KS_THREADS / 32; ++e) {
+            for (int e = 0; e < NT / 32; ++e) {
                 loc[e] = acc;
-                const dd2 v = tot[lane * (KS_THREADS / 32) + e];
+                const dd2 v = tot[lane * (NT / 32) + e];
                 acc.s = dd_add(acc.s, v.s);
                 acc.sw = dd_add(acc.sw, v.sw);
             }
@@ -474,11 +476,11 @@ kmeans_bucket_kernel(const T* __restrict__ W, int64_t ldw, int64_t r, int c, int
             excl.sw.lo = __shfl_up_sync(0xffffffffu, inc.sw.lo, 1);
             if (lane == 0) excl.s.hi = excl.s.lo = excl.sw.hi = excl.sw.lo = 0.0;
 #pragma unroll
-            for (int e = 0; e < KS_THREADS / 32; ++e) {
+            for (int e = 0; e < NT / 32; ++e) {
                 dd2 v;
                 v.s = dd_add(excl.s, loc[e].s);
                 v.sw = dd_add(excl.sw, loc[e].sw);
-                tot[lane * (KS_THREADS / 32) + e] = v;
+                tot[lane * (NT / 32) + e] = v;
             }
             if (lane == 31) LQ_AT(coarse + nch) = inc;          // grand total
         }
@@ -721,12 +723,19 @@ int launch_kmeans(cudaStream_t st, int sms, const T* W, int64_t ldw, int64_t r, 
         if (init == LQ_INIT_UNIFORM && n >= KB_MIN_N && bsmem <= 216 * 1024) {
             static lq_once_per_device battr_set;
             if (battr_set.first()) {
-                LQ_CUDA_TRY(cudaFuncSetAttribute(kmeans_bucket_kernel<K, T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 216 * 1024));
+                LQ_CUDA_TRY(cudaFuncSetAttribute(kmeans_bucket_kernel<K, T, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, 216 * 1024));
+                LQ_CUDA_TRY(cudaFuncSetAttribute(kmeans_bucket_kernel<K, T, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+            }
+            if (n > 8192 && bsmem <= 200 * 1024) {      // one row fills an SM's shared memory: 512 threads for it
+                kmeans_bucket_kernel<K, T, 512><<<static_cast<unsigned>(r < sms ? r : sms), 512, bsmem, st>>>(
+                    W, ldw, r, static_cast<int>(c), n, s64, grid, n_iter);
+                LQ_LAUNCH_CHECK();
+                return LQ_OK;
             }
             int per_sm = static_cast<int>((228 * 1024) / (bsmem + 10 * 1024));
             per_sm = per_sm < 1 ? 1 : (per_sm > 3 ? 3 : per_sm);
             const int64_t cap = static_cast<int64_t>(sms) * per_sm;
-            kmeans_bucket_kernel<K, T><<<static_cast<unsigned>(r < cap ? r : cap), KS_THREADS, bsmem, st>>>(
+            kmeans_bucket_kernel<K, T, 256><<<static_cast<unsigned>(r < cap ? r : cap), 256, bsmem, st>>>(
                 W, ldw, r, static_cast<int>(c), n, s64, grid, n_iter);
             LQ_LAUNCH_CHECK();
             return LQ_OK;
