@@ -73,9 +73,9 @@ typedef struct {
 /* ---- handle ------------------------------------------------------------------------- */
 
 /* Creates a handle bound to CUDA device `device` (allocates a few bytes of device memory
- * for the status word, one auxiliary stream and three events: lq_prepare_hinv forks part of its
- * work onto that stream and joins it back before it returns control of the caller's stream, so
- * to the caller everything still happens in stream order).  Fails with LQ_ERR_CUDA when no such
+ * for the status word, three streams of different priority and a few events: lq_prepare_hinv forks
+ * its sweep onto those streams and joins them back before it returns control of the caller's stream,
+ * so to the caller everything still happens in stream order; one lq_prepare_hinv per handle at a time).  Fails with LQ_ERR_CUDA when no such
  * device exists. */
 int lq_create(lq_handle** out, int device);
 int lq_destroy(lq_handle* h);
